@@ -1,0 +1,196 @@
+/*
+ * isc.h -- integer smoothing certification on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the Monte-Carlo PREDICT / CERTIFY loop of integer randomized smoothing
+ * (Lin, Lou, Xiong, Shahabi, "Integer-arithmetic-only Certified Robustness for
+ * Quantized Neural Networks", ICCV 2021).  For one uint8 image the loop draws N copies
+ * perturbed with discrete Gaussian noise (Def. 3.3, Eq. 2), evaluates an int8
+ * integer-only classifier f on each copy (Def. 3.4, Eq. 3) and counts the argmax
+ * labels; the counts give the predicted class and the certified l2 radius
+ * (Algorithm 1, Algorithm 2).
+ *
+ * Every step runs in CUDA kernels of this library; there is no CPU fallback.  All
+ * entry points return ISC_OK (0) or a negative isc_status; they never throw or abort,
+ * and on error the output arguments are left untouched.  ABSTAIN is not an error: the
+ * class is reported as -1 and the radius as 0.
+ *
+ * Pointers are HOST pointers unless the argument is documented otherwise.  The caller
+ * owns everything it passes; the library copies what it keeps.  Calls on one model
+ * handle must not overlap in time (the handle owns its device work space); different
+ * handles are independent.  `cuda_stream` is a cudaStream_t passed as void* (NULL =
+ * the default stream); each call returns after its work on that stream has completed.
+ */
+#ifndef ISC_H_
+#define ISC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ISC_OK = 0,
+    ISC_ERR_ARG = -1,          /* null pointer, value out of range                          */
+    ISC_ERR_SHAPE = -2,        /* layer list does not type-check (channels, sizes, tensors) */
+    ISC_ERR_UNSUPPORTED = -3,  /* valid, but outside what the kernels implement             */
+    ISC_ERR_NOMEM = -4,        /* host or device allocation failed                          */
+    ISC_ERR_CUDA = -5,         /* a CUDA call or kernel launch failed                       */
+    ISC_ERR_TIMEOUT = -6       /* a bounded device-side wait expired; results discarded     */
+} isc_status;
+
+typedef enum { ISC_CONV2D = 0, ISC_FC = 1, ISC_GAVGPOOL = 2, ISC_MAXPOOL = 3 } isc_op;
+
+/*
+ * One layer of the quantized base classifier f.  Tensor 0 is the (noisy, saturated)
+ * uint8 network input; layer i reads tensor `in_tensor` (<= i) and writes tensor i+1;
+ * the last tensor holds the n_classes logits.  The paper delegates the layer
+ * arithmetic to the integer-only quantization scheme it cites (Sec. 1 and Sec. 2,
+ * "Model Compression: Quantization"); this library fixes it as follows, with
+ * rs(v, n) = floor(v / 2^n + 1/2) evaluated exactly:
+ *
+ *   conv / FC : acc[o] = bias[o] + sum_{c,r,s} (a[c, y*stride+r-pad, x*stride+s-pad] - zp_in) * w[o,c,r,s]
+ *               (taps outside the image contribute 0), int32 accumulation;
+ *               v = rs(acc * mult[o], 31 + shift[o]);
+ *               if res_tensor >= 0:  v += rs((r[o,y,x] - zp_res) * res_mult, 31 - res_shift);
+ *               out = min(127, max(lo, v + zp_out)),  lo = relu ? max(-128, zp_out) : -128.
+ *   global average pool : s = sum over pixels of (a - zp_in); out = clamp(rs(s * mult[0], 31 + shift[0]) + zp_out).
+ *   max pool  : integer maximum over the taps inside the image; zero-point unchanged.
+ *
+ * Ranges: mult in [2^30, 2^31), shift in [0, 31], res_mult in [2^30, 2^31) when a
+ * residual is present, res_shift in [-4, 4], zero-points in [-128, 127] (zp_in of a
+ * layer reading tensor 0 in [0, 255]).  Weights are symmetric int8 (zero-point 0).
+ */
+typedef struct {
+    int32_t op;                       /* isc_op                                               */
+    int32_t in_tensor, res_tensor;    /* res_tensor = -1: no residual add                     */
+    int32_t cin, cout, kh, kw, stride, pad; /* FC: 1x1 on a 1x1 map; pools: cout = cin        */
+    int32_t relu;                     /* 1: lower clamp is max(-128, zp_out)                  */
+    int32_t zp_in, zp_out, zp_res;
+    const int8_t *w;                  /* [cout][cin][kh][kw]; NULL for pools                  */
+    const int32_t *bias;              /* [cout]; NULL for pools                               */
+    const int32_t *mult;              /* [cout]; pools: [1]                                   */
+    const int8_t *shift;              /* [cout]; pools: [1]                                   */
+    int32_t res_mult, res_shift;
+} isc_layer;
+
+typedef struct isc_model isc_model;   /* opaque; owns the device copies of all parameters    */
+
+/*
+ * isc_load_qmodel -- validate a layer list, repack it for the GPU and upload it.
+ * The base classifier f of Def. 3.4 / Algorithm 1's "base function f".
+ *   layers[n_layers] : as above; may be freed on return.
+ *   in_c, in_h, in_w : shape of the CHW uint8 network input.
+ *   n_classes        : size of the last tensor (must be C x 1 x 1 with C = n_classes).
+ *   out              : receives the handle; release it with isc_free_qmodel.
+ * Errors: ISC_ERR_ARG, ISC_ERR_SHAPE, ISC_ERR_UNSUPPORTED, ISC_ERR_NOMEM, ISC_ERR_CUDA.
+ */
+int isc_load_qmodel(const isc_layer *layers, int n_layers, int in_c, int in_h, int in_w,
+                    int n_classes, isc_model **out);
+
+void isc_free_qmodel(isc_model *m);
+
+/*
+ * isc_predict -- Algorithm 2 (Appendix C): N noisy evaluations, top two vote counts
+ * (n_A, n_B), two-sided exact binomial test of n_A out of n_A + n_B at 1/2; the class
+ * is returned iff the p-value is <= alpha, else -1 (ABSTAIN).
+ *   x_u8       : host, CHW, in_c*in_h*in_w bytes.
+ *   seed, image_id : select the random stream (see isc_sample_counts); phase 2 is used.
+ *   N >= 1, sigma > 0 (noise std in [0,1] pixel units, i.e. 255*sigma pixel levels),
+ *   0 < alpha < 1.
+ *   out_class  : host, one int32.   out_counts : host, n_classes int32, or NULL.
+ */
+int isc_predict(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id,
+                int64_t N, double sigma, double alpha, void *cuda_stream,
+                int32_t *out_class, int32_t *out_counts);
+
+/*
+ * isc_certify -- Algorithm 1: N0 noisy evaluations select the class c_A (phase 0), N
+ * fresh ones count its votes n_A (phase 1); p_A is the one-sided (1 - alpha)
+ * Clopper-Pearson lower bound of n_A out of N; if p_A > 1/2 the result is c_A with
+ * radius sigma * Phi^-1(p_A), Phi the standard normal cdf, else ABSTAIN (-1, 0.0).
+ * The radius is in the same units as sigma.
+ *   out_counts0 / out_counts : host, n_classes int32 each (votes of the two phases), or NULL.
+ */
+int isc_certify(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id,
+                int64_t N0, int64_t N, double sigma, double alpha, void *cuda_stream,
+                int32_t *out_class, double *out_radius,
+                int32_t *out_counts0, int32_t *out_counts);
+
+/*
+ * isc_certify_batch -- Algorithm 1 for n_images images; image i uses image_id0 + i and
+ * gives exactly what isc_certify gives for it.
+ *   x_u8        : [n_images][C][H][W] bytes; a HOST pointer, or a DEVICE pointer when
+ *                 x_on_device != 0 (the images are then read in place).
+ *   out_class[n_images], out_radius[n_images] : host.
+ *   out_counts0 / out_counts : host, [n_images][n_classes] int32, or NULL.
+ */
+int isc_certify_batch(isc_model *m, const uint8_t *x_u8, int x_on_device, int n_images,
+                      uint64_t seed, uint64_t image_id0, int64_t N0, int64_t N,
+                      double sigma, double alpha, void *cuda_stream,
+                      int32_t *out_class, double *out_radius,
+                      int32_t *out_counts0, int32_t *out_counts);
+
+/*
+ * isc_sample_counts -- the Monte-Carlo loop alone (Algorithm 1 steps 1-4, Algorithm 2
+ * steps 1-2) for samples j = first_sample .. first_sample + n_samples - 1 of one image:
+ * draw delta_j, evaluate f(clamp(x + delta_j, 0, 255)), count the argmax label (ties go
+ * to the lowest class index).  Counts over a range equal the sum of the counts over any
+ * partition of it, whatever the launch batch.
+ * Random stream: element e = (c*H + h)*W + w of sample j takes output word (e & 3) of
+ * Philox4x32-10 with key (seed low, seed high) and counter
+ *   (e >> 2, j low 32, image_id low 32, phase | (j >> 32 & 0xFF) << 8 | (image_id >> 32 & 0xFFFF) << 16),
+ * and maps that uniform u to the smallest level z with u < cum[z], where cum is the
+ * 2^-32-grid CDF of Eq. 2 on the integer pixel levels with std 255*sigma, cut at
+ * +-ceil(7*255*sigma).  Requires j < 2^40, image_id < 2^48, 0 <= phase < 256.
+ *   out_counts : host, n_classes int32 (overwritten).
+ *   out_logits : host, [n_samples][n_classes] int8, or NULL.
+ */
+int isc_sample_counts(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id,
+                      int32_t phase, int64_t first_sample, int64_t n_samples, double sigma,
+                      void *cuda_stream, int32_t *out_counts, int8_t *out_logits);
+
+/*
+ * isc_decide_certify / isc_decide_predict -- the host part of Algorithm 1 (steps 2,
+ * 5-9) and Algorithm 2 (steps 2-6) on given vote counts; no GPU work.
+ *   out_p_lower : the lower confidence bound p_A, or NULL.
+ */
+int isc_decide_certify(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N,
+                       double sigma, double alpha, int32_t *out_class, double *out_radius,
+                       double *out_p_lower);
+int isc_decide_predict(const int32_t *counts, int n_classes, double alpha, int32_t *out_class);
+
+/*
+ * isc_noise_table -- the cumulative table of the noise law (Eq. 2) the kernels use for
+ * `sigma`: writes 2*T+1 uint32 entries for levels -T..T to `cum` (host) when
+ * capacity >= 2*T+1, and T to *out_T.  Pass cum = NULL to query T only.
+ */
+int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_T);
+
+/*
+ * isc_debug_tensor -- evaluate sample j of one image and copy tensor `tensor`
+ * (0 = the noisy input, values 0..255; i+1 = output of layer i) to `out` as
+ * [C][H][W] int32 (host).  For layer-by-layer comparison; slow.
+ */
+int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id,
+                     int32_t phase, int64_t j, double sigma, int tensor, void *cuda_stream,
+                     int32_t *out, int64_t capacity);
+
+/*
+ * isc_set_option -- tuning knobs; none changes a result.
+ *   "batch"  : noisy samples per launch (0 = choose automatically).
+ *   "engine" : 0 = automatic, 1 = layer-by-layer kernels only, 2 = require the
+ *              shared-memory-resident tensor-core kernel (ISC_ERR_UNSUPPORTED at the
+ *              next call if the model does not fit it).
+ * isc_get_info reads back: "engine" (the engine the last call used), "gpu_launches"
+ * (kernel launches issued by this handle so far), "macs_per_sample".
+ */
+int isc_set_option(isc_model *m, const char *name, int64_t value);
+int isc_get_info(isc_model *m, const char *name, int64_t *out);
+
+const char *isc_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ISC_H_ */

@@ -1,0 +1,703 @@
+// Host side of libisc: argument checks, model repacking and upload, launch sequencing of the
+// Monte-Carlo loop (Algorithm 1 steps 1-4, Algorithm 2 steps 1-2) and the decision rules.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
+#include <cmath>
+#include <new>
+#include <vector>
+
+#include "isc.h"
+#include "isc_internal.h"
+#include "isc_mega.h"
+
+using namespace isc;
+
+namespace {
+
+inline int pad16(int c) { return (c + 15) & ~15; }
+
+struct HostLayer {           // private copy of one isc_layer with its arrays
+    isc_layer d;
+    std::vector<int8_t> w;
+    std::vector<int32_t> bias, mult;
+    std::vector<int8_t> shift;
+};
+
+struct DevBuf {
+    void *p = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace
+
+struct isc_model {
+    int in_c = 0, in_h = 0, in_w = 0, n_classes = 0;
+    std::vector<HostLayer> layers;
+    std::vector<TShape> shapes;                 // [n_layers + 1]
+    int64_t macs = 0;
+
+    // device parameters of the layer-by-layer engine
+    std::vector<GLayer> glayers;
+    std::vector<void *> param_allocs;
+
+    // activation buffers: tensor t lives in pool buffer tensor_buf[t] (bytes per sample buf_bytes[b])
+    std::vector<int> tensor_buf;
+    std::vector<size_t> buf_bytes;
+    std::vector<DevBuf> bufs;
+    int ws_batch = 0;
+
+    // per-call device scratch
+    uint8_t *d_x = nullptr;       size_t d_x_bytes = 0;
+    int32_t *d_counts = nullptr;  size_t d_counts_n = 0;
+    int8_t *d_logits = nullptr;   size_t d_logits_bytes = 0;
+    uint32_t *d_cum = nullptr;    size_t d_cum_n = 0;
+    double cum_sigma = -1.0;
+    int cum_T = 0;
+
+    isc::MegaPlan *mega = nullptr;
+
+    int64_t opt_batch = 0, opt_engine = 0;
+    int64_t last_engine = 0, launches = 0;
+};
+
+namespace {
+
+#define CK(call)                                      \
+    do {                                              \
+        cudaError_t e_ = (call);                      \
+        if (e_ != cudaSuccess) {                      \
+            cudaGetLastError();                       \
+            return e_ == cudaErrorMemoryAllocation ? ISC_ERR_NOMEM : ISC_ERR_CUDA; \
+        }                                             \
+    } while (0)
+
+int infer_shape(const isc_layer &L, const TShape &in, TShape *out)
+{
+    switch (L.op) {
+    case ISC_CONV2D:
+    case ISC_MAXPOOL:
+        if (L.kh < 1 || L.kw < 1 || L.stride < 1 || L.pad < 0) return ISC_ERR_SHAPE;
+        if (L.cin != in.c) return ISC_ERR_SHAPE;
+        if (in.h + 2 * L.pad < L.kh || in.w + 2 * L.pad < L.kw) return ISC_ERR_SHAPE;
+        if (L.op == ISC_MAXPOOL && L.cout != L.cin) return ISC_ERR_SHAPE;
+        if (L.cout < 1) return ISC_ERR_SHAPE;
+        out->c = L.cout;
+        out->h = (in.h + 2 * L.pad - L.kh) / L.stride + 1;
+        out->w = (in.w + 2 * L.pad - L.kw) / L.stride + 1;
+        break;
+    case ISC_FC:
+        if (in.h != 1 || in.w != 1 || L.cin != in.c || L.cout < 1) return ISC_ERR_SHAPE;
+        out->c = L.cout; out->h = 1; out->w = 1;
+        break;
+    case ISC_GAVGPOOL:
+        if (L.cin != in.c || L.cout != in.c) return ISC_ERR_SHAPE;
+        out->c = in.c; out->h = 1; out->w = 1;
+        break;
+    default:
+        return ISC_ERR_ARG;
+    }
+    out->cp = pad16(out->c);
+    return ISC_OK;
+}
+
+template <typename T>
+int upload(isc_model *m, const std::vector<T> &h, const T **dptr)
+{
+    void *p = nullptr;
+    CK(cudaMalloc(&p, std::max<size_t>(h.size() * sizeof(T), 16)));
+    m->param_allocs.push_back(p);
+    CK(cudaMemcpy(p, h.data(), h.size() * sizeof(T), cudaMemcpyHostToDevice));
+    *dptr = static_cast<const T *>(p);
+    return ISC_OK;
+}
+
+// Validate, copy, infer shapes.  No device work.
+int build_host_model(isc_model *m, const isc_layer *layers, int n_layers)
+{
+    m->shapes.resize((size_t)n_layers + 1);
+    m->shapes[0] = TShape{m->in_c, m->in_h, m->in_w, 4};
+    m->layers.resize((size_t)n_layers);
+    std::vector<int> uses_of_input(1, 0);
+    for (int i = 0; i < n_layers; ++i) {
+        const isc_layer &L = layers[i];
+        if (L.op < ISC_CONV2D || L.op > ISC_MAXPOOL) return ISC_ERR_ARG;
+        if (L.in_tensor < 0 || L.in_tensor > i) return ISC_ERR_SHAPE;
+        if (L.res_tensor < -1 || L.res_tensor > i) return ISC_ERR_SHAPE;
+        const bool weighted = L.op == ISC_CONV2D || L.op == ISC_FC;
+        if (L.res_tensor >= 0 && !weighted) return ISC_ERR_SHAPE;
+        if (!L.mult || !L.shift) return ISC_ERR_ARG;
+        if (weighted && (!L.w || !L.bias)) return ISC_ERR_ARG;
+        int rc = infer_shape(L, m->shapes[(size_t)L.in_tensor], &m->shapes[(size_t)i + 1]);
+        if (rc) return rc;
+        const TShape &os = m->shapes[(size_t)i + 1];
+        if (L.res_tensor >= 0) {
+            const TShape &r = m->shapes[(size_t)L.res_tensor];
+            if (L.res_tensor == 0 || r.c != os.c || r.h != os.h || r.w != os.w) return ISC_ERR_SHAPE;
+            if (L.res_mult < (1 << 30) || L.res_shift < -4 || L.res_shift > 4) return ISC_ERR_ARG;
+            if (L.zp_res < -128 || L.zp_res > 127) return ISC_ERR_ARG;
+        }
+        const int zp_in_lo = L.in_tensor == 0 ? 0 : -128, zp_in_hi = L.in_tensor == 0 ? 255 : 127;
+        if (L.zp_in < zp_in_lo || L.zp_in > zp_in_hi) return ISC_ERR_ARG;
+        if (L.zp_out < -128 || L.zp_out > 127) return ISC_ERR_ARG;
+        if (L.relu != 0 && L.relu != 1) return ISC_ERR_ARG;
+
+        HostLayer &H = m->layers[(size_t)i];
+        H.d = L;
+        const int nch = weighted ? L.cout : 1;
+        H.mult.assign(L.mult, L.mult + nch);
+        H.shift.assign(L.shift, L.shift + nch);
+        for (int c = 0; c < nch; ++c) {
+            if (L.op != ISC_MAXPOOL && H.mult[(size_t)c] < (1 << 30)) return ISC_ERR_ARG;
+            if (H.shift[(size_t)c] < 0 || H.shift[(size_t)c] > 31) return ISC_ERR_ARG;
+        }
+        if (weighted) {
+            const int kh = L.op == ISC_FC ? 1 : L.kh, kw = L.op == ISC_FC ? 1 : L.kw;
+            const size_t per_out = (size_t)L.cin * kh * kw;
+            H.w.assign(L.w, L.w + per_out * L.cout);
+            H.bias.assign(L.bias, L.bias + L.cout);
+            H.d.kh = kh; H.d.kw = kw;
+            if (L.op == ISC_FC) { H.d.stride = 1; H.d.pad = 0; }
+            // worst-case accumulator magnitude must stay inside int32
+            const int amax = 255;                              // |a - zp_in| <= 255 for 8-bit activations
+            for (int o = 0; o < L.cout; ++o) {
+                int64_t s = 0;
+                for (size_t k = 0; k < per_out; ++k) {
+                    const int wv = H.w[(size_t)o * per_out + k];
+                    if (wv == -128) return ISC_ERR_ARG;        // symmetric int8 weights: [-127, 127]
+                    s += std::abs(wv);
+                }
+                const int64_t b = H.bias[(size_t)o];
+                if (s * amax + (b < 0 ? -b : b) >= (1ll << 30)) return ISC_ERR_UNSUPPORTED;
+            }
+            m->macs += (int64_t)os.h * os.w * L.cout * (int64_t)per_out;
+        }
+        H.d.w = nullptr; H.d.bias = nullptr; H.d.mult = nullptr; H.d.shift = nullptr;
+    }
+    const TShape &last = m->shapes[(size_t)n_layers];
+    if (last.c != m->n_classes || last.h != 1 || last.w != 1) return ISC_ERR_SHAPE;
+    return ISC_OK;
+}
+
+// Device parameters and buffer plan of the layer-by-layer engine.
+int build_generic_engine(isc_model *m)
+{
+    const int n = (int)m->layers.size();
+    // tensor 0 exists only inside the first convolution's staging
+    const isc_layer &L0 = m->layers[0].d;
+    if (L0.op != ISC_CONV2D || L0.in_tensor != 0 || L0.cin > 4) return ISC_ERR_UNSUPPORTED;
+    for (int i = 1; i < n; ++i)
+        if (m->layers[(size_t)i].d.in_tensor == 0) return ISC_ERR_UNSUPPORTED;
+
+    m->glayers.resize((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        const HostLayer &H = m->layers[(size_t)i];
+        const isc_layer &L = H.d;
+        const TShape &is = m->shapes[(size_t)L.in_tensor], &os = m->shapes[(size_t)i + 1];
+        GLayer G;
+        memset(&G, 0, sizeof(G));
+        G.op = L.op;
+        G.cin = L.cin; G.cinp = i == 0 ? 4 : is.cp;
+        G.cout = L.cout; G.coutp = os.cp;
+        G.kh = L.kh; G.kw = L.kw; G.stride = L.stride; G.pad = L.pad; G.relu = L.relu;
+        G.zp_in = L.zp_in; G.zp_out = L.zp_out; G.zp_res = L.zp_res;
+        G.res_mult = L.res_mult; G.res_shift = L.res_shift;
+        G.hin = is.h; G.win = is.w; G.hout = os.h; G.wout = os.w;
+        const bool weighted = L.op == ISC_CONV2D || L.op == ISC_FC;
+        std::vector<int32_t> mult((size_t)(weighted ? G.coutp : 1), 1 << 30), shift(mult.size(), 0);
+        for (size_t c = 0; c < H.mult.size(); ++c) { mult[c] = H.mult[c]; shift[c] = H.shift[c]; }
+        int rc = upload(m, mult, &G.mult); if (rc) return rc;
+        rc = upload(m, shift, &G.shift); if (rc) return rc;
+        if (weighted) {
+            const int taps = L.kh * L.kw;
+            std::vector<int32_t> bias((size_t)G.coutp, 0);
+            for (int o = 0; o < L.cout; ++o) {
+                int64_t s = 0;
+                for (int k = 0; k < L.cin * taps; ++k) s += H.w[(size_t)o * L.cin * taps + k];
+                bias[(size_t)o] = (int32_t)(H.bias[(size_t)o] - (int64_t)L.zp_in * s);   // padding value is zp_in
+            }
+            rc = upload(m, bias, &G.bias); if (rc) return rc;
+            std::vector<int8_t> w;
+            if (i == 0) {                                   // [coutp][taps][4]
+                w.assign((size_t)G.coutp * taps * 4, 0);
+                for (int o = 0; o < L.cout; ++o)
+                    for (int c = 0; c < L.cin; ++c)
+                        for (int t = 0; t < taps; ++t)
+                            w[((size_t)o * taps + t) * 4 + c] = H.w[((size_t)o * L.cin + c) * taps + t];
+            } else {                                        // [coutp/16][taps][cinp/16][16 out][16 in]
+                const int c16s = G.cinp / 16;
+                w.assign((size_t)G.coutp * taps * G.cinp, 0);
+                for (int o = 0; o < L.cout; ++o)
+                    for (int c = 0; c < L.cin; ++c)
+                        for (int t = 0; t < taps; ++t) {
+                            const size_t idx = ((((size_t)(o / 16) * taps + t) * c16s + c / 16) * 16 + o % 16) * 16 + c % 16;
+                            w[idx] = H.w[((size_t)o * L.cin + c) * taps + t];
+                        }
+            }
+            rc = upload(m, w, &G.w); if (rc) return rc;
+        }
+        m->glayers[(size_t)i] = G;
+    }
+
+    // buffer plan: greedy reuse by last use
+    std::vector<int> last_use((size_t)n + 1, -1);
+    for (int i = 0; i < n; ++i) {
+        last_use[(size_t)m->layers[(size_t)i].d.in_tensor] = i;
+        if (m->layers[(size_t)i].d.res_tensor >= 0) last_use[(size_t)m->layers[(size_t)i].d.res_tensor] = i;
+    }
+    last_use[(size_t)n] = n;
+    m->tensor_buf.assign((size_t)n + 1, -1);
+    std::vector<int> owner;                                 // pool buffer -> tensor currently in it (or -1)
+    for (int i = 0; i < n; ++i) {
+        const int t = i + 1;
+        const TShape &s = m->shapes[(size_t)t];
+        const size_t need = (size_t)s.h * s.w * s.cp;
+        for (size_t b = 0; b < owner.size(); ++b)           // release buffers whose tensor is dead
+            if (owner[b] >= 0 && last_use[(size_t)owner[b]] < i) owner[b] = -1;
+        int pick = -1;
+        for (size_t b = 0; b < owner.size(); ++b)
+            if (owner[b] < 0 && (pick < 0 || m->buf_bytes[b] > m->buf_bytes[(size_t)pick])) pick = (int)b;
+        if (pick < 0) {
+            owner.push_back(-1);
+            m->buf_bytes.push_back(0);
+            pick = (int)owner.size() - 1;
+        }
+        m->buf_bytes[(size_t)pick] = std::max(m->buf_bytes[(size_t)pick], need);
+        owner[(size_t)pick] = t;
+        m->tensor_buf[(size_t)t] = pick;
+    }
+    m->bufs.resize(owner.size());
+    return ISC_OK;
+}
+
+int ensure_bytes(void **p, size_t *have, size_t need)
+{
+    if (*have >= need && *p) return ISC_OK;
+    if (*p) cudaFree(*p);
+    *p = nullptr; *have = 0;
+    CK(cudaMalloc(p, std::max<size_t>(need, 16)));
+    *have = need;
+    return ISC_OK;
+}
+
+int ensure_workspace(isc_model *m, int batch)
+{
+    if (batch <= m->ws_batch) return ISC_OK;
+    for (size_t b = 0; b < m->bufs.size(); ++b) {
+        if (m->bufs[b].p) cudaFree(m->bufs[b].p);
+        m->bufs[b].p = nullptr;
+    }
+    m->ws_batch = 0;
+    for (size_t b = 0; b < m->bufs.size(); ++b) {
+        CK(cudaMalloc(&m->bufs[b].p, m->buf_bytes[b] * (size_t)batch));
+        m->bufs[b].bytes = m->buf_bytes[b] * (size_t)batch;
+    }
+    m->ws_batch = batch;
+    return ISC_OK;
+}
+
+int ensure_noise_table(isc_model *m, double sigma, cudaStream_t st)
+{
+    if (m->d_cum && m->cum_sigma == sigma) return ISC_OK;
+    std::vector<uint32_t> cum;
+    noise_table(sigma, cum);
+    size_t have = m->d_cum_n * sizeof(uint32_t);
+    void *p = m->d_cum;
+    int rc = ensure_bytes(&p, &have, cum.size() * sizeof(uint32_t));
+    m->d_cum = (uint32_t *)p; m->d_cum_n = have / sizeof(uint32_t);
+    if (rc) return rc;
+    CK(cudaMemcpyAsync(m->d_cum, cum.data(), cum.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+    CK(cudaStreamSynchronize(st));                       // cum is a local vector
+    m->cum_sigma = sigma;
+    m->cum_T = (int)(cum.size() - 1) / 2;
+    return ISC_OK;
+}
+
+int check_stream_args(uint64_t image_id, int32_t phase, int64_t first, int64_t n, double sigma)
+{
+    if (!(sigma > 0.0) || !std::isfinite(sigma) || sigma > 64.0) return ISC_ERR_ARG;
+    if (phase < 0 || phase > 255) return ISC_ERR_ARG;
+    if (image_id >= (1ull << 48)) return ISC_ERR_ARG;
+    if (first < 0 || n < 0 || first + n > (1ll << 40)) return ISC_ERR_ARG;
+    return ISC_OK;
+}
+
+NoiseStream make_stream(const isc_model *m, uint64_t seed, uint64_t image_id, int32_t phase, int64_t first)
+{
+    NoiseStream ns;
+    ns.key0 = (uint32_t)(seed & 0xFFFFFFFFu);
+    ns.key1 = (uint32_t)(seed >> 32);
+    ns.ctr2 = (uint32_t)(image_id & 0xFFFFFFFFu);
+    ns.ctr3_fixed = (uint32_t)phase | (uint32_t)(((image_id >> 32) & 0xFFFFu) << 16);
+    ns.first_sample = first;
+    ns.cum = m->d_cum;
+    ns.T = m->cum_T;
+    return ns;
+}
+
+int choose_engine(isc_model *m)
+{
+    if (m->opt_engine == 1) return 1;
+    if (m->mega) return 2;
+    return m->opt_engine == 2 ? ISC_ERR_UNSUPPORTED : 1;
+}
+
+// Layer-by-layer forward of `batch` samples; leaves the logits in the last tensor's buffer.
+int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int batch, cudaStream_t st,
+                    int stop_after_layer = -1)
+{
+    const int n = (int)m->glayers.size();
+    for (int i = 0; i < n; ++i) {
+        const GLayer &G = m->glayers[(size_t)i];
+        const isc_layer &L = m->layers[(size_t)i].d;
+        int8_t *out = (int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)i + 1]].p;
+        const int8_t *in = i == 0 ? nullptr : (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.in_tensor]].p;
+        const int8_t *res = L.res_tensor >= 0 ? (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.res_tensor]].p : nullptr;
+        cudaError_t e;
+        if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, batch, out, st);
+        else if (L.op == ISC_CONV2D || L.op == ISC_FC) e = launch_conv(G, batch, in, res, out, st);
+        else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, batch, in, out, st);
+        else e = launch_maxpool(G, batch, in, out, st);
+        m->launches += 1;
+        if (e != cudaSuccess) return ISC_ERR_CUDA;
+        if (i == stop_after_layer) break;
+    }
+    return ISC_OK;
+}
+
+size_t generic_bytes_per_sample(const isc_model *m)
+{
+    size_t s = 0;
+    for (size_t b : m->buf_bytes) s += b;
+    return s;
+}
+
+// The Monte-Carlo loop for one image and one phase; adds votes into d_counts (device).
+int run_counts(isc_model *m, const uint8_t *d_x, uint64_t seed, uint64_t image_id, int32_t phase,
+               int64_t first, int64_t n, cudaStream_t st, int32_t *d_counts, int8_t *d_logits)
+{
+    const int engine = choose_engine(m);
+    if (engine < 0) return engine;
+    m->last_engine = engine;
+    if (engine == 2) {
+        NoiseStream ns = make_stream(m, seed, image_id, phase, first);
+        int64_t launches = 0;
+        int rc = isc::mega_run(m->mega, d_x, ns, n, (int)m->opt_batch, d_counts, d_logits, st, &launches);
+        m->launches += launches;
+        return rc;
+    }
+    int64_t cap = m->opt_batch > 0 ? m->opt_batch : 4096;
+    const size_t per = std::max<size_t>(generic_bytes_per_sample(m), 1);
+    cap = std::min<int64_t>(cap, std::max<int64_t>(1, (int64_t)((3ull << 30) / per)));
+    cap = std::min<int64_t>(cap, 32768);
+    const int batch_alloc = (int)std::min<int64_t>(cap, std::max<int64_t>(n, 1));
+    int rc = ensure_workspace(m, batch_alloc);
+    if (rc) return rc;
+    const int last = (int)m->glayers.size();
+    for (int64_t done = 0; done < n; done += cap) {
+        const int b = (int)std::min<int64_t>(cap, n - done);
+        NoiseStream ns = make_stream(m, seed, image_id, phase, first + done);
+        rc = generic_forward(m, d_x, ns, b, st);
+        if (rc) return rc;
+        const int8_t *lg = (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)last]].p;
+        cudaError_t e = launch_votes(lg, m->shapes[(size_t)last].cp, m->n_classes, b, d_counts,
+                                     d_logits ? d_logits + (size_t)done * m->n_classes : nullptr, st);
+        m->launches += 1;
+        if (e != cudaSuccess) return ISC_ERR_CUDA;
+    }
+    return ISC_OK;
+}
+
+int stage_image(isc_model *m, const uint8_t *x, size_t bytes, bool on_device, cudaStream_t st,
+                const uint8_t **d_x)
+{
+    if (on_device) { *d_x = x; return ISC_OK; }
+    void *p = m->d_x; size_t have = m->d_x_bytes;
+    int rc = ensure_bytes(&p, &have, bytes);
+    m->d_x = (uint8_t *)p; m->d_x_bytes = have;
+    if (rc) return rc;
+    CK(cudaMemcpyAsync(m->d_x, x, bytes, cudaMemcpyHostToDevice, st));
+    *d_x = m->d_x;
+    return ISC_OK;
+}
+
+int ensure_counts(isc_model *m, size_t n)
+{
+    void *p = m->d_counts; size_t have = m->d_counts_n * sizeof(int32_t);
+    int rc = ensure_bytes(&p, &have, n * sizeof(int32_t));
+    m->d_counts = (int32_t *)p; m->d_counts_n = have / sizeof(int32_t);
+    return rc;
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+
+extern "C" {
+
+const char *isc_strerror(int code)
+{
+    switch (code) {
+    case ISC_OK: return "ok";
+    case ISC_ERR_ARG: return "invalid argument";
+    case ISC_ERR_SHAPE: return "layer list does not type-check";
+    case ISC_ERR_UNSUPPORTED: return "not supported by the kernels";
+    case ISC_ERR_NOMEM: return "out of memory";
+    case ISC_ERR_CUDA: return "CUDA error";
+    case ISC_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown error";
+    }
+}
+
+int isc_load_qmodel(const isc_layer *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes,
+                    isc_model **out)
+{
+    if (!layers || !out || n_layers < 1 || n_layers > 4096) return ISC_ERR_ARG;
+    if (in_c < 1 || in_h < 1 || in_w < 1 || n_classes < 1 || n_classes > 4096) return ISC_ERR_ARG;
+    if ((int64_t)in_c * in_h * in_w > (1ll << 30)) return ISC_ERR_ARG;
+    isc_model *m = new (std::nothrow) isc_model();
+    if (!m) return ISC_ERR_NOMEM;
+    m->in_c = in_c; m->in_h = in_h; m->in_w = in_w; m->n_classes = n_classes;
+    int rc;
+    try {
+        rc = build_host_model(m, layers, n_layers);
+        if (rc == ISC_OK) rc = build_generic_engine(m);
+        if (rc == ISC_OK) {
+            std::vector<isc::MegaLayerIn> ml(m->layers.size());
+            for (size_t i = 0; i < m->layers.size(); ++i) {
+                const HostLayer &H = m->layers[i];
+                ml[i].d = H.d;
+                ml[i].w = H.w.data(); ml[i].bias = H.bias.data();
+                ml[i].mult = H.mult.data(); ml[i].shift = H.shift.data();
+            }
+            rc = isc::mega_build(ml.data(), (int)ml.size(), in_c, in_h, in_w, n_classes, &m->mega);
+        }
+    } catch (const std::bad_alloc &) {
+        rc = ISC_ERR_NOMEM;
+    }
+    if (rc != ISC_OK) {
+        isc_free_qmodel(m);
+        return rc;
+    }
+    *out = m;
+    return ISC_OK;
+}
+
+void isc_free_qmodel(isc_model *m)
+{
+    if (!m) return;
+    for (void *p : m->param_allocs) cudaFree(p);
+    for (DevBuf &b : m->bufs) if (b.p) cudaFree(b.p);
+    if (m->d_x) cudaFree(m->d_x);
+    if (m->d_counts) cudaFree(m->d_counts);
+    if (m->d_logits) cudaFree(m->d_logits);
+    if (m->d_cum) cudaFree(m->d_cum);
+    isc::mega_free(m->mega);
+    delete m;
+}
+
+int isc_sample_counts(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id, int32_t phase,
+                      int64_t first_sample, int64_t n_samples, double sigma, void *cuda_stream,
+                      int32_t *out_counts, int8_t *out_logits)
+{
+    if (!m || !x_u8 || !out_counts) return ISC_ERR_ARG;
+    int rc = check_stream_args(image_id, phase, first_sample, n_samples, sigma);
+    if (rc) return rc;
+    if (n_samples > (1ll << 31) - 1) return ISC_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t C = (size_t)m->n_classes;
+    if ((rc = ensure_noise_table(m, sigma, st))) return rc;
+    if ((rc = ensure_counts(m, C))) return rc;
+    const uint8_t *d_x;
+    if ((rc = stage_image(m, x_u8, (size_t)m->in_c * m->in_h * m->in_w, false, st, &d_x))) return rc;
+    if (out_logits) {
+        void *p = m->d_logits; size_t have = m->d_logits_bytes;
+        rc = ensure_bytes(&p, &have, (size_t)std::max<int64_t>(n_samples, 1) * C);
+        m->d_logits = (int8_t *)p; m->d_logits_bytes = have;
+        if (rc) return rc;
+    }
+    CK(cudaMemsetAsync(m->d_counts, 0, C * sizeof(int32_t), st));
+    if ((rc = run_counts(m, d_x, seed, image_id, phase, first_sample, n_samples, st, m->d_counts,
+                         out_logits ? m->d_logits : nullptr))) {
+        cudaStreamSynchronize(st);
+        return rc;
+    }
+    std::vector<int32_t> h(C);
+    std::vector<int8_t> hl;
+    CK(cudaMemcpyAsync(h.data(), m->d_counts, C * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    if (out_logits && n_samples > 0) {
+        hl.resize((size_t)n_samples * C);
+        CK(cudaMemcpyAsync(hl.data(), m->d_logits, hl.size(), cudaMemcpyDeviceToHost, st));
+    }
+    CK(cudaStreamSynchronize(st));
+    if (m->mega && (rc = isc::mega_check(m->mega))) return rc;
+    memcpy(out_counts, h.data(), C * sizeof(int32_t));
+    if (out_logits && n_samples > 0) memcpy(out_logits, hl.data(), hl.size());
+    return ISC_OK;
+}
+
+int isc_predict(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id, int64_t N, double sigma,
+                double alpha, void *cuda_stream, int32_t *out_class, int32_t *out_counts)
+{
+    if (!m || !x_u8 || !out_class) return ISC_ERR_ARG;
+    if (N < 1 || !(alpha > 0.0 && alpha < 1.0)) return ISC_ERR_ARG;
+    std::vector<int32_t> counts((size_t)m->n_classes);
+    int rc = isc_sample_counts(m, x_u8, seed, image_id, 2, 0, N, sigma, cuda_stream, counts.data(), nullptr);
+    if (rc) return rc;
+    *out_class = decide_predict(counts.data(), m->n_classes, alpha);
+    if (out_counts) memcpy(out_counts, counts.data(), counts.size() * sizeof(int32_t));
+    return ISC_OK;
+}
+
+int isc_certify_batch(isc_model *m, const uint8_t *x_u8, int x_on_device, int n_images, uint64_t seed,
+                      uint64_t image_id0, int64_t N0, int64_t N, double sigma, double alpha, void *cuda_stream,
+                      int32_t *out_class, double *out_radius, int32_t *out_counts0, int32_t *out_counts)
+{
+    if (!m || !x_u8 || !out_class || !out_radius || n_images < 0) return ISC_ERR_ARG;
+    if (N0 < 1 || N < 1 || !(alpha > 0.0 && alpha < 1.0)) return ISC_ERR_ARG;
+    if (N0 > (1ll << 31) - 1 || N > (1ll << 31) - 1) return ISC_ERR_ARG;
+    int rc = check_stream_args(image_id0 + (uint64_t)std::max(n_images - 1, 0), 0, 0, std::max(N0, N), sigma);
+    if (rc) return rc;
+    if (n_images == 0) return ISC_OK;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t C = (size_t)m->n_classes;
+    const size_t d = (size_t)m->in_c * m->in_h * m->in_w;
+    if ((rc = ensure_noise_table(m, sigma, st))) return rc;
+    if ((rc = ensure_counts(m, 2 * C * (size_t)n_images))) return rc;
+    const uint8_t *d_x;
+    if ((rc = stage_image(m, x_u8, d * (size_t)n_images, x_on_device != 0, st, &d_x))) return rc;
+    CK(cudaMemsetAsync(m->d_counts, 0, 2 * C * (size_t)n_images * sizeof(int32_t), st));
+    for (int i = 0; i < n_images && rc == ISC_OK; ++i) {
+        int32_t *c0 = m->d_counts + (size_t)i * 2 * C;
+        rc = run_counts(m, d_x + (size_t)i * d, seed, image_id0 + (uint64_t)i, 0, 0, N0, st, c0, nullptr);
+        if (rc == ISC_OK)
+            rc = run_counts(m, d_x + (size_t)i * d, seed, image_id0 + (uint64_t)i, 1, 0, N, st, c0 + C, nullptr);
+    }
+    if (rc) { cudaStreamSynchronize(st); return rc; }
+    std::vector<int32_t> h(2 * C * (size_t)n_images);
+    CK(cudaMemcpyAsync(h.data(), m->d_counts, h.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    if (m->mega && (rc = isc::mega_check(m->mega))) return rc;
+    for (int i = 0; i < n_images; ++i) {
+        const int32_t *c0 = h.data() + (size_t)i * 2 * C, *c1 = c0 + C;
+        double radius = 0.0;
+        out_class[i] = decide_certify(c0, c1, m->n_classes, N, sigma, alpha, &radius, nullptr);
+        out_radius[i] = radius;
+        if (out_counts0) memcpy(out_counts0 + (size_t)i * C, c0, C * sizeof(int32_t));
+        if (out_counts) memcpy(out_counts + (size_t)i * C, c1, C * sizeof(int32_t));
+    }
+    return ISC_OK;
+}
+
+int isc_certify(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id, int64_t N0, int64_t N,
+                double sigma, double alpha, void *cuda_stream, int32_t *out_class, double *out_radius,
+                int32_t *out_counts0, int32_t *out_counts)
+{
+    return isc_certify_batch(m, x_u8, 0, 1, seed, image_id, N0, N, sigma, alpha, cuda_stream, out_class,
+                             out_radius, out_counts0, out_counts);
+}
+
+int isc_decide_certify(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N, double sigma,
+                       double alpha, int32_t *out_class, double *out_radius, double *out_p_lower)
+{
+    if (!counts0 || !counts || !out_class || !out_radius || n_classes < 1 || N < 1) return ISC_ERR_ARG;
+    if (!(alpha > 0.0 && alpha < 1.0) || !(sigma > 0.0)) return ISC_ERR_ARG;
+    for (int c = 0; c < n_classes; ++c)
+        if (counts0[c] < 0 || counts[c] < 0 || counts[c] > N) return ISC_ERR_ARG;
+    double radius = 0.0, pl = 0.0;
+    *out_class = decide_certify(counts0, counts, n_classes, N, sigma, alpha, &radius, &pl);
+    *out_radius = radius;
+    if (out_p_lower) *out_p_lower = pl;
+    return ISC_OK;
+}
+
+int isc_decide_predict(const int32_t *counts, int n_classes, double alpha, int32_t *out_class)
+{
+    if (!counts || !out_class || n_classes < 1 || !(alpha > 0.0 && alpha < 1.0)) return ISC_ERR_ARG;
+    for (int c = 0; c < n_classes; ++c)
+        if (counts[c] < 0) return ISC_ERR_ARG;
+    *out_class = decide_predict(counts, n_classes, alpha);
+    return ISC_OK;
+}
+
+int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_T)
+{
+    if (!out_T || !(sigma > 0.0) || !std::isfinite(sigma) || sigma > 64.0) return ISC_ERR_ARG;
+    const int T = noise_halfwidth(sigma);
+    if (cum) {
+        if (capacity < 2 * (int64_t)T + 1) return ISC_ERR_ARG;
+        std::vector<uint32_t> t;
+        noise_table(sigma, t);
+        memcpy(cum, t.data(), t.size() * sizeof(uint32_t));
+    }
+    *out_T = T;
+    return ISC_OK;
+}
+
+int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id, int32_t phase,
+                     int64_t j, double sigma, int tensor, void *cuda_stream, int32_t *out, int64_t capacity)
+{
+    if (!m || !x_u8 || !out || tensor < 0 || tensor > (int)m->layers.size()) return ISC_ERR_ARG;
+    int rc = check_stream_args(image_id, phase, j, 1, sigma);
+    if (rc) return rc;
+    const TShape &s = m->shapes[(size_t)tensor];
+    const size_t n = (size_t)s.c * s.h * s.w;
+    if (capacity < (int64_t)n) return ISC_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if ((rc = ensure_noise_table(m, sigma, st))) return rc;
+    const uint8_t *d_x;
+    if ((rc = stage_image(m, x_u8, (size_t)m->in_c * m->in_h * m->in_w, false, st, &d_x))) return rc;
+    NoiseStream ns = make_stream(m, seed, image_id, phase, j);
+    if (tensor == 0) {
+        int32_t *d_out = nullptr;
+        CK(cudaMalloc((void **)&d_out, n * sizeof(int32_t)));
+        cudaError_t e = launch_noisy_input(d_x, m->in_c, m->in_h, m->in_w, ns, 1, d_out, st);
+        m->launches += 1;
+        if (e == cudaSuccess) e = cudaMemcpyAsync(out, d_out, n * sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        cudaFree(d_out);
+        return e == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
+    }
+    if ((rc = ensure_workspace(m, 1))) return rc;
+    if ((rc = generic_forward(m, d_x, ns, 1, st, tensor - 1))) return rc;
+    std::vector<int8_t> h((size_t)s.h * s.w * s.cp);
+    CK(cudaMemcpyAsync(h.data(), m->bufs[(size_t)m->tensor_buf[(size_t)tensor]].p, h.size(),
+                       cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    for (int c = 0; c < s.c; ++c)
+        for (int y = 0; y < s.h; ++y)
+            for (int x = 0; x < s.w; ++x)
+                out[((size_t)c * s.h + y) * s.w + x] = h[((size_t)y * s.w + x) * s.cp + c];
+    return ISC_OK;
+}
+
+int isc_set_option(isc_model *m, const char *name, int64_t value)
+{
+    if (!m || !name) return ISC_ERR_ARG;
+    if (!strcmp(name, "batch")) {
+        if (value < 0 || value > (1 << 20)) return ISC_ERR_ARG;
+        m->opt_batch = value;
+        return ISC_OK;
+    }
+    if (!strcmp(name, "engine")) {
+        if (value < 0 || value > 2) return ISC_ERR_ARG;
+        m->opt_engine = value;
+        return ISC_OK;
+    }
+    return ISC_ERR_ARG;
+}
+
+int isc_get_info(isc_model *m, const char *name, int64_t *out)
+{
+    if (!m || !name || !out) return ISC_ERR_ARG;
+    if (!strcmp(name, "engine")) *out = m->last_engine;
+    else if (!strcmp(name, "gpu_launches")) *out = m->launches;
+    else if (!strcmp(name, "macs_per_sample")) *out = m->macs;
+    else if (!strcmp(name, "has_resident_engine")) *out = m->mega ? 1 : 0;
+    else return ISC_ERR_ARG;
+    return ISC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,63 @@
+// Internal declarations shared by the host API and the kernel files of libisc.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "isc.h"
+
+namespace isc {
+
+struct TShape {
+    int c, h, w;
+    int cp;  // channels padded to a multiple of 16 (device NHWC layout)
+};
+
+// Where the random stream of one launch starts (Philox4x32-10 key and fixed counter words).
+struct NoiseStream {
+    uint32_t key0, key1;      // seed halves
+    uint32_t ctr2;            // image_id low 32
+    uint32_t ctr3_fixed;      // phase | (image_id >> 32 & 0xFFFF) << 16
+    int64_t first_sample;     // sample id of batch slot 0
+    const uint32_t *cum;      // device, 2T+1 entries
+    int T;
+};
+
+// One layer as the layer-by-layer kernels see it (device pointers).
+struct GLayer {
+    int op;
+    int cin, cinp, cout, coutp;
+    int kh, kw, stride, pad, relu;
+    int zp_in, zp_out, zp_res, res_mult, res_shift;
+    int hin, win, hout, wout;
+    const int8_t *w;        // conv/FC: [coutp/16][kh*kw][cinp/16][16 out][16 in]; first layer: [coutp][kh*kw][4]
+    const int32_t *bias;    // [coutp], folded: bias - zp_in * sum(w)
+    const int32_t *mult;    // [coutp]
+    const int32_t *shift;   // [coutp]
+};
+
+// ---- layer-by-layer engine (isc_generic.cu) ----
+cudaError_t launch_first_conv(const GLayer &L, const uint8_t *x_chw, int in_c, const NoiseStream &ns,
+                              int batch, int8_t *out, cudaStream_t st);
+cudaError_t launch_noisy_input(const uint8_t *x_chw, int in_c, int in_h, int in_w, const NoiseStream &ns,
+                               int batch, int32_t *out_chw, cudaStream_t st);
+cudaError_t launch_conv(const GLayer &L, int batch, const int8_t *in, const int8_t *res, int8_t *out,
+                        cudaStream_t st);
+cudaError_t launch_gavgpool(const GLayer &L, int batch, const int8_t *in, int8_t *out, cudaStream_t st);
+cudaError_t launch_maxpool(const GLayer &L, int batch, const int8_t *in, int8_t *out, cudaStream_t st);
+cudaError_t launch_votes(const int8_t *logits_nhwc, int cp, int n_classes, int batch, int32_t *counts,
+                         int8_t *logits_out, cudaStream_t st);
+
+// ---- host decision rules (isc_decide.cpp) ----
+double lower_conf_bound(int64_t k, int64_t n, double alpha);
+double normal_quantile(double p);
+double binom_pvalue_half(int64_t n_a, int64_t m);
+int32_t decide_certify(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N,
+                       double sigma, double alpha, double *radius, double *p_lower);
+int32_t decide_predict(const int32_t *counts, int n_classes, double alpha);
+int noise_halfwidth(double sigma);
+void noise_table(double sigma, std::vector<uint32_t> &cum);
+
+}  // namespace isc

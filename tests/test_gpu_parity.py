@@ -1,0 +1,220 @@
+"""GPU parity: every value the CUDA library returns through its C ABI is compared, bit for bit,
+with the CPU oracle on the same seeded inputs."""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+import paper_2108_09413_b200 as isc
+
+pytestmark = pytest.mark.gpu
+SEED = wl.NOISE_SEED
+ALPHA = 0.001
+ENGINES = {"layerwise": 1, "auto": 0}
+
+
+def _pair(model):
+    return isc.Model(model), oracle.Model(model)
+
+
+def _tensor_sizes(om):
+    return [oracle.tensor_size(om, k) for k in range(om.n_layers + 1)]
+
+
+@pytest.mark.parametrize("sigma", [0.12, 0.25, 0.5, 1.0])
+def test_noisy_input_matches(sigma):
+    gm, om = _pair(wl.tiny_cnn())
+    x = wl.images(1)[0]
+    for image_id, phase, j in ((0, 0, 0), (5, 1, 77), ((3 << 32) | 9, 2, (1 << 33) + 12345), (1, 255, 99999)):
+        got = gm.debug_tensor(x, SEED, image_id, phase, j, sigma, 0, x.size)
+        np.testing.assert_array_equal(got, oracle.noisy_input(x, SEED, image_id, phase, j, sigma).ravel())
+
+
+def test_tiny_cnn_every_tensor_and_full_certify():
+    model = wl.CONFIGS[0]["model"]()
+    gm, om = _pair(model)
+    x = wl.images(1, seed=wl.CONFIGS[0]["image_seed"])[0]
+    sizes = _tensor_sizes(om)
+    for j in (0, 3, 1000):
+        a0 = oracle.noisy_input(x, SEED, 0, 1, j, 0.25)
+        for k in range(1, om.n_layers + 1):
+            _, exp = oracle.forward(om, a0, dump_tensor=k)
+            got = gm.debug_tensor(x, SEED, 0, 1, j, 0.25, k, sizes[k])
+            np.testing.assert_array_equal(got, exp, err_msg=f"tensor {k} sample {j}")
+    for name, eng in ENGINES.items():
+        gm.set_option("engine", eng)
+        cls, rad, c0, c1 = gm.certify(x, SEED, 0, 100, 1000, 0.25, ALPHA)
+        ecls, erad, ec0, ec1 = oracle.certify(om, x, SEED, 0, 100, 1000, 0.25, ALPHA)
+        np.testing.assert_array_equal(c0, ec0)
+        np.testing.assert_array_equal(c1, ec1)
+        assert (cls, rad) == (ecls, erad), name
+        pc, pcounts = gm.predict(x, SEED, 0, 500, 0.25, ALPHA)
+        epc, epcounts = oracle.predict(om, x, SEED, 0, 500, 0.25, ALPHA)
+        np.testing.assert_array_equal(pcounts, epcounts)
+        assert pc == epc
+
+
+def _logit_parity(model, x, image_id, phase, first, n, sigma, engines=ENGINES):
+    gm, om = _pair(model)
+    ecounts, elog = oracle.sample_counts(om, x, SEED, image_id, phase, first, n, sigma, want_logits=True)
+    for name, eng in engines.items():
+        gm.set_option("engine", eng)
+        counts, log = gm.sample_counts(x, SEED, image_id, phase, first, n, sigma, want_logits=True)
+        bad = np.nonzero((log != elog).any(axis=1))[0]
+        assert bad.size == 0, f"{name}: first mismatching sample {bad[:5]} of {n}"
+        np.testing.assert_array_equal(counts, ecounts, err_msg=name)
+    gm.close()
+
+
+@pytest.mark.parametrize("sigma", [0.12, 0.25, 0.5])
+def test_resnet20_logits_and_prefix_counts(sigma):
+    cfg = wl.CONFIGS[1]
+    xs = wl.images(3, seed=cfg["image_seed"])
+    model = cfg["model"]()
+    for i in (0, 2):
+        _logit_parity(model, xs[i], i, 1, 0, 300, sigma)          # spans several tiles + ragged tail
+    _logit_parity(model, xs[1], 1, 0, 0, 100, sigma)              # the selection phase
+
+
+def test_resnet20_every_tensor():
+    model = wl.resnet20()
+    gm, om = _pair(model)
+    x = wl.images(1, seed=77)[0]
+    sizes = _tensor_sizes(om)
+    a0 = oracle.noisy_input(x, SEED, 4, 1, 9, 0.5)
+    for k in range(1, om.n_layers + 1):
+        _, exp = oracle.forward(om, a0, dump_tensor=k)
+        got = gm.debug_tensor(x, SEED, 4, 1, 9, 0.5, k, sizes[k])
+        np.testing.assert_array_equal(got, exp, err_msg=f"tensor {k}")
+
+
+def test_resnet110_logits_and_prefix_counts():
+    cfg = wl.CONFIGS[2]
+    xs = wl.images(2, seed=cfg["image_seed"])
+    model = cfg["model"]()
+    _logit_parity(model, xs[0], 0, 1, 0, 160, 0.25)
+    _logit_parity(model, xs[1], 1, 1, 99_990, 10, 0.25)          # the tail of N = 100,000
+    _logit_parity(model, xs[1], 1, 0, 0, 40, 1.0)                # sweep sigma of config 4
+
+
+def test_resnet50_logits():
+    cfg = wl.CONFIGS[3]
+    x = wl.images(1, seed=cfg["image_seed"], shape=cfg["shape"])[0]
+    _logit_parity(cfg["model"](), x, 0, 1, 0, 6, 0.5, engines={"auto": 0})
+
+
+def test_partition_and_batch_invariance():
+    model = wl.resnet20()
+    gm = isc.Model(model)
+    x = wl.images(1, seed=3)[0]
+    n = 2500
+    for eng in ENGINES.values():
+        gm.set_option("engine", eng)
+        gm.set_option("batch", 0)
+        full = gm.sample_counts(x, SEED, 7, 1, 0, n, 0.25)
+        assert full.sum() == n
+        parts = sum(gm.sample_counts(x, SEED, 7, 1, a, b - a, 0.25)
+                    for a, b in ((0, 1), (1, 130), (130, 1031), (1031, n)))
+        np.testing.assert_array_equal(full, parts)
+        for batch in (256, 1024, 4096, 16384):
+            gm.set_option("batch", batch)
+            np.testing.assert_array_equal(gm.sample_counts(x, SEED, 7, 1, 0, n, 0.25), full)
+    gm.set_option("batch", 0)
+    assert np.array_equal(gm.sample_counts(x, SEED, 7, 1, 0, 0, 0.25), np.zeros(10, np.int32))
+
+
+def test_certify_batch_equals_single_calls_and_oracle_prefix():
+    cfg = wl.CONFIGS[1]
+    model = cfg["model"]()
+    gm, om = _pair(model)
+    xs = wl.images(4, seed=cfg["image_seed"])
+    cls, rad, c0, c1 = gm.certify_batch(xs, 4, SEED, 10, 100, 700, 0.25, ALPHA)
+    for i in range(4):
+        s = gm.certify(xs[i], SEED, 10 + i, 100, 700, 0.25, ALPHA)
+        assert (s[0], s[1]) == (cls[i], rad[i])
+        np.testing.assert_array_equal(s[2], c0[i]); np.testing.assert_array_equal(s[3], c1[i])
+        e = oracle.certify_decide(c0[i], c1[i], 700, 0.25, ALPHA)
+        assert (e[0], e[1]) == (cls[i], rad[i])
+    e = oracle.certify(om, xs[2], SEED, 12, 100, 700, 0.25, ALPHA)
+    assert (e[0], e[1]) == (cls[2], rad[2])
+    np.testing.assert_array_equal(e[2], c0[2]); np.testing.assert_array_equal(e[3], c1[2])
+    # images resident on the device give the same answer
+    import torch
+    xd = torch.from_numpy(xs).cuda()
+    d = gm.certify_batch(None, 4, SEED, 10, 100, 700, 0.25, ALPHA, device_ptr=xd.data_ptr(),
+                         stream=torch.cuda.current_stream())
+    np.testing.assert_array_equal(d[0], cls); np.testing.assert_array_equal(d[1], rad)
+    np.testing.assert_array_equal(d[3], c1)
+
+
+def test_sigma_to_zero_limit():
+    model = wl.tiny_cnn()
+    gm, om = _pair(model)
+    x = wl.images(1, seed=2)[0]
+    clean = int(np.argmax(oracle.forward(om, x)))
+    cls, rad, c0, c1 = gm.certify(x, 1, 0, 50, 300, 1e-4, ALPHA)
+    assert c1[clean] == 300 and cls == clean
+    assert rad == oracle.certify_decide(c0, c1, 300, 1e-4, ALPHA)[1]
+
+
+def _rand_conv(rng, in_tensor, cin, cout, k, stride, pad, relu, zp_in, zp_out, res_tensor=-1, zp_res=0):
+    return dict(op=wl.OP_CONV2D, in_tensor=in_tensor, res_tensor=res_tensor, cin=cin, cout=cout, kh=k, kw=k,
+                stride=stride, pad=pad, relu=relu, zp_in=zp_in, zp_out=zp_out, zp_res=zp_res,
+                w=rng.integers(-127, 128, (cout, cin, k, k)).astype(np.int8),
+                bias=rng.integers(-30000, 30001, cout).astype(np.int32),
+                mult=rng.integers(2 ** 30, 2 ** 31, cout).astype(np.int32),
+                shift=rng.integers(0, 14, cout).astype(np.int8),
+                res_mult=int(rng.integers(2 ** 30, 2 ** 31)) if res_tensor >= 0 else 0,
+                res_shift=int(rng.integers(-4, 5)) if res_tensor >= 0 else 0)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_odd_shapes_zero_points_and_shifts(seed):
+    """Ragged sizes, channel counts that are not multiples of 16, every zero-point and shift range."""
+    rng = np.random.default_rng(100 + seed)
+    h, w = int(rng.integers(5, 14)), int(rng.integers(5, 14)) // 4 * 4 + 4
+    c1, c2 = int(rng.integers(3, 40)), int(rng.integers(3, 40))
+    zp1, zp2 = int(rng.integers(-128, 100)), int(rng.integers(-128, 100))
+    k0 = int(rng.choice([1, 3, 5]))
+    L = [_rand_conv(rng, 0, 3, c1, k0, 1, k0 // 2, 1, int(rng.integers(0, 200)), zp1),
+         _rand_conv(rng, 1, c1, c2, 3, 2, 1, int(rng.integers(0, 2)), zp1, zp2)]
+    L.append(_rand_conv(rng, 2, c2, c2, 3, 1, 1, 1, zp2, zp1, res_tensor=2, zp_res=zp2))
+    L.append(dict(wl._maxpool(3, c2, 3, 2, 1, zp1)))
+    model = dict(in_shape=(3, h, w), n_classes=7, layers=L)
+    om_tmp = oracle.Model(dict(model, n_classes=1))
+    hw = oracle.tensor_size(om_tmp, 4) // c2
+    L.append(wl._gavgpool(4, c2, hw, zp1))
+    fc = _rand_conv(rng, 5, c2, 7, 1, 1, 0, 0, zp1, int(rng.integers(-20, 20)))
+    fc["op"] = wl.OP_FC
+    L.append(fc)
+    gm, om = _pair(model)
+    x = rng.integers(0, 256, (3, h, w)).astype(np.uint8)
+    sizes = _tensor_sizes(om)
+    a0 = oracle.noisy_input(x, 5, seed, 1, 2, 0.25)
+    for k in range(1, om.n_layers + 1):
+        _, exp = oracle.forward(om, a0, dump_tensor=k)
+        got = gm.debug_tensor(x, 5, seed, 1, 2, 0.25, k, sizes[k])
+        np.testing.assert_array_equal(got, exp, err_msg=f"tensor {k}")
+    ec, el = oracle.sample_counts(om, x, 5, seed, 1, 0, 40, 0.25, want_logits=True)
+    gc, gl = gm.sample_counts(x, 5, seed, 1, 0, 40, 0.25, want_logits=True)
+    np.testing.assert_array_equal(gl, el)
+    np.testing.assert_array_equal(gc, ec)
+
+
+def test_argument_errors_leave_outputs_untouched():
+    gm = isc.Model(wl.tiny_cnn())
+    x = wl.images(1)[0]
+    L = isc.lib()
+    counts = np.full(10, -5, np.int32)
+    for kw in (dict(sigma=0.0), dict(phase=256), dict(n=-1), dict(first=1 << 40)):
+        rc = L.isc_sample_counts(gm._h, x.ctypes.data, 1, 0, kw.get("phase", 1), kw.get("first", 0),
+                                 kw.get("n", 10), kw.get("sigma", 0.25), None, counts.ctypes.data, None)
+        assert rc == -1 and (counts == -5).all()
+    cls, rad = C.c_int32(9), C.c_double(9.0)
+    assert L.isc_certify(gm._h, x.ctypes.data, 1, 0, 0, 10, 0.25, 0.001, None, C.byref(cls), C.byref(rad), None, None) == -1
+    assert L.isc_certify(gm._h, x.ctypes.data, 1, 0, 10, 10, 0.25, 1.0, None, C.byref(cls), C.byref(rad), None, None) == -1
+    assert L.isc_predict(gm._h, None, 1, 0, 10, 0.25, 0.001, None, C.byref(cls), None) == -1
+    assert cls.value == 9 and rad.value == 9.0
+    assert gm.get_info("gpu_launches") >= 0

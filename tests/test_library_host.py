@@ -1,0 +1,106 @@
+"""CPU-only checks of libisc: it loads, exports every declared symbol, rejects bad arguments
+before touching the GPU, and its host decision code agrees with the oracle bit for bit."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+import paper_2108_09413_b200 as isc
+from paper_2108_09413_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_exports_match_header():
+    hdr = open(os.path.join(ROOT, "include", "isc.h")).read()
+    declared = set(re.findall(r"\b(isc_[a-z_0-9]+)\s*\(", hdr))
+    assert declared == set(binding.EXPORTS)
+    L = isc.lib()
+    for name in declared:
+        assert getattr(L, name) is not None
+
+
+def test_strerror():
+    L = isc.lib()
+    assert L.isc_strerror(0) == b"ok"
+    for code in range(-6, 0):
+        assert len(L.isc_strerror(code)) > 3
+    assert L.isc_strerror(-99) == b"unknown error"
+
+
+def test_noise_table_equals_oracle_entry_by_entry():
+    for sigma in (0.12, 0.25, 0.5, 1.0, 0.01, 2.0):
+        np.testing.assert_array_equal(isc.noise_table(sigma), oracle.dgauss_table(sigma))
+    T = C.c_int32()
+    assert isc.lib().isc_noise_table(0.0, None, 0, C.byref(T)) == -1
+    small = np.zeros(4, np.uint32)
+    assert isc.lib().isc_noise_table(0.25, small.ctypes.data, 4, C.byref(T)) == -1
+
+
+def test_decisions_bit_equal_to_oracle():
+    rng = np.random.default_rng(4)
+    for _ in range(40):
+        N = int(rng.choice([100, 1000, 10000, 100000]))
+        nA = int(rng.integers(0, N + 1))
+        rest = N - nA
+        b = int(rng.integers(0, rest + 1))
+        counts = [b, nA, rest - b]
+        c0 = rng.integers(0, 100, 3).tolist()
+        sigma = float(rng.choice([0.12, 0.25, 0.5, 1.0]))
+        got = isc.certify_decide(c0, counts, N, sigma, 0.001)
+        exp = oracle.certify_decide(c0, counts, N, sigma, 0.001)
+        assert got == exp                                    # class, radius and p_lower: identical doubles
+        assert isc.predict_decide(counts, 0.001) == oracle.predict_decide(counts, 0.001)
+    for counts in ([0, 11, 0], [0, 10, 0], [50, 50], [7, 7, 7], [0, 0, 100000]):
+        assert isc.predict_decide(counts, 0.001) == oracle.predict_decide(counts, 0.001)
+    assert isc.certify_decide([0, 1], [0, 100000], 100000, 0.25, 0.001) == \
+        oracle.certify_decide([0, 1], [0, 100000], 100000, 0.25, 0.001)
+
+
+def test_decide_rejects_bad_arguments():
+    L = isc.lib()
+    c = np.array([1, 2], np.int32)
+    cls, rad = C.c_int32(7), C.c_double(7.0)
+    assert L.isc_decide_certify(None, c.ctypes.data, 2, 3, 0.25, 0.001, C.byref(cls), C.byref(rad), None) == -1
+    assert L.isc_decide_certify(c.ctypes.data, c.ctypes.data, 2, 3, 0.25, 1.5, C.byref(cls), C.byref(rad), None) == -1
+    assert L.isc_decide_certify(c.ctypes.data, c.ctypes.data, 2, 1, 0.25, 0.001, C.byref(cls), C.byref(rad), None) == -1
+    assert L.isc_decide_predict(c.ctypes.data, 0, 0.001, C.byref(cls)) == -1
+    assert cls.value == 7 and rad.value == 7.0               # outputs untouched on error
+
+
+def _load(model):
+    arr, keep = binding.layer_array(model["layers"])
+    h = C.c_void_p()
+    rc = isc.lib().isc_load_qmodel(C.cast(arr, C.c_void_p), len(model["layers"]), *model["in_shape"],
+                                   model["n_classes"], C.byref(h))
+    return rc, h
+
+
+def test_load_rejects_malformed_models_without_a_gpu():
+    base = wl.tiny_cnn()
+    h = C.c_void_p()
+    assert isc.lib().isc_load_qmodel(None, 4, 3, 32, 32, 10, C.byref(h)) == -1
+    def variant(kw=None):
+        m = dict(base, layers=[dict(l) for l in base["layers"]])
+        for (i, k), v in (kw or {}).items():
+            m["layers"][i][k] = v
+        return m
+    assert _load(variant({(1, "cin"): 8}))[0] == -2                 # channel mismatch
+    assert _load(variant({(1, "in_tensor"): 3}))[0] == -2           # reads a later tensor
+    assert _load(variant({(0, "op"): 9}))[0] == -1
+    assert _load(variant({(0, "zp_out"): 300}))[0] == -1
+    bad_shift = variant()
+    bad_shift["layers"][0]["shift"] = np.full(16, 40, np.int8)
+    assert _load(bad_shift)[0] == -1
+    bad_mult = variant()
+    bad_mult["layers"][0]["mult"] = np.full(16, 5, np.int32)
+    assert _load(bad_mult)[0] == -1
+    assert _load(dict(base, n_classes=11))[0] == -2                  # last tensor is not the logits
+    no_w = variant()
+    no_w["layers"][0]["w"] = None
+    assert _load(no_w)[0] == -1
+    assert h.value is None
