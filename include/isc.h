@@ -151,6 +151,38 @@ int isc_sample_counts(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t
                       void *cuda_stream, int32_t *out_counts, int8_t *out_logits);
 
 /*
+ * isc_sample_counts_static -- isc_sample_counts for callers that must not allocate device
+ * memory.  (The paper has no counterpart: this is a deployment variant of the same
+ * Monte-Carlo loop, added for such callers.)
+ *
+ * Some hosts of this library may not call cudaMalloc at all once they are running: a
+ * service whose device memory is handed out up front by its own pool, a real-time loop
+ * that cannot afford the implicit device synchronisation of an allocation, a process
+ * running under a memory budget enforced by refusing allocations.  For them this entry
+ * point computes the same vote counts as isc_sample_counts with the layer-by-layer
+ * kernels, but takes every byte of its device work space (activation buffers, noise
+ * table, staged image, counts) from one fixed 32 MiB array that is part of the library
+ * image.  It calls no cudaMalloc / cudaFree and no allocating library routine; the model
+ * handle must have been loaded beforehand (loading does allocate).  Each GPU on which the
+ * library is loaded holds that array until the process exits.
+ *
+ *   arguments  : as isc_sample_counts (x_u8 and out_counts are host pointers); no logits.
+ *   limits     : returns ISC_ERR_UNSUPPORTED, doing nothing, when one sample's activation
+ *                buffers do not fit in the array, when the image exceeds 1 MiB, when the
+ *                noise table exceeds 16384 entries (sigma above about 4.5) or when
+ *                n_classes exceeds 4096.  Any n_samples is accepted: samples are processed
+ *                in batches as large as the array allows.
+ *   first call : the first call made on a device looks up the array's device address (the
+ *                device must be current); make that call before starting a stream capture.
+ *   sharing    : all calls, on all handles and streams, share the one array.  Its contents
+ *                persist between calls (the counts are cleared at the start of each call);
+ *                two calls whose GPU work overlaps in time race on it, so serialise them.
+ */
+int isc_sample_counts_static(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id,
+                             int32_t phase, int64_t first_sample, int64_t n_samples, double sigma,
+                             void *cuda_stream, int32_t *out_counts);
+
+/*
  * isc_decide_certify / isc_decide_predict -- the host part of Algorithm 1 (steps 2,
  * 5-9) and Algorithm 2 (steps 2-6) on given vote counts; no GPU work.
  *   out_p_lower : the lower confidence bound p_A, or NULL.

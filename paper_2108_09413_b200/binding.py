@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
 EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_predict", "isc_certify", "isc_certify_batch",
-           "isc_sample_counts", "isc_decide_certify", "isc_decide_predict", "isc_noise_table",
+           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_noise_table",
            "isc_debug_tensor", "isc_set_option", "isc_get_info", "isc_strerror"]
 
 
@@ -51,6 +51,8 @@ def lib():
                                         C.c_int64, C.c_double, C.c_double, vp, vp, vp, vp, vp]
         L.isc_sample_counts.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int32, C.c_int64, C.c_int64,
                                         C.c_double, vp, vp, vp]
+        L.isc_sample_counts_static.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int32, C.c_int64, C.c_int64,
+                                               C.c_double, vp, vp]
         L.isc_decide_certify.argtypes = [vp, vp, C.c_int, C.c_int64, C.c_double, C.c_double, i32p, f64p, f64p]
         L.isc_decide_predict.argtypes = [vp, C.c_int, C.c_double, i32p]
         L.isc_noise_table.argtypes = [C.c_double, vp, C.c_int64, i32p]
@@ -144,6 +146,16 @@ class Model:
                                        float(sigma), _stream_ptr(stream), _ptr(counts), _ptr(logits)),
                "isc_sample_counts")
         return (counts, logits) if want_logits else counts
+
+    def sample_counts_static(self, x_u8, seed, image_id, phase, first_sample, n_samples, sigma, stream=None):
+        """isc_sample_counts_static: same counts, device work space taken from the library's fixed
+        array instead of cudaMalloc (for callers that may not allocate device memory)."""
+        x = self._x(x_u8)
+        counts = np.zeros(self.n_classes, dtype=np.int32)
+        _check(lib().isc_sample_counts_static(self._h, _ptr(x), seed, image_id, phase, first_sample,
+                                              n_samples, float(sigma), _stream_ptr(stream), _ptr(counts)),
+               "isc_sample_counts_static")
+        return counts
 
     def predict(self, x_u8, seed, image_id, N, sigma, alpha, stream=None):
         x = self._x(x_u8)

@@ -673,6 +673,119 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
     return ISC_OK;
 }
 
+}  // extern "C"
+
+// ------------------------------------------------------------------ allocation-free variant
+//
+// Work space of isc_sample_counts_static: one fixed array in the library's device image.  Every
+// GPU on which the library is loaded carries it from module load until the process exits.
+#define ISC_STATIC_SCRATCH_BYTES (32u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[ISC_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr size_t kStaticCountsBytes = 16u << 10;     // up to 4096 classes
+constexpr size_t kStaticTableBytes = 64u << 10;      // up to 16384 table entries (sigma up to ~4.5)
+constexpr size_t kStaticImageBytes = 1u << 20;       // up to 1 MiB of input image
+constexpr int kMaxDevices = 64;
+unsigned char *g_static_ptr[kMaxDevices];            // device address of the array, per device ordinal
+
+// The symbol name is only a host-side handle; the kernels need the array's device address,
+// which the runtime reports per device.  Done once for each device, with that device current.
+int static_scratch_base(unsigned char **base)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ISC_ERR_CUDA;
+    if (!g_static_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return ISC_ERR_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<unsigned char *>(p);
+    }
+    *base = g_static_ptr[dev];
+    return ISC_OK;
+}
+
+}  // namespace
+
+extern "C" int isc_sample_counts_static(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id,
+                                        int32_t phase, int64_t first_sample, int64_t n_samples, double sigma,
+                                        void *cuda_stream, int32_t *out_counts)
+{
+    if (!m || !x_u8 || !out_counts) return ISC_ERR_ARG;
+    int rc = check_stream_args(image_id, phase, first_sample, n_samples, sigma);
+    if (rc) return rc;
+    if (n_samples > (1ll << 31) - 1) return ISC_ERR_ARG;
+    const size_t C = (size_t)m->n_classes;
+    const size_t d = (size_t)m->in_c * m->in_h * m->in_w;
+    const int T = noise_halfwidth(sigma);
+    const size_t per_sample = generic_bytes_per_sample(m) + 256 * m->buf_bytes.size();
+    const size_t fixed = kStaticCountsBytes + kStaticTableBytes + kStaticImageBytes;
+    // sizes beyond the fixed work space are refused, never silently truncated
+    if (C * sizeof(int32_t) > kStaticCountsBytes) return ISC_ERR_UNSUPPORTED;
+    if ((size_t)(2 * T + 1) * sizeof(uint32_t) > kStaticTableBytes) return ISC_ERR_UNSUPPORTED;
+    if (d > kStaticImageBytes) return ISC_ERR_UNSUPPORTED;
+    if (per_sample > ISC_STATIC_SCRATCH_BYTES - fixed) return ISC_ERR_UNSUPPORTED;
+
+    unsigned char *base = nullptr;
+    if ((rc = static_scratch_base(&base))) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int32_t *d_counts = reinterpret_cast<int32_t *>(base);
+    uint32_t *d_cum = reinterpret_cast<uint32_t *>(base + kStaticCountsBytes);
+    uint8_t *d_x = base + kStaticCountsBytes + kStaticTableBytes;
+    unsigned char *act = base + fixed;
+    const int64_t cap = std::min<int64_t>(32768, (int64_t)((ISC_STATIC_SCRATCH_BYTES - fixed) / per_sample));
+
+    // carve the activation buffers for `cap` samples out of the array (256-byte aligned)
+    std::vector<int8_t *> buf(m->buf_bytes.size());
+    size_t off = 0;
+    for (size_t b = 0; b < buf.size(); ++b) {
+        buf[b] = reinterpret_cast<int8_t *>(act + off);
+        off += (m->buf_bytes[b] * (size_t)cap + 255) & ~(size_t)255;
+    }
+
+    std::vector<uint32_t> cum;
+    noise_table(sigma, cum);
+    // the array keeps whatever the previous call left: the vote counts must start from zero
+    CK(cudaMemsetAsync(d_counts, 0, C * sizeof(int32_t), st));
+    CK(cudaMemcpyAsync(d_cum, cum.data(), cum.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(d_x, x_u8, d, cudaMemcpyHostToDevice, st));
+    const int n_layers = (int)m->glayers.size();
+    for (int64_t done = 0; done < n_samples; done += cap) {
+        const int b = (int)std::min<int64_t>(cap, n_samples - done);
+        NoiseStream ns = make_stream(m, seed, image_id, phase, first_sample + done);
+        ns.cum = d_cum;
+        ns.T = T;
+        for (int i = 0; i < n_layers; ++i) {
+            const GLayer &G = m->glayers[(size_t)i];
+            const isc_layer &L = m->layers[(size_t)i].d;
+            int8_t *out = buf[(size_t)m->tensor_buf[(size_t)i + 1]];
+            const int8_t *in = i == 0 ? nullptr : buf[(size_t)m->tensor_buf[(size_t)L.in_tensor]];
+            const int8_t *res = L.res_tensor >= 0 ? buf[(size_t)m->tensor_buf[(size_t)L.res_tensor]] : nullptr;
+            cudaError_t e;
+            if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, b, out, st);
+            else if (L.op == ISC_CONV2D || L.op == ISC_FC) e = launch_conv(G, b, in, res, out, st);
+            else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, b, in, out, st);
+            else e = launch_maxpool(G, b, in, out, st);
+            m->launches += 1;
+            if (e != cudaSuccess) { cudaStreamSynchronize(st); return ISC_ERR_CUDA; }
+        }
+        cudaError_t e = launch_votes(buf[(size_t)m->tensor_buf[(size_t)n_layers]], m->shapes[(size_t)n_layers].cp,
+                                     m->n_classes, b, d_counts, nullptr, st);
+        m->launches += 1;
+        if (e != cudaSuccess) { cudaStreamSynchronize(st); return ISC_ERR_CUDA; }
+    }
+    std::vector<int32_t> h(C);
+    CK(cudaMemcpyAsync(h.data(), d_counts, C * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    memcpy(out_counts, h.data(), C * sizeof(int32_t));
+    return ISC_OK;
+}
+
+extern "C" {
+
 int isc_set_option(isc_model *m, const char *name, int64_t value)
 {
     if (!m || !name) return ISC_ERR_ARG;
