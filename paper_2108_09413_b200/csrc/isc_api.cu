@@ -650,6 +650,15 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
     const uint8_t *d_x;
     if ((rc = stage_image(m, x_u8, (size_t)m->in_c * m->in_h * m->in_w, false, st, &d_x))) return rc;
     NoiseStream ns = make_stream(m, seed, image_id, phase, j);
+    if (m->opt_engine == 2) {                 // read the tensor back from the resident engine
+        if (!m->mega) return ISC_ERR_UNSUPPORTED;
+        if ((rc = ensure_counts(m, (size_t)m->n_classes))) return rc;
+        std::vector<int32_t> tmp(n);
+        rc = isc::mega_debug_tensor(m->mega, d_x, ns, tensor, tmp.data(), m->d_counts, st, &m->launches);
+        if (rc) return rc;
+        memcpy(out, tmp.data(), n * sizeof(int32_t));
+        return ISC_OK;
+    }
     if (tensor == 0) {
         int32_t *d_out = nullptr;
         CK(cudaMalloc((void **)&d_out, n * sizeof(int32_t)));

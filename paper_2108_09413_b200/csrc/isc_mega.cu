@@ -1,20 +1,1237 @@
+// Shared-memory-resident tensor-core engine (sm_100a) for CIFAR-shaped residual networks.
+//
+// One persistent CTA per SM carries a group of G noisy samples through the whole network:
+// the activations never leave shared memory, every 3x3 / 1x1 convolution is an implicit GEMM
+// on tcgen05 (kind::i8, int32 accumulators in tensor memory), and only vote counts return to
+// global memory.  Per group the CTA runs a list of phases prepared on the host:
+//
+//   FILL   set a freshly allocated activation region to its halo value (the zero-point)
+//   INPUT  draw the discrete Gaussian noise (Def. 3.3, Eq. 2), add it to the image, saturate to
+//          0..255 and write the result straight into the first layer's operand region (Def. 3.4)
+//   CONV   tiles of 128 positions x N output channels: one thread issues the MMAs of a tile,
+//          four epilogue warps requantise it (fixed-point multiplier, shift, zero-points,
+//          residual add, clamp) and write the next layer's operand
+//   TAIL   global average pool, FC, argmax and vote per sample (Algorithm 1 steps 1-4)
+//
+// Activation layout: [channel plane of 16][position][16 bytes]; a position is a pixel of the
+// zero-point-padded image, all samples of the group stacked in one linear index with one halo
+// row/column shared between neighbours, so a filter tap is a constant byte offset and eight
+// consecutive positions are one 8x16-byte core matrix of the no-swizzle K-major operand layout.
+//
+// Every device-side wait is bounded by a wall-clock limit; on expiry the CTA raises an abort
+// flag, all remaining waits fall through, and the host reports ISC_ERR_TIMEOUT.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
+#include <vector>
+
 #include "isc_mega.h"
 
 namespace isc {
 
-struct MegaPlan { int unused; };
+namespace {
 
-int mega_build(const MegaLayerIn *, int, int, int, int, int, MegaPlan **out)
+constexpr int kEpiWarps = 16;
+constexpr int kWarpGroups = kEpiWarps / 4;
+constexpr int kThreads = 32 * (1 + kEpiWarps);
+constexpr int kTmemSlots = 8;
+constexpr int kSlotCols = 64;
+constexpr int kMaxKsteps = 20;
+constexpr int kMaxChunks = 4;
+constexpr int kCtrlBytes = 4096;
+constexpr int kSmemLimit = 227 * 1024;
+constexpr int kFillItemBytes = 8192;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+
+enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
+enum { ERR_NONE = 0, ERR_WAIT_ITEMS = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_EMPTY = 3, ERR_WAIT_FULL = 4,
+       ERR_WAIT_DRAIN = 5 };
+
+struct alignas(16) MPhase {
+    int32_t kind, n_items, item_base, full_sync;
+    // geometry of the positions this phase walks (CONV: its input tensor)
+    int32_t H, W, Wp, HsWp;
+    int32_t P_first, scatter, o_Wp, o_HsWp;
+    uint32_t magic_hswp, magic_wp, pad0, pad1;
+    // FILL
+    uint32_t fill_off, fill_bytes, fill_word, pad2;
+    // CONV
+    uint32_t in_off, n_ksteps, idesc, n_chunks;
+    uint32_t w_off, w_bytes, const_off, conv_index;
+    unsigned long long w_gmem;
+    int32_t tile_base, n_rows;
+    int32_t res_mult, res_n;
+    long long res_R;
+    int32_t a_delta[kMaxKsteps];
+    uint32_t a_lbo[kMaxKsteps];
+    uint32_t out_off[kMaxChunks], res_off[kMaxChunks];
+    int32_t lo[kMaxChunks];
+    uint32_t halo[kMaxChunks], flags[kMaxChunks];   // flags: bit0 explicit lower clamp, bit1 residual
+};
+
+struct FcConst { int32_t mult, n, zp_out, lo, bias, pad0, pad1, pad2; };
+
+struct MegaParams {
+    const MPhase *phases;
+    int32_t n_phases, n_conv, items_per_group, tiles_per_group;
+    int32_t G, n_groups, n_samples, in_c;
+    const uint8_t *x;                 // clean image, CHW
+    NoiseStream ns;
+    uint32_t input_off;               // operand region of the first layer
+    int32_t input_halo;
+    // tail
+    uint32_t tail_in_off, tail_plane_bytes;
+    int32_t tail_C, tail_H, tail_W, tail_Wp, tail_HsWp;
+    int32_t pool_mult, pool_n, pool_zp_in, pool_zp_out, pool_lo;
+    const int8_t *fc_w;               // [n_classes][64]
+    const FcConst *fc_c;
+    int32_t n_classes, fc_pad;
+    int32_t *counts;
+    int8_t *logits;                   // [n_samples][n_classes] or null
+    int32_t *err;
+    // debug
+    int32_t stop_phase;
+    uint32_t dump_off, dump_bytes;
+    uint8_t *dump;
+};
+
+struct Ctrl {
+    unsigned long long full[kTmemSlots], empty[kTmemSlots], wbar[3], drain;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+    uint32_t prog[kEpiWarps];
+    int32_t hist[128];
+};
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
+
+// ------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void st_release(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void named_bar(int id, int n)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// K-major, no-swizzle shared-memory operand descriptor: rows of 16 bytes, 8 rows contiguous,
+// `sbo` bytes between 8-row groups, `lbo` bytes between the two 16-byte halves of K = 32.
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+// saturate four int32 to int8 and pack them (v0 in the low byte)
+__device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3)
+{
+    uint32_t hi, d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi) : "r"(v3), "r"(v2));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v1), "r"(v0), "r"(hi));
+    return d;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c;
+}
+
+__device__ __forceinline__ int noise_level(uint32_t u, const uint32_t *__restrict__ cum, int T)
+{
+    int lo = 0, hi = 2 * T;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (u < __ldg(cum + mid)) hi = mid; else lo = mid + 1;
+    }
+    return lo - T;
+}
+
+// ------------------------------------------------------------------ bounded waits
+
+struct Waiter {
+    Ctrl *ctrl;
+    int32_t *err;
+    __device__ __forceinline__ bool aborted() const { return ctrl->abort_flag != 0; }
+    __device__ __noinline__ void fail(int code)
+    {
+        ctrl->abort_flag = 1;
+        atomicCAS(err, 0, code | (blockIdx.x << 8));
+    }
+    template <typename Pred>
+    __device__ __forceinline__ bool until(Pred pred, int code)
+    {
+        if (pred()) return true;
+        const unsigned long long t0 = globaltimer();
+        for (int spin = 0;; ++spin) {
+            if (pred()) return true;
+            if ((spin & 63) == 63) {
+                if (aborted()) return false;
+                if (globaltimer() - t0 > kWaitLimitNs) { fail(code); return false; }
+            }
+        }
+    }
+};
+
+// number of global item indices g < end with g % kWarpGroups == wg
+__device__ __forceinline__ uint32_t items_of_wg_below(uint32_t end, int wg)
+{
+    return end > (uint32_t)wg ? (end - wg + kWarpGroups - 1) / kWarpGroups : 0u;
+}
+
+// every item with global index < end has been completed by all four warps of its warpgroup
+__device__ __forceinline__ bool all_items_below_done(uint32_t prog_addr, uint32_t end)
+{
+    for (int wg = 0; wg < kWarpGroups; ++wg) {
+        const uint32_t need = items_of_wg_below(end, wg);
+        for (int k = 0; k < 4; ++k)
+            if (ld_acquire(prog_addr + 4 * (wg * 4 + k)) < need) return false;
+    }
+    return true;
+}
+
+__device__ __forceinline__ bool item_done(uint32_t prog_addr, uint32_t g)
+{
+    const int wg = g % kWarpGroups;
+    const uint32_t need = g / kWarpGroups + 1;
+    for (int k = 0; k < 4; ++k)
+        if (ld_acquire(prog_addr + 4 * (wg * 4 + k)) < need) return false;
+    return true;
+}
+
+// ------------------------------------------------------------------ roles
+
+__device__ void issue_weights(const MPhase &ph, uint32_t sbase, uint32_t wbar_addr)
+{
+    mbar_expect_tx(wbar_addr, ph.w_bytes);
+    bulk_g2s(sbase + ph.w_off, reinterpret_cast<const void *>(ph.w_gmem), ph.w_bytes, wbar_addr);
+}
+
+// Warp 0, one thread: weight loads and all tensor-core work of one group.
+__device__ void mma_role(const MegaParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, int it, const int *conv_phase)
+{
+    Waiter w{ctrl, p.err};
+    const uint32_t prog = smem_u32(ctrl->prog);
+    const uint32_t item_off = (uint32_t)it * p.items_per_group;
+    const uint32_t tile_off = (uint32_t)it * p.tiles_per_group;
+    const uint32_t conv_off = (uint32_t)it * p.n_conv;
+    {   // weights of this group's first convolution (everything before the group barrier is complete)
+        const uint32_t cg = conv_off;
+        if (!w.aborted()) issue_weights(p.phases[conv_phase[0]], sbase, smem_u32(&ctrl->wbar[cg % 3]));
+    }
+    for (int ph = 0; ph < p.n_phases && ph <= p.stop_phase; ++ph) {
+        const MPhase &P = p.phases[ph];
+        if (P.kind != PH_CONV) continue;
+        // the phase before last must be complete (shared-memory reuse rule); with full_sync the last one too
+        const uint32_t end = item_off + (P.full_sync ? (uint32_t)P.item_base
+                                                     : (ph >= 1 ? (uint32_t)p.phases[ph - 1].item_base : 0u));
+        if (!w.until([&] { return all_items_below_done(prog, end); }, ERR_WAIT_ITEMS)) return;
+        const uint32_t cg = conv_off + P.conv_index;
+        if ((int)P.conv_index + 1 < p.n_conv && conv_phase[P.conv_index + 1] <= p.stop_phase)
+            issue_weights(p.phases[conv_phase[P.conv_index + 1]], sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
+        {
+            const uint32_t bar = smem_u32(&ctrl->wbar[cg % 3]), par = (cg / 3) & 1;
+            if (!w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_WEIGHTS)) return;
+        }
+        const uint32_t dep_base = item_off + (ph >= 1 ? (uint32_t)p.phases[ph - 1].item_base : 0u);
+        const int dep_n = ph >= 1 ? p.phases[ph - 1].n_items : 0;
+        const uint32_t n_rows = (uint32_t)P.n_rows;
+        for (int t = 0; t < P.n_items; ++t) {
+            if (!P.full_sync && dep_n > 0) {
+                const int t0 = max(t - 1, 0), t1 = min(t + 1, dep_n - 1);
+                if (!w.until([&] {
+                        for (int q = t0; q <= t1; ++q)
+                            if (!item_done(prog, dep_base + q)) return false;
+                        return true;
+                    }, ERR_WAIT_ITEMS)) return;
+            }
+            const uint32_t ts = tile_off + P.tile_base + t, slot = ts % kTmemSlots, use = ts / kTmemSlots;
+            if (use > 0) {
+                const uint32_t bar = smem_u32(&ctrl->empty[slot]), par = (use - 1) & 1;
+                if (!w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_EMPTY)) return;
+            }
+            tc_fence_after();
+            const uint32_t d = tmem + slot * kSlotCols;
+            const uint32_t abase = sbase + P.in_off + (uint32_t)(P.P_first + 128 * t) * 16u;
+            for (uint32_t k = 0; k < P.n_ksteps; ++k) {
+                const uint64_t ad = make_desc(abase + (uint32_t)P.a_delta[k], P.a_lbo[k], 128);
+                const uint64_t bd = make_desc(sbase + P.w_off + k * n_rows * 32u, 128, 256);
+                mma_i8(d, ad, bd, P.idesc, k > 0 ? 1u : 0u);
+            }
+            mma_commit(smem_u32(&ctrl->full[slot]));
+        }
+    }
+}
+
+struct EpiCtx {
+    Ctrl *ctrl;
+    uint32_t sbase, tmem;
+    int warp_e, wg, quarter, lane, tid_wg;
+    uint32_t done;      // items this warp has completed (monotonic)
+};
+
+__device__ __forceinline__ void finish_item(EpiCtx &c)
+{
+    fence_proxy_async();
+    __syncwarp();
+    c.done += 1;
+    if (c.lane == 0) st_release(smem_u32(&c.ctrl->prog[c.warp_e]), c.done);
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+__device__ void fill_item(const MPhase &P, EpiCtx &c, int i)
+{
+    const uint32_t begin = (uint32_t)i * kFillItemBytes;
+    const uint32_t end = min(begin + kFillItemBytes, P.fill_bytes);
+    const uint4 v = make_uint4(P.fill_word, P.fill_word, P.fill_word, P.fill_word);
+    for (uint32_t o = begin + c.tid_wg * 16; o < end; o += 128 * 16) st_shared_v4(c.sbase + P.fill_off + o, v);
+}
+
+// INPUT: one thread = four horizontally adjacent pixels of one sample, all input channels.
+__device__ void input_item(const MegaParams &p, const MPhase &P, EpiCtx &c, int i, int grp)
+{
+    const int wq = P.W >> 2;
+    const int quads = p.G * P.H * wq;
+    const int qi = i * 128 + c.tid_wg;
+    if (qi >= quads) return;
+    const int s = qi / (P.H * wq);
+    const int rem = qi - s * (P.H * wq);
+    const int y = rem / wq, x4 = rem - y * wq;
+    const long long j = p.ns.first_sample + (long long)grp * p.G + s;
+    uint32_t px[4] = {0, 0, 0, 0};
+    for (int ch = 0; ch < p.in_c; ++ch) {
+        const uint32_t e = (uint32_t)((ch * P.H + y) * P.W + 4 * x4);
+        const uint4 ctr = make_uint4(e >> 2, (uint32_t)(j & 0xFFFFFFFFll), p.ns.ctr2,
+                                     p.ns.ctr3_fixed | (uint32_t)(((j >> 32) & 0xFF) << 8));
+        const uint4 r = philox4x32_10(ctr, p.ns.key0, p.ns.key1);
+        const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+        const uint32_t clean = __ldg(reinterpret_cast<const uint32_t *>(p.x + e));
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int v = (int)((clean >> (8 * k)) & 0xFF) + noise_level(u[k], p.ns.cum, p.ns.T);
+            v = min(255, max(0, v));
+            px[k] |= (uint32_t)v << (8 * ch);
+        }
+    }
+    const uint32_t pos = (uint32_t)(s * P.HsWp + (y + 1) * P.Wp + 4 * x4 + 1);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) st_shared_v4(c.sbase + p.input_off + (pos + k) * 16u, make_uint4(px[k], 0, 0, 0));
+}
+
+// CONV epilogue of one tile: thread = one position (tensor-memory lane), 16 channels at a time.
+__device__ void conv_tile(const MPhase &P, EpiCtx &c, int t, uint32_t slot, int G)
+{
+    const uint32_t pos = (uint32_t)(P.P_first + 128 * t + c.quarter * 32 + c.lane);
+    // position -> (sample, row, column) of the padded image
+    const uint32_t s = __umulhi(pos, P.magic_hswp);
+    const uint32_t rem = pos - s * (uint32_t)P.HsWp;
+    const uint32_t y1 = __umulhi(rem, P.magic_wp);
+    const uint32_t x1 = rem - y1 * (uint32_t)P.Wp;
+    const bool interior = (int)s < G && y1 >= 1 && x1 >= 1;
+    bool store = true;
+    uint32_t opos = pos;
+    if (P.scatter) {
+        const uint32_t y = y1 - 1, x = x1 - 1;
+        store = interior && !(y & 1) && !(x & 1);
+        opos = s * (uint32_t)P.o_HsWp + ((y >> 1) + 1) * (uint32_t)P.o_Wp + (x >> 1) + 1;
+    }
+    const uint32_t taddr = c.tmem + ((uint32_t)(c.quarter * 32) << 16) + slot * kSlotCols;
+    const long long res_R = P.res_R;
+    const int res_mult = P.res_mult, res_n = P.res_n;
+    for (uint32_t ch = 0; ch < P.n_chunks; ++ch) {
+        int acc[16];
+        tmem_ld16(taddr + ch * 16, acc);
+        if (ch + 1 == P.n_chunks) {           // accumulator slot may be overwritten from here on
+            tc_fence_before();
+            __syncwarp();
+            if (c.lane == 0) mbar_arrive(smem_u32(&c.ctrl->empty[slot]));
+        }
+        const uint32_t flags = P.flags[ch];
+        uint32_t rw[4] = {0, 0, 0, 0};
+        if (flags & 2) {
+            const uint4 rv = ld_shared_v4(c.sbase + P.res_off[ch] + pos * 16u);
+            rw[0] = rv.x; rw[1] = rv.y; rw[2] = rv.z; rw[3] = rv.w;
+        }
+        const uint32_t cbase = c.sbase + P.const_off + ch * 256u;
+        const int lo = P.lo[ch];
+        int q[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const uint4 cs = ld_shared_v4(cbase + k * 16);   // mult, B low, B high, shift - 1
+            const long long B = (long long)(((unsigned long long)cs.z << 32) | cs.y);
+            const long long v = (long long)acc[k] * (long long)(int)cs.x + B;
+            int y = (int)(v >> 32) >> (int)cs.w;
+            if (flags & 2) {
+                const int r = (int)(int8_t)((rw[k >> 2] >> (8 * (k & 3))) & 0xFF);
+                y += (int)(((long long)r * res_mult + res_R) >> res_n);
+            }
+            if (flags & 1) y = max(y, lo);
+            q[k] = y;
+        }
+        uint4 o = make_uint4(pack4_sat(q[0], q[1], q[2], q[3]), pack4_sat(q[4], q[5], q[6], q[7]),
+                             pack4_sat(q[8], q[9], q[10], q[11]), pack4_sat(q[12], q[13], q[14], q[15]));
+        if (!P.scatter && !interior) o = make_uint4(P.halo[ch], P.halo[ch], P.halo[ch], P.halo[ch]);
+        if (store) st_shared_v4(c.sbase + P.out_off[ch] + opos * 16u, o);
+    }
+}
+
+// TAIL: global average pool, FC, argmax and vote; one warp carries one sample.
+__device__ void tail_sample(const MegaParams &p, EpiCtx &c, int s, int grp)
+{
+    const int hw = p.tail_H * p.tail_W;
+    int pooled[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int ch = c.lane + 32 * h;
+        int q = 0;
+        if (ch < p.tail_C) {
+            const uint32_t base = c.sbase + p.tail_in_off + (uint32_t)(ch >> 4) * p.tail_plane_bytes + (ch & 15);
+            int sum = 0;
+            for (int i = 0; i < hw; ++i) {
+                const int y = i / p.tail_W, x = i - y * p.tail_W;
+                const uint32_t pos = (uint32_t)(s * p.tail_HsWp + (y + 1) * p.tail_Wp + x + 1);
+                int v;
+                asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(base + pos * 16u));
+                sum += v - p.pool_zp_in;
+            }
+            long long v = ((long long)sum * p.pool_mult + (1ll << (p.pool_n - 1))) >> p.pool_n;
+            v += p.pool_zp_out;
+            v = v < p.pool_lo ? p.pool_lo : v;
+            v = v > 127 ? 127 : v;
+            q = (int)v;
+        }
+        pooled[h] = q;
+    }
+    const long long sample = (long long)grp * p.G + s;          // index within this launch
+    const bool counted = s < p.G && sample < p.n_samples;
+    int best_v = -1000, best_o = 0x7fffffff;
+    for (int o0 = 0; o0 < p.n_classes; o0 += 32) {
+        const int o = o0 + c.lane;
+        const bool live = o < p.n_classes;
+        const FcConst k = p.fc_c[live ? o : 0];
+        const int8_t *wrow = p.fc_w + (size_t)(live ? o : 0) * 64;
+        int acc = k.bias;
+        for (int cc = 0; cc < p.tail_C; ++cc) {
+            const int a = __shfl_sync(0xffffffffu, pooled[cc >> 5], cc & 31);
+            acc += a * (int)__ldg(wrow + cc);
+        }
+        long long v = ((long long)acc * k.mult + (1ll << (k.n - 1))) >> k.n;
+        v += k.zp_out;
+        v = v < k.lo ? k.lo : v;
+        v = v > 127 ? 127 : v;
+        if (live) {
+            if ((int)v > best_v) { best_v = (int)v; best_o = o; }
+            if (counted && p.logits) p.logits[sample * p.n_classes + o] = (int8_t)v;
+        }
+    }
+    // lowest index among the maxima
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        const int ov = __shfl_xor_sync(0xffffffffu, best_v, d), oo = __shfl_xor_sync(0xffffffffu, best_o, d);
+        if (ov > best_v || (ov == best_v && oo < best_o)) { best_v = ov; best_o = oo; }
+    }
+    if (counted && c.lane == 0) atomicAdd(&c.ctrl->hist[best_o], 1);
+}
+
+// Epilogue warps: all non-tensor-core work of one group, item by item.
+__device__ void epi_role(const MegaParams &p, EpiCtx &c, int it, int grp)
+{
+    Waiter w{c.ctrl, p.err};
+    const uint32_t prog = smem_u32(c.ctrl->prog);
+    const uint32_t item_off = (uint32_t)it * p.items_per_group;
+    const uint32_t tile_off = (uint32_t)it * p.tiles_per_group;
+    const uint32_t conv_off = (uint32_t)it * p.n_conv;
+    for (int ph = 0; ph < p.n_phases && ph <= p.stop_phase; ++ph) {
+        const MPhase &P = p.phases[ph];
+        const uint32_t first = item_off + P.item_base;
+        const int i0 = (c.wg + kWarpGroups - (int)(first % kWarpGroups)) % kWarpGroups;
+        if (i0 >= P.n_items) continue;
+        bool ok;
+        if (P.kind != PH_CONV) {
+            ok = w.until([&] { return all_items_below_done(prog, first); }, ERR_WAIT_ITEMS);
+        } else {
+            const uint32_t cg = conv_off + P.conv_index;
+            const uint32_t bar = smem_u32(&c.ctrl->wbar[cg % 3]), par = (cg / 3) & 1;
+            ok = w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_WEIGHTS);
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        for (int i = i0; i < P.n_items; i += kWarpGroups) {
+            if (ok) {
+                if (P.kind == PH_FILL) {
+                    fill_item(P, c, i);
+                } else if (P.kind == PH_INPUT) {
+                    input_item(p, P, c, i, grp);
+                } else if (P.kind == PH_CONV) {
+                    const uint32_t ts = tile_off + P.tile_base + i, slot = ts % kTmemSlots;
+                    const uint32_t bar = smem_u32(&c.ctrl->full[slot]), par = (ts / kTmemSlots) & 1;
+                    ok = w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_FULL);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (ok) {
+                        tc_fence_after();
+                        conv_tile(P, c, i, slot, p.G);
+                    }
+                } else {
+                    const int s = i * 4 + (c.warp_e & 3);
+                    tail_sample(p, c, min(s, p.G - 1), grp + (s >= p.G ? (1 << 28) : 0));
+                }
+            }
+            finish_item(c);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) k_mega(const MegaParams p, const int *__restrict__ conv_phase)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
+    const uint32_t sbase = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTmemSlots; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->empty[s]), 4);
+        }
+        for (int s = 0; s < 3; ++s) mbar_init(smem_u32(&ctrl->wbar[s]), 1);
+        mbar_init(smem_u32(&ctrl->drain), 1);
+        ctrl->abort_flag = 0;
+    }
+    for (int i = threadIdx.x; i < 128; i += blockDim.x) ctrl->hist[i] = 0;
+    if (threadIdx.x < kEpiWarps) ctrl->prog[threadIdx.x] = 0;
+    if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), 512);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctrl->tmem_base;
+
+    EpiCtx c;
+    c.ctrl = ctrl; c.sbase = sbase; c.tmem = tmem;
+    c.warp_e = warp - 1; c.wg = (warp - 1) >> 2; c.quarter = warp & 3; c.lane = lane;
+    c.tid_wg = ((warp - 1) & 3) * 32 + lane; c.done = 0;
+
+    int it = 0;
+    for (int grp = blockIdx.x; grp < p.n_groups; grp += gridDim.x, ++it) {
+        if (warp == 0) {
+            if (lane == 0) mma_role(p, ctrl, sbase, tmem, it, conv_phase);
+            __syncwarp();
+        } else {
+            epi_role(p, c, it, grp);
+        }
+        __syncthreads();
+    }
+    if (!ctrl->abort_flag)
+        for (int i = threadIdx.x; i < p.n_classes; i += blockDim.x)
+            if (ctrl->hist[i]) atomicAdd(p.counts + i, ctrl->hist[i]);
+    if (p.dump)
+        for (uint32_t o = threadIdx.x * 16u; o < p.dump_bytes; o += blockDim.x * 16u)
+            *reinterpret_cast<uint4 *>(p.dump + o) = ld_shared_v4(sbase + p.dump_off + o);
+    // no tensor-core work may be in flight when tensor memory is released
+    if (warp == 0 && lane == 0) {
+        Waiter w{ctrl, p.err};
+        mma_commit(smem_u32(&ctrl->drain));
+        const uint32_t bar = smem_u32(&ctrl->drain);
+        w.until([&] { return mbar_test(bar, 0); }, ERR_WAIT_DRAIN);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// =============================================================================== host planner
+
+struct PlanTensor {
+    int C = 0, H = 0, W = 0, planes = 0, halo = 0;
+    int Wp = 0, HsWp = 0, P_first = 0, n_tiles = 0, npa = 0;
+    uint32_t plane_bytes = 0, bytes = 0;
+    int buffer = -1;             // index into buffers
+    int producer_phase = -1;
+    bool scatter_produced = false;
+    int last_use_layer = -1;     // model layer index of the last reader
+};
+
+struct PlanBuffer {
+    uint32_t bytes = 0, off = 0;
+    int birth = 0, death = 0;    // phase indices
+    int halo = 0;
+    int C = 0, H = 0, W = 0;
+    int last_tenant_death_layer = -1;
+    bool last_death_as_conv_operand = false;
+};
+
+struct AllocReq { uint32_t bytes; int birth, death, slack; uint32_t *off; };
+
+void set_geometry(PlanTensor &t, int G)
+{
+    t.planes = (t.C + 15) / 16;
+    t.Wp = t.W + 1;
+    t.HsWp = (t.H + 1) * t.Wp;
+    t.P_first = t.Wp + 1;
+    const int p_last = (G - 1) * t.HsWp + t.H * t.Wp + t.W;
+    t.n_tiles = (p_last - t.P_first + 1 + 127) / 128;
+    t.npa = (t.P_first + 128 * t.n_tiles + t.Wp + 2 + 7) & ~7;
+    t.plane_bytes = (uint32_t)t.npa * 16u;
+    t.bytes = t.plane_bytes * (uint32_t)t.planes;
+}
+
+uint32_t magic_for(uint32_t d, uint32_t limit, bool *ok)
+{
+    const uint32_t m = (uint32_t)(((1ull << 32) + d - 1) / d);
+    for (uint32_t p = 0; p < limit; ++p)
+        if ((uint32_t)(((unsigned long long)p * m) >> 32) != p / d) { *ok = false; break; }
+    return m;
+}
+
+}  // namespace
+
+struct MegaPlan {
+    int G = 0, in_c = 0, in_h = 0, in_w = 0, n_classes = 0;
+    std::vector<MPhase> phases;
+    std::vector<int> conv_phase;
+    int items_per_group = 0, tiles_per_group = 0;
+    uint32_t smem_bytes = 0;
+    MegaParams base;                      // fields that do not change between launches
+    // device copies
+    MPhase *d_phases = nullptr;
+    int *d_conv_phase = nullptr;
+    uint8_t *d_blob = nullptr;
+    int8_t *d_fc_w = nullptr;
+    FcConst *d_fc_c = nullptr;
+    int32_t *d_err = nullptr;
+    uint8_t *d_dump = nullptr;
+    // model tensor id -> where it lives (for the debug read-back)
+    std::vector<PlanTensor> tensors;
+    std::vector<uint32_t> tensor_off;
+    int sm_count = 0;
+    bool attr_set = false;
+};
+
+namespace {
+
+struct ConvNode {
+    int layer;                 // model layer index
+    int fused_layer = -1;      // second layer (1x1 projection) sharing input and stride
+};
+
+bool conv_ok(const isc_layer &L, bool first)
+{
+    if (L.op != ISC_CONV2D) return false;
+    if (L.kh != L.kw || (L.kh != 1 && L.kh != 3)) return false;
+    if (L.pad != (L.kh - 1) / 2) return false;
+    if (L.stride != 1 && L.stride != 2) return false;
+    if (first) { if (L.cin > 4 || L.stride != 1) return false; }
+    else if (L.cin % 16 != 0 || L.cin > 64) return false;
+    if (L.cout % 16 != 0 || L.cout > 64) return false;
+    return true;
+}
+
+// First-fit placement of one request among the allocations that are still busy at its birth.
+bool place(std::vector<AllocReq> &done, AllocReq &r, uint32_t capacity)
+{
+    std::vector<std::pair<uint32_t, uint32_t>> busy;
+    for (const AllocReq &e : done)
+        if (e.death >= r.birth - r.slack) busy.push_back({*e.off, *e.off + e.bytes});
+    std::sort(busy.begin(), busy.end());
+    uint32_t at = kCtrlBytes;
+    for (const auto &b : busy) {
+        if (at + r.bytes <= b.first) break;
+        at = std::max(at, (b.second + 127u) & ~127u);
+    }
+    if (at + r.bytes > capacity) return false;
+    *r.off = at;
+    done.push_back(r);
+    return true;
+}
+
+// Build the phase list for groups of G samples.  Returns false when it does not fit.
+bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, int G,
+                MegaPlan *plan, std::vector<uint8_t> *blob_out, std::vector<uint32_t> *blob_offsets)
+{
+    const int n_conv_layers = n_layers - 2;
+    // ---- tensors of the model (tensor t = output of layer t-1)
+    std::vector<PlanTensor> T((size_t)n_layers + 1);
+    T[0].C = in_c; T[0].H = in_h; T[0].W = in_w; T[0].halo = layers[0].d.zp_in;
+    for (int i = 0; i < n_conv_layers; ++i) {
+        const isc_layer &L = layers[i].d;
+        const PlanTensor &in = T[(size_t)L.in_tensor];
+        PlanTensor &o = T[(size_t)i + 1];
+        o.C = L.cout;
+        o.H = (in.H + 2 * L.pad - L.kh) / L.stride + 1;
+        o.W = (in.W + 2 * L.pad - L.kw) / L.stride + 1;
+        o.halo = L.zp_out;
+        if (L.stride == 2 && ((in.H & 1) || (in.W & 1))) return false;
+    }
+    for (int t = 0; t <= n_conv_layers; ++t) set_geometry(T[(size_t)t], G);
+    for (int i = 0; i < n_layers; ++i) {
+        T[(size_t)layers[i].d.in_tensor].last_use_layer = i;
+        if (layers[i].d.res_tensor >= 0) T[(size_t)layers[i].d.res_tensor].last_use_layer = i;
+    }
+    // ---- conv nodes, fusing a 3x3 with the 1x1 projection that follows it on the same input
+    std::vector<ConvNode> nodes;
+    for (int i = 0; i < n_conv_layers; ++i) {
+        ConvNode nd; nd.layer = i;
+        if (i + 1 < n_conv_layers) {
+            const isc_layer &A = layers[i].d, &B = layers[i + 1].d;
+            if (A.kh == 3 && B.kh == 1 && B.in_tensor == A.in_tensor && B.stride == A.stride && B.res_tensor < 0 &&
+                A.res_tensor < 0 && A.cout + B.cout <= kSlotCols && A.zp_in == B.zp_in &&
+                T[(size_t)i + 1].H == T[(size_t)i + 2].H && T[(size_t)i + 1].W == T[(size_t)i + 2].W) {
+                nd.fused_layer = i + 1;
+                ++i;
+            }
+        }
+        nodes.push_back(nd);
+    }
+    // ---- phase skeleton: FILL(input) INPUT, then per node [FILL per fresh output] CONV, then TAIL
+    struct Skel { int kind; int node; int tensor; };
+    std::vector<Skel> skel;
+    std::vector<PlanBuffer> buffers;
+    std::vector<int> layer_phase((size_t)n_layers, -1);
+    auto new_buffer = [&](int tensor) {
+        PlanBuffer b;
+        b.bytes = T[(size_t)tensor].bytes; b.halo = T[(size_t)tensor].halo;
+        b.C = T[(size_t)tensor].C; b.H = T[(size_t)tensor].H; b.W = T[(size_t)tensor].W;
+        b.birth = (int)skel.size();
+        buffers.push_back(b);
+        T[(size_t)tensor].buffer = (int)buffers.size() - 1;
+        skel.push_back({PH_FILL, -1, tensor});
+    };
+    new_buffer(0);
+    skel.push_back({PH_INPUT, -1, 0});
+    int prev_conv_layer_last = -1;         // last model layer covered by the previous conv phase
+    for (size_t ni = 0; ni < nodes.size(); ++ni) {
+        const ConvNode &nd = nodes[ni];
+        const int lay[2] = {nd.layer, nd.fused_layer};
+        const isc_layer &L0 = layers[nd.layer].d;
+        for (int k = 0; k < 2; ++k) {
+            if (lay[k] < 0) continue;
+            const isc_layer &L = layers[lay[k]].d;
+            const int out_t = lay[k] + 1;
+            PlanTensor &o = T[(size_t)out_t];
+            // (a) in place over the residual operand, when this layer is its last reader
+            if (L.res_tensor >= 0 && L.stride == 1 && T[(size_t)L.res_tensor].last_use_layer == lay[k] &&
+                L.res_tensor != L.in_tensor && T[(size_t)L.res_tensor].halo == o.halo &&
+                T[(size_t)L.res_tensor].bytes == o.bytes) {
+                o.buffer = T[(size_t)L.res_tensor].buffer;
+                continue;
+            }
+            // (b) over a same-shaped tensor whose last reader was the previous conv phase
+            int reuse = -1;
+            if (L.stride == 1 && lay[1] < 0 && prev_conv_layer_last >= 0)
+                for (int t = 1; t <= n_conv_layers && reuse < 0; ++t) {
+                    const PlanTensor &x = T[(size_t)t];
+                    if (x.buffer < 0 || t == out_t || t == L.in_tensor || t == L.res_tensor) continue;
+                    if (x.last_use_layer != prev_conv_layer_last) continue;
+                    if (x.C != o.C || x.H != o.H || x.W != o.W || x.halo != o.halo) continue;
+                    bool newest = true;           // x must be the current tenant of its buffer
+                    for (int u = t + 1; u <= n_conv_layers; ++u)
+                        if (T[(size_t)u].buffer == x.buffer) newest = false;
+                    if (newest) reuse = x.buffer;
+                }
+            if (reuse >= 0) { o.buffer = reuse; continue; }
+            new_buffer(out_t);
+        }
+        (void)L0;
+        for (int k = 0; k < 2; ++k)
+            if (lay[k] >= 0) layer_phase[(size_t)lay[k]] = (int)skel.size();
+        skel.push_back({PH_CONV, (int)ni, -1});
+        prev_conv_layer_last = nd.fused_layer >= 0 ? nd.fused_layer : nd.layer;
+    }
+    const int tail_phase = (int)skel.size();
+    skel.push_back({PH_TAIL, -1, n_conv_layers});
+    layer_phase[(size_t)n_layers - 2] = tail_phase;
+    layer_phase[(size_t)n_layers - 1] = tail_phase;
+    const int n_phases = (int)skel.size();
+    // ---- lifetimes
+    for (int t = 0; t <= n_conv_layers; ++t) {
+        PlanTensor &x = T[(size_t)t];
+        if (x.buffer < 0) return false;
+        int death = x.last_use_layer >= 0 ? layer_phase[(size_t)x.last_use_layer] : -1;
+        if (t >= 1) x.producer_phase = layer_phase[(size_t)t - 1];
+        else x.producer_phase = 1;
+        death = std::max(death, x.producer_phase);
+        buffers[(size_t)x.buffer].death = std::max(buffers[(size_t)x.buffer].death, death);
+    }
+    // ---- weight blobs: conv c is loaded when conv c-1 starts (conv 0 at the start of the group)
+    std::vector<int> conv_phase;
+    for (int ph = 0; ph < n_phases; ++ph)
+        if (skel[(size_t)ph].kind == PH_CONV) conv_phase.push_back(ph);
+    const int n_conv = (int)conv_phase.size();
+    std::vector<uint32_t> w_bytes((size_t)n_conv), w_off((size_t)n_conv), n_rows((size_t)n_conv);
+    std::vector<std::vector<std::pair<int, int>>> ksteps((size_t)n_conv);   // indices into chunk list, -1 = none
+    std::vector<std::vector<int>> chunk_addr((size_t)n_conv);
+    for (int cidx = 0; cidx < n_conv; ++cidx) {
+        const ConvNode &nd = nodes[(size_t)skel[(size_t)conv_phase[(size_t)cidx]].node];
+        const isc_layer &L = layers[nd.layer].d;
+        const PlanTensor &in = T[(size_t)L.in_tensor];
+        const int taps = L.kh * L.kw;
+        std::vector<int> addr;
+        for (int tap = 0; tap < taps; ++tap)
+            for (int pl = 0; pl < in.planes; ++pl) {
+                const int r = tap / L.kw, s = tap % L.kw;
+                addr.push_back(((r - L.pad) * in.Wp + (s - L.pad)) * 16 + pl * (int)in.plane_bytes);
+            }
+        std::vector<std::pair<int, int>> ks;
+        for (size_t a = 0; a < addr.size(); a += 2) {
+            if (a + 1 < addr.size()) {
+                if (addr[a + 1] > addr[a]) ks.push_back({(int)a, (int)a + 1});
+                else ks.push_back({(int)a + 1, (int)a});
+                const int diff = std::abs(addr[a + 1] - addr[a]);
+                if (diff == 0 || diff >= (1 << 18)) return false;
+            } else {
+                ks.push_back({(int)a, -1});
+            }
+        }
+        if ((int)ks.size() > kMaxKsteps) return false;
+        ksteps[(size_t)cidx] = ks;
+        chunk_addr[(size_t)cidx] = addr;
+        n_rows[(size_t)cidx] = (uint32_t)(L.cout + (nd.fused_layer >= 0 ? layers[nd.fused_layer].d.cout : 0));
+        w_bytes[(size_t)cidx] = (uint32_t)ks.size() * n_rows[(size_t)cidx] * 32u + n_rows[(size_t)cidx] * 16u;
+    }
+    // ---- shared-memory placement in order of birth
+    std::vector<AllocReq> reqs, placed;
+    for (PlanBuffer &b : buffers) reqs.push_back({b.bytes, b.birth, b.death, 0, &b.off});
+    for (int cidx = 0; cidx < n_conv; ++cidx)
+        reqs.push_back({w_bytes[(size_t)cidx], cidx == 0 ? 0 : conv_phase[(size_t)cidx - 1], conv_phase[(size_t)cidx],
+                        cidx == 0 ? 0 : 1, &w_off[(size_t)cidx]});
+    std::stable_sort(reqs.begin(), reqs.end(), [](const AllocReq &a, const AllocReq &b) { return a.birth < b.birth; });
+    uint32_t high = kCtrlBytes;
+    for (AllocReq &r : reqs) {
+        if (!place(placed, r, kSmemLimit)) return false;
+        high = std::max(high, *r.off + r.bytes);
+    }
+    // ---- emit phases
+    plan->phases.assign((size_t)n_phases, MPhase{});
+    plan->conv_phase = conv_phase;
+    plan->tensors = T;
+    plan->tensor_off.assign(T.size(), 0);
+    for (int t = 0; t <= n_conv_layers; ++t) plan->tensor_off[(size_t)t] = buffers[(size_t)T[(size_t)t].buffer].off;
+    int item_base = 0, tile_base = 0;
+    blob_out->clear();
+    blob_offsets->assign((size_t)n_conv, 0);
+    bool magic_ok = true;
+    for (int ph = 0; ph < n_phases; ++ph) {
+        MPhase &P = plan->phases[(size_t)ph];
+        const Skel &S = skel[(size_t)ph];
+        P.kind = S.kind;
+        P.item_base = item_base;
+        P.full_sync = 1;
+        if (S.kind == PH_FILL) {
+            const PlanTensor &x = T[(size_t)S.tensor];
+            P.fill_off = plan->tensor_off[(size_t)S.tensor];
+            P.fill_bytes = x.bytes;
+            P.fill_word = (uint32_t)(x.halo & 0xFF) * 0x01010101u;
+            P.n_items = (int)((x.bytes + kFillItemBytes - 1) / kFillItemBytes);
+        } else if (S.kind == PH_INPUT) {
+            const PlanTensor &x = T[0];
+            if (x.W % 4 != 0) return false;
+            P.H = x.H; P.W = x.W; P.Wp = x.Wp; P.HsWp = x.HsWp; P.P_first = x.P_first;
+            P.n_items = (G * x.H * (x.W / 4) + 127) / 128;
+        } else if (S.kind == PH_TAIL) {
+            P.n_items = (G + 3) / 4;
+        } else {
+            const ConvNode &nd = nodes[(size_t)S.node];
+            const int cidx = (int)(std::find(conv_phase.begin(), conv_phase.end(), ph) - conv_phase.begin());
+            const isc_layer &L = layers[nd.layer].d;
+            const PlanTensor &in = T[(size_t)L.in_tensor];
+            P.H = in.H; P.W = in.W; P.Wp = in.Wp; P.HsWp = in.HsWp; P.P_first = in.P_first;
+            P.n_items = in.n_tiles;
+            P.magic_hswp = magic_for((uint32_t)in.HsWp, (uint32_t)in.npa + 256, &magic_ok);
+            P.magic_wp = magic_for((uint32_t)in.Wp, (uint32_t)in.HsWp + 256, &magic_ok);
+            P.scatter = L.stride == 2;
+            const PlanTensor &o0 = T[(size_t)nd.layer + 1];
+            P.o_Wp = o0.Wp; P.o_HsWp = o0.HsWp;
+            P.in_off = plan->tensor_off[(size_t)L.in_tensor];
+            P.n_ksteps = (uint32_t)ksteps[(size_t)cidx].size();
+            P.n_rows = (int)n_rows[(size_t)cidx];
+            P.n_chunks = n_rows[(size_t)cidx] / 16;
+            if (P.n_chunks > kMaxChunks) return false;
+            P.idesc = (2u << 4) | ((L.in_tensor == 0 ? 0u : 1u) << 7) | (1u << 10) |
+                      ((uint32_t)(P.n_rows >> 3) << 17) | ((128u >> 4) << 24);
+            P.w_off = w_off[(size_t)cidx];
+            P.w_bytes = w_bytes[(size_t)cidx];
+            P.const_off = P.w_off + P.n_ksteps * (uint32_t)P.n_rows * 32u;
+            P.conv_index = (uint32_t)cidx;
+            P.tile_base = tile_base;
+            tile_base += P.n_items;
+            for (uint32_t k = 0; k < P.n_ksteps; ++k) {
+                const auto &kp = ksteps[(size_t)cidx][k];
+                P.a_delta[k] = chunk_addr[(size_t)cidx][(size_t)kp.first];
+                P.a_lbo[k] = kp.second >= 0 ? (uint32_t)(chunk_addr[(size_t)cidx][(size_t)kp.second] -
+                                                         chunk_addr[(size_t)cidx][(size_t)kp.first]) : 16u;
+            }
+            // operand reads must stay inside the input region
+            for (uint32_t k = 0; k < P.n_ksteps; ++k) {
+                const long long lo_b = (long long)P.P_first * 16 + P.a_delta[k];
+                const long long hi_b = (long long)(P.P_first + 128 * P.n_items) * 16 + P.a_delta[k] + P.a_lbo[k];
+                if (lo_b < 0) return false;
+                const long long plane_of_hi = (hi_b - 1) / in.plane_bytes;
+                if (plane_of_hi >= in.planes) return false;
+            }
+            // dependencies: tile rule only when the operand was written, tile for tile, by the previous phase
+            const bool prev_is_conv = ph >= 1 && skel[(size_t)ph - 1].kind == PH_CONV;
+            bool tile_rule = prev_is_conv && in.producer_phase == ph - 1 && !in.scatter_produced;
+            if (L.res_tensor >= 0 && T[(size_t)L.res_tensor].producer_phase >= ph - 1) tile_rule = false;
+            if (tile_rule && plan->phases[(size_t)ph - 1].n_items != P.n_items) tile_rule = false;
+            P.full_sync = tile_rule ? 0 : 1;
+            // epilogue chunks and the weight blob
+            const int lay[2] = {nd.layer, nd.fused_layer};
+            std::vector<uint8_t> blob(P.w_bytes, 0);
+            int row0 = 0;
+            int chunk = 0;
+            for (int k2 = 0; k2 < 2; ++k2) {
+                if (lay[k2] < 0) continue;
+                const MegaLayerIn &ML = layers[lay[k2]];
+                const isc_layer &LL = ML.d;
+                PlanTensor &o = T[(size_t)lay[k2] + 1];
+                o.scatter_produced = LL.stride == 2;
+                plan->tensors[(size_t)lay[k2] + 1].scatter_produced = o.scatter_produced;
+                const int taps = LL.kh * LL.kw;
+                if (LL.res_tensor >= 0) {
+                    P.res_mult = LL.res_mult;
+                    P.res_n = 31 - LL.res_shift;
+                    P.res_R = (1ll << (P.res_n - 1)) - (long long)LL.zp_res * LL.res_mult;
+                }
+                for (int pl = 0; pl < o.planes; ++pl, ++chunk) {
+                    P.out_off[chunk] = plan->tensor_off[(size_t)lay[k2] + 1] + (uint32_t)pl * o.plane_bytes;
+                    P.res_off[chunk] = LL.res_tensor >= 0
+                        ? plan->tensor_off[(size_t)LL.res_tensor] + (uint32_t)pl * T[(size_t)LL.res_tensor].plane_bytes : 0u;
+                    const int lo = LL.relu ? std::max(-128, LL.zp_out) : -128;
+                    P.lo[chunk] = lo;
+                    P.halo[chunk] = (uint32_t)(LL.zp_out & 0xFF) * 0x01010101u;
+                    P.flags[chunk] = (lo > -128 ? 1u : 0u) | (LL.res_tensor >= 0 ? 2u : 0u);
+                }
+                for (int oc = 0; oc < LL.cout; ++oc) {
+                    const int n = row0 + oc;
+                    long long wsum = 0;
+                    for (int q = 0; q < LL.cin * taps; ++q) wsum += ML.w[(size_t)oc * LL.cin * taps + q];
+                    for (uint32_t k = 0; k < P.n_ksteps; ++k) {
+                        const auto &kp = ksteps[(size_t)cidx][k];
+                        const int halves[2] = {kp.first, kp.second};
+                        for (int hf = 0; hf < 2; ++hf) {
+                            if (halves[hf] < 0) continue;
+                            const int tap = halves[hf] / in.planes, pl = halves[hf] % in.planes;
+                            int src_tap = tap;
+                            if (k2 == 1) {             // the 1x1 projection rides on the centre tap of the 3x3
+                                if (tap != (L.kh / 2) * L.kw + L.kw / 2) continue;
+                                src_tap = 0;
+                            }
+                            for (int b = 0; b < 16; ++b) {
+                                const int ci = pl * 16 + b;
+                                if (ci >= LL.cin) continue;
+                                const int8_t wv = ML.w[((size_t)oc * LL.cin + ci) * taps + src_tap];
+                                blob[(size_t)k * P.n_rows * 32 + (size_t)(n / 8) * 256 + (size_t)hf * 128 +
+                                     (size_t)(n % 8) * 16 + b] = (uint8_t)wv;
+                            }
+                        }
+                    }
+                    const int sh = ML.shift[oc];
+                    if (sh < 1 || sh > 20) return false;
+                    const int nn = 31 + sh;
+                    const long long biasf = (long long)ML.bias[oc] - (long long)LL.zp_in * wsum;
+                    const long long B = biasf * ML.mult[oc] + (1ll << (nn - 1)) + ((long long)LL.zp_out << nn);
+                    int32_t cst[4] = {ML.mult[oc], (int32_t)(uint32_t)(B & 0xFFFFFFFFll), (int32_t)(B >> 32), nn - 32};
+                    memcpy(&blob[(size_t)P.n_ksteps * P.n_rows * 32 + (size_t)n * 16], cst, 16);
+                }
+                row0 += LL.cout;
+            }
+            (*blob_offsets)[(size_t)cidx] = (uint32_t)blob_out->size();
+            blob_out->insert(blob_out->end(), blob.begin(), blob.end());
+            while (blob_out->size() % 128) blob_out->push_back(0);
+        }
+        item_base += P.n_items;
+    }
+    if (!magic_ok) return false;
+    plan->G = G;
+    plan->items_per_group = item_base;
+    plan->tiles_per_group = tile_base;
+    plan->smem_bytes = (high + 127u) & ~127u;
+    return true;
+}
+
+}  // namespace
+
+int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, MegaPlan **out)
 {
     *out = nullptr;
+    if (n_layers < 3 || n_classes > 128) return ISC_OK;
+    // structure: convolutions, then global average pool, then FC
+    const isc_layer &LP = layers[n_layers - 2].d, &LF = layers[n_layers - 1].d;
+    if (LP.op != ISC_GAVGPOOL || LF.op != ISC_FC) return ISC_OK;
+    if (LP.in_tensor != n_layers - 2 || LF.in_tensor != n_layers - 1) return ISC_OK;
+    if (LP.cin > 64 || LP.cin % 16 != 0 || LF.res_tensor >= 0) return ISC_OK;
+    for (int i = 0; i < n_layers - 2; ++i) {
+        const isc_layer &L = layers[i].d;
+        if (!conv_ok(L, i == 0)) return ISC_OK;
+        if ((i == 0) != (L.in_tensor == 0)) return ISC_OK;
+        if (L.res_tensor == 0) return ISC_OK;
+        // a consumer's zero-point must be the halo value its operand was written with
+        if (L.in_tensor > 0 && L.zp_in != layers[L.in_tensor - 1].d.zp_out) return ISC_OK;
+        if (L.res_tensor > 0 && L.res_tensor > n_layers - 2) return ISC_OK;
+    }
+    if (LP.zp_in != layers[n_layers - 3].d.zp_out) return ISC_OK;
+    for (int i = 1; i < n_layers - 2; ++i)
+        if (layers[i].d.in_tensor > n_layers - 2) return ISC_OK;
+
+    MegaPlan *plan = new MegaPlan();
+    std::vector<uint8_t> blob;
+    std::vector<uint32_t> blob_off;
+    bool ok = false;
+    for (int G = 4; G >= 1 && !ok; --G)
+        ok = plan_for_G(layers, n_layers, in_c, in_h, in_w, n_classes, G, plan, &blob, &blob_off);
+    if (!ok) { delete plan; return ISC_OK; }
+    plan->in_c = in_c; plan->in_h = in_h; plan->in_w = in_w; plan->n_classes = n_classes;
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        cudaGetLastError(); delete plan; return ISC_ERR_CUDA;
+    }
+    if (prop.major != 10 || (size_t)prop.sharedMemPerBlockOptin < plan->smem_bytes) { delete plan; return ISC_OK; }
+    plan->sm_count = prop.multiProcessorCount;
+
+    // FC parameters (bias folded with the pool output's zero-point)
+    const int C = LP.cin;
+    std::vector<int8_t> fcw((size_t)n_classes * 64, 0);
+    std::vector<FcConst> fcc((size_t)n_classes);
+    const MegaLayerIn &MF = layers[n_layers - 1];
+    for (int o = 0; o < n_classes; ++o) {
+        long long wsum = 0;
+        for (int c = 0; c < C; ++c) {
+            fcw[(size_t)o * 64 + c] = MF.w[(size_t)o * C + c];
+            wsum += MF.w[(size_t)o * C + c];
+        }
+        FcConst k{};
+        k.mult = MF.mult[o]; k.n = 31 + MF.shift[o]; k.zp_out = LF.zp_out;
+        k.lo = LF.relu ? std::max(-128, LF.zp_out) : -128;
+        k.bias = (int32_t)(MF.bias[o] - (long long)LF.zp_in * wsum);
+        fcc[(size_t)o] = k;
+    }
+    bool cuda_ok = true;
+    auto up = [&](void **dst, const void *src, size_t bytes) {
+        if (cudaMalloc(dst, std::max<size_t>(bytes, 16)) != cudaSuccess) { cuda_ok = false; *dst = nullptr; return; }
+        if (cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice) != cudaSuccess) cuda_ok = false;
+    };
+    up((void **)&plan->d_blob, blob.data(), blob.size());
+    for (size_t c = 0; c < plan->conv_phase.size(); ++c)
+        plan->phases[(size_t)plan->conv_phase[c]].w_gmem = (unsigned long long)(plan->d_blob + blob_off[c]);
+    up((void **)&plan->d_phases, plan->phases.data(), plan->phases.size() * sizeof(MPhase));
+    up((void **)&plan->d_conv_phase, plan->conv_phase.data(), plan->conv_phase.size() * sizeof(int));
+    up((void **)&plan->d_fc_w, fcw.data(), fcw.size());
+    up((void **)&plan->d_fc_c, fcc.data(), fcc.size() * sizeof(FcConst));
+    int32_t zero = 0;
+    up((void **)&plan->d_err, &zero, sizeof(zero));
+    if (cuda_ok && cudaMalloc((void **)&plan->d_dump, kSmemLimit) != cudaSuccess) cuda_ok = false;
+    if (!cuda_ok) { cudaGetLastError(); mega_free(plan); return ISC_ERR_NOMEM; }
+
+    MegaParams &b = plan->base;
+    memset(&b, 0, sizeof(b));
+    b.phases = plan->d_phases;
+    b.n_phases = (int)plan->phases.size();
+    b.n_conv = (int)plan->conv_phase.size();
+    b.items_per_group = plan->items_per_group;
+    b.tiles_per_group = plan->tiles_per_group;
+    b.G = plan->G;
+    b.in_c = in_c;
+    b.input_off = plan->tensor_off[0];
+    b.input_halo = layers[0].d.zp_in;
+    const PlanTensor &last = plan->tensors[(size_t)n_layers - 2];
+    b.tail_in_off = plan->tensor_off[(size_t)n_layers - 2];
+    b.tail_plane_bytes = last.plane_bytes;
+    b.tail_C = last.C; b.tail_H = last.H; b.tail_W = last.W; b.tail_Wp = last.Wp; b.tail_HsWp = last.HsWp;
+    b.pool_mult = layers[n_layers - 2].mult[0];
+    b.pool_n = 31 + layers[n_layers - 2].shift[0];
+    b.pool_zp_in = LP.zp_in; b.pool_zp_out = LP.zp_out;
+    b.pool_lo = LP.relu ? std::max(-128, LP.zp_out) : -128;
+    b.fc_w = plan->d_fc_w; b.fc_c = plan->d_fc_c;
+    b.n_classes = n_classes;
+    b.err = plan->d_err;
+    b.stop_phase = 1 << 30;
+    *out = plan;
     return ISC_OK;
 }
-void mega_free(MegaPlan *p) { delete p; }
-int mega_run(MegaPlan *, const uint8_t *, const NoiseStream &, int64_t, int, int32_t *, int8_t *, cudaStream_t,
-             int64_t *)
+
+void mega_free(MegaPlan *p)
 {
-    return ISC_ERR_UNSUPPORTED;
+    if (!p) return;
+    cudaFree(p->d_phases); cudaFree(p->d_conv_phase); cudaFree(p->d_blob); cudaFree(p->d_fc_w);
+    cudaFree(p->d_fc_c); cudaFree(p->d_err); cudaFree(p->d_dump);
+    delete p;
 }
-int mega_check(MegaPlan *) { return ISC_OK; }
+
+static int mega_launch(MegaPlan *p, MegaParams &q, cudaStream_t st)
+{
+    if (!p->attr_set) {
+        if (cudaFuncSetAttribute(k_mega, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p->smem_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            return ISC_ERR_CUDA;
+        }
+        p->attr_set = true;
+    }
+    const int grid = std::max(1, std::min(q.n_groups, p->sm_count));
+    k_mega<<<grid, kThreads, p->smem_bytes, st>>>(q, p->d_conv_phase);
+    return cudaGetLastError() == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
+}
+
+int mega_run(MegaPlan *p, const uint8_t *d_x, const NoiseStream &ns, int64_t n, int batch_hint, int32_t *d_counts,
+             int8_t *d_logits, cudaStream_t st, int64_t *launches)
+{
+    const int64_t per_launch = batch_hint > 0 ? batch_hint : (1ll << 30);
+    for (int64_t done = 0; done < n; done += per_launch) {
+        const int64_t m = std::min(per_launch, n - done);
+        MegaParams q = p->base;
+        q.x = d_x;
+        q.ns = ns;
+        q.ns.first_sample = ns.first_sample + done;
+        q.n_samples = (int32_t)m;
+        q.n_groups = (int32_t)((m + p->G - 1) / p->G);
+        q.counts = d_counts;
+        q.logits = d_logits ? d_logits + (size_t)done * p->n_classes : nullptr;
+        int rc = mega_launch(p, q, st);
+        *launches += 1;
+        if (rc) return rc;
+    }
+    return ISC_OK;
+}
+
+int mega_check(MegaPlan *p)
+{
+    int32_t e = 0;
+    if (cudaMemcpy(&e, p->d_err, sizeof(e), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return ISC_ERR_CUDA; }
+    if (e != 0) {
+        cudaMemset(p->d_err, 0, sizeof(e));
+        return ISC_ERR_TIMEOUT;
+    }
+    return ISC_OK;
+}
+
+int mega_tensor_phase(MegaPlan *p, int tensor)
+{
+    if (tensor < 0 || tensor >= (int)p->tensors.size() || p->tensors[(size_t)tensor].buffer < 0) return -1;
+    return p->tensors[(size_t)tensor].producer_phase;
+}
+
+// Runs one group (samples ns.first_sample ..) up to the phase that produces `tensor` and returns that
+// tensor of the first sample as [C][H][W] int32.
+int mega_debug_tensor(MegaPlan *p, const uint8_t *d_x, const NoiseStream &ns, int tensor, int32_t *out_chw,
+                      int32_t *d_counts_scratch, cudaStream_t st, int64_t *launches)
+{
+    const int ph = mega_tensor_phase(p, tensor);
+    if (ph < 0) return ISC_ERR_UNSUPPORTED;
+    const PlanTensor &t = p->tensors[(size_t)tensor];
+    MegaParams q = p->base;
+    q.x = d_x; q.ns = ns; q.n_samples = 1; q.n_groups = 1; q.counts = d_counts_scratch; q.logits = nullptr;
+    q.stop_phase = ph;
+    q.dump_off = p->tensor_off[(size_t)tensor]; q.dump_bytes = t.bytes; q.dump = p->d_dump;
+    int rc = mega_launch(p, q, st);
+    *launches += 1;
+    if (rc) return rc;
+    std::vector<uint8_t> h(t.bytes);
+    if (cudaMemcpyAsync(h.data(), p->d_dump, t.bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ISC_ERR_CUDA; }
+    if ((rc = mega_check(p))) return rc;
+    for (int c = 0; c < t.C; ++c)
+        for (int y = 0; y < t.H; ++y)
+            for (int x = 0; x < t.W; ++x) {
+                const size_t pos = (size_t)(y + 1) * t.Wp + x + 1;
+                const uint8_t b = h[(size_t)(c / 16) * t.plane_bytes + pos * 16 + (c % 16)];
+                out_chw[((size_t)c * t.H + y) * t.W + x] = tensor == 0 ? (int32_t)b : (int32_t)(int8_t)b;
+            }
+    return ISC_OK;
+}
 
 }  // namespace isc

@@ -28,6 +28,12 @@ void mega_free(MegaPlan *p);
 int mega_run(MegaPlan *p, const uint8_t *d_x, const NoiseStream &ns, int64_t n, int batch_hint,
              int32_t *d_counts, int8_t *d_logits, cudaStream_t st, int64_t *launches);
 
+// Debug read-back: runs one group up to the phase producing model tensor `tensor` and returns that
+// tensor of sample ns.first_sample as [C][H][W] int32 (host).  ISC_ERR_UNSUPPORTED if the tensor is
+// not held by this engine.
+int mega_debug_tensor(MegaPlan *p, const uint8_t *d_x, const NoiseStream &ns, int tensor, int32_t *out_chw,
+                      int32_t *d_counts_scratch, cudaStream_t st, int64_t *launches);
+
 // After the stream has been synchronised: ISC_OK, or ISC_ERR_TIMEOUT if a bounded wait expired.
 int mega_check(MegaPlan *p);
 

@@ -12,7 +12,7 @@ import paper_2108_09413_b200 as isc
 pytestmark = pytest.mark.gpu
 SEED = wl.NOISE_SEED
 ALPHA = 0.001
-ENGINES = {"layerwise": 1, "auto": 0}
+ENGINES = {"layerwise": 1, "resident": 2}
 
 
 def _pair(model):
@@ -78,16 +78,32 @@ def test_resnet20_logits_and_prefix_counts(sigma):
     _logit_parity(model, xs[1], 1, 0, 0, 100, sigma)              # the selection phase
 
 
-def test_resnet20_every_tensor():
+@pytest.mark.parametrize("engine", ["layerwise", "resident"])
+def test_resnet20_every_tensor(engine):
     model = wl.resnet20()
     gm, om = _pair(model)
+    gm.set_option("engine", ENGINES[engine])
     x = wl.images(1, seed=77)[0]
     sizes = _tensor_sizes(om)
     a0 = oracle.noisy_input(x, SEED, 4, 1, 9, 0.5)
-    for k in range(1, om.n_layers + 1):
-        _, exp = oracle.forward(om, a0, dump_tensor=k)
+    last = om.n_layers if engine == "layerwise" else om.n_layers - 2     # resident: conv tensors only
+    first = 1 if engine == "layerwise" else 0
+    for k in range(first, last + 1):
+        exp = a0.ravel().astype(np.int32) if k == 0 else oracle.forward(om, a0, dump_tensor=k)[1]
         got = gm.debug_tensor(x, SEED, 4, 1, 9, 0.5, k, sizes[k])
-        np.testing.assert_array_equal(got, exp, err_msg=f"tensor {k}")
+        bad = np.nonzero(got != exp)[0]
+        assert bad.size == 0, f"{engine}: tensor {k}: {bad.size} of {exp.size} differ, first at {bad[:8]}"
+
+
+def test_resident_engine_is_used_for_cifar_resnets():
+    for model in (wl.tiny_cnn(), wl.resnet20(), wl.resnet110()):
+        gm = isc.Model(model)
+        assert gm.get_info("has_resident_engine") == 1, model["name"]
+        gm.sample_counts(wl.images(1)[0], SEED, 0, 1, 0, 8, 0.25)
+        assert gm.get_info("engine") == 2
+        gm.close()
+    gm = isc.Model(wl.resnet50())
+    assert gm.get_info("has_resident_engine") == 0
 
 
 def test_resnet110_logits_and_prefix_counts():
