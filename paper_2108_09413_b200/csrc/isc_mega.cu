@@ -33,13 +33,15 @@ namespace isc {
 
 namespace {
 
-constexpr int kEpiWarps = 16;
+constexpr int kIssuers = 4;                 // warps 0..3: one thread of each issues the MMAs of every 4th tile
+constexpr int kEpiWarps = 16;               // warps 4..19: epilogue, four warpgroups
 constexpr int kWarpGroups = kEpiWarps / 4;
-constexpr int kThreads = 32 * (1 + kEpiWarps);
+constexpr int kThreads = 32 * (kIssuers + kEpiWarps);
 constexpr int kTmemSlots = 8;
 constexpr int kSlotCols = 64;
 constexpr int kMaxKsteps = 20;
 constexpr int kMaxChunks = 4;
+constexpr int kMaxPhases = 136;
 constexpr int kCtrlBytes = 4096;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kFillItemBytes = 8192;
@@ -49,33 +51,64 @@ enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
 enum { ERR_NONE = 0, ERR_WAIT_ITEMS = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_EMPTY = 3, ERR_WAIT_FULL = 4,
        ERR_WAIT_DRAIN = 5 };
 
+// Where and how one group of 16 output channels of a CONV phase is written.
+struct alignas(16) ChunkInfo {
+    uint32_t out_off, res_off;      // byte offsets of the destination / residual channel plane
+    int32_t lo;                     // lower clamp when flags bit 0 is set
+    uint32_t halo;                  // zero-point byte replicated: value of positions outside the image
+    uint32_t flags, pad0, pad1, pad2;   // bit0 explicit lower clamp, bit1 residual add
+};
+
+// Host-side description of a phase (the planner's working form).
 struct alignas(16) MPhase {
     int32_t kind, n_items, item_base, full_sync;
-    // geometry of the positions this phase walks (CONV: its input tensor)
-    int32_t H, W, Wp, HsWp;
+    int32_t H, W, Wp, HsWp;                 // geometry of the positions this phase walks (CONV: its input tensor)
     int32_t P_first, scatter, o_Wp, o_HsWp;
     uint32_t magic_hswp, magic_wp, pad0, pad1;
-    // FILL
     uint32_t fill_off, fill_bytes, fill_word, pad2;
-    // CONV
     uint32_t in_off, n_ksteps, idesc, n_chunks;
     uint32_t w_off, w_bytes, const_off, conv_index;
-    unsigned long long w_gmem;
     int32_t tile_base, n_rows;
     int32_t res_mult, res_n;
     long long res_R;
     int32_t a_delta[kMaxKsteps];
     uint32_t a_lbo[kMaxKsteps];
-    uint32_t out_off[kMaxChunks], res_off[kMaxChunks];
-    int32_t lo[kMaxChunks];
-    uint32_t halo[kMaxChunks], flags[kMaxChunks];   // flags: bit0 explicit lower clamp, bit1 residual
+    ChunkInfo chunk[kMaxChunks];
 };
+
+// ---- what the kernel reads -------------------------------------------------------------------
+
+// One entry per phase, copied to shared memory when the kernel starts.
+//   CONV: a = shared-memory offset of the phase's blob (ConvDesc, weights, per-channel constants)
+//   FILL: a = offset of the region, b = bytes | halo byte << 24
+struct alignas(16) PhaseEntry { uint32_t kind_sync, n_items, a, b; };     // kind | full_sync << 8
+
+// Where the blob of convolution c comes from (global) and goes to (shared).
+struct alignas(16) ConvSrc { unsigned long long gmem; uint32_t bytes_phase, smem_off; };   // bytes | phase << 24
+
+// Head of every blob: everything the issuing threads and the epilogue need to know about the phase.
+struct alignas(16) ConvDesc {
+    uint32_t in_off, n_ksteps, idesc, n_rows;
+    int32_t P_first, HsWp, Wp, scatter;
+    int32_t o_Wp, o_HsWp;
+    uint32_t magic_hswp, magic_wp;
+    uint32_t n_chunks, weights_rel, consts_rel, mode;   // mode: epilogue variant, same for all chunks
+    int32_t res_mult, res_n;
+    long long res_R;
+    ChunkInfo chunk[kMaxChunks];
+    int32_t a_delta[kMaxKsteps];
+    uint32_t a_lbo[kMaxKsteps];
+    uint32_t pad1[4];
+};
+static_assert(sizeof(ConvDesc) % 128 == 0, "blob sections must stay 128-byte aligned");
 
 struct FcConst { int32_t mult, n, zp_out, lo, bias, pad0, pad1, pad2; };
 
 struct MegaParams {
-    const MPhase *phases;
+    const PhaseEntry *ptab;
+    const ConvSrc *conv_src;
     int32_t n_phases, n_conv, items_per_group, tiles_per_group;
+    int32_t in_H, in_W, in_Wp, in_HsWp;
     int32_t G, n_groups, n_samples, in_c;
     const uint8_t *x;                 // clean image, CHW
     NoiseStream ns;
@@ -101,8 +134,9 @@ struct Ctrl {
     unsigned long long full[kTmemSlots], empty[kTmemSlots], wbar[3], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
-    uint32_t prog[kEpiWarps];
+    alignas(16) uint32_t prog[kEpiWarps];          // items completed by each epilogue warp (monotonic)
     int32_t hist[128];
+    PhaseEntry ptab[kMaxPhases];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -129,11 +163,22 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// non-blocking test of a barrier phase
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile("{\n\t.reg .pred p;\n\t"
                  "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// test that parks the thread in hardware for a bounded time when the phase is not complete
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
                  "selp.u32 %0, 1, 0, p;\n\t}"
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
@@ -151,15 +196,28 @@ __device__ __forceinline__ void st_release(uint32_t addr, uint32_t v)
 {
     asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
-__device__ __forceinline__ uint32_t ld_acquire(uint32_t addr)
+__device__ __forceinline__ uint4 ld_acquire_v4(uint32_t addr)
 {
-    uint32_t v;
-    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    uint4 v;
+    asm volatile("ld.acquire.cta.shared::cta.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
-__device__ __forceinline__ void named_bar(int id, int n)
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
 {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -172,11 +230,18 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+// D = A * B (first K-step of a tile) and D += A * B
+__device__ __forceinline__ void mma_i8_first(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc)
 {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
                  "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void mma_i8_acc(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
@@ -193,7 +258,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16])
 
 // K-major, no-swizzle shared-memory operand descriptor: rows of 16 bytes, 8 rows contiguous,
 // `sbo` bytes between 8-row groups, `lbo` bytes between the two 16-byte halves of K = 32.
-__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
+__host__ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
 {
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
            ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
@@ -205,6 +270,33 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3)
     uint32_t hi, d;
     asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi) : "r"(v3), "r"(v2));
     asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v1), "r"(v0), "r"(hi));
+    return d;
+}
+// a * b + c as one 32x32+64 multiply-add
+__device__ __forceinline__ long long mad_wide(int a, int b, long long c)
+{
+    long long d;
+    asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ int hi32(long long v)
+{
+    int lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+    return hi;
+}
+__device__ __forceinline__ int lo32(long long v)
+{
+    int lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+    return lo;
+}
+// byte K of w, sign-extended (one byte-permute with sign replication)
+template <int K>
+__device__ __forceinline__ int sbyte(uint32_t w)
+{
+    int d;
+    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(w), "n"(((8 | K) << 12) | ((8 | K) << 8) | ((8 | K) << 4) | K));
     return d;
 }
 
@@ -242,14 +334,30 @@ struct Waiter {
         ctrl->abort_flag = 1;
         atomicCAS(err, 0, code | (blockIdx.x << 8));
     }
+    // Wait for a phase of an mbarrier.  Each attempt parks the thread in hardware for a bounded time,
+    // so a waiting warp does not compete for issue slots.
+    __device__ __forceinline__ bool barrier(uint32_t bar, uint32_t parity, int code)
+    {
+        if (mbar_test(bar, parity)) return true;
+        const unsigned long long t0 = globaltimer();
+        for (int spin = 0;; ++spin) {
+            if (mbar_try(bar, parity)) return true;
+            if ((spin & 7) == 7) {
+                if (aborted()) return false;
+                if (globaltimer() - t0 > kWaitLimitNs) { fail(code); return false; }
+            }
+        }
+    }
+    // Wait on a predicate over shared-memory progress counters, backing off between polls.
     template <typename Pred>
     __device__ __forceinline__ bool until(Pred pred, int code)
     {
         if (pred()) return true;
         const unsigned long long t0 = globaltimer();
         for (int spin = 0;; ++spin) {
+            __nanosleep(64);
             if (pred()) return true;
-            if ((spin & 63) == 63) {
+            if ((spin & 31) == 31) {
                 if (aborted()) return false;
                 if (globaltimer() - t0 > kWaitLimitNs) { fail(code); return false; }
             }
@@ -263,89 +371,182 @@ __device__ __forceinline__ uint32_t items_of_wg_below(uint32_t end, int wg)
     return end > (uint32_t)wg ? (end - wg + kWarpGroups - 1) / kWarpGroups : 0u;
 }
 
+// all four warps of warpgroup wg have completed at least `need` items (one 16-byte acquire read)
+__device__ __forceinline__ bool wg_reached(uint32_t prog_addr, int wg, uint32_t need)
+{
+    const uint4 v = ld_acquire_v4(prog_addr + 16 * wg);
+    return v.x >= need && v.y >= need && v.z >= need && v.w >= need;
+}
+
 // every item with global index < end has been completed by all four warps of its warpgroup
 __device__ __forceinline__ bool all_items_below_done(uint32_t prog_addr, uint32_t end)
 {
-    for (int wg = 0; wg < kWarpGroups; ++wg) {
-        const uint32_t need = items_of_wg_below(end, wg);
-        for (int k = 0; k < 4; ++k)
-            if (ld_acquire(prog_addr + 4 * (wg * 4 + k)) < need) return false;
-    }
-    return true;
+    bool ok = true;
+#pragma unroll
+    for (int wg = 0; wg < kWarpGroups; ++wg) ok = ok && wg_reached(prog_addr, wg, items_of_wg_below(end, wg));
+    return ok;
 }
 
 __device__ __forceinline__ bool item_done(uint32_t prog_addr, uint32_t g)
 {
-    const int wg = g % kWarpGroups;
-    const uint32_t need = g / kWarpGroups + 1;
-    for (int k = 0; k < 4; ++k)
-        if (ld_acquire(prog_addr + 4 * (wg * 4 + k)) < need) return false;
+    return wg_reached(prog_addr, g % kWarpGroups, g / kWarpGroups + 1);
+}
+
+// ------------------------------------------------------------------ issuing threads
+
+__device__ __forceinline__ void issue_weights(const ConvSrc *src, uint32_t sbase, uint32_t wbar_addr)
+{
+    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
+    const void *gmem = reinterpret_cast<const void *>(((unsigned long long)v.y << 32) | v.x);
+    const uint32_t bytes = v.z & 0xFFFFFFu;
+    mbar_expect_tx(wbar_addr, bytes);
+    bulk_g2s(sbase + v.w, gmem, bytes, wbar_addr);
+}
+
+struct IssueArgs {
+    uint32_t desc, a0, w0, n_rows, idesc, dep_base, ts0;
+    int n_items, dep_n, issuer;
+};
+
+// Issue loop of one CONV phase with KS K-steps per tile, for the tiles of one issuing thread.  The low
+// words of the operand descriptors stay in registers; the next tile of this thread is kIssuers * 128
+// positions further, i.e. kIssuers * 128 units of the A descriptors' start-address field.  The body is
+// kept as short as possible: the issuing thread is alone in its warp, so every instruction it executes
+// is on the critical path of the tensor pipe.
+template <int KS>
+__device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem, const IssueArgs &ia)
+{
+    const uint32_t prog = smem_u32(ctrl->prog);
+    const int t_first = (int)((ia.issuer + kIssuers - (ia.ts0 % kIssuers)) % kIssuers);
+    uint32_t alo[KS], blo[KS];
+    const uint32_t ahi = (uint32_t)(make_desc(0, 0, 128) >> 32), bhi = (uint32_t)(make_desc(0, 128, 256) >> 32);
+#pragma unroll
+    for (int k = 0; k < KS; ++k) {
+        const uint32_t delta = lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * k);
+        const uint32_t lbo = lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * k);
+        alo[k] = (uint32_t)make_desc(ia.a0 + delta, lbo, 128) + 128u * (uint32_t)t_first;
+        blo[k] = (uint32_t)make_desc(ia.w0 + (uint32_t)k * ia.n_rows * 32u, 128, 256);
+    }
+    const uint32_t full0 = smem_u32(&ctrl->full[0]), empty0 = smem_u32(&ctrl->empty[0]);
+    const uint32_t idesc = ia.idesc;
+    const int n_items = ia.n_items, dep_n = ia.dep_n;
+    const uint32_t dep_base = ia.dep_base;
+    int known = 0;                           // tiles 0..known-1 of the producing phase are complete
+    uint32_t ts = ia.ts0 + (uint32_t)t_first;
+    for (int t = t_first; t < n_items; t += kIssuers, ts += kIssuers) {
+        const int need = min(t + 2, dep_n);
+        while (known < need) {
+            const uint32_t g = dep_base + known;
+            if (!w.until([&] { return item_done(prog, g); }, ERR_WAIT_ITEMS)) return false;
+            ++known;
+        }
+        const uint32_t slot = ts % kTmemSlots, use = ts / kTmemSlots;
+        if (use > 0 && !w.barrier(empty0 + 8 * slot, (use - 1) & 1, ERR_WAIT_EMPTY)) return false;
+        tc_fence_after();
+        const uint32_t d = tmem + slot * kSlotCols;
+#pragma unroll
+        for (int k = 0; k < KS; ++k) {
+            const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)alo[k];
+            const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)blo[k];
+            if (k == 0) mma_i8_first(d, ad, bd, idesc);
+            else mma_i8_acc(d, ad, bd, idesc);
+            alo[k] += 128u * kIssuers;
+        }
+        mma_commit(full0 + 8 * slot);
+    }
     return true;
 }
 
-// ------------------------------------------------------------------ roles
-
-__device__ void issue_weights(const MPhase &ph, uint32_t sbase, uint32_t wbar_addr)
+// Same for an arbitrary number of K-steps (descriptors rebuilt from shared memory for every tile).
+__device__ __noinline__ bool issue_phase_any(Waiter w, Ctrl *ctrl, uint32_t tmem, const IssueArgs &ia, uint32_t n_ksteps)
 {
-    mbar_expect_tx(wbar_addr, ph.w_bytes);
-    bulk_g2s(sbase + ph.w_off, reinterpret_cast<const void *>(ph.w_gmem), ph.w_bytes, wbar_addr);
+    const uint32_t prog = smem_u32(ctrl->prog);
+    const int t_first = (int)((ia.issuer + kIssuers - (ia.ts0 % kIssuers)) % kIssuers);
+    int known = 0;
+    uint32_t ts = ia.ts0 + (uint32_t)t_first;
+    for (int t = t_first; t < ia.n_items; t += kIssuers, ts += kIssuers) {
+        const int need = min(t + 2, ia.dep_n);
+        while (known < need) {
+            const uint32_t g = ia.dep_base + known;
+            if (!w.until([&] { return item_done(prog, g); }, ERR_WAIT_ITEMS)) return false;
+            ++known;
+        }
+        const uint32_t slot = ts % kTmemSlots, use = ts / kTmemSlots;
+        if (use > 0 && !w.barrier(smem_u32(&ctrl->empty[slot]), (use - 1) & 1, ERR_WAIT_EMPTY)) return false;
+        tc_fence_after();
+        const uint32_t d = tmem + slot * kSlotCols;
+        for (uint32_t k = 0; k < n_ksteps; ++k) {
+            const uint32_t delta = lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * k);
+            const uint32_t lbo = lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * k);
+            const uint64_t ad = make_desc(ia.a0 + delta + 2048u * (uint32_t)t, lbo, 128);
+            const uint64_t bd = make_desc(ia.w0 + k * ia.n_rows * 32u, 128, 256);
+            if (k == 0) mma_i8_first(d, ad, bd, ia.idesc);
+            else mma_i8_acc(d, ad, bd, ia.idesc);
+        }
+        mma_commit(smem_u32(&ctrl->full[slot]));
+    }
+    return true;
 }
 
-// Warp 0, one thread: weight loads and all tensor-core work of one group.
-__device__ void mma_role(const MegaParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, int it, const int *conv_phase)
+// One thread of each of warps 0..3: the tensor-core work of one group (issuer 0 also loads the weights).
+__device__ __noinline__ void mma_role(const MegaParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, int it, int issuer)
 {
     Waiter w{ctrl, p.err};
     const uint32_t prog = smem_u32(ctrl->prog);
+    const uint32_t ptab = smem_u32(ctrl->ptab);
     const uint32_t item_off = (uint32_t)it * p.items_per_group;
     const uint32_t tile_off = (uint32_t)it * p.tiles_per_group;
     const uint32_t conv_off = (uint32_t)it * p.n_conv;
-    {   // weights of this group's first convolution (everything before the group barrier is complete)
-        const uint32_t cg = conv_off;
-        if (!w.aborted()) issue_weights(p.phases[conv_phase[0]], sbase, smem_u32(&ctrl->wbar[cg % 3]));
-    }
-    for (int ph = 0; ph < p.n_phases && ph <= p.stop_phase; ++ph) {
-        const MPhase &P = p.phases[ph];
-        if (P.kind != PH_CONV) continue;
-        // the phase before last must be complete (shared-memory reuse rule); with full_sync the last one too
-        const uint32_t end = item_off + (P.full_sync ? (uint32_t)P.item_base
-                                                     : (ph >= 1 ? (uint32_t)p.phases[ph - 1].item_base : 0u));
-        if (!w.until([&] { return all_items_below_done(prog, end); }, ERR_WAIT_ITEMS)) return;
-        const uint32_t cg = conv_off + P.conv_index;
-        if ((int)P.conv_index + 1 < p.n_conv && conv_phase[P.conv_index + 1] <= p.stop_phase)
-            issue_weights(p.phases[conv_phase[P.conv_index + 1]], sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
-        {
-            const uint32_t bar = smem_u32(&ctrl->wbar[cg % 3]), par = (cg / 3) & 1;
-            if (!w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_WEIGHTS)) return;
+    const int n_phases = p.n_phases, stop_phase = p.stop_phase, n_conv = p.n_conv;
+    const ConvSrc *conv_src = p.conv_src;
+    // weights of this group's first convolution (everything before the group barrier is complete)
+    if (issuer == 0 && !w.aborted()) issue_weights(conv_src, sbase, smem_u32(&ctrl->wbar[conv_off % 3]));
+    int item_base = 0, prev_item_base = 0, prev_n_items = 0;
+    uint32_t conv_index = 0, tile_base = 0;
+    for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
+        const uint4 e = ld_shared_v4(ptab + 16 * ph);
+        const int kind = e.x & 0xFF, full_sync = (e.x >> 8) & 1, n_items = (int)e.y;
+        if (kind == PH_CONV) {
+            // the phase before last must be complete (shared-memory reuse rule); with full_sync the last one too
+            const uint32_t end = item_off + (uint32_t)(full_sync ? item_base : prev_item_base);
+            if (!w.until([&] { return all_items_below_done(prog, end); }, ERR_WAIT_ITEMS)) return;
+            const uint32_t cg = conv_off + conv_index;
+            if (issuer == 0 && (int)conv_index + 1 < n_conv) {
+                const ConvSrc *nxt = conv_src + conv_index + 1;
+                if ((int)(__ldg(&nxt->bytes_phase) >> 24) <= stop_phase)
+                    issue_weights(nxt, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
+            }
+            if (!w.barrier(smem_u32(&ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS)) return;
+            // phase parameters from the head of the blob
+            const uint32_t desc = sbase + e.z;
+            const uint4 h = ld_shared_v4(desc);                        // in_off, n_ksteps, idesc, n_rows
+            IssueArgs ia;
+            ia.desc = desc;
+            ia.a0 = sbase + h.x + lds32(desc + offsetof(ConvDesc, P_first)) * 16u;
+            ia.w0 = desc + lds32(desc + offsetof(ConvDesc, weights_rel));
+            ia.n_rows = h.w; ia.idesc = h.z; ia.n_items = n_items;
+            ia.dep_base = item_off + (uint32_t)prev_item_base;
+            ia.dep_n = full_sync ? 0 : prev_n_items;
+            ia.ts0 = tile_off + tile_base;
+            ia.issuer = issuer;
+            bool ok;
+            switch (h.y) {
+            case 1: ok = issue_phase<1>(w, ctrl, tmem, ia); break;
+            case 5: ok = issue_phase<5>(w, ctrl, tmem, ia); break;
+            case 9: ok = issue_phase<9>(w, ctrl, tmem, ia); break;
+            case 18: ok = issue_phase<18>(w, ctrl, tmem, ia); break;
+            default: ok = issue_phase_any(w, ctrl, tmem, ia, h.y); break;
+            }
+            if (!ok) return;
+            conv_index += 1;
+            tile_base += (uint32_t)n_items;
         }
-        const uint32_t dep_base = item_off + (ph >= 1 ? (uint32_t)p.phases[ph - 1].item_base : 0u);
-        const int dep_n = ph >= 1 ? p.phases[ph - 1].n_items : 0;
-        const uint32_t n_rows = (uint32_t)P.n_rows;
-        for (int t = 0; t < P.n_items; ++t) {
-            if (!P.full_sync && dep_n > 0) {
-                const int t0 = max(t - 1, 0), t1 = min(t + 1, dep_n - 1);
-                if (!w.until([&] {
-                        for (int q = t0; q <= t1; ++q)
-                            if (!item_done(prog, dep_base + q)) return false;
-                        return true;
-                    }, ERR_WAIT_ITEMS)) return;
-            }
-            const uint32_t ts = tile_off + P.tile_base + t, slot = ts % kTmemSlots, use = ts / kTmemSlots;
-            if (use > 0) {
-                const uint32_t bar = smem_u32(&ctrl->empty[slot]), par = (use - 1) & 1;
-                if (!w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_EMPTY)) return;
-            }
-            tc_fence_after();
-            const uint32_t d = tmem + slot * kSlotCols;
-            const uint32_t abase = sbase + P.in_off + (uint32_t)(P.P_first + 128 * t) * 16u;
-            for (uint32_t k = 0; k < P.n_ksteps; ++k) {
-                const uint64_t ad = make_desc(abase + (uint32_t)P.a_delta[k], P.a_lbo[k], 128);
-                const uint64_t bd = make_desc(sbase + P.w_off + k * n_rows * 32u, 128, 256);
-                mma_i8(d, ad, bd, P.idesc, k > 0 ? 1u : 0u);
-            }
-            mma_commit(smem_u32(&ctrl->full[slot]));
-        }
+        prev_item_base = item_base; prev_n_items = n_items;
+        item_base += n_items;
     }
 }
+
+// ------------------------------------------------------------------ epilogue warps
 
 struct EpiCtx {
     Ctrl *ctrl;
@@ -362,128 +563,191 @@ __device__ __forceinline__ void finish_item(EpiCtx &c)
     if (c.lane == 0) st_release(smem_u32(&c.ctrl->prog[c.warp_e]), c.done);
 }
 
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
+__device__ void fill_item(uint32_t fill_off, uint32_t bytes_halo, const EpiCtx &c, int i)
 {
-    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-
-__device__ void fill_item(const MPhase &P, EpiCtx &c, int i)
-{
+    const uint32_t fill_bytes = bytes_halo & 0xFFFFFFu, word = (bytes_halo >> 24) * 0x01010101u;
     const uint32_t begin = (uint32_t)i * kFillItemBytes;
-    const uint32_t end = min(begin + kFillItemBytes, P.fill_bytes);
-    const uint4 v = make_uint4(P.fill_word, P.fill_word, P.fill_word, P.fill_word);
-    for (uint32_t o = begin + c.tid_wg * 16; o < end; o += 128 * 16) st_shared_v4(c.sbase + P.fill_off + o, v);
+    const uint32_t end = min(begin + kFillItemBytes, fill_bytes);
+    const uint4 v = make_uint4(word, word, word, word);
+    for (uint32_t o = begin + c.tid_wg * 16; o < end; o += 128 * 16) st_shared_v4(c.sbase + fill_off + o, v);
 }
 
 // INPUT: one thread = four horizontally adjacent pixels of one sample, all input channels.
-__device__ void input_item(const MegaParams &p, const MPhase &P, EpiCtx &c, int i, int grp)
+__device__ void input_item(const MegaParams &p, const EpiCtx &c, int i, int grp)
 {
-    const int wq = P.W >> 2;
-    const int quads = p.G * P.H * wq;
+    const int H = p.in_H, W = p.in_W, Wp = p.in_Wp, HsWp = p.in_HsWp, G = p.G, in_c = p.in_c;
+    const int wq = W >> 2;
+    const int quads = G * H * wq;
     const int qi = i * 128 + c.tid_wg;
     if (qi >= quads) return;
-    const int s = qi / (P.H * wq);
-    const int rem = qi - s * (P.H * wq);
+    const int s = qi / (H * wq);
+    const int rem = qi - s * (H * wq);
     const int y = rem / wq, x4 = rem - y * wq;
-    const long long j = p.ns.first_sample + (long long)grp * p.G + s;
+    const long long j = p.ns.first_sample + (long long)grp * G + s;
+    const uint32_t *__restrict__ cum = p.ns.cum;
+    const int T = p.ns.T;
+    const uint32_t key0 = p.ns.key0, key1 = p.ns.key1, ctr2 = p.ns.ctr2;
+    const uint32_t ctr3 = p.ns.ctr3_fixed | (uint32_t)(((j >> 32) & 0xFF) << 8);
+    const uint8_t *__restrict__ x = p.x;
     uint32_t px[4] = {0, 0, 0, 0};
-    for (int ch = 0; ch < p.in_c; ++ch) {
-        const uint32_t e = (uint32_t)((ch * P.H + y) * P.W + 4 * x4);
-        const uint4 ctr = make_uint4(e >> 2, (uint32_t)(j & 0xFFFFFFFFll), p.ns.ctr2,
-                                     p.ns.ctr3_fixed | (uint32_t)(((j >> 32) & 0xFF) << 8));
-        const uint4 r = philox4x32_10(ctr, p.ns.key0, p.ns.key1);
+    for (int ch = 0; ch < in_c; ++ch) {
+        const uint32_t e = (uint32_t)((ch * H + y) * W + 4 * x4);
+        const uint4 r = philox4x32_10(make_uint4(e >> 2, (uint32_t)(j & 0xFFFFFFFFll), ctr2, ctr3), key0, key1);
         const uint32_t u[4] = {r.x, r.y, r.z, r.w};
-        const uint32_t clean = __ldg(reinterpret_cast<const uint32_t *>(p.x + e));
+        const uint32_t clean = __ldg(reinterpret_cast<const uint32_t *>(x + e));
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            int v = (int)((clean >> (8 * k)) & 0xFF) + noise_level(u[k], p.ns.cum, p.ns.T);
+            int v = (int)((clean >> (8 * k)) & 0xFF) + noise_level(u[k], cum, T);
             v = min(255, max(0, v));
             px[k] |= (uint32_t)v << (8 * ch);
         }
     }
-    const uint32_t pos = (uint32_t)(s * P.HsWp + (y + 1) * P.Wp + 4 * x4 + 1);
+    const uint32_t pos = (uint32_t)(s * HsWp + (y + 1) * Wp + 4 * x4 + 1);
+    const uint32_t dst = c.sbase + p.input_off;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) st_shared_v4(c.sbase + p.input_off + (pos + k) * 16u, make_uint4(px[k], 0, 0, 0));
+    for (int k = 0; k < 4; ++k) st_shared_v4(dst + (pos + k) * 16u, make_uint4(px[k], 0, 0, 0));
+}
+
+// What the epilogue warps keep in registers for the whole of a CONV phase.
+struct ConvRegs {
+    int P_first, HsWp, Wp, scatter, o_Wp, o_HsWp, G;
+    uint32_t magic_hswp, magic_wp, const_addr, n_chunks, chunks;
+    int res_mult, res_sh;          // res_sh = n - 32 when n >= 32, else n
+    long long res_R;
+    uint32_t mode;                 // bit0 explicit lower clamp, bit1 residual, bit2 residual shift >= 32
+};
+
+// desc = shared-memory address of the phase's ConvDesc
+__device__ __forceinline__ ConvRegs load_conv_regs(uint32_t desc, int G)
+{
+    ConvRegs r;
+    const uint4 g0 = ld_shared_v4(desc + offsetof(ConvDesc, P_first));      // P_first, HsWp, Wp, scatter
+    const uint4 g1 = ld_shared_v4(desc + offsetof(ConvDesc, o_Wp));         // o_Wp, o_HsWp, magic_hswp, magic_wp
+    const uint4 g2 = ld_shared_v4(desc + offsetof(ConvDesc, n_chunks));     // n_chunks, weights_rel, consts_rel, mode
+    const uint4 g3 = ld_shared_v4(desc + offsetof(ConvDesc, res_mult));     // res_mult, res_n, res_R
+    r.P_first = (int)g0.x; r.HsWp = (int)g0.y; r.Wp = (int)g0.z; r.scatter = (int)g0.w;
+    r.o_Wp = (int)g1.x; r.o_HsWp = (int)g1.y; r.magic_hswp = g1.z; r.magic_wp = g1.w;
+    r.n_chunks = g2.x; r.const_addr = desc + g2.z; r.mode = g2.w;
+    r.res_mult = (int)g3.x; r.res_sh = (int)g3.y >= 32 ? (int)g3.y - 32 : (int)g3.y;
+    r.res_R = (long long)(((unsigned long long)g3.w << 32) | g3.z);
+    r.G = G;
+    r.chunks = desc + offsetof(ConvDesc, chunk);
+    return r;
+}
+
+// One output channel:
+//   main    : y = floor((acc * mult + B) / 2^(32 + s)); B holds the folded bias, the rounding half and the
+//             output zero-point, so this is rs(acc' * mult, 31 + shift) + zp_out exactly
+//   residual: y += floor((r * res_mult + R) / 2^n), R = 2^(n-1) - zp_res * res_mult   (kResHigh: n >= 32)
+template <bool kRes, bool kResHigh, bool kLo, int K>
+__device__ __forceinline__ int requant1(int acc, uint32_t caddr, uint32_t rword, const ConvRegs &R, int lo)
+{
+    const uint4 cs = ld_shared_v4(caddr);            // mult, B low, B high, s = shift - 1
+    const long long B = (long long)(((unsigned long long)cs.z << 32) | cs.y);
+    int y = hi32(mad_wide(acc, (int)cs.x, B)) >> (int)cs.w;
+    if (kRes) {
+        const long long t = mad_wide(sbyte<K>(rword), R.res_mult, R.res_R);
+        y += kResHigh ? (hi32(t) >> R.res_sh) : (int)__funnelshift_r((uint32_t)lo32(t), (uint32_t)hi32(t), R.res_sh);
+    }
+    if (kLo) y = max(y, lo);
+    return y;
+}
+
+template <bool kRes, bool kResHigh, bool kLo>
+__device__ __forceinline__ uint32_t requant4(int a0, int a1, int a2, int a3, uint32_t caddr, uint32_t rword,
+                                             const ConvRegs &R, int lo)
+{
+    const int y0 = requant1<kRes, kResHigh, kLo, 0>(a0, caddr, rword, R, lo);
+    const int y1 = requant1<kRes, kResHigh, kLo, 1>(a1, caddr + 16, rword, R, lo);
+    const int y2 = requant1<kRes, kResHigh, kLo, 2>(a2, caddr + 32, rword, R, lo);
+    const int y3 = requant1<kRes, kResHigh, kLo, 3>(a3, caddr + 48, rword, R, lo);
+    return pack4_sat(y0, y1, y2, y3);
 }
 
 // CONV epilogue of one tile: thread = one position (tensor-memory lane), 16 channels at a time.
-__device__ void conv_tile(const MPhase &P, EpiCtx &c, int t, uint32_t slot, int G)
+template <bool kRes, bool kResHigh, bool kLo>
+__device__ __forceinline__ void conv_tile(const ConvRegs &R, const EpiCtx &c, int t, uint32_t slot)
 {
-    const uint32_t pos = (uint32_t)(P.P_first + 128 * t + c.quarter * 32 + c.lane);
+    const uint32_t pos = (uint32_t)(R.P_first + 128 * t + c.quarter * 32 + c.lane);
     // position -> (sample, row, column) of the padded image
-    const uint32_t s = __umulhi(pos, P.magic_hswp);
-    const uint32_t rem = pos - s * (uint32_t)P.HsWp;
-    const uint32_t y1 = __umulhi(rem, P.magic_wp);
-    const uint32_t x1 = rem - y1 * (uint32_t)P.Wp;
-    const bool interior = (int)s < G && y1 >= 1 && x1 >= 1;
+    const uint32_t s = __umulhi(pos, R.magic_hswp);
+    const uint32_t rem = pos - s * (uint32_t)R.HsWp;
+    const uint32_t y1 = __umulhi(rem, R.magic_wp);
+    const uint32_t x1 = rem - y1 * (uint32_t)R.Wp;
+    const bool interior = (int)s < R.G && y1 >= 1 && x1 >= 1;
     bool store = true;
     uint32_t opos = pos;
-    if (P.scatter) {
+    if (R.scatter) {
         const uint32_t y = y1 - 1, x = x1 - 1;
         store = interior && !(y & 1) && !(x & 1);
-        opos = s * (uint32_t)P.o_HsWp + ((y >> 1) + 1) * (uint32_t)P.o_Wp + (x >> 1) + 1;
+        opos = s * (uint32_t)R.o_HsWp + ((y >> 1) + 1) * (uint32_t)R.o_Wp + (x >> 1) + 1;
     }
+    const bool keep = R.scatter || interior;          // otherwise the position holds the halo value
     const uint32_t taddr = c.tmem + ((uint32_t)(c.quarter * 32) << 16) + slot * kSlotCols;
-    const long long res_R = P.res_R;
-    const int res_mult = P.res_mult, res_n = P.res_n;
-    for (uint32_t ch = 0; ch < P.n_chunks; ++ch) {
+    for (uint32_t ch = 0; ch < R.n_chunks; ++ch) {
         int acc[16];
         tmem_ld16(taddr + ch * 16, acc);
-        if (ch + 1 == P.n_chunks) {           // accumulator slot may be overwritten from here on
+        if (ch + 1 == R.n_chunks) {           // accumulator slot may be overwritten from here on
             tc_fence_before();
             __syncwarp();
             if (c.lane == 0) mbar_arrive(smem_u32(&c.ctrl->empty[slot]));
         }
-        const uint32_t flags = P.flags[ch];
-        uint32_t rw[4] = {0, 0, 0, 0};
-        if (flags & 2) {
-            const uint4 rv = ld_shared_v4(c.sbase + P.res_off[ch] + pos * 16u);
-            rw[0] = rv.x; rw[1] = rv.y; rw[2] = rv.z; rw[3] = rv.w;
-        }
-        const uint32_t cbase = c.sbase + P.const_off + ch * 256u;
-        const int lo = P.lo[ch];
-        int q[16];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            const uint4 cs = ld_shared_v4(cbase + k * 16);   // mult, B low, B high, shift - 1
-            const long long B = (long long)(((unsigned long long)cs.z << 32) | cs.y);
-            const long long v = (long long)acc[k] * (long long)(int)cs.x + B;
-            int y = (int)(v >> 32) >> (int)cs.w;
-            if (flags & 2) {
-                const int r = (int)(int8_t)((rw[k >> 2] >> (8 * (k & 3))) & 0xFF);
-                y += (int)(((long long)r * res_mult + res_R) >> res_n);
-            }
-            if (flags & 1) y = max(y, lo);
-            q[k] = y;
-        }
-        uint4 o = make_uint4(pack4_sat(q[0], q[1], q[2], q[3]), pack4_sat(q[4], q[5], q[6], q[7]),
-                             pack4_sat(q[8], q[9], q[10], q[11]), pack4_sat(q[12], q[13], q[14], q[15]));
-        if (!P.scatter && !interior) o = make_uint4(P.halo[ch], P.halo[ch], P.halo[ch], P.halo[ch]);
-        if (store) st_shared_v4(c.sbase + P.out_off[ch] + opos * 16u, o);
+        const uint4 ci = ld_shared_v4(R.chunks + ch * (uint32_t)sizeof(ChunkInfo));   // out_off, res_off, lo, halo
+        const uint32_t cbase = R.const_addr + ch * 256u;
+        uint4 rv = make_uint4(0, 0, 0, 0);
+        if (kRes) rv = ld_shared_v4(c.sbase + ci.y + pos * 16u);
+        const int lo = (int)ci.z;
+        uint4 o;
+        o.x = requant4<kRes, kResHigh, kLo>(acc[0], acc[1], acc[2], acc[3], cbase, rv.x, R, lo);
+        o.y = requant4<kRes, kResHigh, kLo>(acc[4], acc[5], acc[6], acc[7], cbase + 64, rv.y, R, lo);
+        o.z = requant4<kRes, kResHigh, kLo>(acc[8], acc[9], acc[10], acc[11], cbase + 128, rv.z, R, lo);
+        o.w = requant4<kRes, kResHigh, kLo>(acc[12], acc[13], acc[14], acc[15], cbase + 192, rv.w, R, lo);
+        if (!keep) o = make_uint4(ci.w, ci.w, ci.w, ci.w);
+        if (store) st_shared_v4(c.sbase + ci.x + opos * 16u, o);
     }
 }
 
-// TAIL: global average pool, FC, argmax and vote; one warp carries one sample.
-__device__ void tail_sample(const MegaParams &p, EpiCtx &c, int s, int grp)
+// All tiles of one CONV phase that belong to this warpgroup.
+template <bool kRes, bool kResHigh, bool kLo>
+__device__ __noinline__ void conv_phase_tiles(Waiter w, EpiCtx &c_io, const ConvRegs &R_in, int i0, int n_items, uint32_t ts0)
 {
-    const int hw = p.tail_H * p.tail_W;
+    // private copies: values reached through references would be re-read after every barrier or fence
+    EpiCtx c = c_io;
+    const ConvRegs R = R_in;
+    const uint32_t full0 = smem_u32(&c.ctrl->full[0]);
+    bool ok = true;
+    for (int i = i0; i < n_items; i += kWarpGroups) {
+        if (ok) {
+            const uint32_t ts = ts0 + (uint32_t)i, slot = ts % kTmemSlots;
+            ok = w.barrier(full0 + 8 * slot, (ts / kTmemSlots) & 1, ERR_WAIT_FULL);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                conv_tile<kRes, kResHigh, kLo>(R, c, i, slot);
+            }
+        }
+        finish_item(c);
+    }
+    c_io.done = c.done;
+}
+
+// TAIL: global average pool, FC, argmax and vote; one warp carries one sample.
+__device__ void tail_sample(const MegaParams &p, const EpiCtx &c, int s, bool counted_slot, int grp)
+{
+    const int tail_H = p.tail_H, tail_W = p.tail_W, tail_C = p.tail_C, tail_Wp = p.tail_Wp, tail_HsWp = p.tail_HsWp;
+    const int n_classes = p.n_classes;
+    const int hw = tail_H * tail_W;
     int pooled[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int ch = c.lane + 32 * h;
         int q = 0;
-        if (ch < p.tail_C) {
+        if (ch < tail_C) {
             const uint32_t base = c.sbase + p.tail_in_off + (uint32_t)(ch >> 4) * p.tail_plane_bytes + (ch & 15);
             int sum = 0;
             for (int i = 0; i < hw; ++i) {
-                const int y = i / p.tail_W, x = i - y * p.tail_W;
-                const uint32_t pos = (uint32_t)(s * p.tail_HsWp + (y + 1) * p.tail_Wp + x + 1);
+                const int y = i / tail_W, x = i - y * tail_W;
+                const uint32_t pos = (uint32_t)(s * tail_HsWp + (y + 1) * tail_Wp + x + 1);
                 int v;
                 asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(base + pos * 16u));
                 sum += v - p.pool_zp_in;
@@ -497,15 +761,15 @@ __device__ void tail_sample(const MegaParams &p, EpiCtx &c, int s, int grp)
         pooled[h] = q;
     }
     const long long sample = (long long)grp * p.G + s;          // index within this launch
-    const bool counted = s < p.G && sample < p.n_samples;
+    const bool counted = counted_slot && sample < p.n_samples;
     int best_v = -1000, best_o = 0x7fffffff;
-    for (int o0 = 0; o0 < p.n_classes; o0 += 32) {
+    for (int o0 = 0; o0 < n_classes; o0 += 32) {
         const int o = o0 + c.lane;
-        const bool live = o < p.n_classes;
+        const bool live = o < n_classes;
         const FcConst k = p.fc_c[live ? o : 0];
         const int8_t *wrow = p.fc_w + (size_t)(live ? o : 0) * 64;
         int acc = k.bias;
-        for (int cc = 0; cc < p.tail_C; ++cc) {
+        for (int cc = 0; cc < tail_C; ++cc) {
             const int a = __shfl_sync(0xffffffffu, pooled[cc >> 5], cc & 31);
             acc += a * (int)__ldg(wrow + cc);
         }
@@ -515,7 +779,7 @@ __device__ void tail_sample(const MegaParams &p, EpiCtx &c, int s, int grp)
         v = v > 127 ? 127 : v;
         if (live) {
             if ((int)v > best_v) { best_v = (int)v; best_o = o; }
-            if (counted && p.logits) p.logits[sample * p.n_classes + o] = (int8_t)v;
+            if (counted && p.logits) p.logits[sample * n_classes + o] = (int8_t)v;
         }
     }
     // lowest index among the maxima
@@ -528,45 +792,57 @@ __device__ void tail_sample(const MegaParams &p, EpiCtx &c, int s, int grp)
 }
 
 // Epilogue warps: all non-tensor-core work of one group, item by item.
-__device__ void epi_role(const MegaParams &p, EpiCtx &c, int it, int grp)
+__device__ __noinline__ void epi_role(const MegaParams &p, EpiCtx &c, int it, int grp)
 {
     Waiter w{c.ctrl, p.err};
     const uint32_t prog = smem_u32(c.ctrl->prog);
+    const uint32_t ptab = smem_u32(c.ctrl->ptab);
     const uint32_t item_off = (uint32_t)it * p.items_per_group;
     const uint32_t tile_off = (uint32_t)it * p.tiles_per_group;
     const uint32_t conv_off = (uint32_t)it * p.n_conv;
-    for (int ph = 0; ph < p.n_phases && ph <= p.stop_phase; ++ph) {
-        const MPhase &P = p.phases[ph];
-        const uint32_t first = item_off + P.item_base;
+    const int n_phases = p.n_phases, stop_phase = p.stop_phase, G = p.G;
+    uint32_t item_base = 0, conv_index = 0, tile_base = 0;
+    for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
+        const uint4 e = ld_shared_v4(ptab + 16 * ph);
+        const int kind = e.x & 0xFF, n_items = (int)e.y;
+        const uint32_t first = item_off + item_base;
+        const uint32_t my_conv = conv_index, my_tile_base = tile_base;
+        item_base += (uint32_t)n_items;
+        if (kind == PH_CONV) { conv_index += 1; tile_base += (uint32_t)n_items; }
         const int i0 = (c.wg + kWarpGroups - (int)(first % kWarpGroups)) % kWarpGroups;
-        if (i0 >= P.n_items) continue;
+        if (i0 >= n_items) continue;
         bool ok;
-        if (P.kind != PH_CONV) {
-            ok = w.until([&] { return all_items_below_done(prog, first); }, ERR_WAIT_ITEMS);
-        } else {
-            const uint32_t cg = conv_off + P.conv_index;
-            const uint32_t bar = smem_u32(&c.ctrl->wbar[cg % 3]), par = (cg / 3) & 1;
-            ok = w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_WEIGHTS);
-        }
-        ok = __all_sync(0xffffffffu, ok);
-        for (int i = i0; i < P.n_items; i += kWarpGroups) {
+        if (kind == PH_CONV) {
+            const uint32_t cg = conv_off + my_conv;
+            ok = w.barrier(smem_u32(&c.ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS);
+            ok = __all_sync(0xffffffffu, ok);
             if (ok) {
-                if (P.kind == PH_FILL) {
-                    fill_item(P, c, i);
-                } else if (P.kind == PH_INPUT) {
-                    input_item(p, P, c, i, grp);
-                } else if (P.kind == PH_CONV) {
-                    const uint32_t ts = tile_off + P.tile_base + i, slot = ts % kTmemSlots;
-                    const uint32_t bar = smem_u32(&c.ctrl->full[slot]), par = (ts / kTmemSlots) & 1;
-                    ok = w.until([&] { return mbar_test(bar, par); }, ERR_WAIT_FULL);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (ok) {
-                        tc_fence_after();
-                        conv_tile(P, c, i, slot, p.G);
-                    }
+                const ConvRegs R = load_conv_regs(c.sbase + e.z, G);
+                const uint32_t ts0 = tile_off + my_tile_base;
+                switch (R.mode & 7u) {
+                case 0: conv_phase_tiles<false, false, false>(w, c, R, i0, n_items, ts0); break;
+                case 1: conv_phase_tiles<false, false, true>(w, c, R, i0, n_items, ts0); break;
+                case 2: conv_phase_tiles<true, false, false>(w, c, R, i0, n_items, ts0); break;
+                case 3: conv_phase_tiles<true, false, true>(w, c, R, i0, n_items, ts0); break;
+                case 6: conv_phase_tiles<true, true, false>(w, c, R, i0, n_items, ts0); break;
+                default: conv_phase_tiles<true, true, true>(w, c, R, i0, n_items, ts0); break;
+                }
+            } else {
+                for (int i = i0; i < n_items; i += kWarpGroups) finish_item(c);
+            }
+            continue;
+        }
+        ok = w.until([&] { return all_items_below_done(prog, first); }, ERR_WAIT_ITEMS);
+        ok = __all_sync(0xffffffffu, ok);
+        for (int i = i0; i < n_items; i += kWarpGroups) {
+            if (ok) {
+                if (kind == PH_FILL) {
+                    fill_item(e.z, e.w, c, i);
+                } else if (kind == PH_INPUT) {
+                    input_item(p, c, i, grp);
                 } else {
                     const int s = i * 4 + (c.warp_e & 3);
-                    tail_sample(p, c, min(s, p.G - 1), grp + (s >= p.G ? (1 << 28) : 0));
+                    tail_sample(p, c, min(s, G - 1), s < G, grp);
                 }
             }
             finish_item(c);
@@ -574,7 +850,7 @@ __device__ void epi_role(const MegaParams &p, EpiCtx &c, int it, int grp)
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 1) k_mega(const MegaParams p, const int *__restrict__ conv_phase)
+__global__ void __launch_bounds__(kThreads, 1) k_mega(const __grid_constant__ MegaParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
@@ -586,11 +862,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_mega(const MegaParams p, const 
             mbar_init(smem_u32(&ctrl->empty[s]), 4);
         }
         for (int s = 0; s < 3; ++s) mbar_init(smem_u32(&ctrl->wbar[s]), 1);
-        mbar_init(smem_u32(&ctrl->drain), 1);
+        mbar_init(smem_u32(&ctrl->drain), kIssuers);
         ctrl->abort_flag = 0;
     }
     for (int i = threadIdx.x; i < 128; i += blockDim.x) ctrl->hist[i] = 0;
     if (threadIdx.x < kEpiWarps) ctrl->prog[threadIdx.x] = 0;
+    for (int i = threadIdx.x; i < p.n_phases; i += blockDim.x) ctrl->ptab[i] = p.ptab[i];
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), 512);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -601,13 +878,13 @@ __global__ void __launch_bounds__(kThreads, 1) k_mega(const MegaParams p, const 
 
     EpiCtx c;
     c.ctrl = ctrl; c.sbase = sbase; c.tmem = tmem;
-    c.warp_e = warp - 1; c.wg = (warp - 1) >> 2; c.quarter = warp & 3; c.lane = lane;
-    c.tid_wg = ((warp - 1) & 3) * 32 + lane; c.done = 0;
+    c.warp_e = warp - kIssuers; c.wg = (warp - kIssuers) >> 2; c.quarter = warp & 3; c.lane = lane;
+    c.tid_wg = ((warp - kIssuers) & 3) * 32 + lane; c.done = 0;
 
     int it = 0;
     for (int grp = blockIdx.x; grp < p.n_groups; grp += gridDim.x, ++it) {
-        if (warp == 0) {
-            if (lane == 0) mma_role(p, ctrl, sbase, tmem, it, conv_phase);
+        if (warp < kIssuers) {
+            if (lane == 0) mma_role(p, ctrl, sbase, tmem, it, warp);
             __syncwarp();
         } else {
             epi_role(p, c, it, grp);
@@ -621,11 +898,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_mega(const MegaParams p, const 
         for (uint32_t o = threadIdx.x * 16u; o < p.dump_bytes; o += blockDim.x * 16u)
             *reinterpret_cast<uint4 *>(p.dump + o) = ld_shared_v4(sbase + p.dump_off + o);
     // no tensor-core work may be in flight when tensor memory is released
-    if (warp == 0 && lane == 0) {
+    if (warp < kIssuers && lane == 0) {
         Waiter w{ctrl, p.err};
         mma_commit(smem_u32(&ctrl->drain));
-        const uint32_t bar = smem_u32(&ctrl->drain);
-        w.until([&] { return mbar_test(bar, 0); }, ERR_WAIT_DRAIN);
+        w.barrier(smem_u32(&ctrl->drain), 0, ERR_WAIT_DRAIN);
     }
     tc_fence_before();
     __syncthreads();
@@ -687,8 +963,8 @@ struct MegaPlan {
     uint32_t smem_bytes = 0;
     MegaParams base;                      // fields that do not change between launches
     // device copies
-    MPhase *d_phases = nullptr;
-    int *d_conv_phase = nullptr;
+    PhaseEntry *d_ptab = nullptr;
+    ConvSrc *d_conv_src = nullptr;
     uint8_t *d_blob = nullptr;
     int8_t *d_fc_w = nullptr;
     FcConst *d_fc_c = nullptr;
@@ -836,6 +1112,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
     layer_phase[(size_t)n_layers - 2] = tail_phase;
     layer_phase[(size_t)n_layers - 1] = tail_phase;
     const int n_phases = (int)skel.size();
+    if (n_phases > kMaxPhases || n_phases >= 256) return false;
     // ---- lifetimes
     for (int t = 0; t <= n_conv_layers; ++t) {
         PlanTensor &x = T[(size_t)t];
@@ -880,7 +1157,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         ksteps[(size_t)cidx] = ks;
         chunk_addr[(size_t)cidx] = addr;
         n_rows[(size_t)cidx] = (uint32_t)(L.cout + (nd.fused_layer >= 0 ? layers[nd.fused_layer].d.cout : 0));
-        w_bytes[(size_t)cidx] = (uint32_t)ks.size() * n_rows[(size_t)cidx] * 32u + n_rows[(size_t)cidx] * 16u;
+        w_bytes[(size_t)cidx] = (uint32_t)sizeof(ConvDesc) + (uint32_t)ks.size() * n_rows[(size_t)cidx] * 32u + n_rows[(size_t)cidx] * 16u;
     }
     // ---- shared-memory placement in order of birth
     std::vector<AllocReq> reqs, placed;
@@ -944,7 +1221,9 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
                       ((uint32_t)(P.n_rows >> 3) << 17) | ((128u >> 4) << 24);
             P.w_off = w_off[(size_t)cidx];
             P.w_bytes = w_bytes[(size_t)cidx];
-            P.const_off = P.w_off + P.n_ksteps * (uint32_t)P.n_rows * 32u;
+            const uint32_t weights_rel = (uint32_t)sizeof(ConvDesc);
+            const uint32_t consts_rel = weights_rel + P.n_ksteps * (uint32_t)P.n_rows * 32u;
+            P.const_off = P.w_off + consts_rel;
             P.conv_index = (uint32_t)cidx;
             P.tile_base = tile_base;
             tile_base += P.n_items;
@@ -987,13 +1266,14 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
                     P.res_R = (1ll << (P.res_n - 1)) - (long long)LL.zp_res * LL.res_mult;
                 }
                 for (int pl = 0; pl < o.planes; ++pl, ++chunk) {
-                    P.out_off[chunk] = plan->tensor_off[(size_t)lay[k2] + 1] + (uint32_t)pl * o.plane_bytes;
-                    P.res_off[chunk] = LL.res_tensor >= 0
+                    ChunkInfo &ci = P.chunk[chunk];
+                    ci.out_off = plan->tensor_off[(size_t)lay[k2] + 1] + (uint32_t)pl * o.plane_bytes;
+                    ci.res_off = LL.res_tensor >= 0
                         ? plan->tensor_off[(size_t)LL.res_tensor] + (uint32_t)pl * T[(size_t)LL.res_tensor].plane_bytes : 0u;
                     const int lo = LL.relu ? std::max(-128, LL.zp_out) : -128;
-                    P.lo[chunk] = lo;
-                    P.halo[chunk] = (uint32_t)(LL.zp_out & 0xFF) * 0x01010101u;
-                    P.flags[chunk] = (lo > -128 ? 1u : 0u) | (LL.res_tensor >= 0 ? 2u : 0u);
+                    ci.lo = lo;
+                    ci.halo = (uint32_t)(LL.zp_out & 0xFF) * 0x01010101u;
+                    ci.flags = (lo > -128 ? 1u : 0u) | (LL.res_tensor >= 0 ? 2u : 0u);
                 }
                 for (int oc = 0; oc < LL.cout; ++oc) {
                     const int n = row0 + oc;
@@ -1014,7 +1294,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
                                 const int ci = pl * 16 + b;
                                 if (ci >= LL.cin) continue;
                                 const int8_t wv = ML.w[((size_t)oc * LL.cin + ci) * taps + src_tap];
-                                blob[(size_t)k * P.n_rows * 32 + (size_t)(n / 8) * 256 + (size_t)hf * 128 +
+                                blob[weights_rel + (size_t)k * P.n_rows * 32 + (size_t)(n / 8) * 256 + (size_t)hf * 128 +
                                      (size_t)(n % 8) * 16 + b] = (uint8_t)wv;
                             }
                         }
@@ -1025,10 +1305,23 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
                     const long long biasf = (long long)ML.bias[oc] - (long long)LL.zp_in * wsum;
                     const long long B = biasf * ML.mult[oc] + (1ll << (nn - 1)) + ((long long)LL.zp_out << nn);
                     int32_t cst[4] = {ML.mult[oc], (int32_t)(uint32_t)(B & 0xFFFFFFFFll), (int32_t)(B >> 32), nn - 32};
-                    memcpy(&blob[(size_t)P.n_ksteps * P.n_rows * 32 + (size_t)n * 16], cst, 16);
+                    memcpy(&blob[consts_rel + (size_t)n * 16], cst, 16);
                 }
                 row0 += LL.cout;
             }
+            for (uint32_t q = 1; q < P.n_chunks; ++q)
+                if (P.chunk[q].flags != P.chunk[0].flags) return false;      // one epilogue variant per phase
+            ConvDesc D;
+            memset(&D, 0, sizeof(D));
+            D.in_off = P.in_off; D.n_ksteps = P.n_ksteps; D.idesc = P.idesc; D.n_rows = (uint32_t)P.n_rows;
+            D.P_first = P.P_first; D.HsWp = P.HsWp; D.Wp = P.Wp; D.scatter = P.scatter;
+            D.o_Wp = P.o_Wp; D.o_HsWp = P.o_HsWp; D.magic_hswp = P.magic_hswp; D.magic_wp = P.magic_wp;
+            D.n_chunks = P.n_chunks; D.weights_rel = weights_rel; D.consts_rel = consts_rel;
+            D.mode = (P.chunk[0].flags & 3u) | ((P.chunk[0].flags & 2u) && P.res_n >= 32 ? 4u : 0u);
+            D.res_mult = P.res_mult; D.res_n = P.res_n; D.res_R = P.res_R;
+            for (int q = 0; q < kMaxChunks; ++q) D.chunk[q] = P.chunk[q];
+            for (int q = 0; q < kMaxKsteps; ++q) { D.a_delta[q] = P.a_delta[q]; D.a_lbo[q] = P.a_lbo[q]; }
+            memcpy(blob.data(), &D, sizeof(D));
             (*blob_offsets)[(size_t)cidx] = (uint32_t)blob_out->size();
             blob_out->insert(blob_out->end(), blob.begin(), blob.end());
             while (blob_out->size() % 128) blob_out->push_back(0);
@@ -1107,10 +1400,23 @@ int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
         if (cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice) != cudaSuccess) cuda_ok = false;
     };
     up((void **)&plan->d_blob, blob.data(), blob.size());
-    for (size_t c = 0; c < plan->conv_phase.size(); ++c)
-        plan->phases[(size_t)plan->conv_phase[c]].w_gmem = (unsigned long long)(plan->d_blob + blob_off[c]);
-    up((void **)&plan->d_phases, plan->phases.data(), plan->phases.size() * sizeof(MPhase));
-    up((void **)&plan->d_conv_phase, plan->conv_phase.data(), plan->conv_phase.size() * sizeof(int));
+    std::vector<PhaseEntry> ptab(plan->phases.size());
+    for (size_t i = 0; i < ptab.size(); ++i) {
+        const MPhase &P = plan->phases[i];
+        ptab[i].kind_sync = (uint32_t)P.kind | ((uint32_t)(P.full_sync ? 1 : 0) << 8);
+        ptab[i].n_items = (uint32_t)P.n_items;
+        ptab[i].a = P.kind == PH_CONV ? P.w_off : P.fill_off;
+        ptab[i].b = P.kind == PH_FILL ? (P.fill_bytes | ((P.fill_word & 0xFFu) << 24)) : 0u;
+    }
+    std::vector<ConvSrc> csrc(plan->conv_phase.size());
+    for (size_t c = 0; c < csrc.size(); ++c) {
+        const MPhase &P = plan->phases[(size_t)plan->conv_phase[c]];
+        csrc[c].gmem = (unsigned long long)(plan->d_blob + blob_off[c]);
+        csrc[c].bytes_phase = P.w_bytes | ((uint32_t)plan->conv_phase[c] << 24);
+        csrc[c].smem_off = P.w_off;
+    }
+    up((void **)&plan->d_ptab, ptab.data(), ptab.size() * sizeof(PhaseEntry));
+    up((void **)&plan->d_conv_src, csrc.data(), csrc.size() * sizeof(ConvSrc));
     up((void **)&plan->d_fc_w, fcw.data(), fcw.size());
     up((void **)&plan->d_fc_c, fcc.data(), fcc.size() * sizeof(FcConst));
     int32_t zero = 0;
@@ -1120,7 +1426,9 @@ int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
 
     MegaParams &b = plan->base;
     memset(&b, 0, sizeof(b));
-    b.phases = plan->d_phases;
+    b.ptab = plan->d_ptab;
+    b.conv_src = plan->d_conv_src;
+    b.in_H = plan->tensors[0].H; b.in_W = plan->tensors[0].W; b.in_Wp = plan->tensors[0].Wp; b.in_HsWp = plan->tensors[0].HsWp;
     b.n_phases = (int)plan->phases.size();
     b.n_conv = (int)plan->conv_phase.size();
     b.items_per_group = plan->items_per_group;
@@ -1148,7 +1456,7 @@ int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
 void mega_free(MegaPlan *p)
 {
     if (!p) return;
-    cudaFree(p->d_phases); cudaFree(p->d_conv_phase); cudaFree(p->d_blob); cudaFree(p->d_fc_w);
+    cudaFree(p->d_ptab); cudaFree(p->d_conv_src); cudaFree(p->d_blob); cudaFree(p->d_fc_w);
     cudaFree(p->d_fc_c); cudaFree(p->d_err); cudaFree(p->d_dump);
     delete p;
 }
@@ -1163,7 +1471,7 @@ static int mega_launch(MegaPlan *p, MegaParams &q, cudaStream_t st)
         p->attr_set = true;
     }
     const int grid = std::max(1, std::min(q.n_groups, p->sm_count));
-    k_mega<<<grid, kThreads, p->smem_bytes, st>>>(q, p->d_conv_phase);
+    k_mega<<<grid, kThreads, p->smem_bytes, st>>>(q);
     return cudaGetLastError() == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
 }
 
