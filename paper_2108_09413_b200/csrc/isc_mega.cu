@@ -34,11 +34,18 @@ namespace isc {
 namespace {
 
 constexpr int kIssuers = 4;                 // warps 0..3: one thread of each issues the MMAs of every 4th tile
-constexpr int kEpiWarps = 16;               // warps 4..19: epilogue, four warpgroups
+constexpr int kEpiWarps = 8;                // warps 4..11: epilogue, two warpgroups of "fat" threads (168 registers)
 constexpr int kWarpGroups = kEpiWarps / 4;
 constexpr int kThreads = 32 * (kIssuers + kEpiWarps);
-constexpr int kTmemSlots = 8;
-constexpr int kSlotCols = 64;
+// Four accumulator slots of 128 tensor-memory columns, one super-tile each: four tiles of up to 32 output
+// channels (narrow) or two tiles of up to 64 (wide).  Slot s is written by issuing thread s and read by
+// warpgroup s mod 2; super-tiles take the slots in turn over the whole run of the kernel.
+constexpr int kSlots = 4, kSlotCols = 128;
+constexpr int kSupNarrow = 4, kTileColsNarrow = 32;
+constexpr int kSupWide = 2, kTileColsWide = 64;
+constexpr int kMaxFusedCols = kTileColsWide;
+static_assert(kSlots == kIssuers, "one issuing thread per accumulator slot");
+static_assert(kWarpGroups == 2, "slot s belongs to warpgroup s mod 2");
 constexpr int kMaxKsteps = 20;
 constexpr int kMaxChunks = 4;
 constexpr int kMaxPhases = 136;
@@ -68,8 +75,9 @@ struct alignas(16) MPhase {
     uint32_t fill_off, fill_bytes, fill_word, pad2;
     uint32_t in_off, n_ksteps, idesc, n_chunks;
     uint32_t w_off, w_bytes, const_off, conv_index;
-    int32_t tile_base, n_rows;
+    int32_t n_tiles, n_rows;
     int32_t res_mult, res_n;
+    int32_t wide, pad3;                     // accumulator layout: 0 narrow slots, 1 wide slots
     long long res_R;
     int32_t a_delta[kMaxKsteps];
     uint32_t a_lbo[kMaxKsteps];
@@ -79,9 +87,10 @@ struct alignas(16) MPhase {
 // ---- what the kernel reads -------------------------------------------------------------------
 
 // One entry per phase, copied to shared memory when the kernel starts.
-//   CONV: a = shared-memory offset of the phase's blob (ConvDesc, weights, per-channel constants)
+//   CONV: n_items = super-tiles, a = shared-memory offset of the phase's blob (ConvDesc, weights,
+//         per-channel constants), b = tiles
 //   FILL: a = offset of the region, b = bytes | halo byte << 24
-struct alignas(16) PhaseEntry { uint32_t kind_sync, n_items, a, b; };     // kind | full_sync << 8
+struct alignas(16) PhaseEntry { uint32_t kind_sync, n_items, a, b; };     // kind | full_sync << 8 | chunks << 16 | wide << 24
 
 // Where the blob of convolution c comes from (global) and goes to (shared).
 struct alignas(16) ConvSrc { unsigned long long gmem; uint32_t bytes_phase, smem_off; };   // bytes | phase << 24
@@ -107,7 +116,7 @@ struct FcConst { int32_t mult, n, zp_out, lo, bias, pad0, pad1, pad2; };
 struct MegaParams {
     const PhaseEntry *ptab;
     const ConvSrc *conv_src;
-    int32_t n_phases, n_conv, items_per_group, tiles_per_group;
+    int32_t n_phases, n_conv, items_per_group, supers_per_group;
     int32_t in_H, in_W, in_Wp, in_HsWp;
     int32_t G, n_groups, n_samples, in_c;
     const uint8_t *x;                 // clean image, CHW
@@ -131,7 +140,7 @@ struct MegaParams {
 };
 
 struct Ctrl {
-    unsigned long long full[kTmemSlots], empty[kTmemSlots], wbar[3], drain;
+    unsigned long long full[kSlots], empty[kSlots], done[kSlots], wbar[3], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
     alignas(16) uint32_t prog[kEpiWarps];          // items completed by each epilogue warp (monotonic)
@@ -219,6 +228,10 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
+__device__ __forceinline__ void named_bar(int id, int n)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
@@ -231,22 +244,46 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 // D = A * B (first K-step of a tile) and D += A * B
+// True in exactly one lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred = 0;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\t@p mov.u32 %0, 1;\n\t}" : "+r"(pred));
+    return pred != 0;
+}
+// A value every lane of the warp holds, in a form the compiler knows to be the same in all lanes.
+__device__ __forceinline__ uint32_t warp_uniform(uint32_t v) { return __shfl_sync(0xffffffffu, v, 0); }
+
+// The tensor-core instructions below are issued by one elected lane of a converged warp; their operands are
+// computed by the whole warp from warp-uniform values.
 __device__ __forceinline__ void mma_i8_first(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc)
 {
+    if (!elect_one()) return;
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
                  "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
 }
 __device__ __forceinline__ void mma_i8_acc(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc)
 {
+    if (!elect_one()) return;
     asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
                  "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
+    if (!elect_one()) return;
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// asynchronous 16-column load of this thread's tensor-memory lane; the registers are valid after tmem_ld_wait()
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, int (&v)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -273,6 +310,18 @@ __device__ __forceinline__ uint32_t pack4_sat(int v0, int v1, int v2, int v3)
     return d;
 }
 // a * b + c as one 32x32+64 multiply-add
+// Per-channel requantisation constants as stored in the blob: the 64-bit addend, then multiplier and shift.
+// Loading the addend as one 64-bit register keeps it in an aligned register pair without any packing code.
+struct ChanConst { long long B; int mult, s; };
+__device__ __forceinline__ ChanConst ld_chan_const(uint32_t addr)
+{
+    long long b, ms;
+    asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(b), "=l"(ms) : "r"(addr));
+    ChanConst c;
+    c.B = b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(c.mult), "=r"(c.s) : "l"(ms));
+    return c;
+}
 __device__ __forceinline__ long long mad_wide(int a, int b, long long c)
 {
     long long d;
@@ -365,32 +414,20 @@ struct Waiter {
     }
 };
 
-// number of global item indices g < end with g % kWarpGroups == wg
-__device__ __forceinline__ uint32_t items_of_wg_below(uint32_t end, int wg)
-{
-    return end > (uint32_t)wg ? (end - wg + kWarpGroups - 1) / kWarpGroups : 0u;
-}
-
-// all four warps of warpgroup wg have completed at least `need` items (one 16-byte acquire read)
-__device__ __forceinline__ bool wg_reached(uint32_t prog_addr, int wg, uint32_t need)
-{
-    const uint4 v = ld_acquire_v4(prog_addr + 16 * wg);
-    return v.x >= need && v.y >= need && v.z >= need && v.w >= need;
-}
-
-// every item with global index < end has been completed by all four warps of its warpgroup
-__device__ __forceinline__ bool all_items_below_done(uint32_t prog_addr, uint32_t end)
+// Every epilogue warp publishes the index of the next item it has work in: all counters >= need means items
+// 0..need-1 are complete.  One 16-byte acquire read per warpgroup.
+__device__ __forceinline__ bool all_reached(uint32_t prog_addr, uint32_t need)
 {
     bool ok = true;
 #pragma unroll
-    for (int wg = 0; wg < kWarpGroups; ++wg) ok = ok && wg_reached(prog_addr, wg, items_of_wg_below(end, wg));
+    for (int g = 0; g < kWarpGroups; ++g) {
+        const uint4 a = ld_acquire_v4(prog_addr + 16 * g);
+        ok = ok && a.x >= need && a.y >= need && a.z >= need && a.w >= need;
+    }
     return ok;
 }
-
-__device__ __forceinline__ bool item_done(uint32_t prog_addr, uint32_t g)
-{
-    return wg_reached(prog_addr, g % kWarpGroups, g / kWarpGroups + 1);
-}
+__device__ __forceinline__ bool all_items_below_done(uint32_t prog_addr, uint32_t end) { return all_reached(prog_addr, end); }
+__device__ __forceinline__ bool item_done(uint32_t prog_addr, uint32_t g) { return all_reached(prog_addr, g + 1); }
 
 // ------------------------------------------------------------------ issuing threads
 
@@ -404,55 +441,87 @@ __device__ __forceinline__ void issue_weights(const ConvSrc *src, uint32_t sbase
 }
 
 struct IssueArgs {
-    uint32_t desc, a0, w0, n_rows, idesc, dep_base, ts0;
-    int n_items, dep_n, issuer;
+    uint32_t desc, a0, w0, n_rows, idesc, dep_base, dep_ss0, ss0;
+    int n_super, n_tiles, dep_n, issuer, wide;
 };
 
-// Issue loop of one CONV phase with KS K-steps per tile, for the tiles of one issuing thread.  The low
-// words of the operand descriptors stay in registers; the next tile of this thread is kIssuers * 128
-// positions further, i.e. kIssuers * 128 units of the A descriptors' start-address field.  The body is
-// kept as short as possible: the issuing thread is alone in its warp, so every instruction it executes
-// is on the critical path of the tensor pipe.
+// Wait until the epilogue warps have published `target` as their progress, i.e. until the producing phase's
+// super-tiles up to sequence number ss_last are stored.  The progress counters decide; the per-slot `done`
+// barriers only serve to park the warp in hardware until something relevant has happened, instead of polling.
+// (A barrier phase can alias when the slot is two uses ahead; then the wait merely returns early or runs into
+// its hardware time limit, and the counters are read again.)
+__device__ __forceinline__ bool dep_wait(Waiter w, Ctrl *ctrl, uint32_t prog, uint32_t target, uint32_t ss_last)
+{
+    if (all_reached(prog, target)) return true;
+    const uint32_t done0 = smem_u32(&ctrl->done[0]);
+    const unsigned long long t0 = globaltimer();
+    for (int spin = 0;; ++spin) {
+        mbar_try(done0 + 8 * (ss_last % kSlots), (ss_last / kSlots) & 1);
+        if (all_reached(prog, target)) return true;
+        if (ss_last > 0) mbar_try(done0 + 8 * ((ss_last - 1) % kSlots), ((ss_last - 1) / kSlots) & 1);   // other warpgroup
+        if (all_reached(prog, target)) return true;
+        __nanosleep(32);
+        if ((spin & 3) == 3) {
+            if (w.aborted()) return false;
+            if (globaltimer() - t0 > kWaitLimitNs) { w.fail(ERR_WAIT_ITEMS); return false; }
+        }
+    }
+}
+
+// Issue loop of one CONV phase with KS K-steps per tile.  Issuing thread k owns the super-tiles whose sequence
+// number is k mod 4 and accumulator slot k, so the four threads work on different super-tiles at different
+// times and the fixed cost per super-tile (dependency check, slot wait, commit) is paid once per two or four
+// tiles.  The low words of the operand descriptors stay in registers; tile t is 128 t positions, i.e. 128 t
+// units of the A descriptors' start-address field, further.  The body is kept as short as possible: the
+// issuing thread is alone in its warp, so every instruction it executes delays the tensor pipe.
 template <int KS>
 __device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem, const IssueArgs &ia)
 {
     const uint32_t prog = smem_u32(ctrl->prog);
-    const int t_first = (int)((ia.issuer + kIssuers - (ia.ts0 % kIssuers)) % kIssuers);
     uint32_t alo[KS], blo[KS];
     const uint32_t ahi = (uint32_t)(make_desc(0, 0, 128) >> 32), bhi = (uint32_t)(make_desc(0, 128, 256) >> 32);
 #pragma unroll
     for (int k = 0; k < KS; ++k) {
-        const uint32_t delta = lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * k);
-        const uint32_t lbo = lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * k);
-        alo[k] = (uint32_t)make_desc(ia.a0 + delta, lbo, 128) + 128u * (uint32_t)t_first;
+        const uint32_t delta = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * k));
+        const uint32_t lbo = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * k));
+        alo[k] = (uint32_t)make_desc(ia.a0 + delta, lbo, 128);
         blo[k] = (uint32_t)make_desc(ia.w0 + (uint32_t)k * ia.n_rows * 32u, 128, 256);
     }
-    const uint32_t full0 = smem_u32(&ctrl->full[0]), empty0 = smem_u32(&ctrl->empty[0]);
-    const uint32_t idesc = ia.idesc;
-    const int n_items = ia.n_items, dep_n = ia.dep_n;
-    const uint32_t dep_base = ia.dep_base;
-    int known = 0;                           // tiles 0..known-1 of the producing phase are complete
-    uint32_t ts = ia.ts0 + (uint32_t)t_first;
-    for (int t = t_first; t < n_items; t += kIssuers, ts += kIssuers) {
-        const int need = min(t + 2, dep_n);
-        while (known < need) {
-            const uint32_t g = dep_base + known;
-            if (!w.until([&] { return item_done(prog, g); }, ERR_WAIT_ITEMS)) return false;
-            ++known;
+    const int sup = ia.wide ? kSupWide : kSupNarrow;
+    const uint32_t tile_cols = ia.wide ? kTileColsWide : kTileColsNarrow;
+    const uint32_t slot = (uint32_t)ia.issuer;
+    const uint32_t full = smem_u32(&ctrl->full[slot]), empty = smem_u32(&ctrl->empty[slot]);
+    const uint32_t d0 = tmem + slot * kSlotCols;
+    const uint32_t idesc = ia.idesc, dep_base = ia.dep_base;
+    const int n_super = ia.n_super, n_tiles = ia.n_tiles, dep_n = ia.dep_n;
+    uint32_t done_upto = 0;                  // producing-phase items 0..done_upto-1 are known complete
+    int st = (int)(((uint32_t)ia.issuer + kIssuers - (ia.ss0 % kIssuers)) % kIssuers);
+    for (; st < n_super; st += kIssuers) {
+        const uint32_t use = (ia.ss0 + (uint32_t)st) / kSlots;      // how often this slot has been filled before
+        if (dep_n > 0) {                     // every tile of the producing phase up to this super-tile's last + 1
+            const uint32_t need = (uint32_t)min(st + 1, dep_n - 1) + 1u;
+            if (need > done_upto) {
+                if (!dep_wait(w, ctrl, prog, dep_base + need, ia.dep_ss0 + need - 1)) return false;
+                done_upto = need;
+            }
         }
-        const uint32_t slot = ts % kTmemSlots, use = ts / kTmemSlots;
-        if (use > 0 && !w.barrier(empty0 + 8 * slot, (use - 1) & 1, ERR_WAIT_EMPTY)) return false;
+        if (use > 0 && !w.barrier(empty, (use - 1) & 1, ERR_WAIT_EMPTY)) return false;
         tc_fence_after();
-        const uint32_t d = tmem + slot * kSlotCols;
+        const uint32_t astep = 128u * (uint32_t)(st * sup);
 #pragma unroll
-        for (int k = 0; k < KS; ++k) {
-            const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)alo[k];
-            const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)blo[k];
-            if (k == 0) mma_i8_first(d, ad, bd, idesc);
-            else mma_i8_acc(d, ad, bd, idesc);
-            alo[k] += 128u * kIssuers;
+        for (int j = 0; j < kSupNarrow; ++j) {
+            if (j < sup && st * sup + j < n_tiles) {
+                const uint32_t d = d0 + (uint32_t)j * tile_cols;
+#pragma unroll
+                for (int k = 0; k < KS; ++k) {
+                    const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[k] + astep + 128u * (uint32_t)j);
+                    const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)blo[k];
+                    if (k == 0) mma_i8_first(d, ad, bd, idesc);
+                    else mma_i8_acc(d, ad, bd, idesc);
+                }
+            }
         }
-        mma_commit(full0 + 8 * slot);
+        mma_commit(full);
     }
     return true;
 }
@@ -461,73 +530,86 @@ __device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem,
 __device__ __noinline__ bool issue_phase_any(Waiter w, Ctrl *ctrl, uint32_t tmem, const IssueArgs &ia, uint32_t n_ksteps)
 {
     const uint32_t prog = smem_u32(ctrl->prog);
-    const int t_first = (int)((ia.issuer + kIssuers - (ia.ts0 % kIssuers)) % kIssuers);
-    int known = 0;
-    uint32_t ts = ia.ts0 + (uint32_t)t_first;
-    for (int t = t_first; t < ia.n_items; t += kIssuers, ts += kIssuers) {
-        const int need = min(t + 2, ia.dep_n);
-        while (known < need) {
-            const uint32_t g = ia.dep_base + known;
-            if (!w.until([&] { return item_done(prog, g); }, ERR_WAIT_ITEMS)) return false;
-            ++known;
+    const int sup = ia.wide ? kSupWide : kSupNarrow;
+    const uint32_t tile_cols = ia.wide ? kTileColsWide : kTileColsNarrow;
+    const uint32_t slot = (uint32_t)ia.issuer;
+    uint32_t done_upto = 0;
+    int st = (int)(((uint32_t)ia.issuer + kIssuers - (ia.ss0 % kIssuers)) % kIssuers);
+    for (; st < ia.n_super; st += kIssuers) {
+        const uint32_t use = (ia.ss0 + (uint32_t)st) / kSlots;
+        if (ia.dep_n > 0) {
+            const uint32_t need = (uint32_t)min(st + 1, ia.dep_n - 1) + 1u;
+            if (need > done_upto) {
+                if (!dep_wait(w, ctrl, prog, ia.dep_base + need, ia.dep_ss0 + need - 1)) return false;
+                done_upto = need;
+            }
         }
-        const uint32_t slot = ts % kTmemSlots, use = ts / kTmemSlots;
         if (use > 0 && !w.barrier(smem_u32(&ctrl->empty[slot]), (use - 1) & 1, ERR_WAIT_EMPTY)) return false;
         tc_fence_after();
-        const uint32_t d = tmem + slot * kSlotCols;
-        for (uint32_t k = 0; k < n_ksteps; ++k) {
-            const uint32_t delta = lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * k);
-            const uint32_t lbo = lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * k);
-            const uint64_t ad = make_desc(ia.a0 + delta + 2048u * (uint32_t)t, lbo, 128);
-            const uint64_t bd = make_desc(ia.w0 + k * ia.n_rows * 32u, 128, 256);
-            if (k == 0) mma_i8_first(d, ad, bd, ia.idesc);
-            else mma_i8_acc(d, ad, bd, ia.idesc);
+        for (int j = 0; j < sup; ++j) {
+            const int t = st * sup + j;
+            if (t >= ia.n_tiles) break;
+            const uint32_t d = tmem + slot * kSlotCols + (uint32_t)j * tile_cols;
+            for (uint32_t k = 0; k < n_ksteps; ++k) {
+                const uint32_t delta = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * k));
+                const uint32_t lbo = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * k));
+                const uint64_t ad = make_desc(ia.a0 + delta + 2048u * (uint32_t)t, lbo, 128);
+                const uint64_t bd = make_desc(ia.w0 + k * ia.n_rows * 32u, 128, 256);
+                if (k == 0) mma_i8_first(d, ad, bd, ia.idesc);
+                else mma_i8_acc(d, ad, bd, ia.idesc);
+            }
         }
         mma_commit(smem_u32(&ctrl->full[slot]));
     }
     return true;
 }
 
-// One thread of each of warps 0..3: the tensor-core work of one group (issuer 0 also loads the weights).
+// Warps 0..3, all lanes converged: the tensor-core work of one group (issuer 0 also loads the weights).
 __device__ __noinline__ void mma_role(const MegaParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, int it, int issuer)
 {
     Waiter w{ctrl, p.err};
     const uint32_t prog = smem_u32(ctrl->prog);
     const uint32_t ptab = smem_u32(ctrl->ptab);
     const uint32_t item_off = (uint32_t)it * p.items_per_group;
-    const uint32_t tile_off = (uint32_t)it * p.tiles_per_group;
     const uint32_t conv_off = (uint32_t)it * p.n_conv;
     const int n_phases = p.n_phases, stop_phase = p.stop_phase, n_conv = p.n_conv;
+    uint32_t ss_next = (uint32_t)it * p.supers_per_group;      // sequence number of the phase's first super-tile
     const ConvSrc *conv_src = p.conv_src;
     // weights of this group's first convolution (everything before the group barrier is complete)
-    if (issuer == 0 && !w.aborted()) issue_weights(conv_src, sbase, smem_u32(&ctrl->wbar[conv_off % 3]));
+    const bool leader = issuer == 0 && elect_one();         // the one thread that starts the weight copies
+    if (leader && !w.aborted()) issue_weights(conv_src, sbase, smem_u32(&ctrl->wbar[conv_off % 3]));
+    __syncwarp();
     int item_base = 0, prev_item_base = 0, prev_n_items = 0;
-    uint32_t conv_index = 0, tile_base = 0;
+    uint32_t conv_index = 0;
     for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
-        const uint4 e = ld_shared_v4(ptab + 16 * ph);
-        const int kind = e.x & 0xFF, full_sync = (e.x >> 8) & 1, n_items = (int)e.y;
+        uint4 e = ld_shared_v4(ptab + 16 * ph);
+        e.x = warp_uniform(e.x); e.y = warp_uniform(e.y); e.z = warp_uniform(e.z); e.w = warp_uniform(e.w);
+        const int kind = e.x & 0xFF, full_sync = (e.x >> 8) & 1, n_items = (int)e.y, wide = (e.x >> 24) & 1;
         if (kind == PH_CONV) {
             // the phase before last must be complete (shared-memory reuse rule); with full_sync the last one too
             const uint32_t end = item_off + (uint32_t)(full_sync ? item_base : prev_item_base);
             if (!w.until([&] { return all_items_below_done(prog, end); }, ERR_WAIT_ITEMS)) return;
             const uint32_t cg = conv_off + conv_index;
-            if (issuer == 0 && (int)conv_index + 1 < n_conv) {
+            if (leader && (int)conv_index + 1 < n_conv) {
                 const ConvSrc *nxt = conv_src + conv_index + 1;
                 if ((int)(__ldg(&nxt->bytes_phase) >> 24) <= stop_phase)
                     issue_weights(nxt, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
             }
+            __syncwarp();
             if (!w.barrier(smem_u32(&ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS)) return;
             // phase parameters from the head of the blob
             const uint32_t desc = sbase + e.z;
-            const uint4 h = ld_shared_v4(desc);                        // in_off, n_ksteps, idesc, n_rows
+            uint4 h = ld_shared_v4(desc);                              // in_off, n_ksteps, idesc, n_rows
+            h.x = warp_uniform(h.x); h.y = warp_uniform(h.y); h.z = warp_uniform(h.z); h.w = warp_uniform(h.w);
             IssueArgs ia;
             ia.desc = desc;
-            ia.a0 = sbase + h.x + lds32(desc + offsetof(ConvDesc, P_first)) * 16u;
-            ia.w0 = desc + lds32(desc + offsetof(ConvDesc, weights_rel));
-            ia.n_rows = h.w; ia.idesc = h.z; ia.n_items = n_items;
+            ia.a0 = sbase + h.x + warp_uniform(lds32(desc + offsetof(ConvDesc, P_first))) * 16u;
+            ia.w0 = desc + warp_uniform(lds32(desc + offsetof(ConvDesc, weights_rel)));
+            ia.n_rows = h.w; ia.idesc = h.z; ia.n_super = n_items; ia.n_tiles = (int)e.w;
             ia.dep_base = item_off + (uint32_t)prev_item_base;
             ia.dep_n = full_sync ? 0 : prev_n_items;
-            ia.ts0 = tile_off + tile_base;
+            ia.dep_ss0 = ss_next - (uint32_t)prev_n_items;     // the producing phase is the conv phase just before
+            ia.ss0 = ss_next; ia.wide = wide;
             ia.issuer = issuer;
             bool ok;
             switch (h.y) {
@@ -539,7 +621,7 @@ __device__ __noinline__ void mma_role(const MegaParams &p, Ctrl *ctrl, uint32_t 
             }
             if (!ok) return;
             conv_index += 1;
-            tile_base += (uint32_t)n_items;
+            ss_next += (uint32_t)n_items;
         }
         prev_item_base = item_base; prev_n_items = n_items;
         item_base += n_items;
@@ -552,15 +634,21 @@ struct EpiCtx {
     Ctrl *ctrl;
     uint32_t sbase, tmem;
     int warp_e, wg, quarter, lane, tid_wg;
-    uint32_t done;      // items this warp has completed (monotonic)
 };
 
-__device__ __forceinline__ void finish_item(EpiCtx &c)
+// Progress counter of a warp: the index of the next item it still has work in.  Every item below the minimum
+// over all warps is therefore complete.  `finish_item` publishes after work (shared-memory writes are fenced for
+// the tensor core's reads first), `skip_to` when there was none.
+__device__ __forceinline__ void finish_item(const EpiCtx &c, uint32_t next_item)
 {
     fence_proxy_async();
     __syncwarp();
-    c.done += 1;
-    if (c.lane == 0) st_release(smem_u32(&c.ctrl->prog[c.warp_e]), c.done);
+    if (c.lane == 0) st_release(smem_u32(&c.ctrl->prog[c.warp_e]), next_item);
+}
+__device__ __forceinline__ void skip_to(const EpiCtx &c, uint32_t next_item)
+{
+    __syncwarp();
+    if (c.lane == 0) st_release(smem_u32(&c.ctrl->prog[c.warp_e]), next_item);
 }
 
 __device__ void fill_item(uint32_t fill_off, uint32_t bytes_halo, const EpiCtx &c, int i)
@@ -640,11 +728,9 @@ __device__ __forceinline__ ConvRegs load_conv_regs(uint32_t desc, int G)
 //             output zero-point, so this is rs(acc' * mult, 31 + shift) + zp_out exactly
 //   residual: y += floor((r * res_mult + R) / 2^n), R = 2^(n-1) - zp_res * res_mult   (kResHigh: n >= 32)
 template <bool kRes, bool kResHigh, bool kLo, int K>
-__device__ __forceinline__ int requant1(int acc, uint32_t caddr, uint32_t rword, const ConvRegs &R, int lo)
+__device__ __forceinline__ int requant1(int acc, const ChanConst &cs, uint32_t rword, const ConvRegs &R, int lo)
 {
-    const uint4 cs = ld_shared_v4(caddr);            // mult, B low, B high, s = shift - 1
-    const long long B = (long long)(((unsigned long long)cs.z << 32) | cs.y);
-    int y = hi32(mad_wide(acc, (int)cs.x, B)) >> (int)cs.w;
+    int y = hi32(mad_wide(acc, cs.mult, cs.B)) >> cs.s;
     if (kRes) {
         const long long t = mad_wide(sbyte<K>(rword), R.res_mult, R.res_R);
         y += kResHigh ? (hi32(t) >> R.res_sh) : (int)__funnelshift_r((uint32_t)lo32(t), (uint32_t)hi32(t), R.res_sh);
@@ -653,82 +739,142 @@ __device__ __forceinline__ int requant1(int acc, uint32_t caddr, uint32_t rword,
     return y;
 }
 
-template <bool kRes, bool kResHigh, bool kLo>
-__device__ __forceinline__ uint32_t requant4(int a0, int a1, int a2, int a3, uint32_t caddr, uint32_t rword,
-                                             const ConvRegs &R, int lo)
-{
-    const int y0 = requant1<kRes, kResHigh, kLo, 0>(a0, caddr, rword, R, lo);
-    const int y1 = requant1<kRes, kResHigh, kLo, 1>(a1, caddr + 16, rword, R, lo);
-    const int y2 = requant1<kRes, kResHigh, kLo, 2>(a2, caddr + 32, rword, R, lo);
-    const int y3 = requant1<kRes, kResHigh, kLo, 3>(a3, caddr + 48, rword, R, lo);
-    return pack4_sat(y0, y1, y2, y3);
-}
+// Where the positions of this thread (one per tile of the super-tile) are, and where their results go.
+template <int SUP>
+struct Spots {
+    uint32_t pos[SUP], opos[SUP];
+    uint32_t keep, store;            // bit j: tile j keeps its computed value (else halo) / is stored at all
+};
 
-// CONV epilogue of one tile: thread = one position (tensor-memory lane), 16 channels at a time.
-template <bool kRes, bool kResHigh, bool kLo>
-__device__ __forceinline__ void conv_tile(const ConvRegs &R, const EpiCtx &c, int t, uint32_t slot)
+template <int SUP>
+__device__ __forceinline__ Spots<SUP> locate(const ConvRegs &R, const EpiCtx &c, int st, int n_tiles)
 {
-    const uint32_t pos = (uint32_t)(R.P_first + 128 * t + c.quarter * 32 + c.lane);
-    // position -> (sample, row, column) of the padded image
-    const uint32_t s = __umulhi(pos, R.magic_hswp);
-    const uint32_t rem = pos - s * (uint32_t)R.HsWp;
-    const uint32_t y1 = __umulhi(rem, R.magic_wp);
-    const uint32_t x1 = rem - y1 * (uint32_t)R.Wp;
-    const bool interior = (int)s < R.G && y1 >= 1 && x1 >= 1;
-    bool store = true;
-    uint32_t opos = pos;
-    if (R.scatter) {
-        const uint32_t y = y1 - 1, x = x1 - 1;
-        store = interior && !(y & 1) && !(x & 1);
-        opos = s * (uint32_t)R.o_HsWp + ((y >> 1) + 1) * (uint32_t)R.o_Wp + (x >> 1) + 1;
-    }
-    const bool keep = R.scatter || interior;          // otherwise the position holds the halo value
-    const uint32_t taddr = c.tmem + ((uint32_t)(c.quarter * 32) << 16) + slot * kSlotCols;
-    for (uint32_t ch = 0; ch < R.n_chunks; ++ch) {
-        int acc[16];
-        tmem_ld16(taddr + ch * 16, acc);
-        if (ch + 1 == R.n_chunks) {           // accumulator slot may be overwritten from here on
-            tc_fence_before();
-            __syncwarp();
-            if (c.lane == 0) mbar_arrive(smem_u32(&c.ctrl->empty[slot]));
+    Spots<SUP> sp;
+    sp.keep = 0; sp.store = 0;
+#pragma unroll
+    for (int j = 0; j < SUP; ++j) {
+        const int t = st * SUP + j;
+        // a tile beyond the phase's last one is never stored; it borrows the last tile's addresses so that
+        // every read stays inside the tensor's region
+        const uint32_t pos = (uint32_t)(R.P_first + 128 * min(t, n_tiles - 1) + c.quarter * 32 + c.lane);
+        // position -> (sample, row, column) of the padded image
+        const uint32_t s = __umulhi(pos, R.magic_hswp);
+        const uint32_t rem = pos - s * (uint32_t)R.HsWp;
+        const uint32_t y1 = __umulhi(rem, R.magic_wp);
+        const uint32_t x1 = rem - y1 * (uint32_t)R.Wp;
+        const bool interior = (int)s < R.G && y1 >= 1 && x1 >= 1;
+        bool store = t < n_tiles;
+        uint32_t opos = pos;
+        if (R.scatter) {
+            const uint32_t y = y1 - 1, x = x1 - 1;
+            store = store && interior && !(y & 1) && !(x & 1);
+            opos = s * (uint32_t)R.o_HsWp + ((y >> 1) + 1) * (uint32_t)R.o_Wp + (x >> 1) + 1;
         }
-        const uint4 ci = ld_shared_v4(R.chunks + ch * (uint32_t)sizeof(ChunkInfo));   // out_off, res_off, lo, halo
-        const uint32_t cbase = R.const_addr + ch * 256u;
+        sp.pos[j] = pos; sp.opos[j] = opos;
+        if (R.scatter || interior) sp.keep |= 1u << j;
+        if (store) sp.store |= 1u << j;
+    }
+    return sp;
+}
+
+// Requantise one 16-channel chunk of the tiles of a super-tile (16 SUP accumulators per thread) and store it.
+// The per-channel constants are read once and applied to all SUP positions.
+template <bool kRes, bool kResHigh, bool kLo, int SUP>
+__device__ __forceinline__ void chunk_compute(const int (&acc)[SUP][16], const ConvRegs &R, const EpiCtx &c,
+                                              const Spots<SUP> &sp, uint32_t ch)
+{
+    const uint4 ci = ld_shared_v4(R.chunks + ch * (uint32_t)sizeof(ChunkInfo));   // out_off, res_off, lo, halo
+    const uint32_t cbase = R.const_addr + ch * 256u;
+    const int lo = (int)ci.z;
+    uint32_t rw[SUP][4];
+#pragma unroll
+    for (int j = 0; j < SUP; ++j) {
         uint4 rv = make_uint4(0, 0, 0, 0);
-        if (kRes) rv = ld_shared_v4(c.sbase + ci.y + pos * 16u);
-        const int lo = (int)ci.z;
-        uint4 o;
-        o.x = requant4<kRes, kResHigh, kLo>(acc[0], acc[1], acc[2], acc[3], cbase, rv.x, R, lo);
-        o.y = requant4<kRes, kResHigh, kLo>(acc[4], acc[5], acc[6], acc[7], cbase + 64, rv.y, R, lo);
-        o.z = requant4<kRes, kResHigh, kLo>(acc[8], acc[9], acc[10], acc[11], cbase + 128, rv.z, R, lo);
-        o.w = requant4<kRes, kResHigh, kLo>(acc[12], acc[13], acc[14], acc[15], cbase + 192, rv.w, R, lo);
-        if (!keep) o = make_uint4(ci.w, ci.w, ci.w, ci.w);
-        if (store) st_shared_v4(c.sbase + ci.x + opos * 16u, o);
+        if (kRes) rv = ld_shared_v4(c.sbase + ci.y + sp.pos[j] * 16u);
+        rw[j][0] = rv.x; rw[j][1] = rv.y; rw[j][2] = rv.z; rw[j][3] = rv.w;
+    }
+    uint32_t out[SUP][4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const ChanConst c0 = ld_chan_const(cbase + (4 * g + 0) * 16), c1 = ld_chan_const(cbase + (4 * g + 1) * 16);
+        const ChanConst c2 = ld_chan_const(cbase + (4 * g + 2) * 16), c3 = ld_chan_const(cbase + (4 * g + 3) * 16);
+#pragma unroll
+        for (int j = 0; j < SUP; ++j) {
+            const int y0 = requant1<kRes, kResHigh, kLo, 0>(acc[j][4 * g + 0], c0, rw[j][g], R, lo);
+            const int y1 = requant1<kRes, kResHigh, kLo, 1>(acc[j][4 * g + 1], c1, rw[j][g], R, lo);
+            const int y2 = requant1<kRes, kResHigh, kLo, 2>(acc[j][4 * g + 2], c2, rw[j][g], R, lo);
+            const int y3 = requant1<kRes, kResHigh, kLo, 3>(acc[j][4 * g + 3], c3, rw[j][g], R, lo);
+            out[j][g] = pack4_sat(y0, y1, y2, y3);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < SUP; ++j) {
+        uint4 o = make_uint4(out[j][0], out[j][1], out[j][2], out[j][3]);
+        if (!((sp.keep >> j) & 1u)) o = make_uint4(ci.w, ci.w, ci.w, ci.w);
+        if ((sp.store >> j) & 1u) st_shared_v4(c.sbase + ci.x + sp.opos[j] * 16u, o);
     }
 }
 
-// All tiles of one CONV phase that belong to this warpgroup.
+// The super-tiles of one CONV phase that fall to this warpgroup: those whose sequence number, hence slot, is
+// the warpgroup's index mod 2.  The loops over pairs of tiles and over 16-channel chunks are kept rolled on
+// purpose: their body (32 outputs per thread) is a few KB of code, so the two epilogue warps and the issuing
+// warp of a scheduler all run out of its instruction cache; a fully unrolled super-tile does not fit and
+// leaves the warps waiting for instruction fetches.  The slot is released after the warp's last read of it,
+// so the tensor cores refill it while the last chunk is still being requantised; the warpgroups never meet.
 template <bool kRes, bool kResHigh, bool kLo>
-__device__ __noinline__ void conv_phase_tiles(Waiter w, EpiCtx &c_io, const ConvRegs &R_in, int i0, int n_items, uint32_t ts0)
+__device__ __noinline__ void conv_phase_items(Waiter w, const EpiCtx &c_in, const ConvRegs &R_in, int n_super, int n_tiles,
+                                              uint32_t ss0, uint32_t first_item, int sup)
 {
     // private copies: values reached through references would be re-read after every barrier or fence
-    EpiCtx c = c_io;
+    const EpiCtx c = c_in;
     const ConvRegs R = R_in;
-    const uint32_t full0 = smem_u32(&c.ctrl->full[0]);
+    const uint32_t tile_cols = (uint32_t)kSlotCols / (uint32_t)sup;
+    const int n_pairs = sup >> 1;
+    const uint32_t full0 = smem_u32(&c.ctrl->full[0]), empty0 = smem_u32(&c.ctrl->empty[0]);
+    const uint32_t done0 = smem_u32(&c.ctrl->done[0]);
+    const uint32_t lane_base = c.tmem + ((uint32_t)(c.quarter * 32) << 16);
+    const uint32_t n_chunks = R.n_chunks;
     bool ok = true;
-    for (int i = i0; i < n_items; i += kWarpGroups) {
-        if (ok) {
-            const uint32_t ts = ts0 + (uint32_t)i, slot = ts % kTmemSlots;
-            ok = w.barrier(full0 + 8 * slot, (ts / kTmemSlots) & 1, ERR_WAIT_FULL);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                conv_tile<kRes, kResHigh, kLo>(R, c, i, slot);
+    for (int st = (int)(((uint32_t)c.wg + 2u - (ss0 & 1u)) & 1u); st < n_super; st += kWarpGroups) {
+        const uint32_t ss = ss0 + (uint32_t)st, slot = ss % kSlots;
+        if (ok) ok = w.barrier(full0 + 8 * slot, (ss / kSlots) & 1, ERR_WAIT_FULL);
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+        const uint32_t slot_addr = lane_base + slot * kSlotCols;
+#pragma unroll 1
+        for (int pr = 0; pr < n_pairs; ++pr) {
+            const Spots<2> sp = locate<2>(R, c, st * n_pairs + pr, n_tiles);
+            const uint32_t pair_addr = slot_addr + (uint32_t)(2 * pr) * tile_cols;
+#pragma unroll 1
+            for (uint32_t ch = 0; ch < n_chunks; ++ch) {
+                int acc[2][16];
+                tmem_ld16_issue(pair_addr + ch * 16, acc[0]);
+                tmem_ld16_issue(pair_addr + tile_cols + ch * 16, acc[1]);
+                tmem_ld_wait();
+                if (pr + 1 == n_pairs && ch + 1 == n_chunks) {      // last read of the slot by this warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (c.lane == 0) mbar_arrive(empty0 + 8 * slot);
+                }
+                if (ok) chunk_compute<kRes, kResHigh, kLo, 2>(acc, R, c, sp, ch);
             }
         }
-        finish_item(c);
+        finish_item(c, first_item + (uint32_t)min(st + kWarpGroups, n_super));
+        if (c.lane == 0) mbar_arrive(done0 + 8 * slot);
     }
-    c_io.done = c.done;
+}
+
+__device__ __forceinline__ void conv_phase_dispatch(Waiter w, const EpiCtx &c, const ConvRegs &R, int n_super, int n_tiles,
+                                                    uint32_t ss0, uint32_t first, int sup)
+{
+    switch (R.mode & 7u) {
+    case 0: conv_phase_items<false, false, false>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
+    case 1: conv_phase_items<false, false, true>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
+    case 2: conv_phase_items<true, false, false>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
+    case 3: conv_phase_items<true, false, true>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
+    case 6: conv_phase_items<true, true, false>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
+    default: conv_phase_items<true, true, true>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
+    }
 }
 
 // TAIL: global average pool, FC, argmax and vote; one warp carries one sample.
@@ -791,50 +937,49 @@ __device__ void tail_sample(const MegaParams &p, const EpiCtx &c, int s, bool co
     if (counted && c.lane == 0) atomicAdd(&c.ctrl->hist[best_o], 1);
 }
 
-// Epilogue warps: all non-tensor-core work of one group, item by item.
+// Epilogue warps: all non-tensor-core work of one group.  Item g of a FILL / INPUT / TAIL phase belongs to
+// warpgroup g mod 2; CONV items are split as described above.  A warp only visits the items it has work in and
+// publishes, as its progress, the index of the next such item.
 __device__ __noinline__ void epi_role(const MegaParams &p, EpiCtx &c, int it, int grp)
 {
     Waiter w{c.ctrl, p.err};
     const uint32_t prog = smem_u32(c.ctrl->prog);
     const uint32_t ptab = smem_u32(c.ctrl->ptab);
     const uint32_t item_off = (uint32_t)it * p.items_per_group;
-    const uint32_t tile_off = (uint32_t)it * p.tiles_per_group;
     const uint32_t conv_off = (uint32_t)it * p.n_conv;
     const int n_phases = p.n_phases, stop_phase = p.stop_phase, G = p.G;
-    uint32_t item_base = 0, conv_index = 0, tile_base = 0;
+    uint32_t item_base = 0, conv_index = 0;
+    uint32_t ss_next = (uint32_t)it * p.supers_per_group;
     for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
         const uint4 e = ld_shared_v4(ptab + 16 * ph);
         const int kind = e.x & 0xFF, n_items = (int)e.y;
-        const uint32_t first = item_off + item_base;
-        const uint32_t my_conv = conv_index, my_tile_base = tile_base;
+        const uint32_t first = item_off + item_base, end = first + (uint32_t)n_items;
         item_base += (uint32_t)n_items;
-        if (kind == PH_CONV) { conv_index += 1; tile_base += (uint32_t)n_items; }
-        const int i0 = (c.wg + kWarpGroups - (int)(first % kWarpGroups)) % kWarpGroups;
-        if (i0 >= n_items) continue;
         bool ok;
         if (kind == PH_CONV) {
-            const uint32_t cg = conv_off + my_conv;
+            const bool wide = (e.x >> 24) & 1;
+            const uint32_t cg = conv_off + conv_index, ss0 = ss_next;
+            conv_index += 1;
+            ss_next += (uint32_t)n_items;
+            // first item with work for this warpgroup
+            const uint32_t own = ((uint32_t)c.wg + 2u - (ss0 & 1u)) & 1u;
+            skip_to(c, min(first + own, end));
+            if (first + own >= end) continue;
             ok = w.barrier(smem_u32(&c.ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS);
             ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                const ConvRegs R = load_conv_regs(c.sbase + e.z, G);
-                const uint32_t ts0 = tile_off + my_tile_base;
-                switch (R.mode & 7u) {
-                case 0: conv_phase_tiles<false, false, false>(w, c, R, i0, n_items, ts0); break;
-                case 1: conv_phase_tiles<false, false, true>(w, c, R, i0, n_items, ts0); break;
-                case 2: conv_phase_tiles<true, false, false>(w, c, R, i0, n_items, ts0); break;
-                case 3: conv_phase_tiles<true, false, true>(w, c, R, i0, n_items, ts0); break;
-                case 6: conv_phase_tiles<true, true, false>(w, c, R, i0, n_items, ts0); break;
-                default: conv_phase_tiles<true, true, true>(w, c, R, i0, n_items, ts0); break;
-                }
-            } else {
-                for (int i = i0; i < n_items; i += kWarpGroups) finish_item(c);
-            }
+            if (!ok) { skip_to(c, end); continue; }
+            const ConvRegs R = load_conv_regs(c.sbase + e.z, G);
+            const int n_tiles = (int)e.w;
+            conv_phase_dispatch(w, c, R, n_items, n_tiles, ss0, first, wide ? kSupWide : kSupNarrow);
             continue;
         }
+        const uint32_t own = ((uint32_t)c.wg + kWarpGroups - (first % kWarpGroups)) % kWarpGroups;
+        skip_to(c, min(first + own, end));
+        if (first + own >= end) continue;
         ok = w.until([&] { return all_items_below_done(prog, first); }, ERR_WAIT_ITEMS);
         ok = __all_sync(0xffffffffu, ok);
-        for (int i = i0; i < n_items; i += kWarpGroups) {
+        for (uint32_t g = first + own; g < end; g += kWarpGroups) {
+            const int i = (int)(g - first);
             if (ok) {
                 if (kind == PH_FILL) {
                     fill_item(e.z, e.w, c, i);
@@ -845,7 +990,7 @@ __device__ __noinline__ void epi_role(const MegaParams &p, EpiCtx &c, int it, in
                     tail_sample(p, c, min(s, G - 1), s < G, grp);
                 }
             }
-            finish_item(c);
+            finish_item(c, min(g + kWarpGroups, end));
         }
     }
 }
@@ -855,11 +1000,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_mega(const __grid_constant__ Me
     extern __shared__ __align__(128) uint8_t smem[];
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = (int)warp_uniform(threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kTmemSlots; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), 1);
-            mbar_init(smem_u32(&ctrl->empty[s]), 4);
+        for (int s = 0; s < kSlots; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);             // the super-tile's issuing thread
+            mbar_init(smem_u32(&ctrl->empty[s]), 4);            // the four warps of the slot's warpgroup
+            mbar_init(smem_u32(&ctrl->done[s]), 4);             // the same, when the super-tile's outputs are stored
         }
         for (int s = 0; s < 3; ++s) mbar_init(smem_u32(&ctrl->wbar[s]), 1);
         mbar_init(smem_u32(&ctrl->drain), kIssuers);
@@ -879,13 +1025,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_mega(const __grid_constant__ Me
     EpiCtx c;
     c.ctrl = ctrl; c.sbase = sbase; c.tmem = tmem;
     c.warp_e = warp - kIssuers; c.wg = (warp - kIssuers) >> 2; c.quarter = warp & 3; c.lane = lane;
-    c.tid_wg = ((warp - kIssuers) & 3) * 32 + lane; c.done = 0;
+    c.tid_wg = ((warp - kIssuers) & 3) * 32 + lane;
 
     int it = 0;
     for (int grp = blockIdx.x; grp < p.n_groups; grp += gridDim.x, ++it) {
         if (warp < kIssuers) {
-            if (lane == 0) mma_role(p, ctrl, sbase, tmem, it, warp);
-            __syncwarp();
+            mma_role(p, ctrl, sbase, tmem, it, warp);
         } else {
             epi_role(p, c, it, grp);
         }
@@ -898,9 +1043,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_mega(const __grid_constant__ Me
         for (uint32_t o = threadIdx.x * 16u; o < p.dump_bytes; o += blockDim.x * 16u)
             *reinterpret_cast<uint4 *>(p.dump + o) = ld_shared_v4(sbase + p.dump_off + o);
     // no tensor-core work may be in flight when tensor memory is released
-    if (warp < kIssuers && lane == 0) {
+    if (warp < kIssuers) {
         Waiter w{ctrl, p.err};
-        mma_commit(smem_u32(&ctrl->drain));
+        __syncwarp();
+        mma_commit(smem_u32(&ctrl->drain));          // by the lane that issued this warp's tensor-core work
         w.barrier(smem_u32(&ctrl->drain), 0, ERR_WAIT_DRAIN);
     }
     tc_fence_before();
@@ -959,7 +1105,7 @@ struct MegaPlan {
     int G = 0, in_c = 0, in_h = 0, in_w = 0, n_classes = 0;
     std::vector<MPhase> phases;
     std::vector<int> conv_phase;
-    int items_per_group = 0, tiles_per_group = 0;
+    int items_per_group = 0, supers_per_group = 0;
     uint32_t smem_bytes = 0;
     MegaParams base;                      // fields that do not change between launches
     // device copies
@@ -1044,7 +1190,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         if (i + 1 < n_conv_layers) {
             const isc_layer &A = layers[i].d, &B = layers[i + 1].d;
             if (A.kh == 3 && B.kh == 1 && B.in_tensor == A.in_tensor && B.stride == A.stride && B.res_tensor < 0 &&
-                A.res_tensor < 0 && A.cout + B.cout <= kSlotCols && A.zp_in == B.zp_in &&
+                A.res_tensor < 0 && A.cout + B.cout <= kMaxFusedCols && A.zp_in == B.zp_in &&
                 T[(size_t)i + 1].H == T[(size_t)i + 2].H && T[(size_t)i + 1].W == T[(size_t)i + 2].W) {
                 nd.fused_layer = i + 1;
                 ++i;
@@ -1177,7 +1323,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
     plan->tensors = T;
     plan->tensor_off.assign(T.size(), 0);
     for (int t = 0; t <= n_conv_layers; ++t) plan->tensor_off[(size_t)t] = buffers[(size_t)T[(size_t)t].buffer].off;
-    int item_base = 0, tile_base = 0;
+    int item_base = 0, super_base = 0, last_wide = -1;
     blob_out->clear();
     blob_offsets->assign((size_t)n_conv, 0);
     bool magic_ok = true;
@@ -1206,7 +1352,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             const isc_layer &L = layers[nd.layer].d;
             const PlanTensor &in = T[(size_t)L.in_tensor];
             P.H = in.H; P.W = in.W; P.Wp = in.Wp; P.HsWp = in.HsWp; P.P_first = in.P_first;
-            P.n_items = in.n_tiles;
+            P.n_tiles = in.n_tiles;
             P.magic_hswp = magic_for((uint32_t)in.HsWp, (uint32_t)in.npa + 256, &magic_ok);
             P.magic_wp = magic_for((uint32_t)in.Wp, (uint32_t)in.HsWp + 256, &magic_ok);
             P.scatter = L.stride == 2;
@@ -1225,8 +1371,11 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             const uint32_t consts_rel = weights_rel + P.n_ksteps * (uint32_t)P.n_rows * 32u;
             P.const_off = P.w_off + consts_rel;
             P.conv_index = (uint32_t)cidx;
-            P.tile_base = tile_base;
-            tile_base += P.n_items;
+            P.wide = P.n_rows > kTileColsNarrow ? 1 : 0;
+            if (P.n_rows > kTileColsWide) return false;
+            const int sup = P.wide ? kSupWide : kSupNarrow;
+            P.n_items = (in.n_tiles + sup - 1) / sup;             // one item per super-tile
+            super_base += P.n_items;
             for (uint32_t k = 0; k < P.n_ksteps; ++k) {
                 const auto &kp = ksteps[(size_t)cidx][k];
                 P.a_delta[k] = chunk_addr[(size_t)cidx][(size_t)kp.first];
@@ -1236,7 +1385,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             // operand reads must stay inside the input region
             for (uint32_t k = 0; k < P.n_ksteps; ++k) {
                 const long long lo_b = (long long)P.P_first * 16 + P.a_delta[k];
-                const long long hi_b = (long long)(P.P_first + 128 * P.n_items) * 16 + P.a_delta[k] + P.a_lbo[k];
+                const long long hi_b = (long long)(P.P_first + 128 * P.n_tiles) * 16 + P.a_delta[k] + P.a_lbo[k];
                 if (lo_b < 0) return false;
                 const long long plane_of_hi = (hi_b - 1) / in.plane_bytes;
                 if (plane_of_hi >= in.planes) return false;
@@ -1245,7 +1394,9 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             const bool prev_is_conv = ph >= 1 && skel[(size_t)ph - 1].kind == PH_CONV;
             bool tile_rule = prev_is_conv && in.producer_phase == ph - 1 && !in.scatter_produced;
             if (L.res_tensor >= 0 && T[(size_t)L.res_tensor].producer_phase >= ph - 1) tile_rule = false;
-            if (tile_rule && plan->phases[(size_t)ph - 1].n_items != P.n_items) tile_rule = false;
+            if (tile_rule && plan->phases[(size_t)ph - 1].n_tiles != P.n_tiles) tile_rule = false;
+            if (P.wide != last_wide) tile_rule = false;      // super-tiles of another size: no item-for-item rule
+            last_wide = P.wide;
             P.full_sync = tile_rule ? 0 : 1;
             // epilogue chunks and the weight blob
             const int lay[2] = {nd.layer, nd.fused_layer};
@@ -1304,7 +1455,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
                     const int nn = 31 + sh;
                     const long long biasf = (long long)ML.bias[oc] - (long long)LL.zp_in * wsum;
                     const long long B = biasf * ML.mult[oc] + (1ll << (nn - 1)) + ((long long)LL.zp_out << nn);
-                    int32_t cst[4] = {ML.mult[oc], (int32_t)(uint32_t)(B & 0xFFFFFFFFll), (int32_t)(B >> 32), nn - 32};
+                    int32_t cst[4] = {(int32_t)(uint32_t)(B & 0xFFFFFFFFll), (int32_t)(B >> 32), ML.mult[oc], nn - 32};
                     memcpy(&blob[consts_rel + (size_t)n * 16], cst, 16);
                 }
                 row0 += LL.cout;
@@ -1331,7 +1482,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
     if (!magic_ok) return false;
     plan->G = G;
     plan->items_per_group = item_base;
-    plan->tiles_per_group = tile_base;
+    plan->supers_per_group = super_base;
     plan->smem_bytes = (high + 127u) & ~127u;
     return true;
 }
@@ -1403,10 +1554,12 @@ int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
     std::vector<PhaseEntry> ptab(plan->phases.size());
     for (size_t i = 0; i < ptab.size(); ++i) {
         const MPhase &P = plan->phases[i];
-        ptab[i].kind_sync = (uint32_t)P.kind | ((uint32_t)(P.full_sync ? 1 : 0) << 8);
+        ptab[i].kind_sync = (uint32_t)P.kind | ((uint32_t)(P.full_sync ? 1 : 0) << 8) |
+                            (P.kind == PH_CONV ? (P.n_chunks << 16) | ((uint32_t)P.wide << 24) : 0u);
         ptab[i].n_items = (uint32_t)P.n_items;
         ptab[i].a = P.kind == PH_CONV ? P.w_off : P.fill_off;
-        ptab[i].b = P.kind == PH_FILL ? (P.fill_bytes | ((P.fill_word & 0xFFu) << 24)) : 0u;
+        ptab[i].b = P.kind == PH_FILL ? (P.fill_bytes | ((P.fill_word & 0xFFu) << 24))
+                                      : P.kind == PH_CONV ? (uint32_t)P.n_tiles : 0u;
     }
     std::vector<ConvSrc> csrc(plan->conv_phase.size());
     for (size_t c = 0; c < csrc.size(); ++c) {
@@ -1432,7 +1585,7 @@ int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
     b.n_phases = (int)plan->phases.size();
     b.n_conv = (int)plan->conv_phase.size();
     b.items_per_group = plan->items_per_group;
-    b.tiles_per_group = plan->tiles_per_group;
+    b.supers_per_group = plan->supers_per_group;
     b.G = plan->G;
     b.in_c = in_c;
     b.input_off = plan->tensor_off[0];
