@@ -33,19 +33,20 @@ namespace isc {
 
 namespace {
 
-constexpr int kIssuers = 4;                 // warps 0..3: one thread of each issues the MMAs of every 4th tile
+constexpr int kIssuers = 4;                 // warps 0..3: an elected lane of each issues the MMAs of every 4th tile
 constexpr int kEpiWarps = 8;                // warps 4..11: epilogue, two warpgroups of "fat" threads (168 registers)
 constexpr int kWarpGroups = kEpiWarps / 4;
 constexpr int kThreads = 32 * (kIssuers + kEpiWarps);
-// Four accumulator slots of 128 tensor-memory columns, one super-tile each: four tiles of up to 32 output
-// channels (narrow) or two tiles of up to 64 (wide).  Slot s is written by issuing thread s and read by
-// warpgroup s mod 2; super-tiles take the slots in turn over the whole run of the kernel.
-constexpr int kSlots = 4, kSlotCols = 128;
-constexpr int kSupNarrow = 4, kTileColsNarrow = 32;
-constexpr int kSupWide = 2, kTileColsWide = 64;
-constexpr int kMaxFusedCols = kTileColsWide;
-static_assert(kSlots == kIssuers, "one issuing thread per accumulator slot");
-static_assert(kWarpGroups == 2, "slot s belongs to warpgroup s mod 2");
+// Tensor memory is used as two halves of 256 columns.  A CONV phase is cut into rounds of consecutive tiles
+// (as many as fit a half: 16, 8 or 4 tiles of 16, 32 or 64 columns); rounds take the halves in turn over the
+// whole run of the kernel.  The four issuing warps share the tiles of a round; the eight epilogue warps share
+// its outputs.  FILL, INPUT and TAIL phases are rounds of their own without tensor-core work, so that one
+// sequence number orders everything that happens to a group.
+constexpr int kHalves = 2, kHalfCols = 256;
+constexpr int kMaxFusedCols = 64;
+// accumulator columns of a tile with n output channels
+__host__ __device__ constexpr int tile_columns(int n) { return n <= 16 ? 16 : n <= 32 ? 32 : 64; }
+static_assert(kWarpGroups == 2, "the epilogue splits a round's work between two warpgroups");
 constexpr int kMaxKsteps = 20;
 constexpr int kMaxChunks = 4;
 constexpr int kMaxPhases = 136;
@@ -77,7 +78,7 @@ struct alignas(16) MPhase {
     uint32_t w_off, w_bytes, const_off, conv_index;
     int32_t n_tiles, n_rows;
     int32_t res_mult, res_n;
-    int32_t wide, pad3;                     // accumulator layout: 0 narrow slots, 1 wide slots
+    int32_t n_rounds, tiles_per_round;      // CONV: how the tiles are cut into rounds
     long long res_R;
     int32_t a_delta[kMaxKsteps];
     uint32_t a_lbo[kMaxKsteps];
@@ -87,10 +88,10 @@ struct alignas(16) MPhase {
 // ---- what the kernel reads -------------------------------------------------------------------
 
 // One entry per phase, copied to shared memory when the kernel starts.
-//   CONV: n_items = super-tiles, a = shared-memory offset of the phase's blob (ConvDesc, weights,
-//         per-channel constants), b = tiles
+//   CONV: n_items = rounds | tiles per round << 8 | accumulator columns per tile << 16, a = shared-memory offset of
+//         the phase's blob (ConvDesc, weights, per-channel constants), b = tiles
 //   FILL: a = offset of the region, b = bytes | halo byte << 24
-struct alignas(16) PhaseEntry { uint32_t kind_sync, n_items, a, b; };     // kind | full_sync << 8 | chunks << 16 | wide << 24
+struct alignas(16) PhaseEntry { uint32_t kind_sync, n_items, a, b; };     // kind | full_sync << 8 | chunks << 16
 
 // Where the blob of convolution c comes from (global) and goes to (shared).
 struct alignas(16) ConvSrc { unsigned long long gmem; uint32_t bytes_phase, smem_off; };   // bytes | phase << 24
@@ -116,7 +117,7 @@ struct FcConst { int32_t mult, n, zp_out, lo, bias, pad0, pad1, pad2; };
 struct MegaParams {
     const PhaseEntry *ptab;
     const ConvSrc *conv_src;
-    int32_t n_phases, n_conv, items_per_group, supers_per_group;
+    int32_t n_phases, n_conv, rounds_per_group, pad_r;
     int32_t in_H, in_W, in_Wp, in_HsWp;
     int32_t G, n_groups, n_samples, in_c;
     const uint8_t *x;                 // clean image, CHW
@@ -140,10 +141,9 @@ struct MegaParams {
 };
 
 struct Ctrl {
-    unsigned long long full[kSlots], empty[kSlots], done[kSlots], wbar[3], drain;
+    unsigned long long full[kHalves], done[kHalves], wbar[3], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
-    alignas(16) uint32_t prog[kEpiWarps];          // items completed by each epilogue warp (monotonic)
     int32_t hist[128];
     PhaseEntry ptab[kMaxPhases];
 };
@@ -416,20 +416,27 @@ struct Waiter {
 
 // Every epilogue warp publishes the index of the next item it has work in: all counters >= need means items
 // 0..need-1 are complete.  One 16-byte acquire read per warpgroup.
-__device__ __forceinline__ bool all_reached(uint32_t prog_addr, uint32_t need)
-{
-    bool ok = true;
-#pragma unroll
-    for (int g = 0; g < kWarpGroups; ++g) {
-        const uint4 a = ld_acquire_v4(prog_addr + 16 * g);
-        ok = ok && a.x >= need && a.y >= need && a.z >= need && a.w >= need;
-    }
-    return ok;
-}
-__device__ __forceinline__ bool all_items_below_done(uint32_t prog_addr, uint32_t end) { return all_reached(prog_addr, end); }
-__device__ __forceinline__ bool item_done(uint32_t prog_addr, uint32_t g) { return all_reached(prog_addr, g + 1); }
+// ------------------------------------------------------------------ rounds
+//
+// Everything that happens to a group is a sequence of rounds, numbered over the whole run of the kernel:
+// a CONV phase contributes n_rounds of them (consecutive tiles), every other phase one.  Round r uses
+// tensor-memory half r & 1 and the barrier pair full[r & 1] / done[r & 1]; each of the two completes exactly
+// once per round (also for rounds without tensor-core work), so the parity to wait for is (r >> 1) & 1.
+//   full[h]: the four issuing warps have committed their tiles of the round (or simply arrived)
+//   done[h]: the eight epilogue warps have stored the round's outputs (and no longer read the half)
+// A role only ever waits for the latest or the one-before-latest completion of a barrier, so a parity is
+// never ambiguous.  Rounds complete in order.  Round r may start when round r - 2 is complete (its half is
+// free) and its operands are there: `dep`, the latest round whose outputs it reads, is r - 1 at most.
 
-// ------------------------------------------------------------------ issuing threads
+// dependency of round k (tiles [k tpr, (k+1) tpr)) of a CONV phase whose first round is `first`:
+//   with full_sync, everything before the phase; else the producing phase (the one just before, cut into rounds
+//   the same way) up to its round k + 1, because a tile reads one tile beyond itself
+__device__ __forceinline__ uint32_t round_dep(uint32_t first, int k, int n_rounds, bool full_sync)
+{
+    return full_sync ? first - 1u : first - (uint32_t)n_rounds + (uint32_t)min(k + 1, n_rounds - 1);
+}
+
+// ------------------------------------------------------------------ issuing warps
 
 __device__ __forceinline__ void issue_weights(const ConvSrc *src, uint32_t sbase, uint32_t wbar_addr)
 {
@@ -441,43 +448,25 @@ __device__ __forceinline__ void issue_weights(const ConvSrc *src, uint32_t sbase
 }
 
 struct IssueArgs {
-    uint32_t desc, a0, w0, n_rows, idesc, dep_base, dep_ss0, ss0;
-    int n_super, n_tiles, dep_n, issuer, wide;
+    uint32_t desc, a0, w0, n_rows, idesc, first, tile_cols;
+    int n_rounds, tpr, n_tiles, issuer, full_sync;
 };
 
-// Wait until the epilogue warps have published `target` as their progress, i.e. until the producing phase's
-// super-tiles up to sequence number ss_last are stored.  The progress counters decide; the per-slot `done`
-// barriers only serve to park the warp in hardware until something relevant has happened, instead of polling.
-// (A barrier phase can alias when the slot is two uses ahead; then the wait merely returns early or runs into
-// its hardware time limit, and the counters are read again.)
-__device__ __forceinline__ bool dep_wait(Waiter w, Ctrl *ctrl, uint32_t prog, uint32_t target, uint32_t ss_last)
+// wait until round r may be issued: its half is free (round r - 2 complete) and round `dep` is complete
+__device__ __forceinline__ bool round_start_wait(Waiter w, Ctrl *ctrl, uint32_t r, uint32_t dep)
 {
-    if (all_reached(prog, target)) return true;
-    const uint32_t done0 = smem_u32(&ctrl->done[0]);
-    const unsigned long long t0 = globaltimer();
-    for (int spin = 0;; ++spin) {
-        mbar_try(done0 + 8 * (ss_last % kSlots), (ss_last / kSlots) & 1);
-        if (all_reached(prog, target)) return true;
-        if (ss_last > 0) mbar_try(done0 + 8 * ((ss_last - 1) % kSlots), ((ss_last - 1) / kSlots) & 1);   // other warpgroup
-        if (all_reached(prog, target)) return true;
-        __nanosleep(32);
-        if ((spin & 3) == 3) {
-            if (w.aborted()) return false;
-            if (globaltimer() - t0 > kWaitLimitNs) { w.fail(ERR_WAIT_ITEMS); return false; }
-        }
-    }
+    const uint32_t h = r & 1u;
+    if (r >= 2u && !w.barrier(smem_u32(&ctrl->done[h]), ((r - 2u) >> 1) & 1u, ERR_WAIT_EMPTY)) return false;
+    if (r >= 1u && dep == r - 1u && !w.barrier(smem_u32(&ctrl->done[h ^ 1u]), ((r - 1u) >> 1) & 1u, ERR_WAIT_ITEMS)) return false;
+    return true;
 }
 
-// Issue loop of one CONV phase with KS K-steps per tile.  Issuing thread k owns the super-tiles whose sequence
-// number is k mod 4 and accumulator slot k, so the four threads work on different super-tiles at different
-// times and the fixed cost per super-tile (dependency check, slot wait, commit) is paid once per two or four
-// tiles.  The low words of the operand descriptors stay in registers; tile t is 128 t positions, i.e. 128 t
-// units of the A descriptors' start-address field, further.  The body is kept as short as possible: the
-// issuing thread is alone in its warp, so every instruction it executes delays the tensor pipe.
+// The rounds of one CONV phase with KS K-steps per tile.  The issuing warp takes every fourth tile of a round.
+// The low words of the operand descriptors stay in registers; tile t is 128 t positions, i.e. 128 t units of the
+// A descriptors' start-address field, further.
 template <int KS>
 __device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem, const IssueArgs &ia)
 {
-    const uint32_t prog = smem_u32(ctrl->prog);
     uint32_t alo[KS], blo[KS];
     const uint32_t ahi = (uint32_t)(make_desc(0, 0, 128) >> 32), bhi = (uint32_t)(make_desc(0, 128, 256) >> 32);
 #pragma unroll
@@ -487,41 +476,26 @@ __device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem,
         alo[k] = (uint32_t)make_desc(ia.a0 + delta, lbo, 128);
         blo[k] = (uint32_t)make_desc(ia.w0 + (uint32_t)k * ia.n_rows * 32u, 128, 256);
     }
-    const int sup = ia.wide ? kSupWide : kSupNarrow;
-    const uint32_t tile_cols = ia.wide ? kTileColsWide : kTileColsNarrow;
-    const uint32_t slot = (uint32_t)ia.issuer;
-    const uint32_t full = smem_u32(&ctrl->full[slot]), empty = smem_u32(&ctrl->empty[slot]);
-    const uint32_t d0 = tmem + slot * kSlotCols;
-    const uint32_t idesc = ia.idesc, dep_base = ia.dep_base;
-    const int n_super = ia.n_super, n_tiles = ia.n_tiles, dep_n = ia.dep_n;
-    uint32_t done_upto = 0;                  // producing-phase items 0..done_upto-1 are known complete
-    int st = (int)(((uint32_t)ia.issuer + kIssuers - (ia.ss0 % kIssuers)) % kIssuers);
-    for (; st < n_super; st += kIssuers) {
-        const uint32_t use = (ia.ss0 + (uint32_t)st) / kSlots;      // how often this slot has been filled before
-        if (dep_n > 0) {                     // every tile of the producing phase up to this super-tile's last + 1
-            const uint32_t need = (uint32_t)min(st + 1, dep_n - 1) + 1u;
-            if (need > done_upto) {
-                if (!dep_wait(w, ctrl, prog, dep_base + need, ia.dep_ss0 + need - 1)) return false;
-                done_upto = need;
-            }
-        }
-        if (use > 0 && !w.barrier(empty, (use - 1) & 1, ERR_WAIT_EMPTY)) return false;
+    const uint32_t idesc = ia.idesc, tile_cols = ia.tile_cols;
+    const int n_tiles = ia.n_tiles, tpr = ia.tpr, issuer = ia.issuer;
+    for (int k = 0; k < ia.n_rounds; ++k) {
+        const uint32_t r = ia.first + (uint32_t)k, h = r & 1u;
+        if (!round_start_wait(w, ctrl, r, round_dep(ia.first, k, ia.n_rounds, ia.full_sync))) return false;
         tc_fence_after();
-        const uint32_t astep = 128u * (uint32_t)(st * sup);
+        const int t0 = k * tpr, t1 = min(n_tiles, t0 + tpr);
+        const uint32_t d0 = tmem + h * kHalfCols;
+#pragma unroll 1
+        for (int t = t0 + issuer; t < t1; t += kIssuers) {
+            const uint32_t d = d0 + (uint32_t)(t - t0) * tile_cols;
 #pragma unroll
-        for (int j = 0; j < kSupNarrow; ++j) {
-            if (j < sup && st * sup + j < n_tiles) {
-                const uint32_t d = d0 + (uint32_t)j * tile_cols;
-#pragma unroll
-                for (int k = 0; k < KS; ++k) {
-                    const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[k] + astep + 128u * (uint32_t)j);
-                    const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)blo[k];
-                    if (k == 0) mma_i8_first(d, ad, bd, idesc);
-                    else mma_i8_acc(d, ad, bd, idesc);
-                }
+            for (int q = 0; q < KS; ++q) {
+                const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[q] + 128u * (uint32_t)t);
+                const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)blo[q];
+                if (q == 0) mma_i8_first(d, ad, bd, idesc);
+                else mma_i8_acc(d, ad, bd, idesc);
             }
         }
-        mma_commit(full);
+        mma_commit(smem_u32(&ctrl->full[h]));        // arrives at once when this warp had no tile in the round
     }
     return true;
 }
@@ -529,102 +503,92 @@ __device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem,
 // Same for an arbitrary number of K-steps (descriptors rebuilt from shared memory for every tile).
 __device__ __noinline__ bool issue_phase_any(Waiter w, Ctrl *ctrl, uint32_t tmem, const IssueArgs &ia, uint32_t n_ksteps)
 {
-    const uint32_t prog = smem_u32(ctrl->prog);
-    const int sup = ia.wide ? kSupWide : kSupNarrow;
-    const uint32_t tile_cols = ia.wide ? kTileColsWide : kTileColsNarrow;
-    const uint32_t slot = (uint32_t)ia.issuer;
-    uint32_t done_upto = 0;
-    int st = (int)(((uint32_t)ia.issuer + kIssuers - (ia.ss0 % kIssuers)) % kIssuers);
-    for (; st < ia.n_super; st += kIssuers) {
-        const uint32_t use = (ia.ss0 + (uint32_t)st) / kSlots;
-        if (ia.dep_n > 0) {
-            const uint32_t need = (uint32_t)min(st + 1, ia.dep_n - 1) + 1u;
-            if (need > done_upto) {
-                if (!dep_wait(w, ctrl, prog, ia.dep_base + need, ia.dep_ss0 + need - 1)) return false;
-                done_upto = need;
-            }
-        }
-        if (use > 0 && !w.barrier(smem_u32(&ctrl->empty[slot]), (use - 1) & 1, ERR_WAIT_EMPTY)) return false;
+    for (int k = 0; k < ia.n_rounds; ++k) {
+        const uint32_t r = ia.first + (uint32_t)k, h = r & 1u;
+        if (!round_start_wait(w, ctrl, r, round_dep(ia.first, k, ia.n_rounds, ia.full_sync))) return false;
         tc_fence_after();
-        for (int j = 0; j < sup; ++j) {
-            const int t = st * sup + j;
-            if (t >= ia.n_tiles) break;
-            const uint32_t d = tmem + slot * kSlotCols + (uint32_t)j * tile_cols;
-            for (uint32_t k = 0; k < n_ksteps; ++k) {
-                const uint32_t delta = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * k));
-                const uint32_t lbo = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * k));
+        const int t0 = k * ia.tpr, t1 = min(ia.n_tiles, t0 + ia.tpr);
+        for (int t = t0 + ia.issuer; t < t1; t += kIssuers) {
+            const uint32_t d = tmem + h * kHalfCols + (uint32_t)(t - t0) * ia.tile_cols;
+            for (uint32_t q = 0; q < n_ksteps; ++q) {
+                const uint32_t delta = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_delta) + 4 * q));
+                const uint32_t lbo = warp_uniform(lds32(ia.desc + offsetof(ConvDesc, a_lbo) + 4 * q));
                 const uint64_t ad = make_desc(ia.a0 + delta + 2048u * (uint32_t)t, lbo, 128);
-                const uint64_t bd = make_desc(ia.w0 + k * ia.n_rows * 32u, 128, 256);
-                if (k == 0) mma_i8_first(d, ad, bd, ia.idesc);
+                const uint64_t bd = make_desc(ia.w0 + q * ia.n_rows * 32u, 128, 256);
+                if (q == 0) mma_i8_first(d, ad, bd, ia.idesc);
                 else mma_i8_acc(d, ad, bd, ia.idesc);
             }
         }
-        mma_commit(smem_u32(&ctrl->full[slot]));
+        mma_commit(smem_u32(&ctrl->full[h]));
     }
     return true;
 }
 
-// Warps 0..3, all lanes converged: the tensor-core work of one group (issuer 0 also loads the weights).
+// Warps 0..3, all lanes converged: the tensor-core work of one group
 __device__ __noinline__ void mma_role(const MegaParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, int it, int issuer)
 {
     Waiter w{ctrl, p.err};
-    const uint32_t prog = smem_u32(ctrl->prog);
     const uint32_t ptab = smem_u32(ctrl->ptab);
-    const uint32_t item_off = (uint32_t)it * p.items_per_group;
     const uint32_t conv_off = (uint32_t)it * p.n_conv;
     const int n_phases = p.n_phases, stop_phase = p.stop_phase, n_conv = p.n_conv;
-    uint32_t ss_next = (uint32_t)it * p.supers_per_group;      // sequence number of the phase's first super-tile
     const ConvSrc *conv_src = p.conv_src;
-    // weights of this group's first convolution (everything before the group barrier is complete)
     const bool leader = issuer == 0 && elect_one();         // the one thread that starts the weight copies
-    if (leader && !w.aborted()) issue_weights(conv_src, sbase, smem_u32(&ctrl->wbar[conv_off % 3]));
-    __syncwarp();
-    int item_base = 0, prev_item_base = 0, prev_n_items = 0;
+    uint32_t r_next = (uint32_t)it * p.rounds_per_group;      // sequence number of the next round
     uint32_t conv_index = 0;
+    bool first_round = true;
     for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
         uint4 e = ld_shared_v4(ptab + 16 * ph);
         e.x = warp_uniform(e.x); e.y = warp_uniform(e.y); e.z = warp_uniform(e.z); e.w = warp_uniform(e.w);
-        const int kind = e.x & 0xFF, full_sync = (e.x >> 8) & 1, n_items = (int)e.y, wide = (e.x >> 24) & 1;
-        if (kind == PH_CONV) {
-            // the phase before last must be complete (shared-memory reuse rule); with full_sync the last one too
-            const uint32_t end = item_off + (uint32_t)(full_sync ? item_base : prev_item_base);
-            if (!w.until([&] { return all_items_below_done(prog, end); }, ERR_WAIT_ITEMS)) return;
-            const uint32_t cg = conv_off + conv_index;
-            if (leader && (int)conv_index + 1 < n_conv) {
-                const ConvSrc *nxt = conv_src + conv_index + 1;
-                if ((int)(__ldg(&nxt->bytes_phase) >> 24) <= stop_phase)
-                    issue_weights(nxt, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
+        const int kind = e.x & 0xFF, full_sync = (e.x >> 8) & 1;
+        if (kind != PH_CONV) {
+            // a round without tensor-core work: keep the barriers in step
+            const uint32_t r = r_next++;
+            if (!round_start_wait(w, ctrl, r, r - 1u)) return;
+            if (first_round) {
+                // everything of the previous group is complete: the ring slot of this group's first weights is free
+                if (leader && !w.aborted()) issue_weights(conv_src, sbase, smem_u32(&ctrl->wbar[conv_off % 3]));
+                __syncwarp();
+                first_round = false;
             }
+            if (elect_one()) mbar_arrive(smem_u32(&ctrl->full[r & 1u]));
             __syncwarp();
-            if (!w.barrier(smem_u32(&ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS)) return;
-            // phase parameters from the head of the blob
-            const uint32_t desc = sbase + e.z;
-            uint4 h = ld_shared_v4(desc);                              // in_off, n_ksteps, idesc, n_rows
-            h.x = warp_uniform(h.x); h.y = warp_uniform(h.y); h.z = warp_uniform(h.z); h.w = warp_uniform(h.w);
-            IssueArgs ia;
-            ia.desc = desc;
-            ia.a0 = sbase + h.x + warp_uniform(lds32(desc + offsetof(ConvDesc, P_first))) * 16u;
-            ia.w0 = desc + warp_uniform(lds32(desc + offsetof(ConvDesc, weights_rel)));
-            ia.n_rows = h.w; ia.idesc = h.z; ia.n_super = n_items; ia.n_tiles = (int)e.w;
-            ia.dep_base = item_off + (uint32_t)prev_item_base;
-            ia.dep_n = full_sync ? 0 : prev_n_items;
-            ia.dep_ss0 = ss_next - (uint32_t)prev_n_items;     // the producing phase is the conv phase just before
-            ia.ss0 = ss_next; ia.wide = wide;
-            ia.issuer = issuer;
-            bool ok;
-            switch (h.y) {
-            case 1: ok = issue_phase<1>(w, ctrl, tmem, ia); break;
-            case 5: ok = issue_phase<5>(w, ctrl, tmem, ia); break;
-            case 9: ok = issue_phase<9>(w, ctrl, tmem, ia); break;
-            case 18: ok = issue_phase<18>(w, ctrl, tmem, ia); break;
-            default: ok = issue_phase_any(w, ctrl, tmem, ia, h.y); break;
-            }
-            if (!ok) return;
-            conv_index += 1;
-            ss_next += (uint32_t)n_items;
+            continue;
         }
-        prev_item_base = item_base; prev_n_items = n_items;
-        item_base += n_items;
+        const int n_rounds = (int)(e.y & 0xFF), tpr = (int)((e.y >> 8) & 0xFF);
+        const uint32_t cg = conv_off + conv_index;
+        // operands and the ring slot of the next weights: wait for the first round's start conditions here, so
+        // that the copy of the next phase's weights is under way before this phase's tiles are issued
+        if (!round_start_wait(w, ctrl, r_next, round_dep(r_next, 0, n_rounds, full_sync))) return;
+        if (leader && (int)conv_index + 1 < n_conv) {
+            const ConvSrc *nxt = conv_src + conv_index + 1;
+            if ((int)(__ldg(&nxt->bytes_phase) >> 24) <= stop_phase)
+                issue_weights(nxt, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
+        }
+        __syncwarp();
+        if (!w.barrier(smem_u32(&ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS)) return;
+        // phase parameters from the head of the blob
+        const uint32_t desc = sbase + e.z;
+        uint4 h = ld_shared_v4(desc);                              // in_off, n_ksteps, idesc, n_rows
+        h.x = warp_uniform(h.x); h.y = warp_uniform(h.y); h.z = warp_uniform(h.z); h.w = warp_uniform(h.w);
+        IssueArgs ia;
+        ia.desc = desc;
+        ia.a0 = sbase + h.x + warp_uniform(lds32(desc + offsetof(ConvDesc, P_first))) * 16u;
+        ia.w0 = desc + warp_uniform(lds32(desc + offsetof(ConvDesc, weights_rel)));
+        ia.n_rows = h.w; ia.idesc = h.z; ia.n_rounds = n_rounds; ia.tpr = tpr; ia.n_tiles = (int)e.w;
+        ia.tile_cols = (e.y >> 16) & 0xFF;
+        ia.first = r_next; ia.full_sync = full_sync; ia.issuer = issuer;
+        bool ok;
+        switch (h.y) {
+        case 1: ok = issue_phase<1>(w, ctrl, tmem, ia); break;
+        case 5: ok = issue_phase<5>(w, ctrl, tmem, ia); break;
+        case 9: ok = issue_phase<9>(w, ctrl, tmem, ia); break;
+        case 18: ok = issue_phase<18>(w, ctrl, tmem, ia); break;
+        default: ok = issue_phase_any(w, ctrl, tmem, ia, h.y); break;
+        }
+        if (!ok) return;
+        conv_index += 1;
+        r_next += (uint32_t)n_rounds;
+        first_round = false;
     }
 }
 
@@ -635,21 +599,6 @@ struct EpiCtx {
     uint32_t sbase, tmem;
     int warp_e, wg, quarter, lane, tid_wg;
 };
-
-// Progress counter of a warp: the index of the next item it still has work in.  Every item below the minimum
-// over all warps is therefore complete.  `finish_item` publishes after work (shared-memory writes are fenced for
-// the tensor core's reads first), `skip_to` when there was none.
-__device__ __forceinline__ void finish_item(const EpiCtx &c, uint32_t next_item)
-{
-    fence_proxy_async();
-    __syncwarp();
-    if (c.lane == 0) st_release(smem_u32(&c.ctrl->prog[c.warp_e]), next_item);
-}
-__device__ __forceinline__ void skip_to(const EpiCtx &c, uint32_t next_item)
-{
-    __syncwarp();
-    if (c.lane == 0) st_release(smem_u32(&c.ctrl->prog[c.warp_e]), next_item);
-}
 
 __device__ void fill_item(uint32_t fill_off, uint32_t bytes_halo, const EpiCtx &c, int i)
 {
@@ -815,65 +764,69 @@ __device__ __forceinline__ void chunk_compute(const int (&acc)[SUP][16], const C
     }
 }
 
-// The super-tiles of one CONV phase that fall to this warpgroup: those whose sequence number, hence slot, is
-// the warpgroup's index mod 2.  The loops over pairs of tiles and over 16-channel chunks are kept rolled on
-// purpose: their body (32 outputs per thread) is a few KB of code, so the two epilogue warps and the issuing
-// warp of a scheduler all run out of its instruction cache; a fully unrolled super-tile does not fit and
-// leaves the warps waiting for instruction fetches.  The slot is released after the warp's last read of it,
-// so the tensor cores refill it while the last chunk is still being requantised; the warpgroups never meet.
+// End of a round for an epilogue warp: its shared-memory writes become visible to the tensor cores' reads, its
+// tensor-memory reads are ordered before the arrival, and the round counts as complete once all eight warps are here.
+__device__ __forceinline__ void round_done(const EpiCtx &c, uint32_t r)
+{
+    tc_fence_before();
+    fence_proxy_async();
+    __syncwarp();
+    if (c.lane == 0) mbar_arrive(smem_u32(&c.ctrl->done[r & 1u]));
+}
+
+// The rounds of one CONV phase.  A warp owns 32 rows (its tensor-memory lanes) of every tile; the two warpgroups
+// split a round's tiles pair by pair when the phase has one 16-channel chunk, and chunk by chunk otherwise, so
+// that both have the same amount of work in every round.  The loops over pairs and chunks are kept rolled on
+// purpose: their body (32 outputs per thread) is a few KB of code and stays in the instruction cache; a fully
+// unrolled round does not and leaves the warps waiting for instruction fetches.
 template <bool kRes, bool kResHigh, bool kLo>
-__device__ __noinline__ void conv_phase_items(Waiter w, const EpiCtx &c_in, const ConvRegs &R_in, int n_super, int n_tiles,
-                                              uint32_t ss0, uint32_t first_item, int sup)
+__device__ __noinline__ void conv_phase_rounds(Waiter w, const EpiCtx &c_in, const ConvRegs &R_in, int n_rounds, int tpr,
+                                               int n_tiles, uint32_t first, uint32_t tile_cols)
 {
     // private copies: values reached through references would be re-read after every barrier or fence
     const EpiCtx c = c_in;
     const ConvRegs R = R_in;
-    const uint32_t tile_cols = (uint32_t)kSlotCols / (uint32_t)sup;
-    const int n_pairs = sup >> 1;
-    const uint32_t full0 = smem_u32(&c.ctrl->full[0]), empty0 = smem_u32(&c.ctrl->empty[0]);
-    const uint32_t done0 = smem_u32(&c.ctrl->done[0]);
     const uint32_t lane_base = c.tmem + ((uint32_t)(c.quarter * 32) << 16);
     const uint32_t n_chunks = R.n_chunks;
+    const bool by_chunk = (n_chunks & 1u) == 0;
+    const uint32_t ch0 = by_chunk ? (uint32_t)c.wg : 0u, ch_step = by_chunk ? (uint32_t)kWarpGroups : 1u;
     bool ok = true;
-    for (int st = (int)(((uint32_t)c.wg + 2u - (ss0 & 1u)) & 1u); st < n_super; st += kWarpGroups) {
-        const uint32_t ss = ss0 + (uint32_t)st, slot = ss % kSlots;
-        if (ok) ok = w.barrier(full0 + 8 * slot, (ss / kSlots) & 1, ERR_WAIT_FULL);
+    for (int k = 0; k < n_rounds; ++k) {
+        const uint32_t r = first + (uint32_t)k, h = r & 1u;
+        const int t0 = k * tpr, t1 = min(n_tiles, t0 + tpr);
+        if (ok) ok = w.barrier(smem_u32(&c.ctrl->full[h]), (r >> 1) & 1u, ERR_WAIT_FULL);
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
-        const uint32_t slot_addr = lane_base + slot * kSlotCols;
+        const uint32_t half_addr = lane_base + h * kHalfCols;
+        const int n_pairs = (t1 - t0 + 1) >> 1;
 #pragma unroll 1
-        for (int pr = 0; pr < n_pairs; ++pr) {
-            const Spots<2> sp = locate<2>(R, c, st * n_pairs + pr, n_tiles);
-            const uint32_t pair_addr = slot_addr + (uint32_t)(2 * pr) * tile_cols;
+        for (int pr = by_chunk ? 0 : c.wg; pr < n_pairs; pr += by_chunk ? 1 : kWarpGroups) {
+            // t0 is even, so pair pr of the round is pair t0 / 2 + pr of the phase; tiles from t1 on are not stored
+            const Spots<2> sp = locate<2>(R, c, (t0 >> 1) + pr, t1);
+            const uint32_t pair_addr = half_addr + (uint32_t)(2 * pr) * tile_cols;
 #pragma unroll 1
-            for (uint32_t ch = 0; ch < n_chunks; ++ch) {
+            for (uint32_t ch = ch0; ch < n_chunks; ch += ch_step) {
                 int acc[2][16];
                 tmem_ld16_issue(pair_addr + ch * 16, acc[0]);
                 tmem_ld16_issue(pair_addr + tile_cols + ch * 16, acc[1]);
                 tmem_ld_wait();
-                if (pr + 1 == n_pairs && ch + 1 == n_chunks) {      // last read of the slot by this warp
-                    tc_fence_before();
-                    __syncwarp();
-                    if (c.lane == 0) mbar_arrive(empty0 + 8 * slot);
-                }
                 if (ok) chunk_compute<kRes, kResHigh, kLo, 2>(acc, R, c, sp, ch);
             }
         }
-        finish_item(c, first_item + (uint32_t)min(st + kWarpGroups, n_super));
-        if (c.lane == 0) mbar_arrive(done0 + 8 * slot);
+        round_done(c, r);
     }
 }
 
-__device__ __forceinline__ void conv_phase_dispatch(Waiter w, const EpiCtx &c, const ConvRegs &R, int n_super, int n_tiles,
-                                                    uint32_t ss0, uint32_t first, int sup)
+__device__ __forceinline__ void conv_phase_dispatch(Waiter w, const EpiCtx &c, const ConvRegs &R, int n_rounds, int tpr,
+                                                    int n_tiles, uint32_t first, uint32_t tile_cols)
 {
     switch (R.mode & 7u) {
-    case 0: conv_phase_items<false, false, false>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
-    case 1: conv_phase_items<false, false, true>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
-    case 2: conv_phase_items<true, false, false>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
-    case 3: conv_phase_items<true, false, true>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
-    case 6: conv_phase_items<true, true, false>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
-    default: conv_phase_items<true, true, true>(w, c, R, n_super, n_tiles, ss0, first, sup); break;
+    case 0: conv_phase_rounds<false, false, false>(w, c, R, n_rounds, tpr, n_tiles, first, tile_cols); break;
+    case 1: conv_phase_rounds<false, false, true>(w, c, R, n_rounds, tpr, n_tiles, first, tile_cols); break;
+    case 2: conv_phase_rounds<true, false, false>(w, c, R, n_rounds, tpr, n_tiles, first, tile_cols); break;
+    case 3: conv_phase_rounds<true, false, true>(w, c, R, n_rounds, tpr, n_tiles, first, tile_cols); break;
+    case 6: conv_phase_rounds<true, true, false>(w, c, R, n_rounds, tpr, n_tiles, first, tile_cols); break;
+    default: conv_phase_rounds<true, true, true>(w, c, R, n_rounds, tpr, n_tiles, first, tile_cols); break;
     }
 }
 
@@ -938,60 +891,50 @@ __device__ void tail_sample(const MegaParams &p, const EpiCtx &c, int s, bool co
 }
 
 // Epilogue warps: all non-tensor-core work of one group.  Item g of a FILL / INPUT / TAIL phase belongs to
-// warpgroup g mod 2; CONV items are split as described above.  A warp only visits the items it has work in and
-// publishes, as its progress, the index of the next such item.
+// warpgroup g mod 2; the outputs of a CONV round are split as described above.
 __device__ __noinline__ void epi_role(const MegaParams &p, EpiCtx &c, int it, int grp)
 {
     Waiter w{c.ctrl, p.err};
-    const uint32_t prog = smem_u32(c.ctrl->prog);
     const uint32_t ptab = smem_u32(c.ctrl->ptab);
-    const uint32_t item_off = (uint32_t)it * p.items_per_group;
     const uint32_t conv_off = (uint32_t)it * p.n_conv;
     const int n_phases = p.n_phases, stop_phase = p.stop_phase, G = p.G;
-    uint32_t item_base = 0, conv_index = 0;
-    uint32_t ss_next = (uint32_t)it * p.supers_per_group;
+    uint32_t r_next = (uint32_t)it * p.rounds_per_group, conv_index = 0;
     for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
         const uint4 e = ld_shared_v4(ptab + 16 * ph);
-        const int kind = e.x & 0xFF, n_items = (int)e.y;
-        const uint32_t first = item_off + item_base, end = first + (uint32_t)n_items;
-        item_base += (uint32_t)n_items;
+        const int kind = e.x & 0xFF;
         bool ok;
         if (kind == PH_CONV) {
-            const bool wide = (e.x >> 24) & 1;
-            const uint32_t cg = conv_off + conv_index, ss0 = ss_next;
+            const int n_rounds = (int)(e.y & 0xFF), tpr = (int)((e.y >> 8) & 0xFF);
+            const uint32_t cg = conv_off + conv_index, first = r_next;
             conv_index += 1;
-            ss_next += (uint32_t)n_items;
-            // first item with work for this warpgroup
-            const uint32_t own = ((uint32_t)c.wg + 2u - (ss0 & 1u)) & 1u;
-            skip_to(c, min(first + own, end));
-            if (first + own >= end) continue;
+            r_next += (uint32_t)n_rounds;
             ok = w.barrier(smem_u32(&c.ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) { skip_to(c, end); continue; }
+            if (!ok) {                       // keep the barriers in step so that nobody waits for this warp
+                for (int k = 0; k < n_rounds; ++k) round_done(c, first + (uint32_t)k);
+                continue;
+            }
             const ConvRegs R = load_conv_regs(c.sbase + e.z, G);
-            const int n_tiles = (int)e.w;
-            conv_phase_dispatch(w, c, R, n_items, n_tiles, ss0, first, wide ? kSupWide : kSupNarrow);
+            conv_phase_dispatch(w, c, R, n_rounds, tpr, (int)e.w, first, (e.y >> 16) & 0xFF);
             continue;
         }
-        const uint32_t own = ((uint32_t)c.wg + kWarpGroups - (first % kWarpGroups)) % kWarpGroups;
-        skip_to(c, min(first + own, end));
-        if (first + own >= end) continue;
-        ok = w.until([&] { return all_items_below_done(prog, first); }, ERR_WAIT_ITEMS);
+        // a round of its own: every earlier round must be complete in all warps, then the items are shared out
+        const uint32_t r = r_next++;
+        const int n_items = (int)e.y;
+        ok = r == 0u || w.barrier(smem_u32(&c.ctrl->done[(r & 1u) ^ 1u]), ((r - 1u) >> 1) & 1u, ERR_WAIT_ITEMS);
         ok = __all_sync(0xffffffffu, ok);
-        for (uint32_t g = first + own; g < end; g += kWarpGroups) {
-            const int i = (int)(g - first);
-            if (ok) {
-                if (kind == PH_FILL) {
-                    fill_item(e.z, e.w, c, i);
-                } else if (kind == PH_INPUT) {
-                    input_item(p, c, i, grp);
-                } else {
-                    const int s = i * 4 + (c.warp_e & 3);
-                    tail_sample(p, c, min(s, G - 1), s < G, grp);
-                }
+        for (int i = c.wg; i < n_items; i += kWarpGroups) {
+            if (!ok) break;
+            if (kind == PH_FILL) {
+                fill_item(e.z, e.w, c, i);
+            } else if (kind == PH_INPUT) {
+                input_item(p, c, i, grp);
+            } else {
+                const int s = i * 4 + (c.warp_e & 3);
+                tail_sample(p, c, min(s, G - 1), s < G, grp);
             }
-            finish_item(c, min(g + kWarpGroups, end));
         }
+        round_done(c, r);
     }
 }
 
@@ -1002,17 +945,15 @@ __global__ void __launch_bounds__(kThreads, 1) k_mega(const __grid_constant__ Me
     const uint32_t sbase = smem_u32(smem);
     const int warp = (int)warp_uniform(threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSlots; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), 1);             // the super-tile's issuing thread
-            mbar_init(smem_u32(&ctrl->empty[s]), 4);            // the four warps of the slot's warpgroup
-            mbar_init(smem_u32(&ctrl->done[s]), 4);             // the same, when the super-tile's outputs are stored
+        for (int s = 0; s < kHalves; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), kIssuers);      // every issuing warp commits (or arrives) once per round
+            mbar_init(smem_u32(&ctrl->done[s]), kEpiWarps);     // every epilogue warp arrives once per round
         }
         for (int s = 0; s < 3; ++s) mbar_init(smem_u32(&ctrl->wbar[s]), 1);
         mbar_init(smem_u32(&ctrl->drain), kIssuers);
         ctrl->abort_flag = 0;
     }
     for (int i = threadIdx.x; i < 128; i += blockDim.x) ctrl->hist[i] = 0;
-    if (threadIdx.x < kEpiWarps) ctrl->prog[threadIdx.x] = 0;
     for (int i = threadIdx.x; i < p.n_phases; i += blockDim.x) ctrl->ptab[i] = p.ptab[i];
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), 512);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1105,7 +1046,7 @@ struct MegaPlan {
     int G = 0, in_c = 0, in_h = 0, in_w = 0, n_classes = 0;
     std::vector<MPhase> phases;
     std::vector<int> conv_phase;
-    int items_per_group = 0, supers_per_group = 0;
+    int rounds_per_group = 0;
     uint32_t smem_bytes = 0;
     MegaParams base;                      // fields that do not change between launches
     // device copies
@@ -1323,7 +1264,7 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
     plan->tensors = T;
     plan->tensor_off.assign(T.size(), 0);
     for (int t = 0; t <= n_conv_layers; ++t) plan->tensor_off[(size_t)t] = buffers[(size_t)T[(size_t)t].buffer].off;
-    int item_base = 0, super_base = 0, last_wide = -1;
+    int item_base = 0, round_base = 0, last_cols = -1;
     blob_out->clear();
     blob_offsets->assign((size_t)n_conv, 0);
     bool magic_ok = true;
@@ -1371,11 +1312,16 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             const uint32_t consts_rel = weights_rel + P.n_ksteps * (uint32_t)P.n_rows * 32u;
             P.const_off = P.w_off + consts_rel;
             P.conv_index = (uint32_t)cidx;
-            P.wide = P.n_rows > kTileColsNarrow ? 1 : 0;
-            if (P.n_rows > kTileColsWide) return false;
-            const int sup = P.wide ? kSupWide : kSupNarrow;
-            P.n_items = (in.n_tiles + sup - 1) / sup;             // one item per super-tile
-            super_base += P.n_items;
+            // rounds: at most half of tensor memory each, at least two per phase so that the tensor cores work on
+            // one half while the other is requantised, an even number of tiles in all but the last
+            if (P.n_rows > kMaxFusedCols) return false;
+            const int tile_cols = tile_columns(P.n_rows), per_half = kHalfCols / tile_cols;
+            int n_rounds = std::max((in.n_tiles + per_half - 1) / per_half, in.n_tiles >= 2 ? 2 : 1);
+            P.tiles_per_round = ((in.n_tiles + n_rounds - 1) / n_rounds + 1) & ~1;
+            P.n_rounds = (in.n_tiles + P.tiles_per_round - 1) / P.tiles_per_round;
+            if (P.tiles_per_round > per_half || P.n_rounds > 255) return false;
+            P.n_items = P.n_rounds;
+            round_base += P.n_rounds;
             for (uint32_t k = 0; k < P.n_ksteps; ++k) {
                 const auto &kp = ksteps[(size_t)cidx][k];
                 P.a_delta[k] = chunk_addr[(size_t)cidx][(size_t)kp.first];
@@ -1395,8 +1341,8 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             bool tile_rule = prev_is_conv && in.producer_phase == ph - 1 && !in.scatter_produced;
             if (L.res_tensor >= 0 && T[(size_t)L.res_tensor].producer_phase >= ph - 1) tile_rule = false;
             if (tile_rule && plan->phases[(size_t)ph - 1].n_tiles != P.n_tiles) tile_rule = false;
-            if (P.wide != last_wide) tile_rule = false;      // super-tiles of another size: no item-for-item rule
-            last_wide = P.wide;
+            if (tile_cols != last_cols) tile_rule = false;   // rounds of another size: no round-for-round rule
+            last_cols = tile_cols;
             P.full_sync = tile_rule ? 0 : 1;
             // epilogue chunks and the weight blob
             const int lay[2] = {nd.layer, nd.fused_layer};
@@ -1477,12 +1423,12 @@ bool plan_for_G(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             blob_out->insert(blob_out->end(), blob.begin(), blob.end());
             while (blob_out->size() % 128) blob_out->push_back(0);
         }
+        if (S.kind != PH_CONV) round_base += 1;
         item_base += P.n_items;
     }
     if (!magic_ok) return false;
     plan->G = G;
-    plan->items_per_group = item_base;
-    plan->supers_per_group = super_base;
+    plan->rounds_per_group = round_base;
     plan->smem_bytes = (high + 127u) & ~127u;
     return true;
 }
@@ -1555,8 +1501,10 @@ int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
     for (size_t i = 0; i < ptab.size(); ++i) {
         const MPhase &P = plan->phases[i];
         ptab[i].kind_sync = (uint32_t)P.kind | ((uint32_t)(P.full_sync ? 1 : 0) << 8) |
-                            (P.kind == PH_CONV ? (P.n_chunks << 16) | ((uint32_t)P.wide << 24) : 0u);
-        ptab[i].n_items = (uint32_t)P.n_items;
+                            (P.kind == PH_CONV ? (P.n_chunks << 16) : 0u);
+        ptab[i].n_items = P.kind == PH_CONV ? (uint32_t)P.n_rounds | ((uint32_t)P.tiles_per_round << 8) |
+                                                  ((uint32_t)tile_columns(P.n_rows) << 16)
+                                            : (uint32_t)P.n_items;
         ptab[i].a = P.kind == PH_CONV ? P.w_off : P.fill_off;
         ptab[i].b = P.kind == PH_FILL ? (P.fill_bytes | ((P.fill_word & 0xFFu) << 24))
                                       : P.kind == PH_CONV ? (uint32_t)P.n_tiles : 0u;
@@ -1584,8 +1532,7 @@ int mega_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
     b.in_H = plan->tensors[0].H; b.in_W = plan->tensors[0].W; b.in_Wp = plan->tensors[0].Wp; b.in_HsWp = plan->tensors[0].HsWp;
     b.n_phases = (int)plan->phases.size();
     b.n_conv = (int)plan->conv_phase.size();
-    b.items_per_group = plan->items_per_group;
-    b.supers_per_group = plan->supers_per_group;
+    b.rounds_per_group = plan->rounds_per_group;
     b.G = plan->G;
     b.in_c = in_c;
     b.input_off = plan->tensor_off[0];
