@@ -1,0 +1,1490 @@
+// Line-tiled shared-memory-resident tensor-core engine (sm_100a) for CIFAR-shaped residual networks.
+//
+// One persistent CTA per SM carries a group of four noisy samples through the whole network.  Activations
+// stay in shared memory, every convolution is an implicit GEMM on tcgen05 (kind::i8, int32 accumulators in
+// tensor memory) and only vote counts return to global memory (Algorithm 1 steps 1-4, Algorithm 2 steps 1-2).
+//
+// Layout.  A tensor of C channels and H x W pixels (W = 32, 16 or 8) is stored per plane of 16 channels as
+// "lines" of 128 positions of 16 bytes.  Position x * I + b * 4 + s of line l holds pixel (row l + b * L, column x)
+// of sample s, where I = 128 / W positions belong to one column, I / 4 row bands b share a line and L = H / (I / 4)
+// is the number of lines.  Lines are I positions apart from each other (a gap that always holds the zero-point:
+// the left and right padding of every row), there is one more line above and below (the padding rows of the
+// first and last band; for the other bands these two lines hold copies of the neighbouring band's edge rows,
+// written together with the originals), so
+//   * the horizontal neighbours of all 128 positions of a line are the same 128 positions moved by +-I, and
+//   * the vertical neighbours of all 128 positions of line l are the same 128 positions of line l +- 1.
+// A line is therefore an M = 128 operand tile whose nine filter taps are plain address offsets, with every one
+// of its rows a real output pixel.
+//
+// Stacked convolutions.  For a 3x3, stride-1 convolution the three vertical taps are stacked along N: one MMA
+// chain over input line p (K = three horizontal taps x input channels) accumulates into the accumulator
+// columns of output lines p-1, p, p+1 at once (N = 3 x cout), because the accumulators of consecutive output
+// lines are consecutive column blocks of tensor memory.  The epilogue zeroes a line's columns after reading
+// them.  This triples N for the small channel counts where an MMA is bound by fetching its 128 x 32-byte A
+// operand.  Strided and 1x1 convolutions, and those with cout = 64, run unstacked: one chain per output line
+// over all taps.
+//
+// Roles.  Warp 16 issues the MMAs of one convolution after the other (a table of operations prepared on the
+// host: input line, accumulator columns, which lines of the previous convolution it must wait for, which
+// output lines it completes).  Warps 0..15 requantise: four sets of four warps (one per 32-lane quarter of
+// tensor memory) share the output lines of a convolution in the order in which they complete.  Producer and
+// consumer meet on one mbarrier pair per output line (accumulators ready / line stored), so consecutive
+// convolutions overlap line by line.  Input noise (Def. 3.3, Eq. 2; Def. 3.4), halo fills and the pool / FC /
+// argmax tail are CTA-wide phases between barriers.
+//
+// Every device-side wait is bounded by a wall-clock limit; on expiry the CTA raises an abort flag, all
+// remaining waits fall through, and the host reports ISC_ERR_TIMEOUT.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <map>
+#include <vector>
+
+#include "isc_line.h"
+#include "isc_tc.cuh"
+
+namespace isc {
+
+using namespace tc;
+
+namespace {
+
+#ifdef ISC_TRACE
+// Timeline instrumentation, compiled only with -DISC_TRACE: CTA 0 records (warp and event, tag, SM clock).
+constexpr unsigned kTraceMax = 32768;
+__device__ unsigned long long g_ltrace[3 * kTraceMax];
+__device__ unsigned int g_ltrace_n, g_ltrace_lo, g_ltrace_hi;
+__device__ __forceinline__ void ltrace(int ev, uint32_t cg, uint32_t tag)
+{
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && cg >= g_ltrace_lo && cg < g_ltrace_hi) {
+        const unsigned i = atomicAdd(&g_ltrace_n, 1u);
+        if (i < kTraceMax) {
+            g_ltrace[3 * i] = (unsigned long long)(ev | ((threadIdx.x >> 5) << 8));
+            g_ltrace[3 * i + 1] = ((unsigned long long)cg << 16) | tag;
+            g_ltrace[3 * i + 2] = (unsigned long long)clock64();
+        }
+    }
+}
+#else
+#define ltrace(ev, cg, tag) ((void)0)
+#endif
+
+constexpr int kG = 4;                       // samples per group
+constexpr int kEpiWarps = 16;               // warps 0..15: epilogue; set = warp / 4, tensor-memory quarter = warp % 4
+constexpr int kSets = kEpiWarps / 4;
+constexpr int kIssuerWarp = kEpiWarps;      // warp 16: MMA issue and weight copies
+constexpr int kThreads = 32 * (kEpiWarps + 1);
+constexpr int kEpiThreads = 32 * kEpiWarps;
+constexpr int kMaxKsteps = 18;
+constexpr int kMaxPhases = 160;
+constexpr int kMaxBars = 192;
+constexpr int kMaxLines = 32;               // output lines of one convolution
+constexpr int kCtrlBytes = 5120;
+constexpr int kSmemLimit = 227 * 1024;
+constexpr int kTmemCols = 512;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+
+enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
+enum { ERR_NONE = 0, ERR_WAIT_DONE = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_FULL = 4, ERR_WAIT_DRAIN = 5 };
+enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8 };
+enum { OPF_WAIT_ALL = 1 };
+
+// ---- what the kernel reads -------------------------------------------------------------------
+
+// One entry per phase, copied to shared memory when the kernel starts.
+//   CONV: a = shared-memory offset of the blob      FILL: a = offset, b = bytes, c = halo byte
+struct alignas(16) PhaseEntry { uint32_t kind, a, b, c; };
+
+// Where the blob of convolution c comes from (global) and goes to (shared).
+struct alignas(16) ConvSrc { unsigned long long gmem; uint32_t bytes_phase, smem_off; };   // bytes | phase << 24
+
+// One MMA chain: input line, accumulator columns, dependencies and completions.
+struct alignas(16) LOp {
+    uint8_t a_line1;        // input line + 1 (line -1 is the padding line above)
+    uint8_t b_block;        // first weight block (stacked: 2 - vertical tap of the lowest output line)
+    uint8_t n_blocks;       // N = n_blocks * cout
+    uint8_t flags;          // OPF_WAIT_ALL: every line of the previous convolution
+    uint16_t d_col;         // first accumulator column within the bank
+    uint8_t n_wait, n_commit;
+    uint8_t wait[4];        // output lines of the previous convolution that must be stored
+    uint8_t commit[4];      // output lines of this convolution whose accumulators are complete after the chain
+};
+static_assert(sizeof(LOp) == 16, "one operation is one 16-byte load");
+
+// Head of every blob: everything the issuing thread and the epilogue need to know about the convolution.
+struct alignas(16) LConvDesc {
+    uint32_t n_ops, n_passes, n_ksteps, flags;
+    uint32_t a_base, pitch16, bblock16, n_banks;            // a_base: line -1, lane 0, plane 0 of the input
+    uint32_t idesc[3], cols;                                // instruction descriptors for 1, 2, 3 blocks; columns per line
+    uint32_t d_base[2], bar_full, bar_done;                 // accumulator bank bases; barrier indices of this class
+    uint32_t use_local, uses_per_group, n_lines, n_chunks;
+    uint32_t w_rel, c_rel, ops_rel, passes_rel;
+    // epilogue: where results go (line 0, lane 0, plane 0), geometry of the output and of the scattered input
+    uint32_t out_base, out_plane, out_pitch16, out_n_lines;
+    uint32_t out_log_lines, out_nb, out_logI, res_base;
+    uint32_t res_plane, in_logI, in_I, in_n_lines;
+    int32_t lo; uint32_t res_m2, res_r2_lo, res_r2_hi;
+    int32_t a_delta[kMaxKsteps];
+    uint32_t a_lbo[kMaxKsteps];
+};
+static_assert(sizeof(LConvDesc) % 16 == 0, "blob sections stay 16-byte aligned");
+
+struct FcConst { int32_t mult, n, zp_out, lo, bias, pad0, pad1, pad2; };
+
+struct LineParams {
+    const PhaseEntry *ptab;
+    const ConvSrc *conv_src;
+    const uint8_t *bar_counts;
+    int32_t n_bars, n_phases, n_conv, n_groups;
+    int32_t n_samples, in_c, in_H, in_W;
+    const uint8_t *x;                 // clean image, CHW
+    NoiseStream ns;
+    uint32_t input_base, input_pitch16;   // line 0, lane 0 of the first layer's operand region
+    // tail
+    uint32_t tail_base, tail_plane, tail_pitch16, tail_logI;
+    int32_t tail_C, tail_H, tail_W, tail_n_lines;
+    int32_t pool_mult, pool_n, pool_zp_in, pool_zp_out, pool_lo;
+    const int8_t *fc_w;               // [n_classes][64]
+    const FcConst *fc_c;
+    int32_t n_classes;
+    int32_t *counts;
+    int8_t *logits;                   // [n_samples][n_classes] or null
+    int32_t *err;
+    // debug
+    int32_t stop_phase;
+    uint32_t dump_off, dump_bytes;
+    uint8_t *dump;
+};
+
+struct Ctrl {
+    unsigned long long bars[kMaxBars];
+    unsigned long long wbar[3], drain;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+    int32_t hist[128];
+    PhaseEntry ptab[kMaxPhases];
+};
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
+
+// ------------------------------------------------------------------ device helpers
+
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void commit_to(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_st16_zero(uint32_t taddr)
+{
+    const int z = 0;
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+                 ::"r"(taddr), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ long long mad_wide_u(uint32_t a, uint32_t b, long long c)
+{
+    long long d;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+// byte K of w, zero-extended
+template <int K>
+__device__ __forceinline__ uint32_t ubyte(uint32_t w)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(w), "n"(0x4440 | K));
+    return d;
+}
+
+struct Waiter {
+    Ctrl *ctrl;
+    int32_t *err;
+    __device__ __forceinline__ bool aborted() const { return ctrl->abort_flag != 0; }
+    // the error word: wait kind | index of the barrier within the control block << 8 | parity waited for << 20 | CTA << 21
+    __device__ __noinline__ void fail(int code, uint32_t bar, uint32_t parity)
+    {
+        ctrl->abort_flag = 1;
+        const uint32_t idx = (bar - smem_u32(ctrl)) >> 3;
+        atomicCAS(err, 0, (int)((uint32_t)code | ((idx & 0xFFFu) << 8) | ((parity & 1u) << 20) | (blockIdx.x << 21)));
+    }
+    // Wait for a phase of an mbarrier.  Each attempt parks the thread in hardware for a bounded time,
+    // so a waiting warp does not compete for issue slots.
+    __device__ __forceinline__ bool barrier(uint32_t bar, uint32_t parity, int code)
+    {
+        if (mbar_test(bar, parity)) return true;
+        const unsigned long long t0 = globaltimer();
+        for (int spin = 0;; ++spin) {
+            if (mbar_try(bar, parity)) return true;
+            if ((spin & 7) == 7) {
+                if (aborted()) return false;
+                if (globaltimer() - t0 > kWaitLimitNs) { fail(code, bar, parity); return false; }
+            }
+        }
+    }
+};
+
+// ------------------------------------------------------------------ issuing thread
+
+struct PrevConv { uint32_t done_addr, parity, n_lines; };      // n_lines = 0: nothing to wait for
+
+struct IssueCtx {
+    uint32_t desc, ops, n_ops, a0, w0, pitch16, bblock16, kstep_bytes, d0, stacked, full_addr, cg;
+    uint32_t idesc[3];
+};
+
+template <int KS>
+__device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const PrevConv &prev, uint32_t n_ksteps)
+{
+    constexpr int NK = KS > 0 ? KS : 1;
+    uint32_t alo[NK], blo[NK];
+    const uint32_t ahi = (uint32_t)(make_desc(0, 0, 128) >> 32), bhi = (uint32_t)(make_desc(0, 128, 256) >> 32);
+    if (KS > 0) {
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const uint32_t delta = lds32(ic.desc + offsetof(LConvDesc, a_delta) + 4 * k);
+            const uint32_t lbo = lds32(ic.desc + offsetof(LConvDesc, a_lbo) + 4 * k);
+            alo[k] = (uint32_t)make_desc(ic.a0 + delta, lbo, 128);
+            blo[k] = (uint32_t)make_desc(ic.w0 + (uint32_t)k * ic.kstep_bytes, 128, 256);
+        }
+    }
+    uint4 o = ld_shared_v4(ic.ops);
+    for (uint32_t i = 0; i < ic.n_ops; ++i) {
+        const uint4 cur = o;
+        if (i + 1 < ic.n_ops) o = ld_shared_v4(ic.ops + 16 * (i + 1));
+        const uint32_t a_line1 = cur.x & 0xFF, b_block = (cur.x >> 8) & 0xFF, n_blocks = (cur.x >> 16) & 0xFF, flags = cur.x >> 24;
+        const uint32_t d_col = cur.y & 0xFFFF, n_wait = (cur.y >> 16) & 0xFF, n_commit = cur.y >> 24;
+        if (prev.n_lines) {
+            if (flags & OPF_WAIT_ALL) {
+                for (uint32_t l = 0; l < prev.n_lines; ++l)
+                    if (!w.barrier(prev.done_addr + 8 * l, prev.parity, ERR_WAIT_DONE)) return false;
+            }
+            for (uint32_t q = 0; q < n_wait; ++q)
+                if (!w.barrier(prev.done_addr + 8 * ((cur.z >> (8 * q)) & 0xFF), prev.parity, ERR_WAIT_DONE)) return false;
+        }
+        ltrace(1, ic.cg, a_line1);
+        tc_fence_after();
+        const uint32_t d = ic.d0 + d_col, idesc = ic.idesc[n_blocks - 1];
+        const uint32_t a_add = a_line1 * ic.pitch16, b_add = b_block * ic.bblock16;
+        if (KS > 0) {
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[k] + a_add);
+                const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)(blo[k] + b_add);
+                mma_i8(d, ad, bd, idesc, ic.stacked | (uint32_t)(k > 0));
+            }
+        } else {
+            for (uint32_t k = 0; k < n_ksteps; ++k) {
+                const uint32_t delta = lds32(ic.desc + offsetof(LConvDesc, a_delta) + 4 * k);
+                const uint32_t lbo = lds32(ic.desc + offsetof(LConvDesc, a_lbo) + 4 * k);
+                const uint64_t ad = make_desc(ic.a0 + delta + a_add * 16u, lbo, 128);
+                const uint64_t bd = make_desc(ic.w0 + k * ic.kstep_bytes + b_add * 16u, 128, 256);
+                mma_i8(d, ad, bd, idesc, ic.stacked | (uint32_t)(k > 0));
+            }
+        }
+        for (uint32_t q = 0; q < n_commit; ++q) commit_to(ic.full_addr + 8 * ((cur.w >> (8 * q)) & 0xFF));
+        ltrace(2, ic.cg, a_line1);
+    }
+    return true;
+}
+
+__device__ __forceinline__ void issue_weights(const ConvSrc *src, uint32_t sbase, uint32_t wbar_addr)
+{
+    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
+    const void *gmem = reinterpret_cast<const void *>(((unsigned long long)v.y << 32) | v.x);
+    const uint32_t bytes = v.z & 0xFFFFFFu;
+    mbar_expect_tx(wbar_addr, bytes);
+    bulk_g2s(sbase + (v.w & 0x7FFFFFFFu), gmem, bytes, wbar_addr);
+}
+
+// One convolution, by lane 0 of the issuing warp.  Returns false after a wait has expired.
+__device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, uint32_t blob_off,
+                                         uint32_t cg, int conv_index, int it, PrevConv &prev)
+{
+    Waiter w{ctrl, p.err};
+    // The next blob's place was last used by the convolution before the previous one, which is complete; a blob
+    // marked late takes the place of something the previous convolution still uses and is copied further down.
+    bool late_copy = false;
+    if (conv_index + 1 < p.n_conv) {
+        const ConvSrc *nxt = p.conv_src + conv_index + 1;
+        if ((int)(__ldg(&nxt->bytes_phase) >> 24) <= p.stop_phase) {
+            late_copy = (__ldg(&nxt->smem_off) >> 31) != 0;
+            if (!late_copy) issue_weights(nxt, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
+        }
+    }
+    if (!w.barrier(smem_u32(&ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS)) return false;
+    const uint32_t desc = sbase + blob_off;
+    const uint4 h0 = ld_shared_v4(desc);                                    // n_ops, n_passes, n_ksteps, flags
+    const uint4 h1 = ld_shared_v4(desc + offsetof(LConvDesc, a_base));      // a_base, pitch16, bblock16, n_banks
+    const uint4 h2 = ld_shared_v4(desc + offsetof(LConvDesc, idesc));       // idesc[3], cols
+    const uint4 h3 = ld_shared_v4(desc + offsetof(LConvDesc, d_base));      // d_base[2], bar_full, bar_done
+    const uint4 h4 = ld_shared_v4(desc + offsetof(LConvDesc, use_local));   // use_local, uses_per_group, n_lines, n_chunks
+    const uint4 h5 = ld_shared_v4(desc + offsetof(LConvDesc, w_rel));       // w_rel, c_rel, ops_rel, passes_rel
+    const uint32_t use = (uint32_t)it * h4.y + h4.x;
+    IssueCtx ic;
+    ic.desc = desc; ic.ops = desc + h5.z; ic.n_ops = h0.x;
+    ic.a0 = sbase + h1.x; ic.w0 = desc + h5.x; ic.pitch16 = h1.y; ic.bblock16 = h1.z;
+    ic.d0 = tmem + ((h1.w > 1 && (use & 1u)) ? h3.y : h3.x);
+    ic.stacked = (h0.w & CF_STACKED) ? 1u : 0u;
+    ic.kstep_bytes = (ic.stacked ? 3u : 1u) * h2.w * 32u;
+    ic.full_addr = smem_u32(&ctrl->bars[h3.z]);
+    ic.idesc[0] = h2.x; ic.idesc[1] = h2.y; ic.idesc[2] = h2.z;
+    ic.cg = cg;
+    bool ok;
+    switch (h0.z) {
+    case 1: ok = issue_ops<1>(w, ic, prev, 1); break;
+    case 2: ok = issue_ops<2>(w, ic, prev, 2); break;
+    case 3: ok = issue_ops<3>(w, ic, prev, 3); break;
+    case 5: ok = issue_ops<5>(w, ic, prev, 5); break;
+    case 9: ok = issue_ops<9>(w, ic, prev, 9); break;
+    case 18: ok = issue_ops<18>(w, ic, prev, 18); break;
+    default: ok = issue_ops<0>(w, ic, prev, h0.z); break;
+    }
+    if (!ok) return false;
+    // Every line of the previous convolution has been waited for by one of the operations above (the planner
+    // sees to it), exactly once: that convolution is complete, and whatever reads its output later, or reuses
+    // what it read, needs no wait of its own.
+    if (late_copy) issue_weights(p.conv_src + conv_index + 1, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
+    prev.done_addr = smem_u32(&ctrl->bars[h3.w]);
+    prev.parity = use & 1u;
+    prev.n_lines = h4.z;
+    return true;
+}
+
+// ------------------------------------------------------------------ epilogue warps
+
+struct EpiCtx {
+    Ctrl *ctrl;
+    uint32_t sbase, tmem_lane;          // tensor-memory address of this warp's 32 lanes, column 0
+    int warp, set, quarter, lane, tid;
+    uint32_t lane_idx;                  // position within a line: quarter * 32 + lane
+};
+
+// What an epilogue warp keeps in registers for the whole of a convolution.
+struct EpiConv {
+    uint32_t flags, d0, cols, full_addr, done_addr, parity;
+    uint32_t const_addr, out_base, out_plane, out_pitch16, out_n_lines, out_log_lines, out_nb, out_logI;
+    uint32_t res_base, res_plane, in_logI, in_I, in_n_lines;
+    int32_t lo;
+    uint32_t res_m2;
+    long long res_r2;
+};
+
+// Per-channel requantisation constants as stored in the blob: the 64-bit addend, then multiplier and shift.
+//   y = floor((acc * mult + B) / 2^(32 + s)); B holds the folded bias, the rounding half and the output
+//   zero-point, so this is rs(acc' * mult, 31 + shift) + zp_out exactly.
+//   residual: y += floor((u * m2 + R2) / 2^32) with u = r + 128 the residual byte as an unsigned number,
+//   m2 = res_mult * 2^(32-n) and R2 the rounding half and the zero-points folded: rs((r - zp_res) * res_mult, n).
+template <bool kRes, bool kLo, int K>
+__device__ __forceinline__ int requant1(int acc, const ChanConst &cs, uint32_t rword, const EpiConv &E)
+{
+    int y = hi32(mad_wide(acc, cs.mult, cs.B)) >> cs.s;
+    if (kRes) y += hi32(mad_wide_u(ubyte<K>(rword), E.res_m2, E.res_r2));
+    if (kLo) y = max(y, E.lo);
+    return y;
+}
+
+// Stores one position's 16 channels of a plane, with the copies that the line layout asks for.
+__device__ __forceinline__ void store_out(const EpiConv &E, const EpiCtx &c, uint32_t ch, uint32_t line, uint4 o)
+{
+    uint32_t oline = line, olane = c.lane_idx;
+    bool keep = true;
+    if (E.flags & CF_SCATTER) {
+        // stride 2: `line` is the ordinal of an even input line; even columns and even rows survive
+        const uint32_t x_i = c.lane_idx >> E.in_logI, band_i = (c.lane_idx & (E.in_I - 1u)) >> 2, s = c.lane_idx & 3u;
+        const uint32_t r_i = 2u * line + band_i * E.in_n_lines;
+        keep = !(x_i & 1u) && !(r_i & 1u);
+        const uint32_t r_o = r_i >> 1, x_o = x_i >> 1;
+        oline = r_o & (E.out_n_lines - 1u);
+        olane = (x_o << E.out_logI) + ((r_o >> E.out_log_lines) << 2) + s;
+    }
+    if (!keep) return;
+    const uint32_t addr = E.out_base + ch * E.out_plane + (oline * E.out_pitch16 + olane) * 16u;
+    st_shared_v4(addr, o);
+    const uint32_t band = (olane >> 2) & (E.out_nb - 1u);
+    // first row of a lower band: also the row below the band above it; last row of an upper band: the row above the next
+    if (oline == 0 && band >= 1) st_shared_v4(addr + (E.out_n_lines * E.out_pitch16 - 4u) * 16u, o);
+    if (oline == E.out_n_lines - 1u && band + 1u < E.out_nb) st_shared_v4(addr - (E.out_n_lines * E.out_pitch16 - 4u) * 16u, o);
+}
+
+// One pass: SUP output lines, one 16-channel chunk.
+template <bool kRes, bool kLo, int SUP>
+__device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCtx &c, uint32_t pw, bool &ok, uint32_t cg)
+{
+    uint32_t line[SUP];
+#pragma unroll
+    for (int j = 0; j < SUP; ++j) line[j] = (pw >> (8 * j)) & 0xFFu;
+    const uint32_t ch = (pw >> 16) & 0xFFu;
+#pragma unroll
+    for (int j = 0; j < SUP; ++j)
+        if (ok) ok = w.barrier(E.full_addr + 8u * line[j], E.parity, ERR_WAIT_FULL);
+    ok = __all_sync(0xffffffffu, ok);
+    ltrace(3, cg, line[0] | (ch << 8));
+    tc_fence_after();
+    int acc[SUP][16];
+    uint32_t taddr[SUP];
+#pragma unroll
+    for (int j = 0; j < SUP; ++j) {
+        taddr[j] = c.tmem_lane + E.d0 + line[j] * E.cols + ch * 16u;
+        tmem_ld16_issue(taddr[j], acc[j]);
+    }
+    uint32_t rw[SUP][4];
+#pragma unroll
+    for (int j = 0; j < SUP; ++j) {
+        uint4 rv = make_uint4(0, 0, 0, 0);
+        if (kRes) rv = ld_shared_v4(E.res_base + ch * E.res_plane + (line[j] * E.out_pitch16 + c.lane_idx) * 16u);
+        rw[j][0] = rv.x ^ 0x80808080u; rw[j][1] = rv.y ^ 0x80808080u; rw[j][2] = rv.z ^ 0x80808080u; rw[j][3] = rv.w ^ 0x80808080u;
+    }
+    tmem_ld_wait();
+    // every accumulator column is left at zero: stacked chains accumulate from their first K-step on
+#pragma unroll
+    for (int j = 0; j < SUP; ++j) tmem_st16_zero(taddr[j]);
+    if (ok) {
+        const uint32_t cbase = E.const_addr + ch * 256u;
+        uint32_t out[SUP][4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const ChanConst c0 = ld_chan_const(cbase + (4 * g + 0) * 16), c1 = ld_chan_const(cbase + (4 * g + 1) * 16);
+            const ChanConst c2 = ld_chan_const(cbase + (4 * g + 2) * 16), c3 = ld_chan_const(cbase + (4 * g + 3) * 16);
+#pragma unroll
+            for (int j = 0; j < SUP; ++j) {
+                const int y0 = requant1<kRes, kLo, 0>(acc[j][4 * g + 0], c0, rw[j][g], E);
+                const int y1 = requant1<kRes, kLo, 1>(acc[j][4 * g + 1], c1, rw[j][g], E);
+                const int y2 = requant1<kRes, kLo, 2>(acc[j][4 * g + 2], c2, rw[j][g], E);
+                const int y3 = requant1<kRes, kLo, 3>(acc[j][4 * g + 3], c3, rw[j][g], E);
+                out[j][g] = pack4_sat(y0, y1, y2, y3);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < SUP; ++j) store_out(E, c, ch, line[j], make_uint4(out[j][0], out[j][1], out[j][2], out[j][3]));
+    }
+    tmem_st_wait();
+    // the stores become visible to the tensor cores' reads, the tensor-memory accesses are ordered before the arrival
+    tc_fence_before();
+    fence_proxy_async();
+    __syncwarp();
+    if (c.lane == 0) {
+#pragma unroll
+        for (int j = 0; j < SUP; ++j) mbar_arrive(E.done_addr + 8u * line[j]);
+    }
+    ltrace(4, cg, line[0] | (ch << 8));
+}
+
+template <bool kRes, bool kLo>
+__device__ __noinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes,
+                                             uint32_t last_line, uint32_t cg)
+{
+    const EpiConv E = E_in;
+    const EpiCtx c = c_in;
+    bool ok = true;
+#pragma unroll 1
+    for (uint32_t i = (uint32_t)c.set; i < n_passes; i += kSets) {
+        const uint32_t pw = lds32(passes + 4u * i);
+        if ((pw >> 24) == 2u) epi_pass<kRes, kLo, 2>(w, E, c, pw, ok, cg);
+        else epi_pass<kRes, kLo, 1>(w, E, c, pw, ok, cg);
+    }
+    // Every warp leaves a convolution only after its last accumulators are complete, hence all of them: a later
+    // wait for the next use of any of these barriers then always refers to the phase that is still open.
+    if (ok) w.barrier(E.full_addr + 8u * last_line, E.parity, ERR_WAIT_FULL);
+}
+
+__device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint32_t blob_off, uint32_t cg, int it)
+{
+    Waiter w{c.ctrl, p.err};
+    bool ok = w.barrier(smem_u32(&c.ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) return;                    // the abort flag is up: every other wait falls through as well
+    const uint32_t desc = c.sbase + blob_off;
+    const uint4 h0 = ld_shared_v4(desc);
+    const uint4 h1 = ld_shared_v4(desc + offsetof(LConvDesc, a_base));
+    const uint4 h2 = ld_shared_v4(desc + offsetof(LConvDesc, idesc));
+    const uint4 h3 = ld_shared_v4(desc + offsetof(LConvDesc, d_base));
+    const uint4 h4 = ld_shared_v4(desc + offsetof(LConvDesc, use_local));
+    const uint4 h5 = ld_shared_v4(desc + offsetof(LConvDesc, w_rel));
+    const uint4 h6 = ld_shared_v4(desc + offsetof(LConvDesc, out_base));       // out_base, out_plane, out_pitch16, out_n_lines
+    const uint4 h7 = ld_shared_v4(desc + offsetof(LConvDesc, out_log_lines));  // out_log_lines, out_nb, out_logI, res_base
+    const uint4 h8 = ld_shared_v4(desc + offsetof(LConvDesc, res_plane));      // res_plane, in_logI, in_I, in_n_lines
+    const uint4 h9 = ld_shared_v4(desc + offsetof(LConvDesc, lo));             // lo, res_m2, res_r2
+    const uint32_t use = (uint32_t)it * h4.y + h4.x;
+    EpiConv E;
+    E.flags = h0.w;
+    E.d0 = (h1.w > 1 && (use & 1u)) ? h3.y : h3.x;
+    E.cols = h2.w;
+    E.full_addr = smem_u32(&c.ctrl->bars[h3.z]);
+    E.done_addr = smem_u32(&c.ctrl->bars[h3.w]);
+    E.parity = use & 1u;
+    E.const_addr = desc + h5.y;
+    E.out_base = c.sbase + h6.x; E.out_plane = h6.y; E.out_pitch16 = h6.z; E.out_n_lines = h6.w;
+    E.out_log_lines = h7.x; E.out_nb = h7.y; E.out_logI = h7.z; E.res_base = c.sbase + h7.w;
+    E.res_plane = h8.x; E.in_logI = h8.y; E.in_I = h8.z; E.in_n_lines = h8.w;
+    E.lo = (int32_t)h9.x; E.res_m2 = h9.y;
+    E.res_r2 = (long long)(((unsigned long long)h9.w << 32) | h9.z);
+    const uint32_t passes = desc + h5.w, n_passes = h0.y;
+    // the line whose accumulators complete last closes the pass list
+    const uint32_t last_pw = lds32(passes + 4u * (n_passes - 1u));
+    const uint32_t last_line = (last_pw >> 24) == 2u ? (last_pw >> 8) & 0xFFu : last_pw & 0xFFu;
+    switch (E.flags & (CF_RES | CF_LO)) {
+    case 0: epi_conv_passes<false, false>(w, E, c, passes, n_passes, last_line, cg); break;
+    case CF_RES: epi_conv_passes<true, false>(w, E, c, passes, n_passes, last_line, cg); break;
+    case CF_LO: epi_conv_passes<false, true>(w, E, c, passes, n_passes, last_line, cg); break;
+    default: epi_conv_passes<true, true>(w, E, c, passes, n_passes, last_line, cg); break;
+    }
+}
+
+// FILL: the region takes its halo value everywhere
+__device__ void fill_phase(const EpiCtx &c, uint32_t off, uint32_t bytes, uint32_t halo)
+{
+    const uint32_t word = (halo & 0xFFu) * 0x01010101u;
+    const uint4 v = make_uint4(word, word, word, word);
+    for (uint32_t o = (uint32_t)c.tid * 16u; o < bytes; o += kEpiThreads * 16u) st_shared_v4(c.sbase + off + o, v);
+}
+
+// INPUT: one thread = four horizontally adjacent pixels of one sample, all input channels (Def. 3.3, Def. 3.4).
+__device__ void input_phase(const LineParams &p, const EpiCtx &c, int grp)
+{
+    const int H = p.in_H, W = p.in_W, in_c = p.in_c;
+    const int wq = W >> 2;
+    const int quads = kG * H * wq;
+    const uint32_t *__restrict__ cum = p.ns.cum;
+    const int T = p.ns.T;
+    const uint32_t key0 = p.ns.key0, key1 = p.ns.key1, ctr2 = p.ns.ctr2;
+    const uint8_t *__restrict__ x = p.x;
+    for (int qi = c.tid; qi < quads; qi += kEpiThreads) {
+        // consecutive threads take consecutive samples: their stores fall into one 64-byte run
+        const int s = qi & (kG - 1);
+        const int rem = qi >> 2;
+        const int y = rem / wq, x4 = rem - y * wq;
+        const long long j = p.ns.first_sample + (long long)grp * kG + s;
+        const uint32_t ctr3 = p.ns.ctr3_fixed | (uint32_t)(((j >> 32) & 0xFF) << 8);
+        uint32_t px[4] = {0, 0, 0, 0};
+        for (int ch = 0; ch < in_c; ++ch) {
+            const uint32_t e = (uint32_t)((ch * H + y) * W + 4 * x4);
+            const uint4 r = philox4x32_10(make_uint4(e >> 2, (uint32_t)(j & 0xFFFFFFFFll), ctr2, ctr3), key0, key1);
+            const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+            const uint32_t clean = __ldg(reinterpret_cast<const uint32_t *>(x + e));
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                int v = (int)((clean >> (8 * k)) & 0xFF) + noise_level(u[k], cum, T);
+                v = min(255, max(0, v));
+                px[k] |= (uint32_t)v << (8 * ch);
+            }
+        }
+        // the input has one row band: line = row, position = column * 4 + sample
+        const uint32_t pos = (uint32_t)y * p.input_pitch16 + (uint32_t)(4 * x4) * kG + (uint32_t)s;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) st_shared_v4(c.sbase + p.input_base + (pos + (uint32_t)k * kG) * 16u, make_uint4(px[k], 0, 0, 0));
+    }
+}
+
+// TAIL: global average pool, FC, argmax and vote; one warp carries one sample (Algorithm 1 steps 1-4).
+__device__ void tail_sample(const LineParams &p, const EpiCtx &c, int s, int grp)
+{
+    const int tail_H = p.tail_H, tail_W = p.tail_W, tail_C = p.tail_C, n_lines = p.tail_n_lines;
+    const int n_classes = p.n_classes;
+    const int hw = tail_H * tail_W;
+    int pooled[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int ch = c.lane + 32 * h;
+        int q = 0;
+        if (ch < tail_C) {
+            const uint32_t base = c.sbase + p.tail_base + (uint32_t)(ch >> 4) * p.tail_plane + (ch & 15);
+            int sum = 0;
+            for (int i = 0; i < hw; ++i) {
+                const int y = i / tail_W, x = i - y * tail_W;
+                const int line = y % n_lines, band = y / n_lines;
+                const uint32_t pos = (uint32_t)line * p.tail_pitch16 + ((uint32_t)x << p.tail_logI) + (uint32_t)(band * 4 + s);
+                int v;
+                asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(base + pos * 16u));
+                sum += v - p.pool_zp_in;
+            }
+            long long v = ((long long)sum * p.pool_mult + (1ll << (p.pool_n - 1))) >> p.pool_n;
+            v += p.pool_zp_out;
+            v = v < p.pool_lo ? p.pool_lo : v;
+            v = v > 127 ? 127 : v;
+            q = (int)v;
+        }
+        pooled[h] = q;
+    }
+    const long long sample = (long long)grp * kG + s;          // index within this launch
+    const bool counted = sample < p.n_samples;
+    int best_v = -1000, best_o = 0x7fffffff;
+    for (int o0 = 0; o0 < n_classes; o0 += 32) {
+        const int o = o0 + c.lane;
+        const bool live = o < n_classes;
+        const FcConst k = p.fc_c[live ? o : 0];
+        const int8_t *wrow = p.fc_w + (size_t)(live ? o : 0) * 64;
+        int acc = k.bias;
+        for (int cc = 0; cc < tail_C; ++cc) {
+            const int a = __shfl_sync(0xffffffffu, pooled[cc >> 5], cc & 31);
+            acc += a * (int)__ldg(wrow + cc);
+        }
+        long long v = ((long long)acc * k.mult + (1ll << (k.n - 1))) >> k.n;
+        v += k.zp_out;
+        v = v < k.lo ? k.lo : v;
+        v = v > 127 ? 127 : v;
+        if (live) {
+            if ((int)v > best_v) { best_v = (int)v; best_o = o; }
+            if (counted && p.logits) p.logits[sample * n_classes + o] = (int8_t)v;
+        }
+    }
+    // lowest index among the maxima
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        const int ov = __shfl_xor_sync(0xffffffffu, best_v, d), oo = __shfl_xor_sync(0xffffffffu, best_o, d);
+        if (ov > best_v || (ov == best_v && oo < best_o)) { best_v = ov; best_o = oo; }
+    }
+    if (counted && c.lane == 0) atomicAdd(&c.ctrl->hist[best_o], 1);
+}
+
+__global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ LineParams p)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
+    const uint32_t sbase = smem_u32(smem);
+    const int warp = (int)warp_uniform(threadIdx.x >> 5), lane = threadIdx.x & 31;
+    for (int i = threadIdx.x; i < p.n_bars; i += blockDim.x) mbar_init(smem_u32(&ctrl->bars[i]), p.bar_counts[i]);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 3; ++s) mbar_init(smem_u32(&ctrl->wbar[s]), 1);
+        mbar_init(smem_u32(&ctrl->drain), 1);
+        ctrl->abort_flag = 0;
+    }
+    for (int i = threadIdx.x; i < 128; i += blockDim.x) ctrl->hist[i] = 0;
+    for (int i = threadIdx.x; i < p.n_phases; i += blockDim.x) ctrl->ptab[i] = p.ptab[i];
+    if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctrl->tmem_base;
+
+    EpiCtx c;
+    c.ctrl = ctrl; c.sbase = sbase;
+    c.warp = warp; c.set = warp >> 2; c.quarter = warp & 3; c.lane = lane; c.tid = threadIdx.x;
+    c.lane_idx = (uint32_t)((warp & 3) * 32 + lane);
+    c.tmem_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const bool issuer = warp == kIssuerWarp;
+    // accumulators of stacked convolutions start from zero
+    if (!issuer) {
+        for (uint32_t col = (uint32_t)c.set * 16u; col < (uint32_t)kTmemCols; col += kSets * 16u) tmem_st16_zero(c.tmem_lane + col);
+        tmem_st_wait();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const uint32_t ptab = smem_u32(ctrl->ptab);
+    const int n_phases = p.n_phases, stop_phase = p.stop_phase;
+    int it = 0;
+    for (int grp = blockIdx.x; grp < p.n_groups; grp += gridDim.x, ++it) {
+        PrevConv prev{0u, 0u, 0u};
+        bool issuer_ok = true;
+        int conv_index = 0;
+        bool first_phase = true;
+        for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
+            const uint4 e = ld_shared_v4(ptab + 16 * ph);
+            if (e.x == PH_CONV) {
+                const uint32_t cg = (uint32_t)it * (uint32_t)p.n_conv + (uint32_t)conv_index;
+                if (issuer) {
+                    if (lane == 0 && issuer_ok && !ctrl->abort_flag)
+                        issuer_ok = issuer_conv(p, ctrl, sbase, tmem, e.y, cg, conv_index, it, prev);
+                    __syncwarp();
+                } else {
+                    epi_conv(p, c, e.y, cg, it);
+                }
+                conv_index += 1;
+                first_phase = false;
+                continue;
+            }
+            // CTA-wide phase: everything before it is complete in all warps
+            tc_fence_before();
+            __syncthreads();
+            tc_fence_after();
+            prev.n_lines = 0;
+            if (first_phase) {
+                // the first blob of the group: everything of the previous group is complete
+                if (issuer && lane == 0 && p.n_conv > 0 && !ctrl->abort_flag &&
+                    (int)(__ldg(&p.conv_src[0].bytes_phase) >> 24) <= stop_phase)
+                    issue_weights(p.conv_src, sbase, smem_u32(&ctrl->wbar[((uint32_t)it * (uint32_t)p.n_conv) % 3]));
+                first_phase = false;
+            }
+            if (!issuer && !ctrl->abort_flag) {
+                if (e.x == PH_FILL) fill_phase(c, e.y, e.z, e.w);
+                else if (e.x == PH_INPUT) input_phase(p, c, grp);
+                else if (warp < kG) tail_sample(p, c, warp, grp);
+            }
+            fence_proxy_async();
+            __syncthreads();
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+    if (!ctrl->abort_flag)
+        for (int i = threadIdx.x; i < p.n_classes; i += blockDim.x)
+            if (ctrl->hist[i]) atomicAdd(p.counts + i, ctrl->hist[i]);
+    if (p.dump)
+        for (uint32_t o = threadIdx.x * 16u; o < p.dump_bytes; o += blockDim.x * 16u)
+            *reinterpret_cast<uint4 *>(p.dump + o) = ld_shared_v4(sbase + p.dump_off + o);
+    // no tensor-core work may be in flight when tensor memory is released
+    if (issuer && lane == 0) {
+        Waiter w{ctrl, p.err};
+        commit_to(smem_u32(&ctrl->drain));
+        w.barrier(smem_u32(&ctrl->drain), 0, ERR_WAIT_DRAIN);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// =============================================================================== host planner
+
+int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+
+// Geometry of one tensor in the line layout.
+struct LGeo {
+    int C = 0, H = 0, W = 0, planes = 0, halo = 0;
+    int I = 0, nb = 0, n_lines = 0, pitch = 0;       // positions per column, row bands, lines, line pitch in positions
+    uint32_t plane_bytes = 0, bytes = 0, line0 = 0;  // line0: byte offset of line 0, lane 0 within a plane
+    int buffer = -1, producer_phase = -1, producer_conv = -1;
+    bool scatter_produced = false;
+    int last_use_layer = -1;
+    bool last_use_as_input = false;
+};
+
+bool set_geometry(LGeo &t)
+{
+    if (t.W != 32 && t.W != 16 && t.W != 8) return false;
+    if (t.H != t.W) return false;
+    t.planes = (t.C + 15) / 16;
+    t.I = 128 / t.W;
+    t.nb = t.I / kG;
+    t.n_lines = t.H / t.nb;
+    t.pitch = 128 + t.I;
+    const int positions = t.I + (t.n_lines + 2) * t.pitch + 8;      // leading gap, lines -1 .. n_lines with their gaps, slack
+    t.plane_bytes = (uint32_t)positions * 16u;
+    t.bytes = t.plane_bytes * (uint32_t)t.planes;
+    t.line0 = (uint32_t)(t.I + t.pitch) * 16u;
+    return true;
+}
+
+struct PlanBuffer { uint32_t bytes = 0, off = 0; int birth = 0, death = 0, halo = 0; };
+struct AllocReq { uint32_t bytes; int birth, death, slack; uint32_t *off; int conv; };
+
+// First-fit placement of one request among the allocations that are still busy at its birth.
+bool place(std::vector<AllocReq> &done, AllocReq &r, uint32_t capacity)
+{
+    std::vector<std::pair<uint32_t, uint32_t>> busy;
+    for (const AllocReq &e : done)
+        if (e.death >= r.birth - r.slack) busy.push_back({*e.off, *e.off + e.bytes});
+    std::sort(busy.begin(), busy.end());
+    uint32_t at = kCtrlBytes;
+    for (const auto &b : busy) {
+        if (at + r.bytes <= b.first) break;
+        at = std::max(at, (b.second + 127u) & ~127u);
+    }
+    if (at + r.bytes > capacity) return false;
+    *r.off = at;
+    done.push_back(r);
+    return true;
+}
+
+// A plan that does not fit is not an error (another engine runs the model); ISC_PLAN_DEBUG=1 says which rule failed.
+#define PLAN_FAIL(id) do { if (getenv("ISC_PLAN_DEBUG")) fprintf(stderr, "line engine: plan rule %d failed\n", id); return false; } while (0)
+
+bool conv_ok(const isc_layer &L, bool first)
+{
+    if (L.op != ISC_CONV2D) return false;
+    if (L.kh != L.kw || (L.kh != 1 && L.kh != 3)) return false;
+    if (L.pad != (L.kh - 1) / 2) return false;
+    if (L.stride != 1 && L.stride != 2) return false;
+    if (first) { if (L.cin > 4 || L.stride != 1) return false; }
+    else if (L.cin % 16 != 0 || L.cin > 64) return false;
+    if (L.cout % 16 != 0 || L.cout > 64) return false;
+    return true;
+}
+
+}  // namespace
+
+struct LinePlan {
+    int in_c = 0, in_h = 0, in_w = 0, n_classes = 0, n_phases = 0, n_conv = 0, n_bars = 0;
+    uint32_t smem_bytes = 0;
+    LineParams base;
+    std::vector<int> phase_kind;
+    std::vector<LGeo> tensors;
+    std::vector<uint32_t> tensor_off;
+    PhaseEntry *d_ptab = nullptr;
+    ConvSrc *d_conv_src = nullptr;
+    uint8_t *d_bar_counts = nullptr;
+    uint8_t *d_blob = nullptr;
+    int8_t *d_fc_w = nullptr;
+    FcConst *d_fc_c = nullptr;
+    int32_t *d_err = nullptr;
+    uint8_t *d_dump = nullptr;
+    int sm_count = 0;
+    bool attr_set = false;
+};
+
+namespace {
+
+// What the planner knows about a convolution phase while it builds the operation and pass tables.
+struct ConvPlan {
+    int layer = -1, phase = -1;
+    int in_tensor = -1, out_tensor = -1;
+    bool stacked = false, scatter = false;
+    int m = 0;                          // output lines (ordinals)
+    int n_chunks = 0, cols = 0, n_banks = 1;
+    int cls = -1, use_local = 0;
+    std::vector<LOp> ops;
+    std::vector<uint32_t> passes;
+    std::vector<int> done_time;         // per output line: index of the pass that stores its last chunk
+    std::vector<int> a_delta;
+    std::vector<uint32_t> a_lbo;
+    std::vector<std::pair<int, int>> kunits;   // per K-step: indices into `units` (second may be -1)
+    struct Unit { int r, s, pl; };             // vertical tap (-1 when stacked), horizontal tap, input plane
+    std::vector<Unit> units;
+};
+
+bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, LinePlan *plan,
+                std::vector<uint8_t> *blob_out, std::vector<uint32_t> *blob_offsets, std::vector<PhaseEntry> *ptab_out,
+                std::vector<ConvSrc> *csrc_out, std::vector<uint8_t> *bar_counts_out)
+{
+    const int n_conv_layers = n_layers - 2;
+    // ---- tensors of the model (tensor t = output of layer t-1)
+    std::vector<LGeo> T((size_t)n_layers + 1);
+    T[0].C = in_c; T[0].H = in_h; T[0].W = in_w; T[0].halo = layers[0].d.zp_in;
+    for (int i = 0; i < n_conv_layers; ++i) {
+        const isc_layer &L = layers[i].d;
+        const LGeo &in = T[(size_t)L.in_tensor];
+        LGeo &o = T[(size_t)i + 1];
+        o.C = L.cout;
+        o.H = (in.H + 2 * L.pad - L.kh) / L.stride + 1;
+        o.W = (in.W + 2 * L.pad - L.kw) / L.stride + 1;
+        o.halo = L.zp_out;
+        if (L.stride == 2 && ((in.H & 1) || (in.W & 1))) PLAN_FAIL(1);
+    }
+    for (int t = 0; t <= n_conv_layers; ++t)
+        if (!set_geometry(T[(size_t)t])) PLAN_FAIL(2);
+    if (T[0].nb != 1) PLAN_FAIL(3);                 // the input writer knows one row band only
+    for (int i = 0; i < n_layers; ++i) {
+        const isc_layer &L = layers[i].d;
+        T[(size_t)L.in_tensor].last_use_layer = i;
+        T[(size_t)L.in_tensor].last_use_as_input = true;
+        if (L.res_tensor >= 0) {
+            T[(size_t)L.res_tensor].last_use_layer = i;
+            T[(size_t)L.res_tensor].last_use_as_input = false;
+        }
+    }
+    // ---- phase skeleton: FILL(input) INPUT, then per convolution [FILL of a fresh output] CONV, then TAIL
+    struct Skel { int kind; int layer; int tensor; };
+    std::vector<Skel> skel;
+    std::vector<PlanBuffer> buffers;
+    std::vector<int> layer_phase((size_t)n_layers, -1);
+    auto new_buffer = [&](int tensor) {
+        PlanBuffer b;
+        b.bytes = T[(size_t)tensor].bytes; b.halo = T[(size_t)tensor].halo;
+        b.birth = (int)skel.size();
+        buffers.push_back(b);
+        T[(size_t)tensor].buffer = (int)buffers.size() - 1;
+        skel.push_back({PH_FILL, -1, tensor});
+    };
+    new_buffer(0);
+    skel.push_back({PH_INPUT, -1, 0});
+    int prev_conv_layer = -1;
+    for (int i = 0; i < n_conv_layers; ++i) {
+        const isc_layer &L = layers[i].d;
+        const int out_t = i + 1;
+        LGeo &o = T[(size_t)out_t];
+        bool placed = false;
+        // (a) in place over the residual operand, when this layer is its last reader
+        if (L.res_tensor >= 0 && L.stride == 1 && T[(size_t)L.res_tensor].last_use_layer == i &&
+            L.res_tensor != L.in_tensor && T[(size_t)L.res_tensor].halo == o.halo &&
+            T[(size_t)L.res_tensor].bytes == o.bytes && T[(size_t)L.res_tensor].W == o.W) {
+            o.buffer = T[(size_t)L.res_tensor].buffer;
+            placed = true;
+        }
+        // (b) over a same-shaped tensor whose last reader was the previous convolution, as its input
+        if (!placed && L.stride == 1 && prev_conv_layer >= 0)
+            for (int t = 1; t <= n_conv_layers && !placed; ++t) {
+                const LGeo &x = T[(size_t)t];
+                if (x.buffer < 0 || t == out_t || t == L.in_tensor || t == L.res_tensor) continue;
+                if (x.last_use_layer != prev_conv_layer || !x.last_use_as_input) continue;
+                if (x.C != o.C || x.H != o.H || x.W != o.W || x.halo != o.halo) continue;
+                bool newest = true;           // x must be the current tenant of its buffer
+                for (int u = t + 1; u <= n_conv_layers; ++u)
+                    if (T[(size_t)u].buffer == x.buffer) newest = false;
+                if (newest) { o.buffer = x.buffer; placed = true; }
+            }
+        if (!placed) new_buffer(out_t);
+        layer_phase[(size_t)i] = (int)skel.size();
+        skel.push_back({PH_CONV, i, -1});
+        prev_conv_layer = i;
+    }
+    const int tail_phase = (int)skel.size();
+    skel.push_back({PH_TAIL, -1, n_conv_layers});
+    layer_phase[(size_t)n_layers - 2] = tail_phase;
+    layer_phase[(size_t)n_layers - 1] = tail_phase;
+    const int n_phases = (int)skel.size();
+    if (n_phases > kMaxPhases) PLAN_FAIL(4);
+    // ---- lifetimes
+    for (int t = 0; t <= n_conv_layers; ++t) {
+        LGeo &x = T[(size_t)t];
+        if (x.buffer < 0) PLAN_FAIL(5);
+        int death = x.last_use_layer >= 0 ? layer_phase[(size_t)x.last_use_layer] : -1;
+        x.producer_phase = t >= 1 ? layer_phase[(size_t)t - 1] : 1;
+        death = std::max(death, x.producer_phase);
+        buffers[(size_t)x.buffer].death = std::max(buffers[(size_t)x.buffer].death, death);
+    }
+    // ---- convolutions: K-steps, operations, passes
+    std::vector<ConvPlan> convs;
+    std::map<std::pair<int, int>, int> class_of;            // (lines, chunks) -> class
+    std::vector<int> class_lines, class_chunks, class_uses;
+    for (int ph = 0; ph < n_phases; ++ph) {
+        if (skel[(size_t)ph].kind != PH_CONV) continue;
+        ConvPlan cp;
+        cp.layer = skel[(size_t)ph].layer; cp.phase = ph;
+        const isc_layer &L = layers[cp.layer].d;
+        cp.in_tensor = L.in_tensor; cp.out_tensor = cp.layer + 1;
+        LGeo &in = T[(size_t)cp.in_tensor];
+        LGeo &out = T[(size_t)cp.out_tensor];
+        out.producer_conv = (int)convs.size();
+        cp.scatter = L.stride == 2;
+        out.scatter_produced = cp.scatter;
+        cp.n_chunks = L.cout / 16; cp.cols = L.cout;
+        if (cp.scatter && (in.n_lines & 1)) PLAN_FAIL(6);
+        cp.m = cp.scatter ? in.n_lines / 2 : in.n_lines;
+        if (cp.m > kMaxLines || cp.m * cp.cols > kTmemCols) PLAN_FAIL(7);
+        cp.stacked = L.kh == 3 && L.stride == 1 && 3 * L.cout <= 128 && in.n_lines >= 2;
+        cp.n_banks = kTmemCols / (cp.m * cp.cols) >= 2 ? 2 : 1;
+        if (L.res_tensor >= 0) {
+            const LGeo &r = T[(size_t)L.res_tensor];
+            if (cp.scatter || r.W != out.W || r.H != out.H || r.C != out.C) PLAN_FAIL(8);
+            const int res_n = 31 - L.res_shift;
+            if (res_n != 31 && res_n != 32) PLAN_FAIL(9);
+        }
+        // K units and steps
+        const int s_lo = L.kw == 3 ? -1 : 0, s_hi = L.kw == 3 ? 1 : 0;
+        if (cp.stacked) {
+            for (int pl = 0; pl < in.planes; ++pl)
+                for (int s = s_lo; s <= s_hi; ++s) cp.units.push_back({-1, s, pl});
+        } else {
+            const int r_lo = L.kh == 3 ? 0 : 1, r_hi = L.kh == 3 ? 2 : 1;
+            for (int pl = 0; pl < in.planes; ++pl)
+                for (int r = r_lo; r <= r_hi; ++r)
+                    for (int s = s_lo; s <= s_hi; ++s) cp.units.push_back({r, s, pl});
+        }
+        auto unit_addr = [&](const ConvPlan::Unit &u) {
+            const int dr = cp.stacked ? 0 : u.r - 1;
+            return (long long)u.pl * in.plane_bytes + ((long long)dr * in.pitch + (long long)u.s * in.I) * 16;
+        };
+        for (size_t a = 0; a < cp.units.size(); a += 2) {
+            if (a + 1 < cp.units.size()) {
+                const long long d = unit_addr(cp.units[a + 1]) - unit_addr(cp.units[a]);
+                if (d <= 0 || d >= (1 << 18)) PLAN_FAIL(10);
+                cp.kunits.push_back({(int)a, (int)a + 1});
+                cp.a_delta.push_back((int)unit_addr(cp.units[a]));
+                cp.a_lbo.push_back((uint32_t)d);
+            } else {
+                cp.kunits.push_back({(int)a, -1});
+                cp.a_delta.push_back((int)unit_addr(cp.units[a]));
+                cp.a_lbo.push_back(16u);
+            }
+        }
+        if ((int)cp.kunits.size() > kMaxKsteps) PLAN_FAIL(11);
+        // class and banks
+        const auto key = std::make_pair(cp.m, cp.n_chunks);
+        if (!class_of.count(key)) {
+            class_of[key] = (int)class_lines.size();
+            class_lines.push_back(cp.m); class_chunks.push_back(cp.n_chunks); class_uses.push_back(0);
+        }
+        cp.cls = class_of[key];
+        cp.use_local = class_uses[(size_t)cp.cls]++;
+        // ---- operations
+        const ConvPlan *pv = (!convs.empty() && convs.back().phase == ph - 1) ? &convs.back() : nullptr;
+        const bool same_class = pv && pv->cls == cp.cls;
+        // the previous convolution produced this one's input, line for line
+        const bool aligned = pv && in.producer_conv == (int)convs.size() - 1 && !pv->scatter;
+        // Same class: the same barriers, and with one bank the same accumulator columns.  An operation then waits for
+        // the previous convolution's lines of the same numbers as the output lines it adds to, so that no line of
+        // this convolution can be stored (and arrive on the line's barrier) before that line of the previous one.
+        const bool slots = same_class;
+        const bool wait_all = pv && !same_class;
+        auto prev_time = [&](int line) { return pv ? pv->done_time[(size_t)line] : 0; };
+        auto src_line = [&](int p) -> int {       // which output line of the producer fills input line p (-1: constant)
+            if (p >= 0 && p < in.n_lines) return p;
+            if (in.nb == 1) return -1;
+            return p < 0 ? in.n_lines - 1 : 0;
+        };
+        struct ProtoOp { int a_line, b_block, n_blocks, d_line; std::vector<int> need; std::vector<int> outs; int ready; };
+        std::vector<ProtoOp> proto;
+        if (cp.stacked) {
+            for (int p = -1; p <= in.n_lines; ++p) {
+                ProtoOp o;
+                o.a_line = p;
+                const int y_lo = std::max(p - 1, 0), y_hi = std::min(p + 1, in.n_lines - 1);
+                o.b_block = y_lo - (p - 1); o.n_blocks = y_hi - y_lo + 1; o.d_line = y_lo;
+                for (int y = y_lo; y <= y_hi; ++y) o.outs.push_back(y);
+                if (aligned && src_line(p) >= 0) o.need.push_back(src_line(p));
+                if (slots) for (int y = y_lo; y <= y_hi; ++y) o.need.push_back(y);
+                proto.push_back(o);
+            }
+        } else {
+            for (int j = 0; j < cp.m; ++j) {
+                ProtoOp o;
+                const int cline = cp.scatter ? 2 * j : j;
+                o.a_line = cline; o.b_block = 0; o.n_blocks = 1; o.d_line = j;
+                o.outs.push_back(j);
+                if (aligned)
+                    for (int r = (L.kh == 3 ? -1 : 0); r <= (L.kh == 3 ? 1 : 0); ++r)
+                        if (src_line(cline + r) >= 0) o.need.push_back(src_line(cline + r));
+                if (slots) o.need.push_back(j);
+                proto.push_back(o);
+            }
+        }
+        for (ProtoOp &o : proto) {
+            o.ready = 0;
+            for (int l : o.need) o.ready = std::max(o.ready, prev_time(l));
+        }
+        std::stable_sort(proto.begin(), proto.end(), [](const ProtoOp &a, const ProtoOp &b) { return a.ready < b.ready; });
+        // completion of each output line = the last operation that contributes to it
+        std::vector<int> last_op((size_t)cp.m, -1);
+        for (size_t i = 0; i < proto.size(); ++i)
+            for (int y : proto[i].outs) last_op[(size_t)y] = (int)i;
+        std::vector<char> waited(pv ? (size_t)pv->m : 0, 0);
+        for (size_t i = 0; i < proto.size(); ++i) {
+            const ProtoOp &o = proto[i];
+            LOp op;
+            memset(&op, 0, sizeof(op));
+            op.a_line1 = (uint8_t)(o.a_line + 1);
+            op.b_block = (uint8_t)o.b_block; op.n_blocks = (uint8_t)o.n_blocks;
+            op.d_col = (uint16_t)(o.d_line * cp.cols);
+            if (i == 0 && wait_all) {
+                op.flags |= OPF_WAIT_ALL;
+                std::fill(waited.begin(), waited.end(), 1);
+            }
+            for (int l : o.need)
+                if (!waited[(size_t)l]) {
+                    if (op.n_wait >= 4) PLAN_FAIL(12);
+                    op.wait[op.n_wait++] = (uint8_t)l;
+                    waited[(size_t)l] = 1;
+                }
+            for (int y : o.outs)
+                if (last_op[(size_t)y] == (int)i) {
+                    if (op.n_commit >= 4) PLAN_FAIL(13);
+                    op.commit[op.n_commit++] = (uint8_t)y;
+                }
+            cp.ops.push_back(op);
+        }
+        // ---- passes in the order of completion
+        std::vector<int> order((size_t)cp.m);
+        for (int y = 0; y < cp.m; ++y) order[(size_t)y] = y;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return last_op[(size_t)a] < last_op[(size_t)b]; });
+        const int sup = cp.m >= 8 ? 2 : 1;
+        cp.done_time.assign((size_t)cp.m, 0);
+        for (int i = 0; i < cp.m; i += sup)
+            for (int ch = 0; ch < cp.n_chunks; ++ch) {
+                const int n = std::min(sup, cp.m - i);
+                uint32_t pw = (uint32_t)order[(size_t)i] | ((uint32_t)ch << 16) | ((uint32_t)n << 24);
+                if (n == 2) pw |= (uint32_t)order[(size_t)i + 1] << 8;
+                for (int q = 0; q < n; ++q) cp.done_time[(size_t)order[(size_t)i + q]] = (int)cp.passes.size() / kSets;
+                cp.passes.push_back(pw);
+            }
+        convs.push_back(cp);
+    }
+    const int n_conv = (int)convs.size();
+    // ---- barriers: per class, one per output line for "accumulators complete" and one for "line stored"
+    std::vector<int> class_full(class_lines.size()), class_done(class_lines.size());
+    bar_counts_out->clear();
+    for (size_t k = 0; k < class_lines.size(); ++k) {
+        class_full[k] = (int)bar_counts_out->size();
+        for (int l = 0; l < class_lines[k]; ++l) bar_counts_out->push_back(1);
+        class_done[k] = (int)bar_counts_out->size();
+        for (int l = 0; l < class_lines[k]; ++l) bar_counts_out->push_back((uint8_t)(4 * class_chunks[k]));
+    }
+    if ((int)bar_counts_out->size() > kMaxBars) PLAN_FAIL(14);
+    // ---- blob sizes and shared-memory placement in order of birth
+    std::vector<uint32_t> w_bytes((size_t)n_conv), w_off((size_t)n_conv), w_rel((size_t)n_conv), c_rel((size_t)n_conv),
+        ops_rel((size_t)n_conv), passes_rel((size_t)n_conv);
+    for (int c = 0; c < n_conv; ++c) {
+        const ConvPlan &cp = convs[(size_t)c];
+        const isc_layer &L = layers[cp.layer].d;
+        const uint32_t rows = (uint32_t)(cp.stacked ? 3 : 1) * (uint32_t)L.cout;
+        uint32_t at = (uint32_t)sizeof(LConvDesc);
+        ops_rel[(size_t)c] = at; at += (uint32_t)cp.ops.size() * 16u;
+        passes_rel[(size_t)c] = at; at += ((uint32_t)cp.passes.size() * 4u + 15u) & ~15u;
+        at = (at + 127u) & ~127u;
+        w_rel[(size_t)c] = at; at += (uint32_t)cp.kunits.size() * rows * 32u;
+        c_rel[(size_t)c] = at; at += (uint32_t)L.cout * 16u;
+        w_bytes[(size_t)c] = (at + 127u) & ~127u;
+    }
+    std::vector<AllocReq> reqs, placed;
+    for (PlanBuffer &b : buffers) reqs.push_back({b.bytes, b.birth, b.death, 0, &b.off, -1});
+    for (int c = 0; c < n_conv; ++c)
+        reqs.push_back({w_bytes[(size_t)c], c == 0 ? 0 : convs[(size_t)c - 1].phase, convs[(size_t)c].phase, c == 0 ? 0 : 1,
+                        &w_off[(size_t)c], c});
+    std::stable_sort(reqs.begin(), reqs.end(), [](const AllocReq &a, const AllocReq &b) { return a.birth < b.birth; });
+    uint32_t high = kCtrlBytes;
+    std::vector<char> late((size_t)n_conv, 0);
+    for (AllocReq &r : reqs) {
+        bool ok = place(placed, r, kSmemLimit);
+        if (!ok && r.conv > 0) {
+            // A blob is normally copied when the convolution before its own starts, while the one before that may
+            // still be in its epilogue (slack 1).  Where that does not fit, it is copied once that one is complete.
+            r.slack = 0;
+            late[(size_t)r.conv] = 1;
+            ok = place(placed, r, kSmemLimit);
+        }
+        if (!ok) {
+            if (getenv("ISC_PLAN_DEBUG")) {
+                fprintf(stderr, "line engine: no room for %u bytes born at phase %d (dies %d); busy then:\n", r.bytes, r.birth, r.death);
+                for (const AllocReq &e : placed)
+                    if (e.death >= r.birth - r.slack)
+                        fprintf(stderr, "  [%u, %u) phases %d..%d\n", *e.off, *e.off + e.bytes, e.birth, e.death);
+            }
+            PLAN_FAIL(15);
+        }
+        high = std::max(high, *r.off + r.bytes);
+        if (getenv("ISC_PLAN_DEBUG") && atoi(getenv("ISC_PLAN_DEBUG")) > 1)
+            fprintf(stderr, "  %s %d: [%u, %u) phases %d..%d\n", r.conv >= 0 ? "blob" : "tensor", r.conv, *r.off, *r.off + r.bytes, r.birth, r.death);
+    }
+    plan->tensors = T;
+    plan->tensor_off.assign(T.size(), 0);
+    for (int t = 0; t <= n_conv_layers; ++t) plan->tensor_off[(size_t)t] = buffers[(size_t)T[(size_t)t].buffer].off;
+    // ---- emit phases and blobs
+    ptab_out->assign((size_t)n_phases, PhaseEntry{0, 0, 0, 0});
+    csrc_out->assign((size_t)n_conv, ConvSrc{0, 0, 0});
+    blob_out->clear();
+    blob_offsets->assign((size_t)n_conv, 0);
+    plan->phase_kind.assign((size_t)n_phases, 0);
+    int conv_at = 0;
+    for (int ph = 0; ph < n_phases; ++ph) {
+        const Skel &S = skel[(size_t)ph];
+        PhaseEntry &E = (*ptab_out)[(size_t)ph];
+        E.kind = (uint32_t)S.kind;
+        plan->phase_kind[(size_t)ph] = S.kind;
+        if (S.kind == PH_FILL) {
+            E.a = plan->tensor_off[(size_t)S.tensor]; E.b = T[(size_t)S.tensor].bytes; E.c = (uint32_t)(T[(size_t)S.tensor].halo & 0xFF);
+            continue;
+        }
+        if (S.kind != PH_CONV) continue;
+        const int c = conv_at++;
+        const ConvPlan &cp = convs[(size_t)c];
+        const MegaLayerIn &ML = layers[cp.layer];
+        const isc_layer &L = ML.d;
+        const LGeo &in = T[(size_t)cp.in_tensor], &out = T[(size_t)cp.out_tensor];
+        E.a = w_off[(size_t)c];
+        std::vector<uint8_t> blob(w_bytes[(size_t)c], 0);
+        LConvDesc D;
+        memset(&D, 0, sizeof(D));
+        D.n_ops = (uint32_t)cp.ops.size(); D.n_passes = (uint32_t)cp.passes.size(); D.n_ksteps = (uint32_t)cp.kunits.size();
+        D.flags = (cp.stacked ? CF_STACKED : 0u) | (L.res_tensor >= 0 ? CF_RES : 0u) | (cp.scatter ? CF_SCATTER : 0u);
+        const int lo = L.relu ? std::max(-128, L.zp_out) : -128;
+        if (lo > -128) D.flags |= CF_LO;
+        D.lo = lo;
+        // operand base: line -1, lane 0, plane 0 of the input
+        D.a_base = plan->tensor_off[(size_t)cp.in_tensor] + in.line0 - (uint32_t)in.pitch * 16u;
+        D.pitch16 = (uint32_t)in.pitch;
+        D.bblock16 = (uint32_t)L.cout * 2u;
+        D.n_banks = (uint32_t)cp.n_banks;
+        const uint32_t a_fmt = cp.in_tensor == 0 ? 0u : 1u;
+        for (int nbk = 1; nbk <= 3; ++nbk)
+            D.idesc[nbk - 1] = (2u << 4) | (a_fmt << 7) | (1u << 10) | ((uint32_t)((nbk * L.cout) >> 3) << 17) | ((128u >> 4) << 24);
+        D.cols = (uint32_t)cp.cols;
+        D.d_base[0] = 0; D.d_base[1] = cp.n_banks > 1 ? (uint32_t)(cp.m * cp.cols) : 0u;
+        D.bar_full = (uint32_t)class_full[(size_t)cp.cls]; D.bar_done = (uint32_t)class_done[(size_t)cp.cls];
+        D.use_local = (uint32_t)cp.use_local; D.uses_per_group = (uint32_t)class_uses[(size_t)cp.cls];
+        D.n_lines = (uint32_t)cp.m; D.n_chunks = (uint32_t)cp.n_chunks;
+        D.w_rel = w_rel[(size_t)c]; D.c_rel = c_rel[(size_t)c]; D.ops_rel = ops_rel[(size_t)c]; D.passes_rel = passes_rel[(size_t)c];
+        D.out_base = plan->tensor_off[(size_t)cp.out_tensor] + out.line0;
+        D.out_plane = out.plane_bytes; D.out_pitch16 = (uint32_t)out.pitch; D.out_n_lines = (uint32_t)out.n_lines;
+        D.out_log_lines = (uint32_t)ilog2(out.n_lines); D.out_nb = (uint32_t)out.nb; D.out_logI = (uint32_t)ilog2(out.I);
+        if ((1 << D.out_log_lines) != out.n_lines) PLAN_FAIL(16);
+        D.in_logI = (uint32_t)ilog2(in.I); D.in_I = (uint32_t)in.I; D.in_n_lines = (uint32_t)in.n_lines;
+        if (L.res_tensor >= 0) {
+            const LGeo &r = T[(size_t)L.res_tensor];
+            D.res_base = plan->tensor_off[(size_t)L.res_tensor] + r.line0;
+            D.res_plane = r.plane_bytes;
+            const int res_n = 31 - L.res_shift;
+            const unsigned long long m2 = (unsigned long long)(uint32_t)L.res_mult << (32 - res_n);
+            if (L.res_mult <= 0 || m2 >= (1ull << 32)) PLAN_FAIL(17);
+            // rs((r - zp) * mult, n) = floor(((u - 128 - zp) * mult + 2^(n-1)) * 2^(32-n) / 2^32), u = r + 128
+            const long long r2 = (((1ll << (res_n - 1)) - (128ll + L.zp_res) * (long long)L.res_mult)) * (1ll << (32 - res_n));
+            D.res_m2 = (uint32_t)m2;
+            D.res_r2_lo = (uint32_t)((unsigned long long)r2 & 0xFFFFFFFFull);
+            D.res_r2_hi = (uint32_t)((unsigned long long)r2 >> 32);
+        }
+        for (size_t k = 0; k < cp.kunits.size(); ++k) { D.a_delta[k] = cp.a_delta[k]; D.a_lbo[k] = cp.a_lbo[k]; }
+        // operand reads stay inside the input's region
+        for (size_t k = 0; k < cp.kunits.size(); ++k)
+            for (const LOp &op : cp.ops) {
+                const long long lo_b = (long long)in.line0 - (long long)in.pitch * 16 + (long long)op.a_line1 * in.pitch * 16 + cp.a_delta[k];
+                const long long hi_b = lo_b + cp.a_lbo[k] + 128 * 16;
+                if (lo_b < 0 || hi_b > (long long)in.bytes) PLAN_FAIL(18);
+            }
+        memcpy(blob.data(), &D, sizeof(D));
+        memcpy(blob.data() + ops_rel[(size_t)c], cp.ops.data(), cp.ops.size() * sizeof(LOp));
+        memcpy(blob.data() + passes_rel[(size_t)c], cp.passes.data(), cp.passes.size() * 4);
+        // weights: per K-step, rows = block * cout + oc (block b = vertical tap 2 - b when stacked)
+        const int taps = L.kh * L.kw;
+        const uint32_t rows = (uint32_t)(cp.stacked ? 3 : 1) * (uint32_t)L.cout;
+        for (size_t k = 0; k < cp.kunits.size(); ++k) {
+            const int halves[2] = {cp.kunits[k].first, cp.kunits[k].second};
+            for (int hf = 0; hf < 2; ++hf) {
+                if (halves[hf] < 0) continue;
+                const ConvPlan::Unit &u = cp.units[(size_t)halves[hf]];
+                for (uint32_t n = 0; n < rows; ++n) {
+                    const int oc = (int)(n % (uint32_t)L.cout), blk = (int)(n / (uint32_t)L.cout);
+                    const int r = cp.stacked ? 2 - blk : u.r;
+                    const int tap = L.kh == 3 ? r * 3 + (u.s + 1) : 0;
+                    for (int b = 0; b < 16; ++b) {
+                        const int ci = u.pl * 16 + b;
+                        if (ci >= L.cin) continue;
+                        const int8_t wv = ML.w[((size_t)oc * L.cin + ci) * taps + tap];
+                        blob[w_rel[(size_t)c] + k * rows * 32 + (size_t)(n / 8) * 256 + (size_t)hf * 128 + (size_t)(n % 8) * 16 + b] = (uint8_t)wv;
+                    }
+                }
+            }
+        }
+        for (int oc = 0; oc < L.cout; ++oc) {
+            long long wsum = 0;
+            for (int q = 0; q < L.cin * taps; ++q) wsum += ML.w[(size_t)oc * L.cin * taps + q];
+            const int sh = ML.shift[oc];
+            if (sh < 1 || sh > 20) PLAN_FAIL(19);
+            const int nn = 31 + sh;
+            const long long biasf = (long long)ML.bias[oc] - (long long)L.zp_in * wsum;
+            const long long B = biasf * ML.mult[oc] + (1ll << (nn - 1)) + ((long long)L.zp_out << nn);
+            int32_t cst[4] = {(int32_t)(uint32_t)(B & 0xFFFFFFFFll), (int32_t)(B >> 32), ML.mult[oc], nn - 32};
+            memcpy(&blob[c_rel[(size_t)c] + (size_t)oc * 16], cst, 16);
+        }
+        (*blob_offsets)[(size_t)c] = (uint32_t)blob_out->size();
+        blob_out->insert(blob_out->end(), blob.begin(), blob.end());
+        (*csrc_out)[(size_t)c].bytes_phase = w_bytes[(size_t)c] | ((uint32_t)ph << 24);
+        (*csrc_out)[(size_t)c].smem_off = w_off[(size_t)c] | (late[(size_t)c] ? 0x80000000u : 0u);
+    }
+    plan->n_phases = n_phases;
+    plan->n_conv = n_conv;
+    plan->n_bars = (int)bar_counts_out->size();
+    plan->smem_bytes = (high + 127u) & ~127u;
+    (void)n_classes;
+    return true;
+}
+
+}  // namespace
+
+int line_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, LinePlan **out)
+{
+    *out = nullptr;
+    if (n_layers < 3 || n_classes > 128) return ISC_OK;
+    // structure: convolutions, then global average pool, then FC
+    const isc_layer &LP = layers[n_layers - 2].d, &LF = layers[n_layers - 1].d;
+    if (LP.op != ISC_GAVGPOOL || LF.op != ISC_FC) return ISC_OK;
+    if (LP.in_tensor != n_layers - 2 || LF.in_tensor != n_layers - 1) return ISC_OK;
+    if (LP.cin > 64 || LP.cin % 16 != 0 || LF.res_tensor >= 0) return ISC_OK;
+    for (int i = 0; i < n_layers - 2; ++i) {
+        const isc_layer &L = layers[i].d;
+        if (!conv_ok(L, i == 0)) return ISC_OK;
+        if ((i == 0) != (L.in_tensor == 0)) return ISC_OK;
+        if (L.res_tensor == 0) return ISC_OK;
+        // a consumer's zero-point must be the halo value its operand was written with
+        if (L.in_tensor > 0 && L.zp_in != layers[L.in_tensor - 1].d.zp_out) return ISC_OK;
+        if (L.in_tensor > i || L.res_tensor > i) return ISC_OK;
+    }
+    if (LP.zp_in != layers[n_layers - 3].d.zp_out) return ISC_OK;
+
+    LinePlan *plan = new LinePlan();
+    std::vector<uint8_t> blob, bar_counts;
+    std::vector<uint32_t> blob_off;
+    std::vector<PhaseEntry> ptab;
+    std::vector<ConvSrc> csrc;
+    if (!build_plan(layers, n_layers, in_c, in_h, in_w, n_classes, plan, &blob, &blob_off, &ptab, &csrc, &bar_counts)) {
+        delete plan;
+        return ISC_OK;
+    }
+    plan->in_c = in_c; plan->in_h = in_h; plan->in_w = in_w; plan->n_classes = n_classes;
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        cudaGetLastError(); delete plan; return ISC_ERR_CUDA;
+    }
+    if (prop.major != 10 || (size_t)prop.sharedMemPerBlockOptin < plan->smem_bytes) { delete plan; return ISC_OK; }
+    plan->sm_count = prop.multiProcessorCount;
+
+    // FC parameters (bias folded with the pool output's zero-point)
+    const int C = LP.cin;
+    std::vector<int8_t> fcw((size_t)n_classes * 64, 0);
+    std::vector<FcConst> fcc((size_t)n_classes);
+    const MegaLayerIn &MF = layers[n_layers - 1];
+    for (int o = 0; o < n_classes; ++o) {
+        long long wsum = 0;
+        for (int c = 0; c < C; ++c) {
+            fcw[(size_t)o * 64 + c] = MF.w[(size_t)o * C + c];
+            wsum += MF.w[(size_t)o * C + c];
+        }
+        FcConst k{};
+        k.mult = MF.mult[o]; k.n = 31 + MF.shift[o]; k.zp_out = LF.zp_out;
+        k.lo = LF.relu ? std::max(-128, LF.zp_out) : -128;
+        k.bias = (int32_t)(MF.bias[o] - (long long)LF.zp_in * wsum);
+        fcc[(size_t)o] = k;
+    }
+    bool cuda_ok = true;
+    auto up = [&](void **dst, const void *src, size_t bytes) {
+        if (cudaMalloc(dst, std::max<size_t>(bytes, 16)) != cudaSuccess) { cuda_ok = false; *dst = nullptr; return; }
+        if (cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice) != cudaSuccess) cuda_ok = false;
+    };
+    up((void **)&plan->d_blob, blob.data(), blob.size());
+    for (size_t c = 0; c < csrc.size(); ++c) csrc[c].gmem = (unsigned long long)(plan->d_blob + blob_off[c]);
+    up((void **)&plan->d_ptab, ptab.data(), ptab.size() * sizeof(PhaseEntry));
+    up((void **)&plan->d_conv_src, csrc.data(), csrc.size() * sizeof(ConvSrc));
+    up((void **)&plan->d_bar_counts, bar_counts.data(), bar_counts.size());
+    up((void **)&plan->d_fc_w, fcw.data(), fcw.size());
+    up((void **)&plan->d_fc_c, fcc.data(), fcc.size() * sizeof(FcConst));
+    int32_t zero = 0;
+    up((void **)&plan->d_err, &zero, sizeof(zero));
+    if (cuda_ok && cudaMalloc((void **)&plan->d_dump, kSmemLimit) != cudaSuccess) cuda_ok = false;
+    if (!cuda_ok) { cudaGetLastError(); line_free(plan); return ISC_ERR_NOMEM; }
+
+    LineParams &b = plan->base;
+    memset(&b, 0, sizeof(b));
+    b.ptab = plan->d_ptab;
+    b.conv_src = plan->d_conv_src;
+    b.bar_counts = plan->d_bar_counts;
+    b.n_bars = plan->n_bars;
+    b.n_phases = plan->n_phases;
+    b.n_conv = plan->n_conv;
+    b.in_c = in_c; b.in_H = in_h; b.in_W = in_w;
+    b.input_base = plan->tensor_off[0] + plan->tensors[0].line0;
+    b.input_pitch16 = (uint32_t)plan->tensors[0].pitch;
+    const LGeo &last = plan->tensors[(size_t)n_layers - 2];
+    b.tail_base = plan->tensor_off[(size_t)n_layers - 2] + last.line0;
+    b.tail_plane = last.plane_bytes; b.tail_pitch16 = (uint32_t)last.pitch; b.tail_logI = (uint32_t)ilog2(last.I);
+    b.tail_C = last.C; b.tail_H = last.H; b.tail_W = last.W; b.tail_n_lines = last.n_lines;
+    b.pool_mult = layers[n_layers - 2].mult[0];
+    b.pool_n = 31 + layers[n_layers - 2].shift[0];
+    b.pool_zp_in = LP.zp_in; b.pool_zp_out = LP.zp_out;
+    b.pool_lo = LP.relu ? std::max(-128, LP.zp_out) : -128;
+    b.fc_w = plan->d_fc_w; b.fc_c = plan->d_fc_c;
+    b.n_classes = n_classes;
+    b.err = plan->d_err;
+    b.stop_phase = 1 << 30;
+    *out = plan;
+    return ISC_OK;
+}
+
+void line_free(LinePlan *p)
+{
+    if (!p) return;
+    cudaFree(p->d_ptab); cudaFree(p->d_conv_src); cudaFree(p->d_bar_counts); cudaFree(p->d_blob); cudaFree(p->d_fc_w);
+    cudaFree(p->d_fc_c); cudaFree(p->d_err); cudaFree(p->d_dump);
+    delete p;
+}
+
+static int line_launch(LinePlan *p, LineParams &q, cudaStream_t st)
+{
+    if (!p->attr_set) {
+        if (cudaFuncSetAttribute(k_line, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p->smem_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            return ISC_ERR_CUDA;
+        }
+        p->attr_set = true;
+    }
+    const int grid = std::max(1, std::min(q.n_groups, p->sm_count));
+#ifdef ISC_TRACE
+    {
+        const char *lo = getenv("ISC_TRACE_LO"), *hi = getenv("ISC_TRACE_HI");
+        const unsigned vlo = lo ? (unsigned)atoi(lo) : 0u, vhi = hi ? (unsigned)atoi(hi) : 0u, zero = 0u;
+        cudaMemcpyToSymbol(g_ltrace_lo, &vlo, sizeof(vlo));
+        cudaMemcpyToSymbol(g_ltrace_hi, &vhi, sizeof(vhi));
+        cudaMemcpyToSymbol(g_ltrace_n, &zero, sizeof(zero));
+    }
+#endif
+    k_line<<<grid, kThreads, p->smem_bytes, st>>>(q);
+    return cudaGetLastError() == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
+}
+
+int line_run(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, int64_t n, int batch_hint, int32_t *d_counts,
+             int8_t *d_logits, cudaStream_t st, int64_t *launches)
+{
+    const int64_t per_launch = batch_hint > 0 ? batch_hint : (1ll << 30);
+    for (int64_t done = 0; done < n; done += per_launch) {
+        const int64_t m = std::min(per_launch, n - done);
+        LineParams q = p->base;
+        q.x = d_x;
+        q.ns = ns;
+        q.ns.first_sample = ns.first_sample + done;
+        q.n_samples = (int32_t)m;
+        q.n_groups = (int32_t)((m + kG - 1) / kG);
+        q.counts = d_counts;
+        q.logits = d_logits ? d_logits + (size_t)done * p->n_classes : nullptr;
+        int rc = line_launch(p, q, st);
+        *launches += 1;
+        if (rc) return rc;
+    }
+    return ISC_OK;
+}
+
+int line_check(LinePlan *p)
+{
+    int32_t e = 0;
+    if (cudaMemcpy(&e, p->d_err, sizeof(e), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return ISC_ERR_CUDA; }
+    if (e != 0) {
+        if (getenv("ISC_PLAN_DEBUG")) fprintf(stderr, "line engine: wait %d on barrier %d parity %d expired in CTA %d\n", e & 0xFF, (e >> 8) & 0xFFF, (e >> 20) & 1, (int)((unsigned)e >> 21));
+        cudaMemset(p->d_err, 0, sizeof(e));
+        return ISC_ERR_TIMEOUT;
+    }
+    return ISC_OK;
+}
+
+// Runs one group (samples ns.first_sample ..) up to the phase that produces `tensor` and returns that
+// tensor of the first sample as [C][H][W] int32.
+int line_debug_tensor(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, int tensor, int32_t *out_chw,
+                      int32_t *d_counts_scratch, cudaStream_t st, int64_t *launches)
+{
+    if (tensor < 0 || tensor >= (int)p->tensors.size() || p->tensors[(size_t)tensor].buffer < 0) return ISC_ERR_UNSUPPORTED;
+    const LGeo &t = p->tensors[(size_t)tensor];
+    LineParams q = p->base;
+    q.x = d_x; q.ns = ns; q.n_samples = 1; q.n_groups = 1; q.counts = d_counts_scratch; q.logits = nullptr;
+    q.stop_phase = t.producer_phase;
+    q.dump_off = p->tensor_off[(size_t)tensor]; q.dump_bytes = t.bytes; q.dump = p->d_dump;
+    int rc = line_launch(p, q, st);
+    *launches += 1;
+    if (rc) return rc;
+    std::vector<uint8_t> h(t.bytes);
+    if (cudaMemcpyAsync(h.data(), p->d_dump, t.bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ISC_ERR_CUDA; }
+    if ((rc = line_check(p))) return rc;
+    for (int c = 0; c < t.C; ++c)
+        for (int y = 0; y < t.H; ++y)
+            for (int x = 0; x < t.W; ++x) {
+                const int line = y % t.n_lines, band = y / t.n_lines;
+                const size_t at = (size_t)(c / 16) * t.plane_bytes + t.line0 +
+                                  ((size_t)line * t.pitch + (size_t)x * t.I + (size_t)band * 4) * 16 + (size_t)(c % 16);
+                const uint8_t b = h[at];
+                out_chw[((size_t)c * t.H + y) * t.W + x] = tensor == 0 ? (int32_t)b : (int32_t)(int8_t)b;
+            }
+    return ISC_OK;
+}
+
+#ifdef ISC_TRACE
+// Copies the recorded triples to the host; returns how many there are.
+extern "C" int isc_line_trace_read(unsigned long long *out, int max_events)
+{
+    unsigned n = 0;
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(&n, g_ltrace_n, sizeof(n));
+    n = std::min(n, std::min(kTraceMax, (unsigned)max_events));
+    cudaMemcpyFromSymbol(out, g_ltrace, (size_t)n * 3 * sizeof(unsigned long long));
+    return (int)n;
+}
+#endif
+
+}  // namespace isc

@@ -1,0 +1,32 @@
+// Line-tiled shared-memory-resident tensor-core engine for CIFAR-shaped residual networks.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "isc.h"
+#include "isc_internal.h"
+#include "isc_mega.h"
+
+namespace isc {
+
+struct LinePlan;
+
+// Builds the plan when the network fits the engine; otherwise *out = nullptr and ISC_OK.
+int line_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes,
+               LinePlan **out);
+void line_free(LinePlan *p);
+
+// Runs samples first..first+n-1 (ns.first_sample = first) and adds their votes to d_counts.
+int line_run(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, int64_t n, int batch_hint,
+             int32_t *d_counts, int8_t *d_logits, cudaStream_t st, int64_t *launches);
+
+// Debug read-back: runs one group up to the phase producing model tensor `tensor` and returns that
+// tensor of sample ns.first_sample as [C][H][W] int32 (host).
+int line_debug_tensor(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, int tensor, int32_t *out_chw,
+                      int32_t *d_counts_scratch, cudaStream_t st, int64_t *launches);
+
+// After the stream has been synchronised: ISC_OK, or ISC_ERR_TIMEOUT if a bounded wait expired.
+int line_check(LinePlan *p);
+
+}  // namespace isc

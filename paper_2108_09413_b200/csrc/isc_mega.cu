@@ -22,6 +22,7 @@
 // flag, all remaining waits fall through, and the host reports ISC_ERR_TIMEOUT.
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -32,6 +33,27 @@
 namespace isc {
 
 namespace {
+
+#ifdef ISC_TRACE
+// Timeline instrumentation, compiled only with -DISC_TRACE: CTA 0 records (warp and event, round, SM clock)
+// for the rounds in [g_trace_lo, g_trace_hi).
+constexpr unsigned kTraceMax = 16384;
+__device__ unsigned long long g_trace[3 * kTraceMax];
+__device__ unsigned int g_trace_n, g_trace_lo, g_trace_hi;
+__device__ __forceinline__ void trace(int ev, uint32_t r)
+{
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && r >= g_trace_lo && r < g_trace_hi) {
+        const unsigned i = atomicAdd(&g_trace_n, 1u);
+        if (i < kTraceMax) {
+            g_trace[3 * i] = (unsigned long long)(ev | ((threadIdx.x >> 5) << 8));
+            g_trace[3 * i + 1] = r;
+            g_trace[3 * i + 2] = (unsigned long long)clock64();
+        }
+    }
+}
+#else
+#define trace(ev, r) ((void)0)
+#endif
 
 constexpr int kIssuers = 4;                 // warps 0..3: an elected lane of each issues the MMAs of every 4th tile
 constexpr int kEpiWarps = 8;                // warps 4..11: epilogue, two warpgroups of "fat" threads (168 registers)
@@ -481,6 +503,7 @@ __device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem,
     for (int k = 0; k < ia.n_rounds; ++k) {
         const uint32_t r = ia.first + (uint32_t)k, h = r & 1u;
         if (!round_start_wait(w, ctrl, r, round_dep(ia.first, k, ia.n_rounds, ia.full_sync))) return false;
+        trace(1, r);
         tc_fence_after();
         const int t0 = k * tpr, t1 = min(n_tiles, t0 + tpr);
         const uint32_t d0 = tmem + h * kHalfCols;
@@ -496,6 +519,7 @@ __device__ __forceinline__ bool issue_phase(Waiter w, Ctrl *ctrl, uint32_t tmem,
             }
         }
         mma_commit(smem_u32(&ctrl->full[h]));        // arrives at once when this warp had no tile in the round
+        trace(2, r);
     }
     return true;
 }
@@ -772,6 +796,7 @@ __device__ __forceinline__ void round_done(const EpiCtx &c, uint32_t r)
     fence_proxy_async();
     __syncwarp();
     if (c.lane == 0) mbar_arrive(smem_u32(&c.ctrl->done[r & 1u]));
+    trace(4, r);
 }
 
 // The rounds of one CONV phase.  A warp owns 32 rows (its tensor-memory lanes) of every tile; the two warpgroups
@@ -796,6 +821,7 @@ __device__ __noinline__ void conv_phase_rounds(Waiter w, const EpiCtx &c_in, con
         const int t0 = k * tpr, t1 = min(n_tiles, t0 + tpr);
         if (ok) ok = w.barrier(smem_u32(&c.ctrl->full[h]), (r >> 1) & 1u, ERR_WAIT_FULL);
         ok = __all_sync(0xffffffffu, ok);
+        trace(3, r);
         tc_fence_after();
         const uint32_t half_addr = lane_base + h * kHalfCols;
         const int n_pairs = (t1 - t0 + 1) >> 1;
@@ -923,6 +949,7 @@ __device__ __noinline__ void epi_role(const MegaParams &p, EpiCtx &c, int it, in
         const int n_items = (int)e.y;
         ok = r == 0u || w.barrier(smem_u32(&c.ctrl->done[(r & 1u) ^ 1u]), ((r - 1u) >> 1) & 1u, ERR_WAIT_ITEMS);
         ok = __all_sync(0xffffffffu, ok);
+        trace(5 + kind, r);
         for (int i = c.wg; i < n_items; i += kWarpGroups) {
             if (!ok) break;
             if (kind == PH_FILL) {
@@ -1571,6 +1598,15 @@ static int mega_launch(MegaPlan *p, MegaParams &q, cudaStream_t st)
         p->attr_set = true;
     }
     const int grid = std::max(1, std::min(q.n_groups, p->sm_count));
+#ifdef ISC_TRACE
+    {
+        const char *lo = getenv("ISC_TRACE_LO"), *hi = getenv("ISC_TRACE_HI");
+        const unsigned vlo = lo ? (unsigned)atoi(lo) : 0u, vhi = hi ? (unsigned)atoi(hi) : 0u, zero = 0u;
+        cudaMemcpyToSymbol(g_trace_lo, &vlo, sizeof(vlo));
+        cudaMemcpyToSymbol(g_trace_hi, &vhi, sizeof(vhi));
+        cudaMemcpyToSymbol(g_trace_n, &zero, sizeof(zero));
+    }
+#endif
     k_mega<<<grid, kThreads, p->smem_bytes, st>>>(q);
     return cudaGetLastError() == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
 }
@@ -1641,5 +1677,18 @@ int mega_debug_tensor(MegaPlan *p, const uint8_t *d_x, const NoiseStream &ns, in
             }
     return ISC_OK;
 }
+
+#ifdef ISC_TRACE
+// Copies the recorded triples to the host; returns how many there are.
+extern "C" int isc_trace_read(unsigned long long *out, int max_events)
+{
+    unsigned n = 0;
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n));
+    n = std::min(n, std::min(kTraceMax, (unsigned)max_events));
+    cudaMemcpyFromSymbol(out, g_trace, (size_t)n * 3 * sizeof(unsigned long long));
+    return (int)n;
+}
+#endif
 
 }  // namespace isc
