@@ -54,23 +54,35 @@ using namespace tc;
 namespace {
 
 #ifdef ISC_TRACE
-// Timeline instrumentation, compiled only with -DISC_TRACE: CTA 0 records (warp and event, tag, SM clock).
-constexpr unsigned kTraceMax = 32768;
-__device__ unsigned long long g_ltrace[3 * kTraceMax];
-__device__ unsigned int g_ltrace_n, g_ltrace_lo, g_ltrace_hi;
-__device__ __forceinline__ void ltrace(int ev, uint32_t cg, uint32_t tag)
+// Timeline instrumentation, compiled only with -DISC_TRACE: CTA 0 records (event, warp, line, chunk, convolution;
+// value) pairs in global memory for the convolutions in [c_trace_lo, c_trace_hi); the slot counter lives in the last
+// 16 bytes of the control block.
+constexpr unsigned kTraceMax = 16384;                // 8 bytes each
+__device__ unsigned int g_ltrace[2 * kTraceMax];
+__device__ unsigned int g_ltrace_n;
+__constant__ unsigned int c_trace_lo, c_trace_hi;
+constexpr unsigned kTraceCounterOff = 7168 - 16;
+__device__ __forceinline__ void ltrace_val(int ev, uint32_t cg, uint32_t tag, uint32_t val)
 {
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && cg >= g_ltrace_lo && cg < g_ltrace_hi) {
-        const unsigned i = atomicAdd(&g_ltrace_n, 1u);
+    extern __shared__ __align__(128) uint8_t trace_smem[];
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && cg >= c_trace_lo && cg < c_trace_hi) {
+        const unsigned i = atomicAdd(reinterpret_cast<unsigned int *>(trace_smem + kTraceCounterOff), 1u);
         if (i < kTraceMax) {
-            g_ltrace[3 * i] = (unsigned long long)(ev | ((threadIdx.x >> 5) << 8));
-            g_ltrace[3 * i + 1] = ((unsigned long long)cg << 16) | tag;
-            g_ltrace[3 * i + 2] = (unsigned long long)clock64();
+            g_ltrace[2 * i] = (unsigned)ev | ((threadIdx.x >> 5) << 4) | ((tag & 0x7FFu) << 9) | ((cg - c_trace_lo) << 20);
+            g_ltrace[2 * i + 1] = val;
         }
     }
 }
+__device__ __forceinline__ void ltrace(int ev, uint32_t cg, uint32_t tag) { ltrace_val(ev, cg, tag, (uint32_t)clock64()); }
+#define LT_CLOCK(v) const uint32_t v = (uint32_t)clock64()
+#define LT_ARRAY(name, n) uint32_t name[n]
+#define LT_SET(name, i, v) do { if ((i) < 40) name[(i)] = (v); } while (0)
 #else
 #define ltrace(ev, cg, tag) ((void)0)
+#define ltrace_val(ev, cg, tag, val) ((void)0)
+#define LT_CLOCK(v) ((void)0)
+#define LT_ARRAY(name, n) ((void)0)
+#define LT_SET(name, i, v) ((void)0)
 #endif
 
 constexpr int kG = 4;                       // samples per group
@@ -81,15 +93,16 @@ constexpr int kThreads = 32 * (kEpiWarps + 1);
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kMaxKsteps = 18;
 constexpr int kMaxPhases = 160;
-constexpr int kMaxBars = 192;
+constexpr int kMaxBars = 128;
 constexpr int kMaxLines = 32;               // output lines of one convolution
-constexpr int kCtrlBytes = 5120;
+constexpr int kCtrlBytes = 7168;
+constexpr int kMaxConv = 128;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
 enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
-enum { ERR_NONE = 0, ERR_WAIT_DONE = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_FULL = 4, ERR_WAIT_DRAIN = 5 };
+enum { ERR_NONE = 0, ERR_WAIT_DONE = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_READY = 3, ERR_WAIT_FULL = 4, ERR_WAIT_DRAIN = 5 };
 enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8 };
 enum { OPF_WAIT_ALL = 1 };
 
@@ -102,18 +115,17 @@ struct alignas(16) PhaseEntry { uint32_t kind, a, b, c; };
 // Where the blob of convolution c comes from (global) and goes to (shared).
 struct alignas(16) ConvSrc { unsigned long long gmem; uint32_t bytes_phase, smem_off; };   // bytes | phase << 24
 
-// One MMA chain: input line, accumulator columns, dependencies and completions.
+// One MMA chain in the form the issuing thread consumes: accumulator columns, what to add to the operand
+// descriptors' start addresses, and the barriers (as byte offsets, 0xFFFF = none) of its dependencies and completions.
 struct alignas(16) LOp {
-    uint8_t a_line1;        // input line + 1 (line -1 is the padding line above)
-    uint8_t b_block;        // first weight block (stacked: 2 - vertical tap of the lowest output line)
-    uint8_t n_blocks;       // N = n_blocks * cout
-    uint8_t flags;          // OPF_WAIT_ALL: every line of the previous convolution
-    uint16_t d_col;         // first accumulator column within the bank
-    uint8_t n_wait, n_commit;
-    uint8_t wait[4];        // output lines of the previous convolution that must be stored
-    uint8_t commit[4];      // output lines of this convolution whose accumulators are complete after the chain
+    uint32_t d_col;         // first accumulator column within the bank
+    uint32_t idesc;         // instruction descriptor (N = blocks * cout)
+    uint32_t a_add, b_add;  // 16-byte units: (input line + 1) * pitch, first weight block * block size
+    uint16_t wait[4];       // 8 * unit of the previous convolution that must be stored
+    uint16_t commit[3];     // 8 * unit of this convolution whose accumulators are complete after the chain
+    uint16_t flags;         // OPF_WAIT_ALL: every line of the previous convolution
 };
-static_assert(sizeof(LOp) == 16, "one operation is one 16-byte load");
+static_assert(sizeof(LOp) == 32, "one operation is two 16-byte loads");
 
 // Head of every blob: everything the issuing thread and the epilogue need to know about the convolution.
 struct alignas(16) LConvDesc {
@@ -128,8 +140,8 @@ struct alignas(16) LConvDesc {
     uint32_t out_log_lines, out_nb, out_logI, res_base;
     uint32_t res_plane, in_logI, in_I, in_n_lines;
     int32_t lo; uint32_t res_m2, res_r2_lo, res_r2_hi;
-    int32_t a_delta[kMaxKsteps];
-    uint32_t a_lbo[kMaxKsteps];
+    uint32_t b_lo0, kstep16, pad0, pad1;       // low word of the first K-step's weight descriptor (shared-memory base 0)
+    uint32_t a_lo[kMaxKsteps + 2];             // low words of the operand descriptors of line -1 (shared-memory base 0)
 };
 static_assert(sizeof(LConvDesc) % 16 == 0, "blob sections stay 16-byte aligned");
 
@@ -165,10 +177,12 @@ struct Ctrl {
     unsigned long long wbar[3], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
+    uint32_t stored[kMaxBars];              // per unit: stores of its 16-channel chunks by a warp, counted over the whole run
     int32_t hist[128];
     PhaseEntry ptab[kMaxPhases];
+    ConvSrc csrc[kMaxConv];
 };
-static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
+static_assert(sizeof(Ctrl) <= kCtrlBytes - 16, "control block too large");
 
 // ------------------------------------------------------------------ device helpers
 
@@ -195,6 +209,27 @@ __device__ __forceinline__ long long mad_wide_u(uint32_t a, uint32_t b, long lon
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
     return d;
 }
+// Per-channel constants of a blob that is complete in shared memory (the address derives from a value read after
+// the wait for the blob): a plain load the compiler may schedule ahead of the tensor-memory wait.
+__device__ __forceinline__ ChanConst ld_chan_const_early(uint32_t addr)
+{
+    long long b, ms;
+    asm("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(b), "=l"(ms) : "r"(addr));
+    ChanConst c;
+    c.B = b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(c.mult), "=r"(c.s) : "l"(ms));
+    return c;
+}
+__device__ __forceinline__ void red_release_add(uint32_t addr, uint32_t v)
+{
+    asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
 // byte K of w, zero-extended
 template <int K>
 __device__ __forceinline__ uint32_t ubyte(uint32_t w)
@@ -220,6 +255,7 @@ struct Waiter {
     __device__ __forceinline__ bool barrier(uint32_t bar, uint32_t parity, int code)
     {
         if (mbar_test(bar, parity)) return true;
+        if (mbar_try(bar, parity)) return true;         // parks the thread; the clock is read only when this gives up
         const unsigned long long t0 = globaltimer();
         for (int spin = 0;; ++spin) {
             if (mbar_try(bar, parity)) return true;
@@ -229,17 +265,31 @@ struct Waiter {
             }
         }
     }
+    // Wait until a counter in shared memory has reached `expected` (counters only grow).
+    __device__ __forceinline__ bool counter(uint32_t addr, uint32_t expected, int code)
+    {
+        if ((int32_t)(ld_acquire_u32(addr) - expected) >= 0) return true;
+        const unsigned long long t0 = globaltimer();
+        for (int spin = 0;; ++spin) {
+            if ((int32_t)(ld_acquire_u32(addr) - expected) >= 0) return true;
+            if ((spin & 15) == 15) {
+                if (aborted()) return false;
+                if (globaltimer() - t0 > kWaitLimitNs) { fail(code, addr, 0); return false; }
+            }
+        }
+    }
 };
 
 // ------------------------------------------------------------------ issuing thread
 
-struct PrevConv { uint32_t done_addr, parity, n_lines; };      // n_lines = 0: nothing to wait for
+struct PrevConv { uint32_t done_addr, expected, n_lines; };    // counters of its units, their value when stored; n_lines = 0: nothing to wait for
 
 struct IssueCtx {
-    uint32_t desc, ops, n_ops, a0, w0, pitch16, bblock16, kstep_bytes, d0, stacked, full_addr, cg;
-    uint32_t idesc[3];
+    uint32_t desc, ops, n_ops, s16, b_lo0, kstep16, d0, stacked, full_addr, cg;
 };
 
+// All operations of one convolution.  The low words of the operand descriptors stay in registers; an operation adds
+// its line and block offsets to their start-address fields.
 template <int KS>
 __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const PrevConv &prev, uint32_t n_ksteps)
 {
@@ -248,56 +298,83 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
     const uint32_t ahi = (uint32_t)(make_desc(0, 0, 128) >> 32), bhi = (uint32_t)(make_desc(0, 128, 256) >> 32);
     if (KS > 0) {
 #pragma unroll
-        for (int k = 0; k < NK; ++k) {
-            const uint32_t delta = lds32(ic.desc + offsetof(LConvDesc, a_delta) + 4 * k);
-            const uint32_t lbo = lds32(ic.desc + offsetof(LConvDesc, a_lbo) + 4 * k);
-            alo[k] = (uint32_t)make_desc(ic.a0 + delta, lbo, 128);
-            blo[k] = (uint32_t)make_desc(ic.w0 + (uint32_t)k * ic.kstep_bytes, 128, 256);
+        for (int k4 = 0; k4 < NK; k4 += 4) {
+            const uint4 v = ld_shared_v4(ic.desc + offsetof(LConvDesc, a_lo) + 4 * k4);
+            const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (k4 + q < NK) alo[k4 + q] = vv[q] + ic.s16;
         }
+#pragma unroll
+        for (int k = 0; k < NK; ++k) blo[k] = ic.b_lo0 + ic.s16 + (uint32_t)k * ic.kstep16;
     }
-    uint4 o = ld_shared_v4(ic.ops);
+    uint32_t at = ic.ops;
+    uint4 n0 = ld_shared_v4(at), n1 = ld_shared_v4(at + 16);
+    LT_ARRAY(tlogA, 40);
+    LT_ARRAY(tlogB, 40);
+    LT_ARRAY(tlogC, 40);
+    LT_ARRAY(tlogD, 40);
     for (uint32_t i = 0; i < ic.n_ops; ++i) {
-        const uint4 cur = o;
-        if (i + 1 < ic.n_ops) o = ld_shared_v4(ic.ops + 16 * (i + 1));
-        const uint32_t a_line1 = cur.x & 0xFF, b_block = (cur.x >> 8) & 0xFF, n_blocks = (cur.x >> 16) & 0xFF, flags = cur.x >> 24;
-        const uint32_t d_col = cur.y & 0xFFFF, n_wait = (cur.y >> 16) & 0xFF, n_commit = cur.y >> 24;
+        LT_CLOCK(tA);
+        const uint4 r0 = n0, r1 = n1;         // d_col, idesc, a_add, b_add | wait 0-1, wait 2-3, commit 0-1, commit 2 and flags
+        at += 32;
+        if (i + 1 < ic.n_ops) { n0 = ld_shared_v4(at); n1 = ld_shared_v4(at + 16); }
+        // units of the previous convolution this operation depends on
         if (prev.n_lines) {
-            if (flags & OPF_WAIT_ALL) {
+            if ((r1.w >> 16) & OPF_WAIT_ALL) {
                 for (uint32_t l = 0; l < prev.n_lines; ++l)
-                    if (!w.barrier(prev.done_addr + 8 * l, prev.parity, ERR_WAIT_DONE)) return false;
+                    if (!w.counter(prev.done_addr + 4 * l, prev.expected, ERR_WAIT_DONE)) return false;
             }
-            for (uint32_t q = 0; q < n_wait; ++q)
-                if (!w.barrier(prev.done_addr + 8 * ((cur.z >> (8 * q)) & 0xFF), prev.parity, ERR_WAIT_DONE)) return false;
+            if ((r1.x & 0xFFFFu) != 0xFFFFu) {
+                if (!w.counter(prev.done_addr + (r1.x & 0xFFFFu), prev.expected, ERR_WAIT_DONE)) return false;
+                if ((r1.x >> 16) != 0xFFFFu) {
+                    if (!w.counter(prev.done_addr + (r1.x >> 16), prev.expected, ERR_WAIT_DONE)) return false;
+                    if ((r1.y & 0xFFFFu) != 0xFFFFu && !w.counter(prev.done_addr + (r1.y & 0xFFFFu), prev.expected, ERR_WAIT_DONE)) return false;
+                    if ((r1.y >> 16) != 0xFFFFu && !w.counter(prev.done_addr + (r1.y >> 16), prev.expected, ERR_WAIT_DONE)) return false;
+                }
+            }
         }
-        ltrace(1, ic.cg, a_line1);
+        LT_CLOCK(tB);
         tc_fence_after();
-        const uint32_t d = ic.d0 + d_col, idesc = ic.idesc[n_blocks - 1];
-        const uint32_t a_add = a_line1 * ic.pitch16, b_add = b_block * ic.bblock16;
+        const uint32_t d = ic.d0 + r0.x;
         if (KS > 0) {
 #pragma unroll
             for (int k = 0; k < NK; ++k) {
-                const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[k] + a_add);
-                const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)(blo[k] + b_add);
-                mma_i8(d, ad, bd, idesc, ic.stacked | (uint32_t)(k > 0));
+                const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[k] + r0.z);
+                const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)(blo[k] + r0.w);
+                mma_i8(d, ad, bd, r0.y, ic.stacked | (uint32_t)(k > 0));
             }
         } else {
             for (uint32_t k = 0; k < n_ksteps; ++k) {
-                const uint32_t delta = lds32(ic.desc + offsetof(LConvDesc, a_delta) + 4 * k);
-                const uint32_t lbo = lds32(ic.desc + offsetof(LConvDesc, a_lbo) + 4 * k);
-                const uint64_t ad = make_desc(ic.a0 + delta + a_add * 16u, lbo, 128);
-                const uint64_t bd = make_desc(ic.w0 + k * ic.kstep_bytes + b_add * 16u, 128, 256);
-                mma_i8(d, ad, bd, idesc, ic.stacked | (uint32_t)(k > 0));
+                const uint32_t a_lo = lds32(ic.desc + offsetof(LConvDesc, a_lo) + 4 * k) + ic.s16;
+                const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(a_lo + r0.z);
+                const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)(ic.b_lo0 + ic.s16 + k * ic.kstep16 + r0.w);
+                mma_i8(d, ad, bd, r0.y, ic.stacked | (uint32_t)(k > 0));
             }
         }
-        for (uint32_t q = 0; q < n_commit; ++q) commit_to(ic.full_addr + 8 * ((cur.w >> (8 * q)) & 0xFF));
-        ltrace(2, ic.cg, a_line1);
+        LT_CLOCK(tC);
+        if ((r1.z & 0xFFFFu) != 0xFFFFu) {
+            commit_to(ic.full_addr + (r1.z & 0xFFFFu));
+            if ((r1.z >> 16) != 0xFFFFu) {
+                commit_to(ic.full_addr + (r1.z >> 16));
+                if ((r1.w & 0xFFFFu) != 0xFFFFu) commit_to(ic.full_addr + (r1.w & 0xFFFFu));
+            }
+        }
+        LT_CLOCK(tD);
+        LT_SET(tlogA, i, tA);
+        LT_SET(tlogB, i, tB);
+        LT_SET(tlogC, i, tC);
+        LT_SET(tlogD, i, tD);
     }
+#ifdef ISC_TRACE
+    for (uint32_t i = 0; i < ic.n_ops && i < 40; ++i) { ltrace_val(1, ic.cg, i, tlogA[i]); ltrace_val(2, ic.cg, i, tlogB[i]); ltrace_val(5, ic.cg, i, tlogC[i]); ltrace_val(6, ic.cg, i, tlogD[i]); }
+#endif
     return true;
 }
 
 __device__ __forceinline__ void issue_weights(const ConvSrc *src, uint32_t sbase, uint32_t wbar_addr)
 {
-    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
+    const uint4 v = *reinterpret_cast<const uint4 *>(src);
     const void *gmem = reinterpret_cast<const void *>(((unsigned long long)v.y << 32) | v.x);
     const uint32_t bytes = v.z & 0xFFFFFFu;
     mbar_expect_tx(wbar_addr, bytes);
@@ -309,33 +386,34 @@ __device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32
                                          uint32_t cg, int conv_index, int it, PrevConv &prev)
 {
     Waiter w{ctrl, p.err};
+    LT_CLOCK(t_enter);
     // The next blob's place was last used by the convolution before the previous one, which is complete; a blob
     // marked late takes the place of something the previous convolution still uses and is copied further down.
     bool late_copy = false;
     if (conv_index + 1 < p.n_conv) {
-        const ConvSrc *nxt = p.conv_src + conv_index + 1;
-        if ((int)(__ldg(&nxt->bytes_phase) >> 24) <= p.stop_phase) {
-            late_copy = (__ldg(&nxt->smem_off) >> 31) != 0;
+        const ConvSrc *nxt = ctrl->csrc + conv_index + 1;
+        if ((int)(nxt->bytes_phase >> 24) <= p.stop_phase) {
+            late_copy = (nxt->smem_off >> 31) != 0;
             if (!late_copy) issue_weights(nxt, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
         }
     }
+    LT_CLOCK(t_wissued);
     if (!w.barrier(smem_u32(&ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS)) return false;
+    LT_CLOCK(t_wbar);
     const uint32_t desc = sbase + blob_off;
     const uint4 h0 = ld_shared_v4(desc);                                    // n_ops, n_passes, n_ksteps, flags
     const uint4 h1 = ld_shared_v4(desc + offsetof(LConvDesc, a_base));      // a_base, pitch16, bblock16, n_banks
-    const uint4 h2 = ld_shared_v4(desc + offsetof(LConvDesc, idesc));       // idesc[3], cols
     const uint4 h3 = ld_shared_v4(desc + offsetof(LConvDesc, d_base));      // d_base[2], bar_full, bar_done
     const uint4 h4 = ld_shared_v4(desc + offsetof(LConvDesc, use_local));   // use_local, uses_per_group, n_lines, n_chunks
     const uint4 h5 = ld_shared_v4(desc + offsetof(LConvDesc, w_rel));       // w_rel, c_rel, ops_rel, passes_rel
+    const uint4 hb = ld_shared_v4(desc + offsetof(LConvDesc, b_lo0));       // b_lo0, kstep16
     const uint32_t use = (uint32_t)it * h4.y + h4.x;
     IssueCtx ic;
     ic.desc = desc; ic.ops = desc + h5.z; ic.n_ops = h0.x;
-    ic.a0 = sbase + h1.x; ic.w0 = desc + h5.x; ic.pitch16 = h1.y; ic.bblock16 = h1.z;
+    ic.s16 = sbase >> 4; ic.b_lo0 = hb.x; ic.kstep16 = hb.y;
     ic.d0 = tmem + ((h1.w > 1 && (use & 1u)) ? h3.y : h3.x);
     ic.stacked = (h0.w & CF_STACKED) ? 1u : 0u;
-    ic.kstep_bytes = (ic.stacked ? 3u : 1u) * h2.w * 32u;
     ic.full_addr = smem_u32(&ctrl->bars[h3.z]);
-    ic.idesc[0] = h2.x; ic.idesc[1] = h2.y; ic.idesc[2] = h2.z;
     ic.cg = cg;
     bool ok;
     switch (h0.z) {
@@ -348,12 +426,14 @@ __device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32
     default: ok = issue_ops<0>(w, ic, prev, h0.z); break;
     }
     if (!ok) return false;
-    // Every line of the previous convolution has been waited for by one of the operations above (the planner
-    // sees to it), exactly once: that convolution is complete, and whatever reads its output later, or reuses
-    // what it read, needs no wait of its own.
-    if (late_copy) issue_weights(p.conv_src + conv_index + 1, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
-    prev.done_addr = smem_u32(&ctrl->bars[h3.w]);
-    prev.parity = use & 1u;
+    LT_CLOCK(t_done);
+    ltrace_val(8, cg, 0, t_enter); ltrace_val(9, cg, 0, t_wissued); ltrace_val(10, cg, 0, t_wbar); ltrace_val(11, cg, 0, t_done);
+    // Every unit of the previous convolution has been waited for on behalf of an operation above (the planner sees
+    // to it): that convolution is complete, and whatever reads its output later, or reuses what it read, needs no
+    // wait of its own.  A blob marked late may now take the place of something it used.
+    if (late_copy) issue_weights(ctrl->csrc + conv_index + 1, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
+    prev.done_addr = smem_u32(&ctrl->stored[h3.w]);
+    prev.expected = 4u * h4.w * (use + 1u);
     prev.n_lines = h4.z;
     return true;
 }
@@ -421,10 +501,8 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
     uint32_t line[SUP];
 #pragma unroll
     for (int j = 0; j < SUP; ++j) line[j] = (pw >> (8 * j)) & 0xFFu;
-    const uint32_t ch = (pw >> 16) & 0xFFu;
-#pragma unroll
-    for (int j = 0; j < SUP; ++j)
-        if (ok) ok = w.barrier(E.full_addr + 8u * line[j], E.parity, ERR_WAIT_FULL);
+    const uint32_t ch = (pw >> 16) & 0xFu, unit = pw >> 24;
+    if (ok) ok = w.barrier(E.full_addr + 8u * unit, E.parity, ERR_WAIT_FULL);
     ok = __all_sync(0xffffffffu, ok);
     ltrace(3, cg, line[0] | (ch << 8));
     tc_fence_after();
@@ -451,8 +529,8 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
         uint32_t out[SUP][4];
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const ChanConst c0 = ld_chan_const(cbase + (4 * g + 0) * 16), c1 = ld_chan_const(cbase + (4 * g + 1) * 16);
-            const ChanConst c2 = ld_chan_const(cbase + (4 * g + 2) * 16), c3 = ld_chan_const(cbase + (4 * g + 3) * 16);
+            const ChanConst c0 = ld_chan_const_early(cbase + (4 * g + 0) * 16), c1 = ld_chan_const_early(cbase + (4 * g + 1) * 16);
+            const ChanConst c2 = ld_chan_const_early(cbase + (4 * g + 2) * 16), c3 = ld_chan_const_early(cbase + (4 * g + 3) * 16);
 #pragma unroll
             for (int j = 0; j < SUP; ++j) {
                 const int y0 = requant1<kRes, kLo, 0>(acc[j][4 * g + 0], c0, rw[j][g], E);
@@ -470,16 +548,13 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
     tc_fence_before();
     fence_proxy_async();
     __syncwarp();
-    if (c.lane == 0) {
-#pragma unroll
-        for (int j = 0; j < SUP; ++j) mbar_arrive(E.done_addr + 8u * line[j]);
-    }
+    if (c.lane == 0) red_release_add(E.done_addr + 4u * unit, 1u);
     ltrace(4, cg, line[0] | (ch << 8));
 }
 
 template <bool kRes, bool kLo>
 __device__ __noinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes,
-                                             uint32_t last_line, uint32_t cg)
+                                             uint32_t last_unit, uint32_t cg)
 {
     const EpiConv E = E_in;
     const EpiCtx c = c_in;
@@ -487,12 +562,12 @@ __device__ __noinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, cons
 #pragma unroll 1
     for (uint32_t i = (uint32_t)c.set; i < n_passes; i += kSets) {
         const uint32_t pw = lds32(passes + 4u * i);
-        if ((pw >> 24) == 2u) epi_pass<kRes, kLo, 2>(w, E, c, pw, ok, cg);
+        if (((pw >> 20) & 0xFu) == 2u) epi_pass<kRes, kLo, 2>(w, E, c, pw, ok, cg);
         else epi_pass<kRes, kLo, 1>(w, E, c, pw, ok, cg);
     }
-    // Every warp leaves a convolution only after its last accumulators are complete, hence all of them: a later
+    // Every warp leaves a convolution only after its last unit's accumulators are complete, hence all of them: a later
     // wait for the next use of any of these barriers then always refers to the phase that is still open.
-    if (ok) w.barrier(E.full_addr + 8u * last_line, E.parity, ERR_WAIT_FULL);
+    if (ok) w.barrier(E.full_addr + 8u * last_unit, E.parity, ERR_WAIT_FULL);
 }
 
 __device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint32_t blob_off, uint32_t cg, int it)
@@ -518,7 +593,7 @@ __device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint
     E.d0 = (h1.w > 1 && (use & 1u)) ? h3.y : h3.x;
     E.cols = h2.w;
     E.full_addr = smem_u32(&c.ctrl->bars[h3.z]);
-    E.done_addr = smem_u32(&c.ctrl->bars[h3.w]);
+    E.done_addr = smem_u32(&c.ctrl->stored[h3.w]);
     E.parity = use & 1u;
     E.const_addr = desc + h5.y;
     E.out_base = c.sbase + h6.x; E.out_plane = h6.y; E.out_pitch16 = h6.z; E.out_n_lines = h6.w;
@@ -527,14 +602,13 @@ __device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint
     E.lo = (int32_t)h9.x; E.res_m2 = h9.y;
     E.res_r2 = (long long)(((unsigned long long)h9.w << 32) | h9.z);
     const uint32_t passes = desc + h5.w, n_passes = h0.y;
-    // the line whose accumulators complete last closes the pass list
-    const uint32_t last_pw = lds32(passes + 4u * (n_passes - 1u));
-    const uint32_t last_line = (last_pw >> 24) == 2u ? (last_pw >> 8) & 0xFFu : last_pw & 0xFFu;
+    // the unit whose accumulators complete last closes the pass list
+    const uint32_t last_unit = lds32(passes + 4u * (n_passes - 1u)) >> 24;
     switch (E.flags & (CF_RES | CF_LO)) {
-    case 0: epi_conv_passes<false, false>(w, E, c, passes, n_passes, last_line, cg); break;
-    case CF_RES: epi_conv_passes<true, false>(w, E, c, passes, n_passes, last_line, cg); break;
-    case CF_LO: epi_conv_passes<false, true>(w, E, c, passes, n_passes, last_line, cg); break;
-    default: epi_conv_passes<true, true>(w, E, c, passes, n_passes, last_line, cg); break;
+    case 0: epi_conv_passes<false, false>(w, E, c, passes, n_passes, last_unit, cg); break;
+    case CF_RES: epi_conv_passes<true, false>(w, E, c, passes, n_passes, last_unit, cg); break;
+    case CF_LO: epi_conv_passes<false, true>(w, E, c, passes, n_passes, last_unit, cg); break;
+    default: epi_conv_passes<true, true>(w, E, c, passes, n_passes, last_unit, cg); break;
     }
 }
 
@@ -658,6 +732,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     }
     for (int i = threadIdx.x; i < 128; i += blockDim.x) ctrl->hist[i] = 0;
     for (int i = threadIdx.x; i < p.n_phases; i += blockDim.x) ctrl->ptab[i] = p.ptab[i];
+    for (int i = threadIdx.x; i < p.n_conv; i += blockDim.x) ctrl->csrc[i] = p.conv_src[i];
+    for (int i = threadIdx.x; i < kMaxBars; i += blockDim.x) ctrl->stored[i] = 0;
+#ifdef ISC_TRACE
+    if (threadIdx.x == 0) *reinterpret_cast<unsigned int *>(smem + kTraceCounterOff) = 0;
+#endif
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -671,9 +750,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     c.warp = warp; c.set = warp >> 2; c.quarter = warp & 3; c.lane = lane; c.tid = threadIdx.x;
     c.lane_idx = (uint32_t)((warp & 3) * 32 + lane);
     c.tmem_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const bool issuer = warp == kIssuerWarp;
+    const bool issuer = warp == kIssuerWarp, epi = warp < kEpiWarps;
     // accumulators of stacked convolutions start from zero
-    if (!issuer) {
+    if (epi) {
         for (uint32_t col = (uint32_t)c.set * 16u; col < (uint32_t)kTmemCols; col += kSets * 16u) tmem_st16_zero(c.tmem_lane + col);
         tmem_st_wait();
     }
@@ -683,10 +762,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
 
     const uint32_t ptab = smem_u32(ctrl->ptab);
     const int n_phases = p.n_phases, stop_phase = p.stop_phase;
+    bool role_ok = true;
     int it = 0;
     for (int grp = blockIdx.x; grp < p.n_groups; grp += gridDim.x, ++it) {
         PrevConv prev{0u, 0u, 0u};
-        bool issuer_ok = true;
         int conv_index = 0;
         bool first_phase = true;
         for (int ph = 0; ph < n_phases && ph <= stop_phase; ++ph) {
@@ -694,8 +773,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
             if (e.x == PH_CONV) {
                 const uint32_t cg = (uint32_t)it * (uint32_t)p.n_conv + (uint32_t)conv_index;
                 if (issuer) {
-                    if (lane == 0 && issuer_ok && !ctrl->abort_flag)
-                        issuer_ok = issuer_conv(p, ctrl, sbase, tmem, e.y, cg, conv_index, it, prev);
+                    if (lane == 0 && role_ok && !ctrl->abort_flag)
+                        role_ok = issuer_conv(p, ctrl, sbase, tmem, e.y, cg, conv_index, it, prev);
                     __syncwarp();
                 } else {
                     epi_conv(p, c, e.y, cg, it);
@@ -712,11 +791,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
             if (first_phase) {
                 // the first blob of the group: everything of the previous group is complete
                 if (issuer && lane == 0 && p.n_conv > 0 && !ctrl->abort_flag &&
-                    (int)(__ldg(&p.conv_src[0].bytes_phase) >> 24) <= stop_phase)
-                    issue_weights(p.conv_src, sbase, smem_u32(&ctrl->wbar[((uint32_t)it * (uint32_t)p.n_conv) % 3]));
+                    (int)(ctrl->csrc[0].bytes_phase >> 24) <= stop_phase)
+                    issue_weights(ctrl->csrc, sbase, smem_u32(&ctrl->wbar[((uint32_t)it * (uint32_t)p.n_conv) % 3]));
                 first_phase = false;
             }
-            if (!issuer && !ctrl->abort_flag) {
+            if (epi && !ctrl->abort_flag) {
                 if (e.x == PH_FILL) fill_phase(c, e.y, e.z, e.w);
                 else if (e.x == PH_INPUT) input_phase(p, c, grp);
                 else if (warp < kG) tail_sample(p, c, warp, grp);
@@ -734,6 +813,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     if (p.dump)
         for (uint32_t o = threadIdx.x * 16u; o < p.dump_bytes; o += blockDim.x * 16u)
             *reinterpret_cast<uint4 *>(p.dump + o) = ld_shared_v4(sbase + p.dump_off + o);
+#ifdef ISC_TRACE
+    if (blockIdx.x == 0 && threadIdx.x == 0) g_ltrace_n = min(*reinterpret_cast<unsigned int *>(smem + kTraceCounterOff), kTraceMax);
+#endif
     // no tensor-core work may be in flight when tensor memory is released
     if (issuer && lane == 0) {
         Waiter w{ctrl, p.err};
@@ -847,6 +929,8 @@ struct ConvPlan {
     std::vector<LOp> ops;
     std::vector<uint32_t> passes;
     std::vector<int> done_time;         // per output line: index of the pass that stores its last chunk
+    int n_units = 0;
+    std::vector<int> unit_of;           // per output line: its unit
     std::vector<int> a_delta;
     std::vector<uint32_t> a_lbo;
     std::vector<std::pair<int, int>> kunits;   // per K-step: indices into `units` (second may be -1)
@@ -1000,24 +1084,16 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             }
         }
         if ((int)cp.kunits.size() > kMaxKsteps) PLAN_FAIL(11);
-        // class and banks
-        const auto key = std::make_pair(cp.m, cp.n_chunks);
-        if (!class_of.count(key)) {
-            class_of[key] = (int)class_lines.size();
-            class_lines.push_back(cp.m); class_chunks.push_back(cp.n_chunks); class_uses.push_back(0);
-        }
-        cp.cls = class_of[key];
-        cp.use_local = class_uses[(size_t)cp.cls]++;
         // ---- operations
         const ConvPlan *pv = (!convs.empty() && convs.back().phase == ph - 1) ? &convs.back() : nullptr;
-        const bool same_class = pv && pv->cls == cp.cls;
+        // same lines and chunks: the same barriers (class) and, with one bank, the same accumulator columns
+        const bool same_class = pv && pv->m == cp.m && pv->n_chunks == cp.n_chunks;
         // the previous convolution produced this one's input, line for line
         const bool aligned = pv && in.producer_conv == (int)convs.size() - 1 && !pv->scatter;
         // Same class: the same barriers, and with one bank the same accumulator columns.  An operation then waits for
         // the previous convolution's lines of the same numbers as the output lines it adds to, so that no line of
         // this convolution can be stored (and arrive on the line's barrier) before that line of the previous one.
         const bool slots = same_class;
-        const bool wait_all = pv && !same_class;
         auto prev_time = [&](int line) { return pv ? pv->done_time[(size_t)line] : 0; };
         auto src_line = [&](int p) -> int {       // which output line of the producer fills input line p (-1: constant)
             if (p >= 0 && p < in.n_lines) return p;
@@ -1059,48 +1135,76 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         std::vector<int> last_op((size_t)cp.m, -1);
         for (size_t i = 0; i < proto.size(); ++i)
             for (int y : proto[i].outs) last_op[(size_t)y] = (int)i;
-        std::vector<char> waited(pv ? (size_t)pv->m : 0, 0);
-        for (size_t i = 0; i < proto.size(); ++i) {
-            const ProtoOp &o = proto[i];
-            LOp op;
-            memset(&op, 0, sizeof(op));
-            op.a_line1 = (uint8_t)(o.a_line + 1);
-            op.b_block = (uint8_t)o.b_block; op.n_blocks = (uint8_t)o.n_blocks;
-            op.d_col = (uint16_t)(o.d_line * cp.cols);
-            if (i == 0 && wait_all) {
-                op.flags |= OPF_WAIT_ALL;
-                std::fill(waited.begin(), waited.end(), 1);
-            }
-            for (int l : o.need)
-                if (!waited[(size_t)l]) {
-                    if (op.n_wait >= 4) PLAN_FAIL(12);
-                    op.wait[op.n_wait++] = (uint8_t)l;
-                    waited[(size_t)l] = 1;
-                }
-            for (int y : o.outs)
-                if (last_op[(size_t)y] == (int)i) {
-                    if (op.n_commit >= 4) PLAN_FAIL(13);
-                    op.commit[op.n_commit++] = (uint8_t)y;
-                }
-            cp.ops.push_back(op);
-        }
-        // ---- passes in the order of completion
+        // ---- units: the lines of a pass, in the order of completion; one barrier pair per unit
         std::vector<int> order((size_t)cp.m);
         for (int y = 0; y < cp.m; ++y) order[(size_t)y] = y;
         std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return last_op[(size_t)a] < last_op[(size_t)b]; });
         const int sup = cp.m >= 8 ? 2 : 1;
+        cp.n_units = (cp.m + sup - 1) / sup;
+        cp.unit_of.assign((size_t)cp.m, 0);
+        std::vector<int> unit_last_op((size_t)cp.n_units, -1);
+        for (int i = 0; i < cp.m; ++i) {
+            const int u = i / sup;
+            cp.unit_of[(size_t)order[(size_t)i]] = u;
+            unit_last_op[(size_t)u] = std::max(unit_last_op[(size_t)u], last_op[(size_t)order[(size_t)i]]);
+        }
+        // class: same number of units and chunks = same barriers
+        const auto key = std::make_pair(cp.n_units, cp.n_chunks);
+        if (!class_of.count(key)) {
+            class_of[key] = (int)class_lines.size();
+            class_lines.push_back(cp.n_units); class_chunks.push_back(cp.n_chunks); class_uses.push_back(0);
+        }
+        cp.cls = class_of[key];
+        cp.use_local = class_uses[(size_t)cp.cls]++;
+        const bool wait_all = pv && pv->cls != cp.cls;
+        std::vector<char> waited(pv ? (size_t)pv->n_units : 0, 0);
+        for (size_t i = 0; i < proto.size(); ++i) {
+            const ProtoOp &o = proto[i];
+            LOp op;
+            memset(&op, 0xFF, sizeof(op));
+            op.flags = 0;
+            op.d_col = (uint32_t)(o.d_line * cp.cols);
+            const uint32_t a_fmt_bit = cp.in_tensor == 0 ? 0u : 1u;
+            op.idesc = (2u << 4) | (a_fmt_bit << 7) | (1u << 10) | ((uint32_t)((o.n_blocks * L.cout) >> 3) << 17) | ((128u >> 4) << 24);
+            op.a_add = (uint32_t)(o.a_line + 1) * (uint32_t)in.pitch;
+            op.b_add = (uint32_t)o.b_block * (uint32_t)L.cout * 2u;
+            if (i == 0 && wait_all) {
+                op.flags |= OPF_WAIT_ALL;
+                std::fill(waited.begin(), waited.end(), 1);
+            }
+            int n_wait = 0, n_commit = 0;
+            for (int l : o.need) {
+                const int u = pv->unit_of[(size_t)l];
+                if (!waited[(size_t)u]) {
+                    if (n_wait >= 4) PLAN_FAIL(12);
+                    op.wait[n_wait++] = (uint16_t)(4 * u);
+                    waited[(size_t)u] = 1;
+                }
+            }
+            for (int u = 0; u < cp.n_units; ++u)
+                if (unit_last_op[(size_t)u] == (int)i) {
+                    if (n_commit >= 3) PLAN_FAIL(13);
+                    op.commit[n_commit++] = (uint16_t)(8 * u);
+                }
+            cp.ops.push_back(op);
+        }
+        if (pv && !wait_all)
+            for (char wtd : waited)
+                if (!wtd) PLAN_FAIL(20);        // the issuing thread must have seen the whole previous convolution stored
+        // ---- passes: unit by unit, chunk by chunk
         cp.done_time.assign((size_t)cp.m, 0);
-        for (int i = 0; i < cp.m; i += sup)
+        for (int u = 0; u < cp.n_units; ++u)
             for (int ch = 0; ch < cp.n_chunks; ++ch) {
-                const int n = std::min(sup, cp.m - i);
-                uint32_t pw = (uint32_t)order[(size_t)i] | ((uint32_t)ch << 16) | ((uint32_t)n << 24);
-                if (n == 2) pw |= (uint32_t)order[(size_t)i + 1] << 8;
-                for (int q = 0; q < n; ++q) cp.done_time[(size_t)order[(size_t)i + q]] = (int)cp.passes.size() / kSets;
+                const int n = std::min(sup, cp.m - u * sup);
+                uint32_t pw = (uint32_t)order[(size_t)u * sup] | ((uint32_t)ch << 16) | ((uint32_t)n << 20) | ((uint32_t)u << 24);
+                if (n == 2) pw |= (uint32_t)order[(size_t)u * sup + 1] << 8;
+                for (int q = 0; q < n; ++q) cp.done_time[(size_t)order[(size_t)u * sup + q]] = (int)cp.passes.size() / kSets;
                 cp.passes.push_back(pw);
             }
         convs.push_back(cp);
     }
     const int n_conv = (int)convs.size();
+    if (n_conv > kMaxConv) PLAN_FAIL(22);
     // ---- barriers: per class, one per output line for "accumulators complete" and one for "line stored"
     std::vector<int> class_full(class_lines.size()), class_done(class_lines.size());
     bar_counts_out->clear();
@@ -1119,7 +1223,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         const isc_layer &L = layers[cp.layer].d;
         const uint32_t rows = (uint32_t)(cp.stacked ? 3 : 1) * (uint32_t)L.cout;
         uint32_t at = (uint32_t)sizeof(LConvDesc);
-        ops_rel[(size_t)c] = at; at += (uint32_t)cp.ops.size() * 16u;
+        ops_rel[(size_t)c] = at; at += (uint32_t)cp.ops.size() * (uint32_t)sizeof(LOp);
         passes_rel[(size_t)c] = at; at += ((uint32_t)cp.passes.size() * 4u + 15u) & ~15u;
         at = (at + 127u) & ~127u;
         w_rel[(size_t)c] = at; at += (uint32_t)cp.kunits.size() * rows * 32u;
@@ -1202,7 +1306,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         D.d_base[0] = 0; D.d_base[1] = cp.n_banks > 1 ? (uint32_t)(cp.m * cp.cols) : 0u;
         D.bar_full = (uint32_t)class_full[(size_t)cp.cls]; D.bar_done = (uint32_t)class_done[(size_t)cp.cls];
         D.use_local = (uint32_t)cp.use_local; D.uses_per_group = (uint32_t)class_uses[(size_t)cp.cls];
-        D.n_lines = (uint32_t)cp.m; D.n_chunks = (uint32_t)cp.n_chunks;
+        D.n_lines = (uint32_t)cp.n_units; D.n_chunks = (uint32_t)cp.n_chunks;
         D.w_rel = w_rel[(size_t)c]; D.c_rel = c_rel[(size_t)c]; D.ops_rel = ops_rel[(size_t)c]; D.passes_rel = passes_rel[(size_t)c];
         D.out_base = plan->tensor_off[(size_t)cp.out_tensor] + out.line0;
         D.out_plane = out.plane_bytes; D.out_pitch16 = (uint32_t)out.pitch; D.out_n_lines = (uint32_t)out.n_lines;
@@ -1222,11 +1326,17 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             D.res_r2_lo = (uint32_t)((unsigned long long)r2 & 0xFFFFFFFFull);
             D.res_r2_hi = (uint32_t)((unsigned long long)r2 >> 32);
         }
-        for (size_t k = 0; k < cp.kunits.size(); ++k) { D.a_delta[k] = cp.a_delta[k]; D.a_lbo[k] = cp.a_lbo[k]; }
+        for (size_t k = 0; k < cp.kunits.size(); ++k) {
+            const long long a = (long long)D.a_base + cp.a_delta[k];
+            if (a < 0 || (a & 15) || (cp.a_lbo[k] & 15u)) PLAN_FAIL(21);
+            D.a_lo[k] = (uint32_t)(a >> 4) | ((cp.a_lbo[k] >> 4) << 16);
+        }
+        D.b_lo0 = ((w_off[(size_t)c] + w_rel[(size_t)c]) >> 4) | ((128u >> 4) << 16);
+        D.kstep16 = (uint32_t)(cp.stacked ? 3 : 1) * (uint32_t)L.cout * 2u;
         // operand reads stay inside the input's region
         for (size_t k = 0; k < cp.kunits.size(); ++k)
             for (const LOp &op : cp.ops) {
-                const long long lo_b = (long long)in.line0 - (long long)in.pitch * 16 + (long long)op.a_line1 * in.pitch * 16 + cp.a_delta[k];
+                const long long lo_b = (long long)in.line0 - (long long)in.pitch * 16 + (long long)op.a_add * 16 + cp.a_delta[k];
                 const long long hi_b = lo_b + cp.a_lbo[k] + 128 * 16;
                 if (lo_b < 0 || hi_b > (long long)in.bytes) PLAN_FAIL(18);
             }
@@ -1402,8 +1512,8 @@ static int line_launch(LinePlan *p, LineParams &q, cudaStream_t st)
     {
         const char *lo = getenv("ISC_TRACE_LO"), *hi = getenv("ISC_TRACE_HI");
         const unsigned vlo = lo ? (unsigned)atoi(lo) : 0u, vhi = hi ? (unsigned)atoi(hi) : 0u, zero = 0u;
-        cudaMemcpyToSymbol(g_ltrace_lo, &vlo, sizeof(vlo));
-        cudaMemcpyToSymbol(g_ltrace_hi, &vhi, sizeof(vhi));
+        cudaMemcpyToSymbol(c_trace_lo, &vlo, sizeof(vlo));
+        cudaMemcpyToSymbol(c_trace_hi, &vhi, sizeof(vhi));
         cudaMemcpyToSymbol(g_ltrace_n, &zero, sizeof(zero));
     }
 #endif
@@ -1475,14 +1585,14 @@ int line_debug_tensor(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, in
 }
 
 #ifdef ISC_TRACE
-// Copies the recorded triples to the host; returns how many there are.
-extern "C" int isc_line_trace_read(unsigned long long *out, int max_events)
+// Copies the recorded pairs of the last launch to the host; returns how many there are.
+extern "C" int isc_line_trace_read(unsigned int *out, int max_events)
 {
     unsigned n = 0;
     cudaDeviceSynchronize();
     cudaMemcpyFromSymbol(&n, g_ltrace_n, sizeof(n));
     n = std::min(n, std::min(kTraceMax, (unsigned)max_events));
-    cudaMemcpyFromSymbol(out, g_ltrace, (size_t)n * 3 * sizeof(unsigned long long));
+    cudaMemcpyFromSymbol(out, g_ltrace, (size_t)n * 2 * sizeof(unsigned int));
     return (int)n;
 }
 #endif
