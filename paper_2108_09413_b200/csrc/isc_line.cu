@@ -61,7 +61,7 @@ constexpr unsigned kTraceMax = 16384;                // 8 bytes each
 __device__ unsigned int g_ltrace[2 * kTraceMax];
 __device__ unsigned int g_ltrace_n;
 __constant__ unsigned int c_trace_lo, c_trace_hi;
-constexpr unsigned kTraceCounterOff = 7168 - 16;
+constexpr unsigned kTraceCounterOff = 9216 - 16;
 __device__ __forceinline__ void ltrace_val(int ev, uint32_t cg, uint32_t tag, uint32_t val)
 {
     extern __shared__ __align__(128) uint8_t trace_smem[];
@@ -88,14 +88,15 @@ __device__ __forceinline__ void ltrace(int ev, uint32_t cg, uint32_t tag) { ltra
 constexpr int kG = 4;                       // samples per group
 constexpr int kEpiWarps = 16;               // warps 0..15: epilogue; set = warp / 4, tensor-memory quarter = warp % 4
 constexpr int kSets = kEpiWarps / 4;
-constexpr int kIssuerWarp = kEpiWarps;      // warp 16: MMA issue and weight copies
-constexpr int kThreads = 32 * (kEpiWarps + 1);
+constexpr int kIssuers = 4;                 // warps 16..19: lane 0 of each issues every fourth MMA chain of a convolution
+constexpr int kLoaderWarp = kEpiWarps + kIssuers;   // warp 20: weight copies
+constexpr int kThreads = 32 * (kEpiWarps + kIssuers + 1);
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kMaxKsteps = 18;
 constexpr int kMaxPhases = 160;
 constexpr int kMaxBars = 128;
 constexpr int kMaxLines = 32;               // output lines of one convolution
-constexpr int kCtrlBytes = 7168;
+constexpr int kCtrlBytes = 9216;
 constexpr int kMaxConv = 128;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kTmemCols = 512;
@@ -104,7 +105,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
 enum { ERR_NONE = 0, ERR_WAIT_DONE = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_READY = 3, ERR_WAIT_FULL = 4, ERR_WAIT_DRAIN = 5 };
 enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8 };
-enum { OPF_WAIT_ALL = 1 };
+enum { OPF_WAIT_ALL = 1, OPF_NULL = 4 };
 
 // ---- what the kernel reads -------------------------------------------------------------------
 
@@ -113,7 +114,13 @@ enum { OPF_WAIT_ALL = 1 };
 struct alignas(16) PhaseEntry { uint32_t kind, a, b, c; };
 
 // Where the blob of convolution c comes from (global) and goes to (shared).
-struct alignas(16) ConvSrc { unsigned long long gmem; uint32_t bytes_phase, smem_off; };   // bytes | phase << 24
+// and which convolution must be complete before the copy may start: the counters stored[dep_first .. + dep_units)
+// must have reached dep_mult * (group * dep_uses + dep_local + 1); dep_units = 0: nothing to wait for.
+struct alignas(16) ConvSrc {
+    unsigned long long gmem;
+    uint32_t bytes_phase, smem_off;                 // bytes | phase << 24; offset | late << 31
+    uint32_t dep_first, dep_units, dep_mult, dep_local_uses;     // dep_local | dep_uses << 16
+};
 
 // One MMA chain in the form the issuing thread consumes: accumulator columns, what to add to the operand
 // descriptors' start addresses, and the barriers (as byte offsets, 0xFFFF = none) of its dependencies and completions.
@@ -123,7 +130,7 @@ struct alignas(16) LOp {
     uint32_t a_add, b_add;  // 16-byte units: (input line + 1) * pitch, first weight block * block size
     uint16_t wait[4];       // 8 * unit of the previous convolution that must be stored
     uint16_t commit[3];     // 8 * unit of this convolution whose accumulators are complete after the chain
-    uint16_t flags;         // OPF_WAIT_ALL: every line of the previous convolution
+    uint16_t flags;         // OPF_WAIT_ALL: every unit of the previous convolution; OPF_NULL: no MMAs, arrivals only
 };
 static_assert(sizeof(LOp) == 32, "one operation is two 16-byte loads");
 
@@ -224,6 +231,12 @@ __device__ __forceinline__ void red_release_add(uint32_t addr, uint32_t v)
 {
     asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+__device__ __forceinline__ uint32_t ld_volatile_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ uint32_t ld_acquire_u32(uint32_t addr)
 {
     uint32_t v;
@@ -268,7 +281,10 @@ struct Waiter {
     // Wait until a counter in shared memory has reached `expected` (counters only grow).
     __device__ __forceinline__ bool counter(uint32_t addr, uint32_t expected, int code)
     {
-        if ((int32_t)(ld_acquire_u32(addr) - expected) >= 0) return true;
+        // The first test is a plain load: an acquiring one costs over a hundred cycles here.  What the counter guards
+        // was made visible to the tensor cores' reads by the storing warp (proxy fence, then a releasing add) and is
+        // read by MMAs that are issued only after the value has been seen.
+        if ((int32_t)(ld_volatile_u32(addr) - expected) >= 0) return true;
         const unsigned long long t0 = globaltimer();
         for (int spin = 0;; ++spin) {
             if ((int32_t)(ld_acquire_u32(addr) - expected) >= 0) return true;
@@ -285,10 +301,10 @@ struct Waiter {
 struct PrevConv { uint32_t done_addr, expected, n_lines; };    // counters of its units, their value when stored; n_lines = 0: nothing to wait for
 
 struct IssueCtx {
-    uint32_t desc, ops, n_ops, s16, b_lo0, kstep16, d0, stacked, full_addr, cg;
+    uint32_t desc, ops, n_ops, s16, b_lo0, kstep16, d0, stacked, full_addr, cg, issuer;
 };
 
-// All operations of one convolution.  The low words of the operand descriptors stay in registers; an operation adds
+// The operations of one convolution that belong to one issuing thread (every kIssuers-th record).  The low words of the operand descriptors stay in registers; an operation adds
 // its line and block offsets to their start-address fields.
 template <int KS>
 __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const PrevConv &prev, uint32_t n_ksteps)
@@ -308,17 +324,17 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
 #pragma unroll
         for (int k = 0; k < NK; ++k) blo[k] = ic.b_lo0 + ic.s16 + (uint32_t)k * ic.kstep16;
     }
-    uint32_t at = ic.ops;
+    uint32_t at = ic.ops + 32u * ic.issuer;           // the table ends with kIssuers spare records: reads run one ahead
     uint4 n0 = ld_shared_v4(at), n1 = ld_shared_v4(at + 16);
     LT_ARRAY(tlogA, 40);
     LT_ARRAY(tlogB, 40);
     LT_ARRAY(tlogC, 40);
     LT_ARRAY(tlogD, 40);
-    for (uint32_t i = 0; i < ic.n_ops; ++i) {
+    for (uint32_t i = ic.issuer; i < ic.n_ops; i += kIssuers) {
         LT_CLOCK(tA);
         const uint4 r0 = n0, r1 = n1;         // d_col, idesc, a_add, b_add | wait 0-1, wait 2-3, commit 0-1, commit 2 and flags
-        at += 32;
-        if (i + 1 < ic.n_ops) { n0 = ld_shared_v4(at); n1 = ld_shared_v4(at + 16); }
+        at += 32u * kIssuers;
+        n0 = ld_shared_v4(at); n1 = ld_shared_v4(at + 16);
         // units of the previous convolution this operation depends on
         if (prev.n_lines) {
             if ((r1.w >> 16) & OPF_WAIT_ALL) {
@@ -337,7 +353,9 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
         LT_CLOCK(tB);
         tc_fence_after();
         const uint32_t d = ic.d0 + r0.x;
-        if (KS > 0) {
+        if ((r1.w >> 16) & OPF_NULL) {
+            // a record that only carries this thread's arrivals on units it did not add to
+        } else if (KS > 0) {
 #pragma unroll
             for (int k = 0; k < NK; ++k) {
                 const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[k] + r0.z);
@@ -367,7 +385,7 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
         LT_SET(tlogD, i, tD);
     }
 #ifdef ISC_TRACE
-    for (uint32_t i = 0; i < ic.n_ops && i < 40; ++i) { ltrace_val(1, ic.cg, i, tlogA[i]); ltrace_val(2, ic.cg, i, tlogB[i]); ltrace_val(5, ic.cg, i, tlogC[i]); ltrace_val(6, ic.cg, i, tlogD[i]); }
+    for (uint32_t i = ic.issuer; i < ic.n_ops && i < 40; i += kIssuers) { ltrace_val(1, ic.cg, i, tlogA[i]); ltrace_val(2, ic.cg, i, tlogB[i]); ltrace_val(5, ic.cg, i, tlogC[i]); ltrace_val(6, ic.cg, i, tlogD[i]); }
 #endif
     return true;
 }
@@ -381,25 +399,30 @@ __device__ __forceinline__ void issue_weights(const ConvSrc *src, uint32_t sbase
     bulk_g2s(sbase + (v.w & 0x7FFFFFFFu), gmem, bytes, wbar_addr);
 }
 
-// One convolution, by lane 0 of the issuing warp.  Returns false after a wait has expired.
-__device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, uint32_t blob_off,
-                                         uint32_t cg, int conv_index, int it, PrevConv &prev)
+// The copy of convolution `target`'s blob, by lane 0 of the loader warp, once the convolution it names is complete:
+// the blob takes the place of things that convolution (or an earlier one) was the last to use.
+__device__ __noinline__ bool loader_copy(const LineParams &p, Ctrl *ctrl, uint32_t sbase, int target, uint32_t cg_target, int it)
 {
     Waiter w{ctrl, p.err};
-    LT_CLOCK(t_enter);
-    // The next blob's place was last used by the convolution before the previous one, which is complete; a blob
-    // marked late takes the place of something the previous convolution still uses and is copied further down.
-    bool late_copy = false;
-    if (conv_index + 1 < p.n_conv) {
-        const ConvSrc *nxt = ctrl->csrc + conv_index + 1;
-        if ((int)(nxt->bytes_phase >> 24) <= p.stop_phase) {
-            late_copy = (nxt->smem_off >> 31) != 0;
-            if (!late_copy) issue_weights(nxt, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
-        }
+    const ConvSrc *src = ctrl->csrc + target;
+    if ((int)(src->bytes_phase >> 24) > p.stop_phase) return true;
+    const uint32_t n = src->dep_units;
+    if (n) {
+        const uint32_t expected = src->dep_mult * ((uint32_t)it * (src->dep_local_uses >> 16) + (src->dep_local_uses & 0xFFFFu) + 1u);
+        const uint32_t first = smem_u32(&ctrl->stored[src->dep_first]);
+        for (uint32_t l = 0; l < n; ++l)
+            if (!w.counter(first + 4 * l, expected, ERR_WAIT_DONE)) return false;
     }
-    LT_CLOCK(t_wissued);
+    issue_weights(src, sbase, smem_u32(&ctrl->wbar[cg_target % 3]));
+    return true;
+}
+
+// One convolution's share of an issuing warp, by its lane 0.  Returns false after a wait has expired.
+__device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32_t sbase, uint32_t tmem, uint32_t blob_off,
+                                         uint32_t cg, int issuer, int it, PrevConv &prev)
+{
+    Waiter w{ctrl, p.err};
     if (!w.barrier(smem_u32(&ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS)) return false;
-    LT_CLOCK(t_wbar);
     const uint32_t desc = sbase + blob_off;
     const uint4 h0 = ld_shared_v4(desc);                                    // n_ops, n_passes, n_ksteps, flags
     const uint4 h1 = ld_shared_v4(desc + offsetof(LConvDesc, a_base));      // a_base, pitch16, bblock16, n_banks
@@ -415,6 +438,7 @@ __device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32
     ic.stacked = (h0.w & CF_STACKED) ? 1u : 0u;
     ic.full_addr = smem_u32(&ctrl->bars[h3.z]);
     ic.cg = cg;
+    ic.issuer = (uint32_t)issuer;
     bool ok;
     switch (h0.z) {
     case 1: ok = issue_ops<1>(w, ic, prev, 1); break;
@@ -426,12 +450,6 @@ __device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32
     default: ok = issue_ops<0>(w, ic, prev, h0.z); break;
     }
     if (!ok) return false;
-    LT_CLOCK(t_done);
-    ltrace_val(8, cg, 0, t_enter); ltrace_val(9, cg, 0, t_wissued); ltrace_val(10, cg, 0, t_wbar); ltrace_val(11, cg, 0, t_done);
-    // Every unit of the previous convolution has been waited for on behalf of an operation above (the planner sees
-    // to it): that convolution is complete, and whatever reads its output later, or reuses what it read, needs no
-    // wait of its own.  A blob marked late may now take the place of something it used.
-    if (late_copy) issue_weights(ctrl->csrc + conv_index + 1, sbase, smem_u32(&ctrl->wbar[(cg + 1) % 3]));
     prev.done_addr = smem_u32(&ctrl->stored[h3.w]);
     prev.expected = 4u * h4.w * (use + 1u);
     prev.n_lines = h4.z;
@@ -727,7 +745,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     for (int i = threadIdx.x; i < p.n_bars; i += blockDim.x) mbar_init(smem_u32(&ctrl->bars[i]), p.bar_counts[i]);
     if (threadIdx.x == 0) {
         for (int s = 0; s < 3; ++s) mbar_init(smem_u32(&ctrl->wbar[s]), 1);
-        mbar_init(smem_u32(&ctrl->drain), 1);
+        mbar_init(smem_u32(&ctrl->drain), kIssuers);
         ctrl->abort_flag = 0;
     }
     for (int i = threadIdx.x; i < 128; i += blockDim.x) ctrl->hist[i] = 0;
@@ -750,7 +768,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     c.warp = warp; c.set = warp >> 2; c.quarter = warp & 3; c.lane = lane; c.tid = threadIdx.x;
     c.lane_idx = (uint32_t)((warp & 3) * 32 + lane);
     c.tmem_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const bool issuer = warp == kIssuerWarp, epi = warp < kEpiWarps;
+    const bool issuer = warp >= kEpiWarps && warp < kEpiWarps + kIssuers, loader = warp == kLoaderWarp, epi = warp < kEpiWarps;
     // accumulators of stacked convolutions start from zero
     if (epi) {
         for (uint32_t col = (uint32_t)c.set * 16u; col < (uint32_t)kTmemCols; col += kSets * 16u) tmem_st16_zero(c.tmem_lane + col);
@@ -774,7 +792,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
                 const uint32_t cg = (uint32_t)it * (uint32_t)p.n_conv + (uint32_t)conv_index;
                 if (issuer) {
                     if (lane == 0 && role_ok && !ctrl->abort_flag)
-                        role_ok = issuer_conv(p, ctrl, sbase, tmem, e.y, cg, conv_index, it, prev);
+                        role_ok = issuer_conv(p, ctrl, sbase, tmem, e.y, cg, warp - kEpiWarps, it, prev);
+                    __syncwarp();
+                } else if (loader) {
+                    if (lane == 0 && role_ok && !ctrl->abort_flag && conv_index + 1 < p.n_conv)
+                        role_ok = loader_copy(p, ctrl, sbase, conv_index + 1, cg + 1u, it);
                     __syncwarp();
                 } else {
                     epi_conv(p, c, e.y, cg, it);
@@ -790,9 +812,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
             prev.n_lines = 0;
             if (first_phase) {
                 // the first blob of the group: everything of the previous group is complete
-                if (issuer && lane == 0 && p.n_conv > 0 && !ctrl->abort_flag &&
-                    (int)(ctrl->csrc[0].bytes_phase >> 24) <= stop_phase)
-                    issue_weights(ctrl->csrc, sbase, smem_u32(&ctrl->wbar[((uint32_t)it * (uint32_t)p.n_conv) % 3]));
+                if (loader && lane == 0 && p.n_conv > 0 && role_ok && !ctrl->abort_flag)
+                    role_ok = loader_copy(p, ctrl, sbase, 0, (uint32_t)it * (uint32_t)p.n_conv, it);
                 first_phase = false;
             }
             if (epi && !ctrl->abort_flag) {
@@ -1157,40 +1178,80 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         cp.cls = class_of[key];
         cp.use_local = class_uses[(size_t)cp.cls]++;
         const bool wait_all = pv && pv->cls != cp.cls;
-        std::vector<char> waited(pv ? (size_t)pv->n_units : 0, 0);
+        // Record i belongs to issuing thread i mod kIssuers; every thread needs a record to carry its arrivals.
+        auto null_op = []() { ProtoOp o; o.a_line = 0; o.b_block = 0; o.n_blocks = 0; o.d_line = 0; o.ready = 0; return o; };
+        while (proto.size() < (size_t)kIssuers) proto.push_back(null_op());
+        // Each thread arrives on every unit's barrier once: after its last record that adds to the unit, or with any
+        // of its records if it has none (at most three arrivals fit a record; empty records are added as needed).
+        std::vector<std::vector<int>> commits;
+        for (int attempt = 0;; ++attempt) {
+            commits.assign(proto.size(), std::vector<int>());
+            bool fits = true;
+            std::vector<std::vector<char>> has((size_t)cp.n_units, std::vector<char>((size_t)kIssuers, 0));
+            for (int u = 0; u < cp.n_units && fits; ++u)
+                for (int wi = 0; wi < kIssuers && fits; ++wi) {
+                    int last = -1;
+                    for (size_t i = (size_t)wi; i < proto.size(); i += kIssuers)
+                        for (int y : proto[i].outs)
+                            if (cp.unit_of[(size_t)y] == u) last = (int)i;
+                    if (last < 0) continue;
+                    if (commits[(size_t)last].size() >= 3) fits = false;
+                    else { commits[(size_t)last].push_back(u); has[(size_t)u][(size_t)wi] = 1; }
+                }
+            for (int u = 0; u < cp.n_units && fits; ++u)
+                for (int wi = 0; wi < kIssuers && fits; ++wi) {
+                    if (has[(size_t)u][(size_t)wi]) continue;
+                    int carrier = -1;
+                    for (size_t i = (size_t)wi; i < proto.size() && carrier < 0; i += kIssuers)
+                        if (commits[i].size() < 3) carrier = (int)i;
+                    if (carrier < 0) fits = false;
+                    else commits[(size_t)carrier].push_back(u);
+                }
+            if (fits) break;
+            if (attempt >= 8) PLAN_FAIL(13);
+            while (proto.size() % kIssuers) proto.push_back(null_op());
+            for (int wi = 0; wi < kIssuers; ++wi) proto.push_back(null_op());
+        }
+        // each thread waits, once, for what its own records need
+        std::vector<std::vector<char>> waited((size_t)kIssuers, std::vector<char>(pv ? (size_t)pv->n_units : 0, 0));
+        std::vector<char> all_waited(pv ? (size_t)pv->n_units : 0, 0);
         for (size_t i = 0; i < proto.size(); ++i) {
             const ProtoOp &o = proto[i];
+            const size_t wi = i % kIssuers;
             LOp op;
             memset(&op, 0xFF, sizeof(op));
-            op.flags = 0;
+            op.flags = o.n_blocks == 0 ? OPF_NULL : 0;
             op.d_col = (uint32_t)(o.d_line * cp.cols);
             const uint32_t a_fmt_bit = cp.in_tensor == 0 ? 0u : 1u;
-            op.idesc = (2u << 4) | (a_fmt_bit << 7) | (1u << 10) | ((uint32_t)((o.n_blocks * L.cout) >> 3) << 17) | ((128u >> 4) << 24);
+            op.idesc = (2u << 4) | (a_fmt_bit << 7) | (1u << 10) | ((uint32_t)((std::max(o.n_blocks, 1) * L.cout) >> 3) << 17) | ((128u >> 4) << 24);
             op.a_add = (uint32_t)(o.a_line + 1) * (uint32_t)in.pitch;
             op.b_add = (uint32_t)o.b_block * (uint32_t)L.cout * 2u;
-            if (i == 0 && wait_all) {
+            if (i < (size_t)kIssuers && wait_all) {
                 op.flags |= OPF_WAIT_ALL;
-                std::fill(waited.begin(), waited.end(), 1);
+                std::fill(waited[wi].begin(), waited[wi].end(), 1);
             }
             int n_wait = 0, n_commit = 0;
-            for (int l : o.need) {
-                const int u = pv->unit_of[(size_t)l];
-                if (!waited[(size_t)u]) {
+            std::vector<int> need_units;
+            for (int l : o.need) need_units.push_back(pv->unit_of[(size_t)l]);
+            // A thread may arrive on a unit's barrier only when the barrier's previous use is over.  Between
+            // convolutions of one class that use is the previous convolution's unit of the same number; anything
+            // older is complete once the previous convolution is (the thread's first record has waited for all of it).
+            if (pv && pv->cls == cp.cls)
+                for (int u : commits[i]) need_units.push_back(u);
+            for (int u : need_units)
+                if (!waited[wi][(size_t)u]) {
                     if (n_wait >= 4) PLAN_FAIL(12);
                     op.wait[n_wait++] = (uint16_t)(4 * u);
-                    waited[(size_t)u] = 1;
+                    waited[wi][(size_t)u] = 1;
+                    all_waited[(size_t)u] = 1;
                 }
-            }
-            for (int u = 0; u < cp.n_units; ++u)
-                if (unit_last_op[(size_t)u] == (int)i) {
-                    if (n_commit >= 3) PLAN_FAIL(13);
-                    op.commit[n_commit++] = (uint16_t)(8 * u);
-                }
+            for (int u : commits[i]) op.commit[n_commit++] = (uint16_t)(8 * u);
             cp.ops.push_back(op);
         }
+        // "this convolution complete" must imply "the previous one complete": between them the threads wait for all its units
         if (pv && !wait_all)
-            for (char wtd : waited)
-                if (!wtd) PLAN_FAIL(20);        // the issuing thread must have seen the whole previous convolution stored
+            for (char wtd : all_waited)
+                if (!wtd) PLAN_FAIL(20);
         // ---- passes: unit by unit, chunk by chunk
         cp.done_time.assign((size_t)cp.m, 0);
         for (int u = 0; u < cp.n_units; ++u)
@@ -1210,7 +1271,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
     bar_counts_out->clear();
     for (size_t k = 0; k < class_lines.size(); ++k) {
         class_full[k] = (int)bar_counts_out->size();
-        for (int l = 0; l < class_lines[k]; ++l) bar_counts_out->push_back(1);
+        for (int l = 0; l < class_lines[k]; ++l) bar_counts_out->push_back((uint8_t)kIssuers);    // one arrival per issuing thread
         class_done[k] = (int)bar_counts_out->size();
         for (int l = 0; l < class_lines[k]; ++l) bar_counts_out->push_back((uint8_t)(4 * class_chunks[k]));
     }
@@ -1223,7 +1284,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         const isc_layer &L = layers[cp.layer].d;
         const uint32_t rows = (uint32_t)(cp.stacked ? 3 : 1) * (uint32_t)L.cout;
         uint32_t at = (uint32_t)sizeof(LConvDesc);
-        ops_rel[(size_t)c] = at; at += (uint32_t)cp.ops.size() * (uint32_t)sizeof(LOp);
+        ops_rel[(size_t)c] = at; at += ((uint32_t)cp.ops.size() + (uint32_t)kIssuers) * (uint32_t)sizeof(LOp);    // spare records: reads run one ahead
         passes_rel[(size_t)c] = at; at += ((uint32_t)cp.passes.size() * 4u + 15u) & ~15u;
         at = (at + 127u) & ~127u;
         w_rel[(size_t)c] = at; at += (uint32_t)cp.kunits.size() * rows * 32u;
@@ -1265,7 +1326,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
     for (int t = 0; t <= n_conv_layers; ++t) plan->tensor_off[(size_t)t] = buffers[(size_t)T[(size_t)t].buffer].off;
     // ---- emit phases and blobs
     ptab_out->assign((size_t)n_phases, PhaseEntry{0, 0, 0, 0});
-    csrc_out->assign((size_t)n_conv, ConvSrc{0, 0, 0});
+    csrc_out->assign((size_t)n_conv, ConvSrc{0, 0, 0, 0, 0, 0, 0});
     blob_out->clear();
     blob_offsets->assign((size_t)n_conv, 0);
     plan->phase_kind.assign((size_t)n_phases, 0);
@@ -1379,6 +1440,20 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         blob_out->insert(blob_out->end(), blob.begin(), blob.end());
         (*csrc_out)[(size_t)c].bytes_phase = w_bytes[(size_t)c] | ((uint32_t)ph << 24);
         (*csrc_out)[(size_t)c].smem_off = w_off[(size_t)c] | (late[(size_t)c] ? 0x80000000u : 0u);
+        {
+            // The copy starts while the convolution before this one runs.  The blob's place was last used by the
+            // convolution three back or an earlier one (for a late blob: two back), which must be complete by then.
+            const int q = late[(size_t)c] ? c - 2 : c - 3;
+            ConvSrc &cs = (*csrc_out)[(size_t)c];
+            cs.dep_first = cs.dep_units = cs.dep_mult = cs.dep_local_uses = 0;
+            if (q >= 0) {
+                const ConvPlan &dq = convs[(size_t)q];
+                cs.dep_first = (uint32_t)class_done[(size_t)dq.cls];
+                cs.dep_units = (uint32_t)dq.n_units;
+                cs.dep_mult = 4u * (uint32_t)dq.n_chunks;
+                cs.dep_local_uses = (uint32_t)dq.use_local | ((uint32_t)class_uses[(size_t)dq.cls] << 16);
+            }
+        }
     }
     plan->n_phases = n_phases;
     plan->n_conv = n_conv;
