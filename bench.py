@@ -142,7 +142,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, choices=sorted(wl.CONFIGS))
     ap.add_argument("--images-per-step", type=int, default=0)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 layer-by-layer, 2 resident tensor-core")
+    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 layer-by-layer, 2 resident tensor-core (flat tiles), 3 resident tensor-core (line tiles)")
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -248,7 +248,8 @@ def main():
         "data": "synthetic",
         "config": {"workload": f"config {args.config}: {model['name']} CERTIFY, {ips} images/step/GPU",
                    "sigma": sigma, "N0": N0, "N": N, "alpha": alpha, "images_per_step": ips,
-                   "engine": {1: "layer-by-layer", 2: "resident tensor-core"}.get(engine, str(engine)),
+                   "engine": {1: "layer-by-layer", 2: "resident tensor-core, flat tiles",
+                              3: "resident tensor-core, line tiles"}.get(engine, str(engine)),
                    "l2": "flushed between steps (256 MiB write)", "macs_per_sample": macs},
         "certified_images_per_sec": value / (N0 + N),
         "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(ips * np.prod(cfg["shape"])),
