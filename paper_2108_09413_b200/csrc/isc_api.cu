@@ -2,6 +2,8 @@
 // Monte-Carlo loop (Algorithm 1 steps 1-4, Algorithm 2 steps 1-2) and the decision rules.
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -71,6 +73,7 @@ namespace {
     do {                                              \
         cudaError_t e_ = (call);                      \
         if (e_ != cudaSuccess) {                      \
+            if (getenv("ISC_DEBUG_CUDA")) fprintf(stderr, "isc: %s: %s\n", #call, cudaGetErrorString(e_)); \
             cudaGetLastError();                       \
             return e_ == cudaErrorMemoryAllocation ? ISC_ERR_NOMEM : ISC_ERR_CUDA; \
         }                                             \

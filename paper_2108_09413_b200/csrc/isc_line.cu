@@ -1593,7 +1593,9 @@ static int line_launch(LinePlan *p, LineParams &q, cudaStream_t st)
     }
 #endif
     k_line<<<grid, kThreads, p->smem_bytes, st>>>(q);
-    return cudaGetLastError() == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess && getenv("ISC_PLAN_DEBUG")) fprintf(stderr, "line engine: launch failed: %s\n", cudaGetErrorString(e));
+    return e == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
 }
 
 int line_run(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, int64_t n, int batch_hint, int32_t *d_counts,
