@@ -1212,6 +1212,14 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             while (proto.size() % kIssuers) proto.push_back(null_op());
             for (int wi = 0; wi < kIssuers; ++wi) proto.push_back(null_op());
         }
+        // No thread may still be reading the table when the convolution is complete (its blob's place may then be
+        // reused): every thread's last record must carry an arrival, so empty records at the end are dropped.
+        while (!proto.empty() && proto.back().n_blocks == 0 && commits.back().empty()) { proto.pop_back(); commits.pop_back(); }
+        for (int wi = 0; wi < kIssuers; ++wi) {
+            int last = -1;
+            for (size_t i = (size_t)wi; i < proto.size(); i += kIssuers) last = (int)i;
+            if (last < 0 || commits[(size_t)last].empty()) PLAN_FAIL(23);
+        }
         // each thread waits, once, for what its own records need
         std::vector<std::vector<char>> waited((size_t)kIssuers, std::vector<char>(pv ? (size_t)pv->n_units : 0, 0));
         std::vector<char> all_waited(pv ? (size_t)pv->n_units : 0, 0);
