@@ -436,7 +436,7 @@ __device__ __noinline__ bool issuer_conv(const LineParams &p, Ctrl *ctrl, uint32
     ic.s16 = sbase >> 4; ic.b_lo0 = hb.x; ic.kstep16 = hb.y;
     ic.d0 = tmem + ((h1.w > 1 && (use & 1u)) ? h3.y : h3.x);
     ic.stacked = (h0.w & CF_STACKED) ? 1u : 0u;
-    ic.full_addr = smem_u32(&ctrl->bars[h3.z]);
+    ic.full_addr = smem_u32(&ctrl->bars[h3.z + (use & 1u) * h4.z]);      // the class has two sets of barriers, used in turn
     ic.cg = cg;
     ic.issuer = (uint32_t)issuer;
     bool ok;
@@ -572,7 +572,7 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
 
 template <bool kRes, bool kLo>
 __device__ __noinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes,
-                                             uint32_t last_unit, uint32_t cg)
+                                             uint32_t cg)
 {
     const EpiConv E = E_in;
     const EpiCtx c = c_in;
@@ -583,9 +583,6 @@ __device__ __noinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, cons
         if (((pw >> 20) & 0xFu) == 2u) epi_pass<kRes, kLo, 2>(w, E, c, pw, ok, cg);
         else epi_pass<kRes, kLo, 1>(w, E, c, pw, ok, cg);
     }
-    // Every warp leaves a convolution only after its last unit's accumulators are complete, hence all of them: a later
-    // wait for the next use of any of these barriers then always refers to the phase that is still open.
-    if (ok) w.barrier(E.full_addr + 8u * last_unit, E.parity, ERR_WAIT_FULL);
 }
 
 __device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint32_t blob_off, uint32_t cg, int it)
@@ -610,9 +607,9 @@ __device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint
     E.flags = h0.w;
     E.d0 = (h1.w > 1 && (use & 1u)) ? h3.y : h3.x;
     E.cols = h2.w;
-    E.full_addr = smem_u32(&c.ctrl->bars[h3.z]);
+    E.full_addr = smem_u32(&c.ctrl->bars[h3.z + (use & 1u) * h4.z]);
     E.done_addr = smem_u32(&c.ctrl->stored[h3.w]);
-    E.parity = use & 1u;
+    E.parity = (use >> 1) & 1u;
     E.const_addr = desc + h5.y;
     E.out_base = c.sbase + h6.x; E.out_plane = h6.y; E.out_pitch16 = h6.z; E.out_n_lines = h6.w;
     E.out_log_lines = h7.x; E.out_nb = h7.y; E.out_logI = h7.z; E.res_base = c.sbase + h7.w;
@@ -620,13 +617,11 @@ __device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint
     E.lo = (int32_t)h9.x; E.res_m2 = h9.y;
     E.res_r2 = (long long)(((unsigned long long)h9.w << 32) | h9.z);
     const uint32_t passes = desc + h5.w, n_passes = h0.y;
-    // the unit whose accumulators complete last closes the pass list
-    const uint32_t last_unit = lds32(passes + 4u * (n_passes - 1u)) >> 24;
     switch (E.flags & (CF_RES | CF_LO)) {
-    case 0: epi_conv_passes<false, false>(w, E, c, passes, n_passes, last_unit, cg); break;
-    case CF_RES: epi_conv_passes<true, false>(w, E, c, passes, n_passes, last_unit, cg); break;
-    case CF_LO: epi_conv_passes<false, true>(w, E, c, passes, n_passes, last_unit, cg); break;
-    default: epi_conv_passes<true, true>(w, E, c, passes, n_passes, last_unit, cg); break;
+    case 0: epi_conv_passes<false, false>(w, E, c, passes, n_passes, cg); break;
+    case CF_RES: epi_conv_passes<true, false>(w, E, c, passes, n_passes, cg); break;
+    case CF_LO: epi_conv_passes<false, true>(w, E, c, passes, n_passes, cg); break;
+    default: epi_conv_passes<true, true>(w, E, c, passes, n_passes, cg); break;
     }
 }
 
@@ -798,7 +793,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
                     if (lane == 0 && role_ok && !ctrl->abort_flag && conv_index + 1 < p.n_conv)
                         role_ok = loader_copy(p, ctrl, sbase, conv_index + 1, cg + 1u, it);
                     __syncwarp();
-                } else {
+                } else if (!ctrl->abort_flag) {
                     epi_conv(p, c, e.y, cg, it);
                 }
                 conv_index += 1;
@@ -1160,7 +1155,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         std::vector<int> order((size_t)cp.m);
         for (int y = 0; y < cp.m; ++y) order[(size_t)y] = y;
         std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return last_op[(size_t)a] < last_op[(size_t)b]; });
-        const int sup = cp.m >= 8 ? 2 : 1;
+        const int sup = cp.m >= 2 ? 2 : 1;
         cp.n_units = (cp.m + sup - 1) / sup;
         cp.unit_of.assign((size_t)cp.m, 0);
         std::vector<int> unit_last_op((size_t)cp.n_units, -1);
@@ -1279,7 +1274,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
     bar_counts_out->clear();
     for (size_t k = 0; k < class_lines.size(); ++k) {
         class_full[k] = (int)bar_counts_out->size();
-        for (int l = 0; l < class_lines[k]; ++l) bar_counts_out->push_back((uint8_t)kIssuers);    // one arrival per issuing thread
+        for (int l = 0; l < 2 * class_lines[k]; ++l) bar_counts_out->push_back((uint8_t)kIssuers);    // two sets, one arrival per issuing thread
         class_done[k] = (int)bar_counts_out->size();
         for (int l = 0; l < class_lines[k]; ++l) bar_counts_out->push_back((uint8_t)(4 * class_chunks[k]));
     }
