@@ -24,13 +24,17 @@
 // operand.  Strided and 1x1 convolutions, and those with cout = 64, run unstacked: one chain per output line
 // over all taps.
 //
-// Roles.  Warp 16 issues the MMAs of one convolution after the other (a table of operations prepared on the
-// host: input line, accumulator columns, which lines of the previous convolution it must wait for, which
-// output lines it completes).  Warps 0..15 requantise: four sets of four warps (one per 32-lane quarter of
-// tensor memory) share the output lines of a convolution in the order in which they complete.  Producer and
-// consumer meet on one mbarrier pair per output line (accumulators ready / line stored), so consecutive
-// convolutions overlap line by line.  Input noise (Def. 3.3, Eq. 2; Def. 3.4), halo fills and the pool / FC /
-// argmax tail are CTA-wide phases between barriers.
+// Roles.  Four issuing warps (lane 0 of each) share the MMA chains of a convolution: the host prepares a table
+// of operations (accumulator columns, descriptor offsets, which units of the previous convolution must be stored,
+// which units complete) in the order in which their inputs become available; operation i belongs to issuing warp
+// i mod 4.  One thread alone cannot feed the tensor pipe: a chain costs it several hundred cycles of issue
+// latency.  Eight epilogue warps requantise: two sets of four warps (one per 32-lane quarter of tensor memory)
+// share the output lines of a convolution, two lines and one 16-channel chunk per pass, in the order in which
+// they complete; eight warps leave each thread 128 registers, which the unrolled requantisation needs (sixteen
+// warps at 80 registers spill and are slower).  A loader warp copies the next convolution's blob once its place is
+// free.  A unit (the lines of a pass) has two mbarriers "accumulators complete", used in turn by the convolutions
+// of a class, and a counter "stored"; consecutive convolutions overlap unit by unit.  Input noise (Def. 3.3,
+// Eq. 2; Def. 3.4), halo fills and the pool / FC / argmax tail are CTA-wide phases between barriers.
 //
 // Every device-side wait is bounded by a wall-clock limit; on expiry the CTA raises an abort flag, all
 // remaining waits fall through, and the host reports ISC_ERR_TIMEOUT.
@@ -86,10 +90,10 @@ __device__ __forceinline__ void ltrace(int ev, uint32_t cg, uint32_t tag) { ltra
 #endif
 
 constexpr int kG = 4;                       // samples per group
-constexpr int kEpiWarps = 16;               // warps 0..15: epilogue; set = warp / 4, tensor-memory quarter = warp % 4
+constexpr int kEpiWarps = 8;                // warps 0..7: epilogue; set = warp / 4, tensor-memory quarter = warp % 4
 constexpr int kSets = kEpiWarps / 4;
-constexpr int kIssuers = 4;                 // warps 16..19: lane 0 of each issues every fourth MMA chain of a convolution
-constexpr int kLoaderWarp = kEpiWarps + kIssuers;   // warp 20: weight copies
+constexpr int kIssuers = 4;                 // the next four warps: lane 0 of each issues every fourth MMA chain of a convolution
+constexpr int kLoaderWarp = kEpiWarps + kIssuers;   // the last warp: weight copies
 constexpr int kThreads = 32 * (kEpiWarps + kIssuers + 1);
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kMaxKsteps = 18;
@@ -571,7 +575,7 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
 }
 
 template <bool kRes, bool kLo>
-__device__ __noinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes,
+__device__ __forceinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes,
                                              uint32_t cg)
 {
     const EpiConv E = E_in;
@@ -585,7 +589,7 @@ __device__ __noinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, cons
     }
 }
 
-__device__ __noinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint32_t blob_off, uint32_t cg, int it)
+__device__ __forceinline__ void epi_conv(const LineParams &p, const EpiCtx &c, uint32_t blob_off, uint32_t cg, int it)
 {
     Waiter w{c.ctrl, p.err};
     bool ok = w.barrier(smem_u32(&c.ctrl->wbar[cg % 3]), (cg / 3) & 1, ERR_WAIT_WEIGHTS);
