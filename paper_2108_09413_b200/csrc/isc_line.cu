@@ -469,15 +469,32 @@ struct EpiCtx {
     uint32_t lane_idx;                  // position within a line: quarter * 32 + lane
 };
 
-// What an epilogue warp keeps in registers for the whole of a convolution.
+// What an epilogue warp keeps in registers for the whole of a convolution: addresses already specialised to the
+// thread (its position within a line, its 32 lanes of tensor memory), so that a pass only adds the offsets of its
+// table record.  The geometry that only strided convolutions need stays in the blob's header.
 struct EpiConv {
-    uint32_t flags, d0, cols, full_addr, done_addr, parity;
-    uint32_t const_addr, out_base, out_plane, out_pitch16, out_n_lines, out_log_lines, out_nb, out_logI;
-    uint32_t res_base, res_plane, in_logI, in_I, in_n_lines;
+    uint32_t flags, desc;
+    uint32_t tmem0;                       // tensor-memory address of this warp's lanes, first column of the bank
+    uint32_t full_addr, done_addr, parity;
+    uint32_t const_addr;
+    uint32_t out_thread, res_thread;      // line 0, this thread's position, plane 0 of the output / residual
+    uint32_t dup_delta;                   // bytes from a band's first row to its copy below the band above; 0: one band
+    uint32_t dup_up, dup_dn;              // this thread's band has a band above / below
     int32_t lo;
     uint32_t res_m2;
     long long res_r2;
 };
+
+// One pass of the table: lines (a unit), chunk, and the offsets they imply.
+struct alignas(16) LPass {
+    uint32_t meta;          // unit | lines << 8 | chunk << 12 | line 0 first / last row of its band << 16, 17 | line 1 << 18, 19
+    uint32_t lines;         // line 0 | line 1 << 8
+    uint32_t tcol[2];       // accumulator columns of the two lines' chunk within the bank
+    uint32_t lp[2];         // byte offset of the two lines within a plane
+    uint32_t ch_out, ch_res;        // byte offset of the chunk's plane in the output / residual
+};
+static_assert(sizeof(LPass) == 32, "one pass is two 16-byte loads");
+
 
 // Per-channel requantisation constants as stored in the blob: the 64-bit addend, then multiplier and shift.
 //   y = floor((acc * mult + B) / 2^(32 + s)); B holds the folded bias, the rounding half and the output
@@ -493,59 +510,51 @@ __device__ __forceinline__ int requant1(int acc, const ChanConst &cs, uint32_t r
     return y;
 }
 
-// Stores one position's 16 channels of a plane, with the copies that the line layout asks for.
-__device__ __forceinline__ void store_out(const EpiConv &E, const EpiCtx &c, uint32_t ch, uint32_t line, uint4 o)
+// Stride 2: stores one position's 16 channels of a plane where the output's layout wants them (`line` is the ordinal
+// of an even input line; even columns and even rows survive), with the copies that the line layout asks for.
+__device__ __noinline__ void store_strided(uint32_t desc, uint32_t sbase, uint32_t lane_idx, uint32_t ch, uint32_t line, uint4 o)
 {
-    uint32_t oline = line, olane = c.lane_idx;
-    bool keep = true;
-    if (E.flags & CF_SCATTER) {
-        // stride 2: `line` is the ordinal of an even input line; even columns and even rows survive
-        const uint32_t x_i = c.lane_idx >> E.in_logI, band_i = (c.lane_idx & (E.in_I - 1u)) >> 2, s = c.lane_idx & 3u;
-        const uint32_t r_i = 2u * line + band_i * E.in_n_lines;
-        keep = !(x_i & 1u) && !(r_i & 1u);
-        const uint32_t r_o = r_i >> 1, x_o = x_i >> 1;
-        oline = r_o & (E.out_n_lines - 1u);
-        olane = (x_o << E.out_logI) + ((r_o >> E.out_log_lines) << 2) + s;
-    }
-    if (!keep) return;
-    const uint32_t addr = E.out_base + ch * E.out_plane + (oline * E.out_pitch16 + olane) * 16u;
+    const uint4 h6 = ld_shared_v4(desc + offsetof(LConvDesc, out_base));       // out_base, out_plane, out_pitch16, out_n_lines
+    const uint4 h7 = ld_shared_v4(desc + offsetof(LConvDesc, out_log_lines));  // out_log_lines, out_nb, out_logI, res_base
+    const uint4 h8 = ld_shared_v4(desc + offsetof(LConvDesc, res_plane));      // res_plane, in_logI, in_I, in_n_lines
+    const uint32_t x_i = lane_idx >> h8.y, band_i = (lane_idx & (h8.z - 1u)) >> 2, s = lane_idx & 3u;
+    const uint32_t r_i = 2u * line + band_i * h8.w;
+    if ((x_i & 1u) || (r_i & 1u)) return;
+    const uint32_t r_o = r_i >> 1, x_o = x_i >> 1;
+    const uint32_t oline = r_o & (h6.w - 1u);
+    const uint32_t olane = (x_o << h7.z) + ((r_o >> h7.x) << 2) + s;
+    const uint32_t addr = sbase + h6.x + ch * h6.y + (oline * h6.z + olane) * 16u;
     st_shared_v4(addr, o);
-    const uint32_t band = (olane >> 2) & (E.out_nb - 1u);
+    const uint32_t band = (olane >> 2) & (h7.y - 1u);
     // first row of a lower band: also the row below the band above it; last row of an upper band: the row above the next
-    if (oline == 0 && band >= 1) st_shared_v4(addr + (E.out_n_lines * E.out_pitch16 - 4u) * 16u, o);
-    if (oline == E.out_n_lines - 1u && band + 1u < E.out_nb) st_shared_v4(addr - (E.out_n_lines * E.out_pitch16 - 4u) * 16u, o);
+    if (oline == 0 && band >= 1) st_shared_v4(addr + (h6.w * h6.z - 4u) * 16u, o);
+    if (oline == h6.w - 1u && band + 1u < h7.y) st_shared_v4(addr - (h6.w * h6.z - 4u) * 16u, o);
 }
 
 // One pass: SUP output lines, one 16-channel chunk.
 template <bool kRes, bool kLo, int SUP>
-__device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCtx &c, uint32_t pw, bool &ok, uint32_t cg)
+__device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCtx &c, uint4 q0, uint4 q1, bool &ok, uint32_t cg)
 {
-    uint32_t line[SUP];
-#pragma unroll
-    for (int j = 0; j < SUP; ++j) line[j] = (pw >> (8 * j)) & 0xFFu;
-    const uint32_t ch = (pw >> 16) & 0xFu, unit = pw >> 24;
+    const uint32_t unit = q0.x & 0xFFu, ch = (q0.x >> 12) & 0xFu;
+    const uint32_t tcol[2] = {q0.z, q0.w}, lp[2] = {q1.x, q1.y};
     if (ok) ok = w.barrier(E.full_addr + 8u * unit, E.parity, ERR_WAIT_FULL);
     ok = __all_sync(0xffffffffu, ok);
-    ltrace(3, cg, line[0] | (ch << 8));
+    ltrace(3, cg, (q0.y & 0xFFu) | (ch << 8));
     tc_fence_after();
     int acc[SUP][16];
-    uint32_t taddr[SUP];
 #pragma unroll
-    for (int j = 0; j < SUP; ++j) {
-        taddr[j] = c.tmem_lane + E.d0 + line[j] * E.cols + ch * 16u;
-        tmem_ld16_issue(taddr[j], acc[j]);
-    }
+    for (int j = 0; j < SUP; ++j) tmem_ld16_issue(E.tmem0 + tcol[j], acc[j]);
     uint32_t rw[SUP][4];
 #pragma unroll
     for (int j = 0; j < SUP; ++j) {
         uint4 rv = make_uint4(0, 0, 0, 0);
-        if (kRes) rv = ld_shared_v4(E.res_base + ch * E.res_plane + (line[j] * E.out_pitch16 + c.lane_idx) * 16u);
+        if (kRes) rv = ld_shared_v4(E.res_thread + lp[j] + q1.w);
         rw[j][0] = rv.x ^ 0x80808080u; rw[j][1] = rv.y ^ 0x80808080u; rw[j][2] = rv.z ^ 0x80808080u; rw[j][3] = rv.w ^ 0x80808080u;
     }
     tmem_ld_wait();
     // every accumulator column is left at zero: stacked chains accumulate from their first K-step on
 #pragma unroll
-    for (int j = 0; j < SUP; ++j) tmem_st16_zero(taddr[j]);
+    for (int j = 0; j < SUP; ++j) tmem_st16_zero(E.tmem0 + tcol[j]);
     if (ok) {
         const uint32_t cbase = E.const_addr + ch * 256u;
         uint32_t out[SUP][4];
@@ -563,7 +572,21 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
             }
         }
 #pragma unroll
-        for (int j = 0; j < SUP; ++j) store_out(E, c, ch, line[j], make_uint4(out[j][0], out[j][1], out[j][2], out[j][3]));
+        for (int j = 0; j < SUP; ++j) {
+            const uint4 o = make_uint4(out[j][0], out[j][1], out[j][2], out[j][3]);
+            if (E.flags & CF_SCATTER) {
+                store_strided(E.desc, c.sbase, c.lane_idx, ch, (q0.y >> (8 * j)) & 0xFFu, o);
+            } else {
+                const uint32_t addr = E.out_thread + lp[j] + q1.z;
+                st_shared_v4(addr, o);
+                if (E.dup_delta) {
+                    // first row of a lower band: also the row below the band above it; last row of an upper band: the
+                    // row above the next band
+                    if (((q0.x >> (16 + 2 * j)) & 1u) & E.dup_up) st_shared_v4(addr + E.dup_delta, o);
+                    if (((q0.x >> (17 + 2 * j)) & 1u) & E.dup_dn) st_shared_v4(addr - E.dup_delta, o);
+                }
+            }
+        }
     }
     tmem_st_wait();
     // the stores become visible to the tensor cores' reads, the tensor-memory accesses are ordered before the arrival
@@ -571,7 +594,7 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
     fence_proxy_async();
     __syncwarp();
     if (c.lane == 0) red_release_add(E.done_addr + 4u * unit, 1u);
-    ltrace(4, cg, line[0] | (ch << 8));
+    ltrace(4, cg, (q0.y & 0xFFu) | (ch << 8));
 }
 
 template <bool kRes, bool kLo>
@@ -583,9 +606,9 @@ __device__ __forceinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, c
     bool ok = true;
 #pragma unroll 1
     for (uint32_t i = (uint32_t)c.set; i < n_passes; i += kSets) {
-        const uint32_t pw = lds32(passes + 4u * i);
-        if (((pw >> 20) & 0xFu) == 2u) epi_pass<kRes, kLo, 2>(w, E, c, pw, ok, cg);
-        else epi_pass<kRes, kLo, 1>(w, E, c, pw, ok, cg);
+        const uint4 q0 = ld_shared_v4(passes + 32u * i), q1 = ld_shared_v4(passes + 32u * i + 16u);
+        if (((q0.x >> 8) & 0xFu) == 2u) epi_pass<kRes, kLo, 2>(w, E, c, q0, q1, ok, cg);
+        else epi_pass<kRes, kLo, 1>(w, E, c, q0, q1, ok, cg);
     }
 }
 
@@ -604,20 +627,22 @@ __device__ __forceinline__ void epi_conv(const LineParams &p, const EpiCtx &c, u
     const uint4 h5 = ld_shared_v4(desc + offsetof(LConvDesc, w_rel));
     const uint4 h6 = ld_shared_v4(desc + offsetof(LConvDesc, out_base));       // out_base, out_plane, out_pitch16, out_n_lines
     const uint4 h7 = ld_shared_v4(desc + offsetof(LConvDesc, out_log_lines));  // out_log_lines, out_nb, out_logI, res_base
-    const uint4 h8 = ld_shared_v4(desc + offsetof(LConvDesc, res_plane));      // res_plane, in_logI, in_I, in_n_lines
     const uint4 h9 = ld_shared_v4(desc + offsetof(LConvDesc, lo));             // lo, res_m2, res_r2
     const uint32_t use = (uint32_t)it * h4.y + h4.x;
     EpiConv E;
     E.flags = h0.w;
-    E.d0 = (h1.w > 1 && (use & 1u)) ? h3.y : h3.x;
-    E.cols = h2.w;
+    E.desc = desc;
+    E.tmem0 = c.tmem_lane + ((h1.w > 1 && (use & 1u)) ? h3.y : h3.x);
     E.full_addr = smem_u32(&c.ctrl->bars[h3.z + (use & 1u) * h4.z]);
     E.done_addr = smem_u32(&c.ctrl->stored[h3.w]);
     E.parity = (use >> 1) & 1u;
     E.const_addr = desc + h5.y;
-    E.out_base = c.sbase + h6.x; E.out_plane = h6.y; E.out_pitch16 = h6.z; E.out_n_lines = h6.w;
-    E.out_log_lines = h7.x; E.out_nb = h7.y; E.out_logI = h7.z; E.res_base = c.sbase + h7.w;
-    E.res_plane = h8.x; E.in_logI = h8.y; E.in_I = h8.z; E.in_n_lines = h8.w;
+    E.out_thread = c.sbase + h6.x + c.lane_idx * 16u;
+    E.res_thread = c.sbase + h7.w + c.lane_idx * 16u;
+    const uint32_t band = (c.lane_idx >> 2) & (h7.y - 1u);
+    E.dup_delta = h7.y > 1u ? (h6.w * h6.z - 4u) * 16u : 0u;
+    E.dup_up = band >= 1u ? 1u : 0u;
+    E.dup_dn = band + 1u < h7.y ? 1u : 0u;
     E.lo = (int32_t)h9.x; E.res_m2 = h9.y;
     E.res_r2 = (long long)(((unsigned long long)h9.w << 32) | h9.z);
     const uint32_t passes = desc + h5.w, n_passes = h0.y;
@@ -947,7 +972,7 @@ struct ConvPlan {
     int n_chunks = 0, cols = 0, n_banks = 1;
     int cls = -1, use_local = 0;
     std::vector<LOp> ops;
-    std::vector<uint32_t> passes;
+    std::vector<LPass> passes;
     std::vector<int> done_time;         // per output line: index of the pass that stores its last chunk
     int n_units = 0;
     std::vector<int> unit_of;           // per output line: its unit
@@ -1264,10 +1289,23 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         for (int u = 0; u < cp.n_units; ++u)
             for (int ch = 0; ch < cp.n_chunks; ++ch) {
                 const int n = std::min(sup, cp.m - u * sup);
-                uint32_t pw = (uint32_t)order[(size_t)u * sup] | ((uint32_t)ch << 16) | ((uint32_t)n << 20) | ((uint32_t)u << 24);
-                if (n == 2) pw |= (uint32_t)order[(size_t)u * sup + 1] << 8;
-                for (int q = 0; q < n; ++q) cp.done_time[(size_t)order[(size_t)u * sup + q]] = (int)cp.passes.size() / kSets;
-                cp.passes.push_back(pw);
+                LPass P;
+                memset(&P, 0, sizeof(P));
+                P.meta = (uint32_t)u | ((uint32_t)n << 8) | ((uint32_t)ch << 12);
+                for (int q = 0; q < n; ++q) {
+                    const int line = order[(size_t)u * sup + q];
+                    P.lines |= (uint32_t)line << (8 * q);
+                    P.tcol[q] = (uint32_t)(line * cp.cols + ch * 16);
+                    P.lp[q] = (uint32_t)(line * out.pitch) * 16u;
+                    if (!cp.scatter) {
+                        if (line == 0) P.meta |= 1u << (16 + 2 * q);
+                        if (line == out.n_lines - 1) P.meta |= 1u << (17 + 2 * q);
+                    }
+                    cp.done_time[(size_t)line] = (int)cp.passes.size() / kSets;
+                }
+                P.ch_out = (uint32_t)ch * out.plane_bytes;
+                P.ch_res = L.res_tensor >= 0 ? (uint32_t)ch * T[(size_t)L.res_tensor].plane_bytes : 0u;
+                cp.passes.push_back(P);
             }
         convs.push_back(cp);
     }
@@ -1292,7 +1330,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         const uint32_t rows = (uint32_t)(cp.stacked ? 3 : 1) * (uint32_t)L.cout;
         uint32_t at = (uint32_t)sizeof(LConvDesc);
         ops_rel[(size_t)c] = at; at += ((uint32_t)cp.ops.size() + (uint32_t)kIssuers) * (uint32_t)sizeof(LOp);    // spare records: reads run one ahead
-        passes_rel[(size_t)c] = at; at += ((uint32_t)cp.passes.size() * 4u + 15u) & ~15u;
+        passes_rel[(size_t)c] = at; at += (uint32_t)cp.passes.size() * (uint32_t)sizeof(LPass);
         at = (at + 127u) & ~127u;
         w_rel[(size_t)c] = at; at += (uint32_t)cp.kunits.size() * rows * 32u;
         c_rel[(size_t)c] = at; at += (uint32_t)L.cout * 16u;
@@ -1410,7 +1448,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
             }
         memcpy(blob.data(), &D, sizeof(D));
         memcpy(blob.data() + ops_rel[(size_t)c], cp.ops.data(), cp.ops.size() * sizeof(LOp));
-        memcpy(blob.data() + passes_rel[(size_t)c], cp.passes.data(), cp.passes.size() * 4);
+        memcpy(blob.data() + passes_rel[(size_t)c], cp.passes.data(), cp.passes.size() * sizeof(LPass));
         // weights: per K-step, rows = block * cout + oc (block b = vertical tap 2 - b when stacked)
         const int taps = L.kh * L.kw;
         const uint32_t rows = (uint32_t)(cp.stacked ? 3 : 1) * (uint32_t)L.cout;
