@@ -308,6 +308,14 @@ int ensure_noise_table(isc_model *m, double sigma, cudaStream_t st)
     if (m->d_cum && m->cum_sigma == sigma) return ISC_OK;
     std::vector<uint32_t> cum;
     noise_table(sigma, cum);
+    // the guide table follows the cumulative one in the same allocation
+    const size_t n_cum = cum.size();
+    for (int j = 0; j <= isc::kNoiseGuide; ++j) {
+        const uint64_t u = (uint64_t)j << (32 - isc::kNoiseGuideBits);
+        uint32_t i = 0;
+        while (i + 1 < n_cum && u >= cum[i]) ++i;        // min{ i : u < cum[i] }, the last entry matching always
+        cum.push_back(i);
+    }
     size_t have = m->d_cum_n * sizeof(uint32_t);
     void *p = m->d_cum;
     int rc = ensure_bytes(&p, &have, cum.size() * sizeof(uint32_t));
@@ -316,7 +324,7 @@ int ensure_noise_table(isc_model *m, double sigma, cudaStream_t st)
     CK(cudaMemcpyAsync(m->d_cum, cum.data(), cum.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
     CK(cudaStreamSynchronize(st));                       // cum is a local vector
     m->cum_sigma = sigma;
-    m->cum_T = (int)(cum.size() - 1) / 2;
+    m->cum_T = (int)(n_cum - 1) / 2;
     return ISC_OK;
 }
 
@@ -339,6 +347,7 @@ NoiseStream make_stream(const isc_model *m, uint64_t seed, uint64_t image_id, in
     ns.first_sample = first;
     ns.cum = m->d_cum;
     ns.T = m->cum_T;
+    ns.guide = m->d_cum ? m->d_cum + (2 * m->cum_T + 1) : nullptr;
     return ns;
 }
 
@@ -782,6 +791,7 @@ extern "C" int isc_sample_counts_static(isc_model *m, const uint8_t *x_u8, uint6
         NoiseStream ns = make_stream(m, seed, image_id, phase, first_sample + done);
         ns.cum = d_cum;
         ns.T = T;
+        ns.guide = nullptr;
         for (int i = 0; i < n_layers; ++i) {
             const GLayer &G = m->glayers[(size_t)i];
             const isc_layer &L = m->layers[(size_t)i].d;

@@ -15,6 +15,8 @@ struct TShape {
     int cp;  // channels padded to a multiple of 16 (device NHWC layout)
 };
 
+constexpr int kNoiseGuideBits = 10, kNoiseGuide = 1 << kNoiseGuideBits;
+
 // Where the random stream of one launch starts (Philox4x32-10 key and fixed counter words).
 struct NoiseStream {
     uint32_t key0, key1;      // seed halves
@@ -23,6 +25,9 @@ struct NoiseStream {
     int64_t first_sample;     // sample id of batch slot 0
     const uint32_t *cum;      // device, 2T+1 entries
     int T;
+    // Optional guide table (device, kNoiseGuide + 1 entries, or null): guide[j] is the search result for the
+    // uniform j << (32 - kNoiseGuideBits), a lower bound of the result for every uniform with these top bits.
+    const uint32_t *guide;
 };
 
 // One layer as the layer-by-layer kernels see it (device pointers).

@@ -659,7 +659,21 @@ __device__ void fill_phase(const EpiCtx &c, uint32_t off, uint32_t bytes, uint32
 {
     const uint32_t word = (halo & 0xFFu) * 0x01010101u;
     const uint4 v = make_uint4(word, word, word, word);
-    for (uint32_t o = (uint32_t)c.tid * 16u; o < bytes; o += kEpiThreads * 16u) st_shared_v4(c.sbase + off + o, v);
+    for (uint32_t o = (uint32_t)c.tid * 16u; o < bytes; o += kThreads * 16u) st_shared_v4(c.sbase + off + o, v);
+}
+
+// Inverse-CDF search min{ z : u < cum[z] } (the last entry always matches) by bisection between the guide table's
+// results for the two uniforms that bracket u's top bits: the same result as the bisection over the whole table,
+// in one or two steps for the bulk of the distribution.
+__device__ __forceinline__ int noise_level_guided(uint32_t u, const uint32_t *__restrict__ cum, const uint32_t *__restrict__ guide, int T)
+{
+    const uint32_t j = u >> (32 - kNoiseGuideBits);
+    uint32_t lo = __ldg(guide + j), hi = __ldg(guide + j + 1);
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (u < __ldg(cum + mid)) hi = mid; else lo = mid + 1;
+    }
+    return (int)lo - T;
 }
 
 // INPUT: one thread = four horizontally adjacent pixels of one sample, all input channels (Def. 3.3, Def. 3.4).
@@ -669,10 +683,11 @@ __device__ void input_phase(const LineParams &p, const EpiCtx &c, int grp)
     const int wq = W >> 2;
     const int quads = kG * H * wq;
     const uint32_t *__restrict__ cum = p.ns.cum;
+    const uint32_t *__restrict__ guide = p.ns.guide;
     const int T = p.ns.T;
     const uint32_t key0 = p.ns.key0, key1 = p.ns.key1, ctr2 = p.ns.ctr2;
     const uint8_t *__restrict__ x = p.x;
-    for (int qi = c.tid; qi < quads; qi += kEpiThreads) {
+    for (int qi = c.tid; qi < quads; qi += kThreads) {
         // consecutive threads take consecutive samples: their stores fall into one 64-byte run
         const int s = qi & (kG - 1);
         const int rem = qi >> 2;
@@ -687,7 +702,7 @@ __device__ void input_phase(const LineParams &p, const EpiCtx &c, int grp)
             const uint32_t clean = __ldg(reinterpret_cast<const uint32_t *>(x + e));
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                int v = (int)((clean >> (8 * k)) & 0xFF) + noise_level(u[k], cum, T);
+                int v = (int)((clean >> (8 * k)) & 0xFF) + (guide ? noise_level_guided(u[k], cum, guide, T) : noise_level(u[k], cum, T));
                 v = min(255, max(0, v));
                 px[k] |= (uint32_t)v << (8 * ch);
             }
@@ -840,7 +855,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
                     role_ok = loader_copy(p, ctrl, sbase, 0, (uint32_t)it * (uint32_t)p.n_conv, it);
                 first_phase = false;
             }
-            if (epi && !ctrl->abort_flag) {
+            if (!ctrl->abort_flag) {           // every warp of the CTA takes part in these phases
                 if (e.x == PH_FILL) fill_phase(c, e.y, e.z, e.w);
                 else if (e.x == PH_INPUT) input_phase(p, c, grp);
                 else if (warp < kG) tail_sample(p, c, warp, grp);
