@@ -143,6 +143,23 @@ def test_partition_and_batch_invariance():
     assert np.array_equal(gm.sample_counts(x, SEED, 7, 1, 0, 0, 0.25), np.zeros(10, np.int32))
 
 
+def test_resnet110_line_engine_many_launches_and_ragged_batches():
+    """Counts must not depend on how the samples are cut into launches (Algorithm 1 counts votes, nothing else):
+    several hundred launches of the line-tiled engine with group counts that do not divide the batch."""
+    gm = isc.Model(wl.resnet110())
+    gm.set_option("engine", ENGINES["line"])
+    xs = wl.images(2, seed=5)
+    for sigma, img in ((0.12, 0), (1.0, 1)):
+        ref = None
+        for batch in (0, 257, 4099):
+            gm.set_option("batch", batch)
+            c = gm.sample_counts(xs[img], SEED, img, 1, 3, 20001, sigma)
+            assert c.sum() == 20001
+            ref = c if ref is None else ref
+            np.testing.assert_array_equal(c, ref, err_msg=f"sigma {sigma} batch {batch}")
+    assert gm.get_info("engine") == 3
+
+
 def test_certify_batch_equals_single_calls_and_oracle_prefix():
     cfg = wl.CONFIGS[1]
     model = cfg["model"]()
