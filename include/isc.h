@@ -200,6 +200,19 @@ int isc_decide_predict(const int32_t *counts, int n_classes, double alpha, int32
 int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_T);
 
 /*
+ * isc_radius_integer -- the integer-only form of the radius (Theorem 3.2 steps 2-3,
+ * Theorem 3.1): the quantile of the one-dimensional discrete Gaussian N_Z(0, (255 sigma)^2)
+ * by lookup in the cumulative table above, for a probability given as a 32-bit fixed-point
+ * fraction p_fx = floor(p * 2^32).  No GPU work, no floating point after the table is built.
+ *   out_q         : the smallest pixel level q in [-T, T] with cum[q + T] >= p_fx (T if none);
+ *                   q / 255 is the radius in [0,1] pixel units, q <= 0 certifies nothing.
+ *   out_q_squared : q * q, the squared integer radius the theorem compares distances with
+ *                   (NULL to skip).
+ * Returns ISC_ERR_ARG for a bad sigma or a NULL out_q; outputs untouched on error.
+ */
+int isc_radius_integer(double sigma, uint32_t p_fx, int32_t *out_q, int64_t *out_q_squared);
+
+/*
  * isc_debug_tensor -- evaluate sample j of one image and copy tensor `tensor`
  * (0 = the noisy input, values 0..255; i+1 = output of layer i) to `out` as
  * [C][H][W] int32 (host).  For layer-by-layer comparison; slow.

@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
 EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_predict", "isc_certify", "isc_certify_batch",
-           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_noise_table",
+           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_noise_table", "isc_radius_integer",
            "isc_debug_tensor", "isc_set_option", "isc_get_info", "isc_strerror"]
 
 
@@ -56,6 +56,7 @@ def lib():
         L.isc_decide_certify.argtypes = [vp, vp, C.c_int, C.c_int64, C.c_double, C.c_double, i32p, f64p, f64p]
         L.isc_decide_predict.argtypes = [vp, C.c_int, C.c_double, i32p]
         L.isc_noise_table.argtypes = [C.c_double, vp, C.c_int64, i32p]
+        L.isc_radius_integer.argtypes = [C.c_double, C.c_uint32, i32p, C.POINTER(C.c_int64)]
         L.isc_debug_tensor.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int32, C.c_int64, C.c_double,
                                        C.c_int, vp, vp, C.c_int64]
         L.isc_set_option.argtypes = [vp, C.c_char_p, C.c_int64]
@@ -214,6 +215,13 @@ def predict_decide(counts, alpha):
     cls = C.c_int32()
     _check(lib().isc_decide_predict(_ptr(c), c.size, float(alpha), C.byref(cls)), "isc_decide_predict")
     return cls.value
+
+
+def radius_integer(sigma, p_fx):
+    """(q, q*q): integer-only quantile of the discrete Gaussian for p_fx = floor(p * 2^32) (Theorem 3.2 steps 2-3)."""
+    q, q2 = C.c_int32(), C.c_int64()
+    _check(lib().isc_radius_integer(float(sigma), int(p_fx), C.byref(q), C.byref(q2)), "isc_radius_integer")
+    return q.value, q2.value
 
 
 def noise_table(sigma):

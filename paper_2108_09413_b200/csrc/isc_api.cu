@@ -658,6 +658,20 @@ int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_
     return ISC_OK;
 }
 
+int isc_radius_integer(double sigma, uint32_t p_fx, int32_t *out_q, int64_t *out_q_squared)
+{
+    if (!out_q || !(sigma > 0.0) || !std::isfinite(sigma) || sigma > 64.0) return ISC_ERR_ARG;
+    std::vector<uint32_t> t;
+    noise_table(sigma, t);
+    const int32_t T = (int32_t)(t.size() - 1) / 2;
+    // the table is non-decreasing: first entry that reaches p_fx
+    const int32_t q = (int32_t)(std::lower_bound(t.begin(), t.end(), p_fx) - t.begin());
+    const int32_t level = q > 2 * T ? T : q - T;
+    *out_q = level;
+    if (out_q_squared) *out_q_squared = (int64_t)level * (int64_t)level;
+    return ISC_OK;
+}
+
 int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id, int32_t phase,
                      int64_t j, double sigma, int tensor, void *cuda_stream, int32_t *out, int64_t capacity)
 {

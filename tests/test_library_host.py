@@ -104,3 +104,23 @@ def test_load_rejects_malformed_models_without_a_gpu():
     no_w["layers"][0]["w"] = None
     assert _load(no_w)[0] == -1
     assert h.value is None
+
+
+def test_integer_radius_equals_oracle_lookup():
+    """Theorem 3.2 steps 2-3: the library's table-lookup quantile and squared radius against the oracle's linear
+    scan of its own table, on a sweep of probabilities (incl. both ends of the table and exact table values)."""
+    rng = np.random.default_rng(7)
+    for sigma in (0.12, 0.25, 0.5, 1.0):
+        cum = oracle.dgauss_table(sigma)
+        T = (cum.size - 1) // 2
+        ps = [0, 1, 2 ** 31, 2 ** 32 - 1, int(0.9889 * 2 ** 32), int(0.99993 * 2 ** 32)]
+        ps += [int(v) for v in cum[[0, 1, T - 1, T, T + 1, cum.size - 2, cum.size - 1]]]
+        ps += [int(v) + 1 for v in cum[[0, T, cum.size - 2]] if int(v) + 1 < 2 ** 32]
+        ps += [int(v) for v in rng.integers(0, 2 ** 32, size=200, dtype=np.uint64)]
+        for p_fx in ps:
+            q, q2 = isc.radius_integer(sigma, p_fx)
+            assert q == oracle.dgauss_quantile_fx(p_fx, cum), (sigma, p_fx)
+            assert q2 == q * q
+    q = C.c_int32(123)
+    assert isc.lib().isc_radius_integer(0.0, 5, C.byref(q), None) == -1 and q.value == 123
+    assert isc.lib().isc_radius_integer(0.25, 5, None, None) == -1
