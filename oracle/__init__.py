@@ -292,3 +292,24 @@ def predict(m: Model, x_u8, seed, image_id, N, sigma, alpha):
     if rc:
         raise ValueError("oracle: bad layer list")
     return cls.value, c
+
+
+def certified_metrics(classes, radii, labels, thresholds):
+    """Certified Percentage and Certified Accuracy at each radius threshold (Sec. 4.1, Evaluation Metrics,
+    the two displayed equations): CP = share of inputs whose certification does not abstain (class != -1);
+    CA(r) = among those, the share with the correct class and a certified radius >= r (0 when nothing certifies).
+    Plain loops over the definition; test infrastructure like the rest of this package."""
+    L = len(classes)
+    certified = 0
+    for i in range(L):
+        if int(classes[i]) != -1:
+            certified += 1
+    cp = certified / L if L else 0.0
+    ca = []
+    for r in thresholds:
+        hit = 0
+        for i in range(L):
+            if int(classes[i]) != -1 and int(classes[i]) == int(labels[i]) and float(radii[i]) >= float(r):
+                hit += 1
+        ca.append(hit / certified if certified else 0.0)
+    return cp, ca

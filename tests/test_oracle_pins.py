@@ -402,6 +402,38 @@ def test_integer_quantile_lookup_tracks_normal_quantile():
             assert abs(q - 255 * sigma * st.norm.ppf(p)) <= 1.5
 
 
+def test_certified_metrics_closed_forms():
+    """Sec. 4.1, Evaluation Metrics: closed forms of the two displayed equations."""
+    L = 40
+    labels = [i % 10 for i in range(L)]
+    # everything certified and correct, radii i / L: CA(r) is the share of radii >= r, CP = 1
+    radii = [i / L for i in range(L)]
+    cp, ca = oracle.certified_metrics(labels, radii, labels, [0.0, 0.25, 0.5, 0.975, 1.0])
+    assert cp == 1.0 and ca == [1.0, 0.75, 0.5, 1 / L, 0.0]
+    # everything abstains: both are 0, whatever the labels
+    cp, ca = oracle.certified_metrics([-1] * L, [0.0] * L, labels, [0.0, 0.5])
+    assert cp == 0.0 and ca == [0.0, 0.0]
+    # half abstain: CP = 1/2 and the denominator of CA is the certified half (the equation's own denominator)
+    classes = [labels[i] if i % 2 == 0 else -1 for i in range(L)]
+    cp, ca = oracle.certified_metrics(classes, [1.0] * L, labels, [0.5, 1.0, 1.5])
+    assert cp == 0.5 and ca == [1.0, 1.0, 0.0]
+    # wrong classes count as certified (CP) but never as accurate (CA)
+    wrong = [(labels[i] + 1) % 10 for i in range(L)]
+    cp, ca = oracle.certified_metrics(wrong, [1.0] * L, labels, [0.0])
+    assert cp == 1.0 and ca == [0.0]
+    # CA is non-increasing in r and invariant under a permutation of the inputs
+    rng = np.random.default_rng(3)
+    classes = rng.integers(-1, 10, size=200)
+    radii = rng.random(200)
+    lab = rng.integers(0, 10, size=200)
+    th = [0.0, 0.1, 0.3, 0.6, 0.9]
+    cp, ca = oracle.certified_metrics(classes, radii, lab, th)
+    assert all(a >= b for a, b in zip(ca, ca[1:]))
+    perm = rng.permutation(200)
+    assert oracle.certified_metrics(classes[perm], radii[perm], lab[perm], th) == (cp, ca)
+    assert oracle.certified_metrics([], [], [], [0.5]) == (0.0, [0.0])
+
+
 # --------------------------------------------------------- whole-loop properties
 
 def test_prefix_partition_and_limit_properties():
