@@ -213,6 +213,21 @@ int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_
 int isc_radius_integer(double sigma, uint32_t p_fx, int32_t *out_q, int64_t *out_q_squared);
 
 /*
+ * isc_certified_metrics -- Certified Percentage and Certified Accuracy over a set of
+ * certification results (Sec. 4.1, Evaluation Metrics, the two displayed equations); host only.
+ *   classes, radii : what isc_certify returned for n inputs (class -1 = ABSTAIN), host arrays [n]
+ *   labels         : ground-truth classes [n]
+ *   r, n_r         : radius thresholds [n_r] (n_r may be 0)
+ *   out_cp         : inputs that did not abstain / n (0 for n = 0)
+ *   out_ca         : [n_r]; for each threshold, inputs that did not abstain, were classified
+ *                    correctly and have radius >= r, divided by the inputs that did not abstain
+ *                    (the denominator the equation prints; 0 when none certified)
+ * Returns ISC_ERR_ARG for NULL arrays with n > 0, negative sizes or a NULL out_cp.
+ */
+int isc_certified_metrics(const int32_t *classes, const double *radii, const int32_t *labels, int64_t n,
+                          const double *r, int n_r, double *out_cp, double *out_ca);
+
+/*
  * isc_debug_tensor -- evaluate sample j of one image and copy tensor `tensor`
  * (0 = the noisy input, values 0..255; i+1 = output of layer i) to `out` as
  * [C][H][W] int32 (host).  For layer-by-layer comparison; slow.

@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
 EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_predict", "isc_certify", "isc_certify_batch",
-           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_noise_table", "isc_radius_integer",
+           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_noise_table", "isc_radius_integer", "isc_certified_metrics",
            "isc_debug_tensor", "isc_set_option", "isc_get_info", "isc_strerror"]
 
 
@@ -57,6 +57,7 @@ def lib():
         L.isc_decide_predict.argtypes = [vp, C.c_int, C.c_double, i32p]
         L.isc_noise_table.argtypes = [C.c_double, vp, C.c_int64, i32p]
         L.isc_radius_integer.argtypes = [C.c_double, C.c_uint32, i32p, C.POINTER(C.c_int64)]
+        L.isc_certified_metrics.argtypes = [vp, vp, vp, C.c_int64, vp, C.c_int, C.POINTER(C.c_double), vp]
         L.isc_debug_tensor.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int32, C.c_int64, C.c_double,
                                        C.c_int, vp, vp, C.c_int64]
         L.isc_set_option.argtypes = [vp, C.c_char_p, C.c_int64]
@@ -215,6 +216,20 @@ def predict_decide(counts, alpha):
     cls = C.c_int32()
     _check(lib().isc_decide_predict(_ptr(c), c.size, float(alpha), C.byref(cls)), "isc_decide_predict")
     return cls.value
+
+
+def certified_metrics(classes, radii, labels, thresholds):
+    """(CP, [CA(r) for r in thresholds]) over certification results (Sec. 4.1, Evaluation Metrics)."""
+    c = np.ascontiguousarray(classes, dtype=np.int32)
+    rd = np.ascontiguousarray(radii, dtype=np.float64)
+    lb = np.ascontiguousarray(labels, dtype=np.int32)
+    th = np.ascontiguousarray(thresholds, dtype=np.float64)
+    ca = np.zeros(th.size, dtype=np.float64)
+    cp = C.c_double()
+    _check(lib().isc_certified_metrics(_ptr(c) if c.size else None, _ptr(rd) if rd.size else None, _ptr(lb) if lb.size else None,
+                                       c.size, _ptr(th) if th.size else None, th.size, C.byref(cp),
+                                       _ptr(ca) if ca.size else None), "isc_certified_metrics")
+    return cp.value, ca.tolist()
 
 
 def radius_integer(sigma, p_fx):

@@ -658,6 +658,24 @@ int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_
     return ISC_OK;
 }
 
+int isc_certified_metrics(const int32_t *classes, const double *radii, const int32_t *labels, int64_t n,
+                          const double *r, int n_r, double *out_cp, double *out_ca)
+{
+    if (!out_cp || n < 0 || n_r < 0 || (n > 0 && (!classes || !radii || !labels)) || (n_r > 0 && (!r || !out_ca)))
+        return ISC_ERR_ARG;
+    int64_t certified = 0;
+    for (int64_t i = 0; i < n; ++i) certified += classes[i] != -1;
+    std::vector<double> ca((size_t)n_r, 0.0);
+    for (int t = 0; t < n_r; ++t) {
+        int64_t hit = 0;
+        for (int64_t i = 0; i < n; ++i) hit += classes[i] != -1 && classes[i] == labels[i] && radii[i] >= r[t];
+        ca[(size_t)t] = certified ? (double)hit / (double)certified : 0.0;
+    }
+    *out_cp = n ? (double)certified / (double)n : 0.0;
+    for (int t = 0; t < n_r; ++t) out_ca[t] = ca[(size_t)t];
+    return ISC_OK;
+}
+
 int isc_radius_integer(double sigma, uint32_t p_fx, int32_t *out_q, int64_t *out_q_squared)
 {
     if (!out_q || !(sigma > 0.0) || !std::isfinite(sigma) || sigma > 64.0) return ISC_ERR_ARG;

@@ -124,3 +124,17 @@ def test_integer_radius_equals_oracle_lookup():
     q = C.c_int32(123)
     assert isc.lib().isc_radius_integer(0.0, 5, C.byref(q), None) == -1 and q.value == 123
     assert isc.lib().isc_radius_integer(0.25, 5, None, None) == -1
+
+
+def test_certified_metrics_equal_oracle():
+    """Certified Percentage / Certified Accuracy (Sec. 4.1): the library's reduction against the oracle's loops."""
+    rng = np.random.default_rng(11)
+    th = [0.0, 0.25, 0.5, 0.75, 1.0, 1.25, 1.5, 1.75, 2.0]
+    for n in (0, 1, 7, 500):
+        classes = rng.integers(-1, 10, size=n)
+        radii = np.where(classes == -1, 0.0, rng.random(n) * 2.0)
+        labels = np.where(rng.random(n) < 0.7, np.maximum(classes, 0), rng.integers(0, 10, size=n))
+        assert isc.certified_metrics(classes, radii, labels, th) == oracle.certified_metrics(classes, radii, labels, th)
+    assert isc.certified_metrics([-1, -1], [0.0, 0.0], [1, 2], []) == (0.0, [])
+    cp = C.c_double(9.0)
+    assert isc.lib().isc_certified_metrics(None, None, None, 3, None, 0, C.byref(cp), None) == -1 and cp.value == 9.0
