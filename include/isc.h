@@ -240,13 +240,12 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
  * isc_set_option -- tuning knobs; none changes a result.
  *   "batch"  : noisy samples per launch (0 = choose automatically).
  *   "engine" : 0 = automatic (the fastest engine the model fits), 1 = layer-by-layer
- *              kernels only, 2 = require the shared-memory-resident tensor-core kernel
- *              with flat position tiles, 3 = require the line-tiled resident kernel
- *              (ISC_ERR_UNSUPPORTED at the next call if the model does not fit the
- *              engine asked for).
+ *              kernels only, 3 = require the line-tiled shared-memory-resident
+ *              tensor-core kernel (ISC_ERR_UNSUPPORTED at the next call if the model
+ *              does not fit it).  2 is not an engine (ISC_ERR_ARG).
  * isc_get_info reads back: "engine" (the engine the last call used), "gpu_launches"
- * (kernel launches issued by this handle so far), "macs_per_sample",
- * "has_resident_engine" and "has_line_engine" (1 if the model fits engine 2 / 3).
+ * (kernel launches issued by this handle so far), "macs_per_sample" and
+ * "has_line_engine" (1 if the model fits engine 3).
  */
 int isc_set_option(isc_model *m, const char *name, int64_t value);
 int isc_get_info(isc_model *m, const char *name, int64_t *out);

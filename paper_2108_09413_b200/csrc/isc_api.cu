@@ -14,7 +14,6 @@
 #include "isc.h"
 #include "isc_internal.h"
 #include "isc_line.h"
-#include "isc_mega.h"
 
 using namespace isc;
 
@@ -60,7 +59,6 @@ struct isc_model {
     double cum_sigma = -1.0;
     int cum_T = 0;
 
-    isc::MegaPlan *mega = nullptr;
     isc::LinePlan *line = nullptr;
 
     int64_t opt_batch = 0, opt_engine = 0;
@@ -354,10 +352,8 @@ NoiseStream make_stream(const isc_model *m, uint64_t seed, uint64_t image_id, in
 int choose_engine(isc_model *m)
 {
     if (m->opt_engine == 1) return 1;
-    if (m->opt_engine == 2) return m->mega ? 2 : ISC_ERR_UNSUPPORTED;
     if (m->opt_engine == 3) return m->line ? 3 : ISC_ERR_UNSUPPORTED;
     if (m->line) return 3;
-    if (m->mega) return 2;
     return 1;
 }
 
@@ -398,11 +394,10 @@ int run_counts(isc_model *m, const uint8_t *d_x, uint64_t seed, uint64_t image_i
     const int engine = choose_engine(m);
     if (engine < 0) return engine;
     m->last_engine = engine;
-    if (engine == 2 || engine == 3) {
+    if (engine == 3) {
         NoiseStream ns = make_stream(m, seed, image_id, phase, first);
         int64_t launches = 0;
-        int rc = engine == 3 ? isc::line_run(m->line, d_x, ns, n, (int)m->opt_batch, d_counts, d_logits, st, &launches)
-                             : isc::mega_run(m->mega, d_x, ns, n, (int)m->opt_batch, d_counts, d_logits, st, &launches);
+        int rc = isc::line_run(m->line, d_x, ns, n, (int)m->opt_batch, d_counts, d_logits, st, &launches);
         m->launches += launches;
         return rc;
     }
@@ -483,15 +478,14 @@ int isc_load_qmodel(const isc_layer *layers, int n_layers, int in_c, int in_h, i
         rc = build_host_model(m, layers, n_layers);
         if (rc == ISC_OK) rc = build_generic_engine(m);
         if (rc == ISC_OK) {
-            std::vector<isc::MegaLayerIn> ml(m->layers.size());
+            std::vector<isc::LayerIn> ml(m->layers.size());
             for (size_t i = 0; i < m->layers.size(); ++i) {
                 const HostLayer &H = m->layers[i];
                 ml[i].d = H.d;
                 ml[i].w = H.w.data(); ml[i].bias = H.bias.data();
                 ml[i].mult = H.mult.data(); ml[i].shift = H.shift.data();
             }
-            rc = isc::mega_build(ml.data(), (int)ml.size(), in_c, in_h, in_w, n_classes, &m->mega);
-            if (rc == ISC_OK) rc = isc::line_build(ml.data(), (int)ml.size(), in_c, in_h, in_w, n_classes, &m->line);
+            rc = isc::line_build(ml.data(), (int)ml.size(), in_c, in_h, in_w, n_classes, &m->line);
         }
     } catch (const std::bad_alloc &) {
         rc = ISC_ERR_NOMEM;
@@ -513,7 +507,6 @@ void isc_free_qmodel(isc_model *m)
     if (m->d_counts) cudaFree(m->d_counts);
     if (m->d_logits) cudaFree(m->d_logits);
     if (m->d_cum) cudaFree(m->d_cum);
-    isc::mega_free(m->mega);
     isc::line_free(m->line);
     delete m;
 }
@@ -552,7 +545,6 @@ int isc_sample_counts(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t
         CK(cudaMemcpyAsync(hl.data(), m->d_logits, hl.size(), cudaMemcpyDeviceToHost, st));
     }
     CK(cudaStreamSynchronize(st));
-    if (m->mega && (rc = isc::mega_check(m->mega))) return rc;
     if (m->line && (rc = isc::line_check(m->line))) return rc;
     memcpy(out_counts, h.data(), C * sizeof(int32_t));
     if (out_logits && n_samples > 0) memcpy(out_logits, hl.data(), hl.size());
@@ -600,7 +592,6 @@ int isc_certify_batch(isc_model *m, const uint8_t *x_u8, int x_on_device, int n_
     std::vector<int32_t> h(2 * C * (size_t)n_images);
     CK(cudaMemcpyAsync(h.data(), m->d_counts, h.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
-    if (m->mega && (rc = isc::mega_check(m->mega))) return rc;
     if (m->line && (rc = isc::line_check(m->line))) return rc;
     for (int i = 0; i < n_images; ++i) {
         const int32_t *c0 = h.data() + (size_t)i * 2 * C, *c1 = c0 + C;
@@ -704,13 +695,11 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
     const uint8_t *d_x;
     if ((rc = stage_image(m, x_u8, (size_t)m->in_c * m->in_h * m->in_w, false, st, &d_x))) return rc;
     NoiseStream ns = make_stream(m, seed, image_id, phase, j);
-    if (m->opt_engine == 2 || m->opt_engine == 3) {       // read the tensor back from a resident engine
-        if (m->opt_engine == 2 ? !m->mega : !m->line) return ISC_ERR_UNSUPPORTED;
+    if (m->opt_engine == 3) {       // read the tensor back from the resident engine
+        if (!m->line) return ISC_ERR_UNSUPPORTED;
         if ((rc = ensure_counts(m, (size_t)m->n_classes))) return rc;
         std::vector<int32_t> tmp(n);
-        rc = m->opt_engine == 3
-            ? isc::line_debug_tensor(m->line, d_x, ns, tensor, tmp.data(), m->d_counts, st, &m->launches)
-            : isc::mega_debug_tensor(m->mega, d_x, ns, tensor, tmp.data(), m->d_counts, st, &m->launches);
+        rc = isc::line_debug_tensor(m->line, d_x, ns, tensor, tmp.data(), m->d_counts, st, &m->launches);
         if (rc) return rc;
         memcpy(out, tmp.data(), n * sizeof(int32_t));
         return ISC_OK;
@@ -813,6 +802,7 @@ extern "C" int isc_sample_counts_static(isc_model *m, const uint8_t *x_u8, uint6
 
     std::vector<uint32_t> cum;
     noise_table(sigma, cum);
+    m->last_engine = 1;
     // the array keeps whatever the previous call left: the vote counts must start from zero
     CK(cudaMemsetAsync(d_counts, 0, C * sizeof(int32_t), st));
     CK(cudaMemcpyAsync(d_cum, cum.data(), cum.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
@@ -861,7 +851,7 @@ int isc_set_option(isc_model *m, const char *name, int64_t value)
         return ISC_OK;
     }
     if (!strcmp(name, "engine")) {
-        if (value < 0 || value > 3) return ISC_ERR_ARG;
+        if (value != 0 && value != 1 && value != 3) return ISC_ERR_ARG;
         m->opt_engine = value;
         return ISC_OK;
     }
@@ -874,7 +864,6 @@ int isc_get_info(isc_model *m, const char *name, int64_t *out)
     if (!strcmp(name, "engine")) *out = m->last_engine;
     else if (!strcmp(name, "gpu_launches")) *out = m->launches;
     else if (!strcmp(name, "macs_per_sample")) *out = m->macs;
-    else if (!strcmp(name, "has_resident_engine")) *out = m->mega ? 1 : 0;
     else if (!strcmp(name, "has_line_engine")) *out = m->line ? 1 : 0;
     else return ISC_ERR_ARG;
     return ISC_OK;

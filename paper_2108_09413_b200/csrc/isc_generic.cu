@@ -1,7 +1,7 @@
 // Layer-by-layer engine: one kernel launch per layer over a batch of noisy samples, int8
 // activations in global memory as [sample][y][x][channel padded to 16].  It runs every layer
 // type of the ABI and any shape; the shared-memory-resident tensor-core engine
-// (isc_mega.cu) takes over for the CIFAR-shaped residual networks it is specialised for.
+// (isc_line.cu) takes over for the CIFAR-shaped residual networks it is specialised for.
 //
 // The noisy copies of the image (Def. 3.4: x + delta, delta ~ discrete Gaussian of Eq. 2)
 // are produced inside the first convolution's input staging and never written to memory.

@@ -43,6 +43,15 @@ struct GLayer {
     const int32_t *shift;   // [coutp]
 };
 
+// One validated layer with its host arrays, as the engines' planners receive it.
+struct LayerIn {
+    isc_layer d;
+    const int8_t *w;
+    const int32_t *bias;
+    const int32_t *mult;
+    const int8_t *shift;
+};
+
 // ---- layer-by-layer engine (isc_generic.cu) ----
 cudaError_t launch_first_conv(const GLayer &L, const uint8_t *x_chw, int in_c, const NoiseStream &ns,
                               int batch, int8_t *out, cudaStream_t st);

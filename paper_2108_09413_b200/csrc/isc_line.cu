@@ -57,38 +57,6 @@ using namespace tc;
 
 namespace {
 
-#ifdef ISC_TRACE
-// Timeline instrumentation, compiled only with -DISC_TRACE: CTA 0 records (event, warp, line, chunk, convolution;
-// value) pairs in global memory for the convolutions in [c_trace_lo, c_trace_hi); the slot counter lives in the last
-// 16 bytes of the control block.
-constexpr unsigned kTraceMax = 16384;                // 8 bytes each
-__device__ unsigned int g_ltrace[2 * kTraceMax];
-__device__ unsigned int g_ltrace_n;
-__constant__ unsigned int c_trace_lo, c_trace_hi;
-constexpr unsigned kTraceCounterOff = 9216 - 16;
-__device__ __forceinline__ void ltrace_val(int ev, uint32_t cg, uint32_t tag, uint32_t val)
-{
-    extern __shared__ __align__(128) uint8_t trace_smem[];
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && cg >= c_trace_lo && cg < c_trace_hi) {
-        const unsigned i = atomicAdd(reinterpret_cast<unsigned int *>(trace_smem + kTraceCounterOff), 1u);
-        if (i < kTraceMax) {
-            g_ltrace[2 * i] = (unsigned)ev | ((threadIdx.x >> 5) << 4) | ((tag & 0x7FFu) << 9) | ((cg - c_trace_lo) << 20);
-            g_ltrace[2 * i + 1] = val;
-        }
-    }
-}
-__device__ __forceinline__ void ltrace(int ev, uint32_t cg, uint32_t tag) { ltrace_val(ev, cg, tag, (uint32_t)clock64()); }
-#define LT_CLOCK(v) const uint32_t v = (uint32_t)clock64()
-#define LT_ARRAY(name, n) uint32_t name[n]
-#define LT_SET(name, i, v) do { if ((i) < 40) name[(i)] = (v); } while (0)
-#else
-#define ltrace(ev, cg, tag) ((void)0)
-#define ltrace_val(ev, cg, tag, val) ((void)0)
-#define LT_CLOCK(v) ((void)0)
-#define LT_ARRAY(name, n) ((void)0)
-#define LT_SET(name, i, v) ((void)0)
-#endif
-
 constexpr int kG = 4;                       // samples per group
 constexpr int kEpiWarps = 8;                // warps 0..7: epilogue; set = warp / 4, tensor-memory quarter = warp % 4
 constexpr int kSets = kEpiWarps / 4;
@@ -330,12 +298,7 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
     }
     uint32_t at = ic.ops + 32u * ic.issuer;           // the table ends with kIssuers spare records: reads run one ahead
     uint4 n0 = ld_shared_v4(at), n1 = ld_shared_v4(at + 16);
-    LT_ARRAY(tlogA, 40);
-    LT_ARRAY(tlogB, 40);
-    LT_ARRAY(tlogC, 40);
-    LT_ARRAY(tlogD, 40);
     for (uint32_t i = ic.issuer; i < ic.n_ops; i += kIssuers) {
-        LT_CLOCK(tA);
         const uint4 r0 = n0, r1 = n1;         // d_col, idesc, a_add, b_add | wait 0-1, wait 2-3, commit 0-1, commit 2 and flags
         at += 32u * kIssuers;
         n0 = ld_shared_v4(at); n1 = ld_shared_v4(at + 16);
@@ -354,7 +317,6 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
                 }
             }
         }
-        LT_CLOCK(tB);
         tc_fence_after();
         const uint32_t d = ic.d0 + r0.x;
         if ((r1.w >> 16) & OPF_NULL) {
@@ -374,7 +336,6 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
                 mma_i8(d, ad, bd, r0.y, ic.stacked | (uint32_t)(k > 0));
             }
         }
-        LT_CLOCK(tC);
         if ((r1.z & 0xFFFFu) != 0xFFFFu) {
             commit_to(ic.full_addr + (r1.z & 0xFFFFu));
             if ((r1.z >> 16) != 0xFFFFu) {
@@ -382,15 +343,7 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
                 if ((r1.w & 0xFFFFu) != 0xFFFFu) commit_to(ic.full_addr + (r1.w & 0xFFFFu));
             }
         }
-        LT_CLOCK(tD);
-        LT_SET(tlogA, i, tA);
-        LT_SET(tlogB, i, tB);
-        LT_SET(tlogC, i, tC);
-        LT_SET(tlogD, i, tD);
     }
-#ifdef ISC_TRACE
-    for (uint32_t i = ic.issuer; i < ic.n_ops && i < 40; i += kIssuers) { ltrace_val(1, ic.cg, i, tlogA[i]); ltrace_val(2, ic.cg, i, tlogB[i]); ltrace_val(5, ic.cg, i, tlogC[i]); ltrace_val(6, ic.cg, i, tlogD[i]); }
-#endif
     return true;
 }
 
@@ -539,7 +492,6 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
     const uint32_t tcol[2] = {q0.z, q0.w}, lp[2] = {q1.x, q1.y};
     if (ok) ok = w.barrier(E.full_addr + 8u * unit, E.parity, ERR_WAIT_FULL);
     ok = __all_sync(0xffffffffu, ok);
-    ltrace(3, cg, (q0.y & 0xFFu) | (ch << 8));
     tc_fence_after();
     int acc[SUP][16];
 #pragma unroll
@@ -594,7 +546,6 @@ __device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCt
     fence_proxy_async();
     __syncwarp();
     if (c.lane == 0) red_release_add(E.done_addr + 4u * unit, 1u);
-    ltrace(4, cg, (q0.y & 0xFFu) | (ch << 8));
 }
 
 template <bool kRes, bool kLo>
@@ -791,9 +742,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     for (int i = threadIdx.x; i < p.n_phases; i += blockDim.x) ctrl->ptab[i] = p.ptab[i];
     for (int i = threadIdx.x; i < p.n_conv; i += blockDim.x) ctrl->csrc[i] = p.conv_src[i];
     for (int i = threadIdx.x; i < kMaxBars; i += blockDim.x) ctrl->stored[i] = 0;
-#ifdef ISC_TRACE
-    if (threadIdx.x == 0) *reinterpret_cast<unsigned int *>(smem + kTraceCounterOff) = 0;
-#endif
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -873,9 +821,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     if (p.dump)
         for (uint32_t o = threadIdx.x * 16u; o < p.dump_bytes; o += blockDim.x * 16u)
             *reinterpret_cast<uint4 *>(p.dump + o) = ld_shared_v4(sbase + p.dump_off + o);
-#ifdef ISC_TRACE
-    if (blockIdx.x == 0 && threadIdx.x == 0) g_ltrace_n = min(*reinterpret_cast<unsigned int *>(smem + kTraceCounterOff), kTraceMax);
-#endif
     // no tensor-core work may be in flight when tensor memory is released
     if (issuer && lane == 0) {
         Waiter w{ctrl, p.err};
@@ -998,7 +943,7 @@ struct ConvPlan {
     std::vector<Unit> units;
 };
 
-bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, LinePlan *plan,
+bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, LinePlan *plan,
                 std::vector<uint8_t> *blob_out, std::vector<uint32_t> *blob_offsets, std::vector<PhaseEntry> *ptab_out,
                 std::vector<ConvSrc> *csrc_out, std::vector<uint8_t> *bar_counts_out)
 {
@@ -1403,7 +1348,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
         if (S.kind != PH_CONV) continue;
         const int c = conv_at++;
         const ConvPlan &cp = convs[(size_t)c];
-        const MegaLayerIn &ML = layers[cp.layer];
+        const LayerIn &ML = layers[cp.layer];
         const isc_layer &L = ML.d;
         const LGeo &in = T[(size_t)cp.in_tensor], &out = T[(size_t)cp.out_tensor];
         E.a = w_off[(size_t)c];
@@ -1525,7 +1470,7 @@ bool build_plan(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int
 
 }  // namespace
 
-int line_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, LinePlan **out)
+int line_build(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, LinePlan **out)
 {
     *out = nullptr;
     if (n_layers < 3 || n_classes > 128) return ISC_OK;
@@ -1568,7 +1513,7 @@ int line_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int 
     const int C = LP.cin;
     std::vector<int8_t> fcw((size_t)n_classes * 64, 0);
     std::vector<FcConst> fcc((size_t)n_classes);
-    const MegaLayerIn &MF = layers[n_layers - 1];
+    const LayerIn &MF = layers[n_layers - 1];
     for (int o = 0; o < n_classes; ++o) {
         long long wsum = 0;
         for (int c = 0; c < C; ++c) {
@@ -1643,15 +1588,6 @@ static int line_launch(LinePlan *p, LineParams &q, cudaStream_t st)
         p->attr_set = true;
     }
     const int grid = std::max(1, std::min(q.n_groups, p->sm_count));
-#ifdef ISC_TRACE
-    {
-        const char *lo = getenv("ISC_TRACE_LO"), *hi = getenv("ISC_TRACE_HI");
-        const unsigned vlo = lo ? (unsigned)atoi(lo) : 0u, vhi = hi ? (unsigned)atoi(hi) : 0u, zero = 0u;
-        cudaMemcpyToSymbol(c_trace_lo, &vlo, sizeof(vlo));
-        cudaMemcpyToSymbol(c_trace_hi, &vhi, sizeof(vhi));
-        cudaMemcpyToSymbol(g_ltrace_n, &zero, sizeof(zero));
-    }
-#endif
     k_line<<<grid, kThreads, p->smem_bytes, st>>>(q);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess && getenv("ISC_PLAN_DEBUG")) fprintf(stderr, "line engine: launch failed: %s\n", cudaGetErrorString(e));
@@ -1721,17 +1657,5 @@ int line_debug_tensor(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, in
     return ISC_OK;
 }
 
-#ifdef ISC_TRACE
-// Copies the recorded pairs of the last launch to the host; returns how many there are.
-extern "C" int isc_line_trace_read(unsigned int *out, int max_events)
-{
-    unsigned n = 0;
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(&n, g_ltrace_n, sizeof(n));
-    n = std::min(n, std::min(kTraceMax, (unsigned)max_events));
-    cudaMemcpyFromSymbol(out, g_ltrace, (size_t)n * 2 * sizeof(unsigned int));
-    return (int)n;
-}
-#endif
 
 }  // namespace isc

@@ -6,14 +6,13 @@
 
 #include "isc.h"
 #include "isc_internal.h"
-#include "isc_mega.h"
 
 namespace isc {
 
 struct LinePlan;
 
 // Builds the plan when the network fits the engine; otherwise *out = nullptr and ISC_OK.
-int line_build(const MegaLayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes,
+int line_build(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes,
                LinePlan **out);
 void line_free(LinePlan *p);
 

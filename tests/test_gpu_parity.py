@@ -12,7 +12,7 @@ import paper_2108_09413_b200 as isc
 pytestmark = pytest.mark.gpu
 SEED = wl.NOISE_SEED
 ALPHA = 0.001
-ENGINES = {"layerwise": 1, "resident": 2, "line": 3}
+ENGINES = {"layerwise": 1, "line": 3}
 
 
 def _pair(model):
@@ -78,7 +78,7 @@ def test_resnet20_logits_and_prefix_counts(sigma):
     _logit_parity(model, xs[1], 1, 0, 0, 100, sigma)              # the selection phase
 
 
-@pytest.mark.parametrize("engine", ["layerwise", "resident", "line"])
+@pytest.mark.parametrize("engine", ["layerwise", "line"])
 def test_resnet20_every_tensor(engine):
     model = wl.resnet20()
     gm, om = _pair(model)
@@ -98,13 +98,11 @@ def test_resnet20_every_tensor(engine):
 def test_resident_engine_is_used_for_cifar_resnets():
     for model in (wl.tiny_cnn(), wl.resnet20(), wl.resnet110()):
         gm = isc.Model(model)
-        assert gm.get_info("has_resident_engine") == 1, model["name"]
         assert gm.get_info("has_line_engine") == 1, model["name"]
         gm.sample_counts(wl.images(1)[0], SEED, 0, 1, 0, 8, 0.25)
         assert gm.get_info("engine") == 3
         gm.close()
     gm = isc.Model(wl.resnet50())
-    assert gm.get_info("has_resident_engine") == 0
     assert gm.get_info("has_line_engine") == 0
 
 

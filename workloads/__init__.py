@@ -214,3 +214,52 @@ CONFIGS = {
             sigmas=(0.12, 0.25, 0.5, 1.0), N0=100, N=100000, alpha=0.001,
             image_seed=0x15171004, batches=(256, 1024, 4096, 16384)),
 }
+
+
+# ---------------------------------------------------------------------------------------------
+# Test models whose votes spread over several classes.
+#
+# A network with random weights puts (almost) every noisy copy of an image in one class, which
+# leaves vote histograms, tie-breaking, ABSTAIN and non-maximal radii unexercised.  The variant
+# below swaps the final FC layer for one with small weights, one multiplier/shift for all
+# classes and a caller-supplied bias vector.  With biases that cancel each class's mean
+# accumulator on one chosen image (``spread_bias.json``, written by ``calibrate_spread.py``
+# beside this file from pooled features the CPU oracle reports), the logits of that image's
+# noisy copies differ by a few units only: votes spread and exact ties for the maximum occur.
+SPREAD_IMAGE_SEED = 0x15172000
+
+
+def with_spread_head(model: dict, bias, seed: int = 0x15173000, delta: int = 4, shift: int = 6) -> dict:
+    rng = SplitMix64(seed)
+    fc = dict(model["layers"][-1])
+    cout, cin = fc["cout"], fc["cin"]
+    fc["w"] = rng.ints(cout * cin, -delta, delta).astype(np.int8).reshape(cout, cin, 1, 1)
+    fc["mult"] = np.full(cout, int(rng.ints(1, 1 << 30, (1 << 31) - 1)[0]), dtype=np.int32)
+    fc["shift"] = np.full(cout, shift, dtype=np.int8)
+    fc["bias"] = np.asarray(bias, dtype=np.int32).reshape(cout)
+    return dict(model, name=model["name"] + "_spread", layers=list(model["layers"][:-1]) + [fc])
+
+
+def spread_image(shape=(3, 32, 32)) -> np.ndarray:
+    """The image the stored biases were balanced on."""
+    return images(1, shape=shape, seed=SPREAD_IMAGE_SEED)[0]
+
+
+# (delta, shift) of the head per base network: the tiny CNN's pooled features move less under noise
+SPREAD_HEADS = {"tiny_cnn": (16, 4), "resnet20": (4, 6), "resnet110": (4, 6)}
+
+
+def spread_base(name: str) -> dict:
+    return {"tiny_cnn": tiny_cnn, "resnet20": resnet20, "resnet110": resnet110}[name]()
+
+
+def spread_model(name: str, boost: int = 0) -> dict:
+    """tiny_cnn / resnet20 / resnet110 with the spread-vote head and its stored biases; `boost` is added to
+    class 0's bias (a favourite class: a majority that is not unanimous)."""
+    import json
+    import os
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "spread_bias.json")) as f:
+        bias = list(json.load(f)[name])
+    bias[0] += boost
+    delta, shift = SPREAD_HEADS[name]
+    return with_spread_head(spread_base(name), bias, delta=delta, shift=shift)
