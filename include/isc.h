@@ -91,6 +91,17 @@ int isc_load_qmodel(const isc_layer *layers, int n_layers, int in_c, int in_h, i
 void isc_free_qmodel(isc_model *m);
 
 /*
+ * isc_plan_resident -- host-only query: would isc_load_qmodel place this network on the
+ * shared-memory-resident tensor-core engine (engine 3)?  Validates the layer list exactly as
+ * isc_load_qmodel does and runs the engine's planner; touches no GPU.
+ *   returns        : 1 = fits, 0 = valid but served by the layer-by-layer kernels, < 0 = isc_status
+ *   out_rule       : 0 when it fits, else the number of the planner rule that refused it (NULL to skip)
+ *   out_smem_bytes : shared memory per CTA the plan needs when it fits (NULL to skip)
+ */
+int isc_plan_resident(const isc_layer *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes,
+                      int32_t *out_rule, int64_t *out_smem_bytes);
+
+/*
  * isc_predict -- Algorithm 2 (Appendix C): N noisy evaluations, top two vote counts
  * (n_A, n_B), two-sided exact binomial test of n_A out of n_A + n_B at 1/2; the class
  * is returned iff the p-value is <= alpha, else -1 (ABSTAIN).

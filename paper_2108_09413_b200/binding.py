@@ -9,7 +9,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
-EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_predict", "isc_certify", "isc_certify_batch",
+EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_plan_resident", "isc_predict", "isc_certify", "isc_certify_batch",
            "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_noise_table", "isc_radius_integer", "isc_certified_metrics",
            "isc_debug_tensor", "isc_set_option", "isc_get_info", "isc_strerror"]
 
@@ -41,6 +41,7 @@ def lib():
         L = C.CDLL(_LIB_PATH)
         vp, i32p, f64p = C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_double)
         L.isc_load_qmodel.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(vp)]
+        L.isc_plan_resident.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i32p, C.POINTER(C.c_int64)]
         L.isc_free_qmodel.argtypes = [vp]
         L.isc_free_qmodel.restype = None
         L.isc_predict.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int64, C.c_double, C.c_double, vp,
@@ -104,6 +105,18 @@ def layer_array(layers):
                 keep.append(a)
                 setattr(s, k, a.ctypes.data)
     return arr, keep
+
+
+def plan_resident(model: dict):
+    """(fits, rule, smem_bytes): isc_plan_resident on a model dict; host only."""
+    arr, keep = layer_array(model["layers"])
+    rule, smem = C.c_int32(), C.c_int64()
+    rc = lib().isc_plan_resident(C.cast(arr, C.c_void_p), len(model["layers"]), *[int(v) for v in model["in_shape"]],
+                                 int(model["n_classes"]), C.byref(rule), C.byref(smem))
+    del keep
+    if rc < 0:
+        raise IscError(rc, "isc_plan_resident")
+    return rc, rule.value, smem.value
 
 
 class Model:

@@ -498,6 +498,35 @@ int isc_load_qmodel(const isc_layer *layers, int n_layers, int in_c, int in_h, i
     return ISC_OK;
 }
 
+int isc_plan_resident(const isc_layer *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes,
+                      int32_t *out_rule, int64_t *out_smem_bytes)
+{
+    if (!layers || n_layers < 1 || n_layers > 4096) return ISC_ERR_ARG;
+    if (in_c < 1 || in_h < 1 || in_w < 1 || n_classes < 1 || n_classes > 4096) return ISC_ERR_ARG;
+    if ((int64_t)in_c * in_h * in_w > (1ll << 30)) return ISC_ERR_ARG;
+    try {
+        isc_model m;
+        m.in_c = in_c; m.in_h = in_h; m.in_w = in_w; m.n_classes = n_classes;
+        int rc = build_host_model(&m, layers, n_layers);
+        if (rc) return rc;
+        std::vector<isc::LayerIn> ml(m.layers.size());
+        for (size_t i = 0; i < m.layers.size(); ++i) {
+            const HostLayer &H = m.layers[i];
+            ml[i].d = H.d;
+            ml[i].w = H.w.data(); ml[i].bias = H.bias.data();
+            ml[i].mult = H.mult.data(); ml[i].shift = H.shift.data();
+        }
+        int rule = 0;
+        uint32_t smem = 0;
+        const int fits = isc::line_plan_probe(ml.data(), (int)ml.size(), in_c, in_h, in_w, n_classes, &rule, &smem);
+        if (out_rule) *out_rule = rule;
+        if (out_smem_bytes) *out_smem_bytes = smem;
+        return fits;
+    } catch (const std::bad_alloc &) {
+        return ISC_ERR_NOMEM;
+    }
+}
+
 void isc_free_qmodel(isc_model *m)
 {
     if (!m) return;

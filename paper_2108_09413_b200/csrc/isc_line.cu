@@ -76,7 +76,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
 enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
 enum { ERR_NONE = 0, ERR_WAIT_DONE = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_READY = 3, ERR_WAIT_FULL = 4, ERR_WAIT_DRAIN = 5 };
-enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8 };
+enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8, CF_GENERAL = 16 };     // CF_GENERAL: the pass that decides everything at run time
 enum { OPF_WAIT_ALL = 1, OPF_NULL = 4 };
 
 // ---- what the kernel reads -------------------------------------------------------------------
@@ -426,14 +426,12 @@ struct EpiCtx {
 // thread (its position within a line, its 32 lanes of tensor memory), so that a pass only adds the offsets of its
 // table record.  The geometry that only strided convolutions need stays in the blob's header.
 struct EpiConv {
-    uint32_t flags, desc;
     uint32_t tmem0;                       // tensor-memory address of this warp's lanes, first column of the bank
     uint32_t full_addr, done_addr, parity;
     uint32_t const_addr;
     uint32_t out_thread, res_thread;      // line 0, this thread's position, plane 0 of the output / residual
     uint32_t dup_delta;                   // bytes from a band's first row to its copy below the band above; 0: one band
     uint32_t dup_up, dup_dn;              // this thread's band has a band above / below
-    int32_t lo;
     uint32_t res_m2;
     long long res_r2;
 };
@@ -443,24 +441,110 @@ struct alignas(16) LPass {
     uint32_t meta;          // unit | lines << 8 | chunk << 12 | line 0 first / last row of its band << 16, 17 | line 1 << 18, 19
     uint32_t lines;         // line 0 | line 1 << 8
     uint32_t tcol[2];       // accumulator columns of the two lines' chunk within the bank
-    uint32_t lp[2];         // byte offset of the two lines within a plane
-    uint32_t ch_out, ch_res;        // byte offset of the chunk's plane in the output / residual
+    uint32_t out[2];        // byte offset of the two lines' chunk (line within its plane + plane) in the output
+    uint32_t res[2];        // the same in the residual operand
 };
 static_assert(sizeof(LPass) == 32, "one pass is two 16-byte loads");
-
 
 // Per-channel requantisation constants as stored in the blob: the 64-bit addend, then multiplier and shift.
 //   y = floor((acc * mult + B) / 2^(32 + s)); B holds the folded bias, the rounding half and the output
 //   zero-point, so this is rs(acc' * mult, 31 + shift) + zp_out exactly.
 //   residual: y += floor((u * m2 + R2) / 2^32) with u = r + 128 the residual byte as an unsigned number,
 //   m2 = res_mult * 2^(32-n) and R2 the rounding half and the zero-points folded: rs((r - zp_res) * res_mult, n).
-template <bool kRes, bool kLo, int K>
-__device__ __forceinline__ int requant1(int acc, const ChanConst &cs, uint32_t rword, const EpiConv &E)
+template <bool kRes, int K>
+__device__ __forceinline__ int requant1(int acc, const ChanConst &cs, uint32_t rword, uint32_t res_m2, long long res_r2)
 {
     int y = hi32(mad_wide(acc, cs.mult, cs.B)) >> cs.s;
-    if (kRes) y += hi32(mad_wide_u(ubyte<K>(rword), E.res_m2, E.res_r2));
-    if (kLo) y = max(y, E.lo);
+    if (kRes) y += hi32(mad_wide_u(ubyte<K>(rword), res_m2, res_r2));
     return y;
+}
+
+__device__ __forceinline__ void st_shared_v4_if(uint32_t addr, uint4 v, uint32_t flag)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t@p st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n\t}"
+                 ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(flag) : "memory");
+}
+
+// The wait of a pass for its unit's accumulators.  The first attempt parks the thread in hardware for a bounded
+// time and nearly always succeeds; the timed loop is kept out of line so that the pass body stays small.
+__device__ __noinline__ bool wait_full_slow(Waiter w, uint32_t bar, uint32_t parity) { return w.barrier(bar, parity, ERR_WAIT_FULL); }
+
+__device__ __forceinline__ bool wait_full(Waiter w, uint32_t bar, uint32_t parity)
+{
+    bool ok = mbar_try(bar, parity);
+    if (!ok) ok = wait_full_slow(w, bar, parity);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// After a pass: the stores become visible to the tensor cores' reads, the tensor-memory accesses are ordered
+// before the arrival, and the warp counts one stored chunk of the unit.
+__device__ __forceinline__ void pass_done(const EpiConv &E, const EpiCtx &c, uint32_t unit)
+{
+    tc_fence_before();
+    fence_proxy_async();
+    __syncwarp();
+    if (c.lane == 0) red_release_add(E.done_addr + 4u * unit, 1u);
+}
+
+// The common pass: two output lines, one 16-channel chunk, results stored where the next convolution reads them.
+// The accumulator columns are left at zero: stacked chains accumulate from their first K-step on.
+template <bool kRes>
+__device__ __forceinline__ void epi_pass2(const EpiConv &E, const EpiCtx &c, uint4 q0, uint4 q1)
+{
+    const uint32_t ch = (q0.x >> 12) & 0xFu;
+    tc_fence_after();
+    int acc0[16], acc1[16];
+    tmem_ld16_issue(E.tmem0 + q0.z, acc0);
+    tmem_ld16_issue(E.tmem0 + q0.w, acc1);
+    uint32_t r0[4] = {0, 0, 0, 0}, r1[4] = {0, 0, 0, 0};
+    if (kRes) {
+        const uint4 a = ld_shared_v4(E.res_thread + q1.z), b = ld_shared_v4(E.res_thread + q1.w);
+        r0[0] = a.x ^ 0x80808080u; r0[1] = a.y ^ 0x80808080u; r0[2] = a.z ^ 0x80808080u; r0[3] = a.w ^ 0x80808080u;
+        r1[0] = b.x ^ 0x80808080u; r1[1] = b.y ^ 0x80808080u; r1[2] = b.z ^ 0x80808080u; r1[3] = b.w ^ 0x80808080u;
+    }
+    tmem_ld_wait();
+    tmem_st16_zero(E.tmem0 + q0.z);
+    tmem_st16_zero(E.tmem0 + q0.w);
+    const uint32_t cbase = E.const_addr + ch * 256u;
+    const uint32_t m2 = E.res_m2;
+    const long long r2 = E.res_r2;
+    uint32_t o0[4], o1[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const ChanConst c0 = ld_chan_const_early(cbase + (4 * g + 0) * 16), c1 = ld_chan_const_early(cbase + (4 * g + 1) * 16);
+        const ChanConst c2 = ld_chan_const_early(cbase + (4 * g + 2) * 16), c3 = ld_chan_const_early(cbase + (4 * g + 3) * 16);
+        o0[g] = pack4_sat(requant1<kRes, 0>(acc0[4 * g + 0], c0, r0[g], m2, r2), requant1<kRes, 1>(acc0[4 * g + 1], c1, r0[g], m2, r2),
+                          requant1<kRes, 2>(acc0[4 * g + 2], c2, r0[g], m2, r2), requant1<kRes, 3>(acc0[4 * g + 3], c3, r0[g], m2, r2));
+        o1[g] = pack4_sat(requant1<kRes, 0>(acc1[4 * g + 0], c0, r1[g], m2, r2), requant1<kRes, 1>(acc1[4 * g + 1], c1, r1[g], m2, r2),
+                          requant1<kRes, 2>(acc1[4 * g + 2], c2, r1[g], m2, r2), requant1<kRes, 3>(acc1[4 * g + 3], c3, r1[g], m2, r2));
+    }
+    const uint4 v0 = make_uint4(o0[0], o0[1], o0[2], o0[3]), v1 = make_uint4(o1[0], o1[1], o1[2], o1[3]);
+    const uint32_t a0 = E.out_thread + q1.x, a1 = E.out_thread + q1.y;
+    st_shared_v4(a0, v0);
+    st_shared_v4(a1, v1);
+    if (E.dup_delta) {
+        // first row of a lower band: also the row below the band above it; last row of an upper band: the row above
+        // the next band
+        st_shared_v4_if(a0 + E.dup_delta, v0, (q0.x >> 16) & E.dup_up);
+        st_shared_v4_if(a0 - E.dup_delta, v0, (q0.x >> 17) & E.dup_dn);
+        st_shared_v4_if(a1 + E.dup_delta, v1, (q0.x >> 18) & E.dup_up);
+        st_shared_v4_if(a1 - E.dup_delta, v1, (q0.x >> 19) & E.dup_dn);
+    }
+    tmem_st_wait();
+    pass_done(E, c, q0.x & 0xFFu);
+}
+
+template <bool kRes>
+__device__ __forceinline__ void epi_conv_fast(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes)
+{
+    const EpiConv E = E_in;
+    const EpiCtx c = c_in;
+#pragma unroll 1
+    for (uint32_t i = (uint32_t)c.set; i < n_passes; i += kSets) {
+        const uint4 q0 = ld_shared_v4(passes + 32u * i), q1 = ld_shared_v4(passes + 32u * i + 16u);
+        if (!wait_full(w, E.full_addr + 8u * (q0.x & 0xFFu), E.parity)) return;     // aborted: every other wait falls through too
+        epi_pass2<kRes>(E, c, q0, q1);
+    }
 }
 
 // Stride 2: stores one position's 16 channels of a plane where the output's layout wants them (`line` is the ordinal
@@ -484,82 +568,52 @@ __device__ __noinline__ void store_strided(uint32_t desc, uint32_t sbase, uint32
     if (oline == h6.w - 1u && band + 1u < h7.y) st_shared_v4(addr - (h6.w * h6.z - 4u) * 16u, o);
 }
 
-// One pass: SUP output lines, one 16-channel chunk.
-template <bool kRes, bool kLo, int SUP>
-__device__ __forceinline__ void epi_pass(Waiter w, const EpiConv &E, const EpiCtx &c, uint4 q0, uint4 q1, bool &ok, uint32_t cg)
+// The general pass (strided convolutions, a lower clamp above -128, a lone line): one line at a time, every
+// property decided at run time.  The networks of the benchmark reach it in their two strided shortcuts only.
+__device__ __noinline__ void epi_conv_general(Waiter w, const EpiConv &E, const EpiCtx &c, uint32_t desc, uint32_t flags, int32_t lo,
+                                              uint32_t passes, uint32_t n_passes)
 {
-    const uint32_t unit = q0.x & 0xFFu, ch = (q0.x >> 12) & 0xFu;
-    const uint32_t tcol[2] = {q0.z, q0.w}, lp[2] = {q1.x, q1.y};
-    if (ok) ok = w.barrier(E.full_addr + 8u * unit, E.parity, ERR_WAIT_FULL);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-    int acc[SUP][16];
+    const bool res = flags & CF_RES, scatter = flags & CF_SCATTER;
+    for (uint32_t i = (uint32_t)c.set; i < n_passes; i += kSets) {
+        const uint4 q0 = ld_shared_v4(passes + 32u * i), q1 = ld_shared_v4(passes + 32u * i + 16u);
+        const uint32_t unit = q0.x & 0xFFu, ch = (q0.x >> 12) & 0xFu, n = (q0.x >> 8) & 0xFu;
+        if (!wait_full(w, E.full_addr + 8u * unit, E.parity)) return;
+        tc_fence_after();
+        for (uint32_t j = 0; j < n; ++j) {
+            const uint32_t tcol = j ? q0.w : q0.z, out = j ? q1.y : q1.x, rs = j ? q1.w : q1.z;
+            int acc[16];
+            tmem_ld16(E.tmem0 + tcol, acc);
+            tmem_st16_zero(E.tmem0 + tcol);
+            uint4 rv = make_uint4(0, 0, 0, 0);
+            if (res) rv = ld_shared_v4(E.res_thread + rs);
+            const uint32_t rw[4] = {rv.x ^ 0x80808080u, rv.y ^ 0x80808080u, rv.z ^ 0x80808080u, rv.w ^ 0x80808080u};
+            uint32_t o[4];
 #pragma unroll
-    for (int j = 0; j < SUP; ++j) tmem_ld16_issue(E.tmem0 + tcol[j], acc[j]);
-    uint32_t rw[SUP][4];
+            for (int g = 0; g < 4; ++g) {
+                int y[4];
 #pragma unroll
-    for (int j = 0; j < SUP; ++j) {
-        uint4 rv = make_uint4(0, 0, 0, 0);
-        if (kRes) rv = ld_shared_v4(E.res_thread + lp[j] + q1.w);
-        rw[j][0] = rv.x ^ 0x80808080u; rw[j][1] = rv.y ^ 0x80808080u; rw[j][2] = rv.z ^ 0x80808080u; rw[j][3] = rv.w ^ 0x80808080u;
-    }
-    tmem_ld_wait();
-    // every accumulator column is left at zero: stacked chains accumulate from their first K-step on
-#pragma unroll
-    for (int j = 0; j < SUP; ++j) tmem_st16_zero(E.tmem0 + tcol[j]);
-    if (ok) {
-        const uint32_t cbase = E.const_addr + ch * 256u;
-        uint32_t out[SUP][4];
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const ChanConst c0 = ld_chan_const_early(cbase + (4 * g + 0) * 16), c1 = ld_chan_const_early(cbase + (4 * g + 1) * 16);
-            const ChanConst c2 = ld_chan_const_early(cbase + (4 * g + 2) * 16), c3 = ld_chan_const_early(cbase + (4 * g + 3) * 16);
-#pragma unroll
-            for (int j = 0; j < SUP; ++j) {
-                const int y0 = requant1<kRes, kLo, 0>(acc[j][4 * g + 0], c0, rw[j][g], E);
-                const int y1 = requant1<kRes, kLo, 1>(acc[j][4 * g + 1], c1, rw[j][g], E);
-                const int y2 = requant1<kRes, kLo, 2>(acc[j][4 * g + 2], c2, rw[j][g], E);
-                const int y3 = requant1<kRes, kLo, 3>(acc[j][4 * g + 3], c3, rw[j][g], E);
-                out[j][g] = pack4_sat(y0, y1, y2, y3);
+                for (int k = 0; k < 4; ++k) {
+                    const ChanConst cs = ld_chan_const_early(E.const_addr + ch * 256u + (4 * g + k) * 16);
+                    int v = hi32(mad_wide(acc[4 * g + k], cs.mult, cs.B)) >> cs.s;
+                    if (res) v += hi32(mad_wide_u((rw[g] >> (8 * k)) & 0xFFu, E.res_m2, E.res_r2));
+                    y[k] = max(v, lo);
+                }
+                o[g] = pack4_sat(y[0], y[1], y[2], y[3]);
             }
-        }
-#pragma unroll
-        for (int j = 0; j < SUP; ++j) {
-            const uint4 o = make_uint4(out[j][0], out[j][1], out[j][2], out[j][3]);
-            if (E.flags & CF_SCATTER) {
-                store_strided(E.desc, c.sbase, c.lane_idx, ch, (q0.y >> (8 * j)) & 0xFFu, o);
+            const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
+            if (scatter) {
+                store_strided(desc, c.sbase, c.lane_idx, ch, (q0.y >> (8 * j)) & 0xFFu, v);
             } else {
-                const uint32_t addr = E.out_thread + lp[j] + q1.z;
-                st_shared_v4(addr, o);
+                const uint32_t addr = E.out_thread + out;
+                st_shared_v4(addr, v);
                 if (E.dup_delta) {
-                    // first row of a lower band: also the row below the band above it; last row of an upper band: the
-                    // row above the next band
-                    if (((q0.x >> (16 + 2 * j)) & 1u) & E.dup_up) st_shared_v4(addr + E.dup_delta, o);
-                    if (((q0.x >> (17 + 2 * j)) & 1u) & E.dup_dn) st_shared_v4(addr - E.dup_delta, o);
+                    if (((q0.x >> (16 + 2 * j)) & 1u) & E.dup_up) st_shared_v4(addr + E.dup_delta, v);
+                    if (((q0.x >> (17 + 2 * j)) & 1u) & E.dup_dn) st_shared_v4(addr - E.dup_delta, v);
                 }
             }
         }
-    }
-    tmem_st_wait();
-    // the stores become visible to the tensor cores' reads, the tensor-memory accesses are ordered before the arrival
-    tc_fence_before();
-    fence_proxy_async();
-    __syncwarp();
-    if (c.lane == 0) red_release_add(E.done_addr + 4u * unit, 1u);
-}
-
-template <bool kRes, bool kLo>
-__device__ __forceinline__ void epi_conv_passes(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes,
-                                             uint32_t cg)
-{
-    const EpiConv E = E_in;
-    const EpiCtx c = c_in;
-    bool ok = true;
-#pragma unroll 1
-    for (uint32_t i = (uint32_t)c.set; i < n_passes; i += kSets) {
-        const uint4 q0 = ld_shared_v4(passes + 32u * i), q1 = ld_shared_v4(passes + 32u * i + 16u);
-        if (((q0.x >> 8) & 0xFu) == 2u) epi_pass<kRes, kLo, 2>(w, E, c, q0, q1, ok, cg);
-        else epi_pass<kRes, kLo, 1>(w, E, c, q0, q1, ok, cg);
+        tmem_st_wait();
+        pass_done(E, c, unit);
     }
 }
 
@@ -572,7 +626,6 @@ __device__ __forceinline__ void epi_conv(const LineParams &p, const EpiCtx &c, u
     const uint32_t desc = c.sbase + blob_off;
     const uint4 h0 = ld_shared_v4(desc);
     const uint4 h1 = ld_shared_v4(desc + offsetof(LConvDesc, a_base));
-    const uint4 h2 = ld_shared_v4(desc + offsetof(LConvDesc, idesc));
     const uint4 h3 = ld_shared_v4(desc + offsetof(LConvDesc, d_base));
     const uint4 h4 = ld_shared_v4(desc + offsetof(LConvDesc, use_local));
     const uint4 h5 = ld_shared_v4(desc + offsetof(LConvDesc, w_rel));
@@ -581,8 +634,6 @@ __device__ __forceinline__ void epi_conv(const LineParams &p, const EpiCtx &c, u
     const uint4 h9 = ld_shared_v4(desc + offsetof(LConvDesc, lo));             // lo, res_m2, res_r2
     const uint32_t use = (uint32_t)it * h4.y + h4.x;
     EpiConv E;
-    E.flags = h0.w;
-    E.desc = desc;
     E.tmem0 = c.tmem_lane + ((h1.w > 1 && (use & 1u)) ? h3.y : h3.x);
     E.full_addr = smem_u32(&c.ctrl->bars[h3.z + (use & 1u) * h4.z]);
     E.done_addr = smem_u32(&c.ctrl->stored[h3.w]);
@@ -594,15 +645,16 @@ __device__ __forceinline__ void epi_conv(const LineParams &p, const EpiCtx &c, u
     E.dup_delta = h7.y > 1u ? (h6.w * h6.z - 4u) * 16u : 0u;
     E.dup_up = band >= 1u ? 1u : 0u;
     E.dup_dn = band + 1u < h7.y ? 1u : 0u;
-    E.lo = (int32_t)h9.x; E.res_m2 = h9.y;
+    E.res_m2 = h9.y;
     E.res_r2 = (long long)(((unsigned long long)h9.w << 32) | h9.z);
     const uint32_t passes = desc + h5.w, n_passes = h0.y;
-    switch (E.flags & (CF_RES | CF_LO)) {
-    case 0: epi_conv_passes<false, false>(w, E, c, passes, n_passes, cg); break;
-    case CF_RES: epi_conv_passes<true, false>(w, E, c, passes, n_passes, cg); break;
-    case CF_LO: epi_conv_passes<false, true>(w, E, c, passes, n_passes, cg); break;
-    default: epi_conv_passes<true, true>(w, E, c, passes, n_passes, cg); break;
+    const uint32_t flags = h0.w;
+    if (flags & CF_GENERAL) {
+        epi_conv_general(w, E, c, desc, flags, (int32_t)h9.x, passes, n_passes);
+        return;
     }
+    if (flags & CF_RES) epi_conv_fast<true>(w, E, c, passes, n_passes);
+    else epi_conv_fast<false>(w, E, c, passes, n_passes);
 }
 
 // FILL: the region takes its halo value everywhere
@@ -885,8 +937,10 @@ bool place(std::vector<AllocReq> &done, AllocReq &r, uint32_t capacity)
     return true;
 }
 
-// A plan that does not fit is not an error (another engine runs the model); ISC_PLAN_DEBUG=1 says which rule failed.
-#define PLAN_FAIL(id) do { if (getenv("ISC_PLAN_DEBUG")) fprintf(stderr, "line engine: plan rule %d failed\n", id); return false; } while (0)
+// A plan that does not fit is not an error (another engine runs the model); the rule that refused it is kept for
+// line_plan_probe, and ISC_PLAN_DEBUG=1 prints it.
+thread_local int g_plan_rule = 0;
+#define PLAN_FAIL(id) do { g_plan_rule = (id); if (getenv("ISC_PLAN_DEBUG")) fprintf(stderr, "line engine: plan rule %d failed\n", id); return false; } while (0)
 
 bool conv_ok(const isc_layer &L, bool first)
 {
@@ -1256,15 +1310,14 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
                     const int line = order[(size_t)u * sup + q];
                     P.lines |= (uint32_t)line << (8 * q);
                     P.tcol[q] = (uint32_t)(line * cp.cols + ch * 16);
-                    P.lp[q] = (uint32_t)(line * out.pitch) * 16u;
+                    P.out[q] = (uint32_t)(line * out.pitch) * 16u + (uint32_t)ch * out.plane_bytes;
+                    P.res[q] = L.res_tensor >= 0 ? (uint32_t)(line * out.pitch) * 16u + (uint32_t)ch * T[(size_t)L.res_tensor].plane_bytes : 0u;
                     if (!cp.scatter) {
                         if (line == 0) P.meta |= 1u << (16 + 2 * q);
                         if (line == out.n_lines - 1) P.meta |= 1u << (17 + 2 * q);
                     }
                     cp.done_time[(size_t)line] = (int)cp.passes.size() / kSets;
                 }
-                P.ch_out = (uint32_t)ch * out.plane_bytes;
-                P.ch_res = L.res_tensor >= 0 ? (uint32_t)ch * T[(size_t)L.res_tensor].plane_bytes : 0u;
                 cp.passes.push_back(P);
             }
         convs.push_back(cp);
@@ -1360,6 +1413,8 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
         const int lo = L.relu ? std::max(-128, L.zp_out) : -128;
         if (lo > -128) D.flags |= CF_LO;
         D.lo = lo;
+        // the fast pass covers pairs of lines stored in place with the saturating pack as the only clamp
+        if (lo > -128 || cp.scatter || (cp.m & 1)) D.flags |= CF_GENERAL;
         // operand base: line -1, lane 0, plane 0 of the input
         D.a_base = plan->tensor_off[(size_t)cp.in_tensor] + in.line0 - (uint32_t)in.pitch * 16u;
         D.pitch16 = (uint32_t)in.pitch;
@@ -1470,25 +1525,54 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
 
 }  // namespace
 
+namespace {
+
+// The structure the engine is built for: convolutions, then global average pool, then FC.
+bool structure_ok(const LayerIn *layers, int n_layers, int n_classes)
+{
+    if (n_layers < 3 || n_classes > 128) PLAN_FAIL(101);
+    const isc_layer &LP = layers[n_layers - 2].d, &LF = layers[n_layers - 1].d;
+    if (LP.op != ISC_GAVGPOOL || LF.op != ISC_FC) PLAN_FAIL(102);
+    if (LP.in_tensor != n_layers - 2 || LF.in_tensor != n_layers - 1) PLAN_FAIL(103);
+    if (LP.cin > 64 || LP.cin % 16 != 0 || LF.res_tensor >= 0) PLAN_FAIL(104);
+    for (int i = 0; i < n_layers - 2; ++i) {
+        const isc_layer &L = layers[i].d;
+        if (!conv_ok(L, i == 0)) PLAN_FAIL(105);
+        if ((i == 0) != (L.in_tensor == 0)) PLAN_FAIL(106);
+        if (L.res_tensor == 0) PLAN_FAIL(107);
+        // a consumer's zero-point must be the halo value its operand was written with
+        if (L.in_tensor > 0 && L.zp_in != layers[L.in_tensor - 1].d.zp_out) PLAN_FAIL(108);
+        if (L.in_tensor > i || L.res_tensor > i) PLAN_FAIL(109);
+    }
+    if (LP.zp_in != layers[n_layers - 3].d.zp_out) PLAN_FAIL(110);
+    return true;
+}
+
+}  // namespace
+
+int line_plan_probe(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, int *rule, uint32_t *smem_bytes)
+{
+    g_plan_rule = 0;
+    *smem_bytes = 0;
+    bool ok = structure_ok(layers, n_layers, n_classes);
+    if (ok) {
+        LinePlan plan;
+        std::vector<uint8_t> blob, bar_counts;
+        std::vector<uint32_t> blob_off;
+        std::vector<PhaseEntry> ptab;
+        std::vector<ConvSrc> csrc;
+        ok = build_plan(layers, n_layers, in_c, in_h, in_w, n_classes, &plan, &blob, &blob_off, &ptab, &csrc, &bar_counts);
+        if (ok) *smem_bytes = plan.smem_bytes;
+    }
+    *rule = ok ? 0 : g_plan_rule;
+    return ok ? 1 : 0;
+}
+
 int line_build(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, LinePlan **out)
 {
     *out = nullptr;
-    if (n_layers < 3 || n_classes > 128) return ISC_OK;
-    // structure: convolutions, then global average pool, then FC
+    if (!structure_ok(layers, n_layers, n_classes)) return ISC_OK;
     const isc_layer &LP = layers[n_layers - 2].d, &LF = layers[n_layers - 1].d;
-    if (LP.op != ISC_GAVGPOOL || LF.op != ISC_FC) return ISC_OK;
-    if (LP.in_tensor != n_layers - 2 || LF.in_tensor != n_layers - 1) return ISC_OK;
-    if (LP.cin > 64 || LP.cin % 16 != 0 || LF.res_tensor >= 0) return ISC_OK;
-    for (int i = 0; i < n_layers - 2; ++i) {
-        const isc_layer &L = layers[i].d;
-        if (!conv_ok(L, i == 0)) return ISC_OK;
-        if ((i == 0) != (L.in_tensor == 0)) return ISC_OK;
-        if (L.res_tensor == 0) return ISC_OK;
-        // a consumer's zero-point must be the halo value its operand was written with
-        if (L.in_tensor > 0 && L.zp_in != layers[L.in_tensor - 1].d.zp_out) return ISC_OK;
-        if (L.in_tensor > i || L.res_tensor > i) return ISC_OK;
-    }
-    if (LP.zp_in != layers[n_layers - 3].d.zp_out) return ISC_OK;
 
     LinePlan *plan = new LinePlan();
     std::vector<uint8_t> blob, bar_counts;

@@ -16,6 +16,11 @@ int line_build(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w
                LinePlan **out);
 void line_free(LinePlan *p);
 
+// Host only: 1 if the planner accepts the network (then *smem_bytes = shared memory per CTA), else 0 and *rule =
+// the number of the rule that refused it.
+int line_plan_probe(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w, int n_classes, int *rule,
+                    uint32_t *smem_bytes);
+
 // Runs samples first..first+n-1 (ns.first_sample = first) and adds their votes to d_counts.
 int line_run(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, int64_t n, int batch_hint,
              int32_t *d_counts, int8_t *d_logits, cudaStream_t st, int64_t *launches);

@@ -145,7 +145,9 @@ def _conv(rng, in_tensor, cin, cout, k, stride, relu, zp_in, zp_out, res_tensor=
 
 def random_cifar_net(seed):
     """32x32 input, three stages of basic blocks with stride-2 transitions and projection shortcuts, global average
-    pool, FC -- with every parameter drawn from the whole range the line-tiled engine accepts."""
+    pool, FC -- with every parameter drawn from the whole range the line-tiled engine accepts.  The tensors that carry
+    a stage's residual stream share one zero-point (the engine adds the residual in place, padding included, and keeps
+    three 72 KB stage-1 tensors in shared memory only that way); everything else is drawn freely."""
     rng = np.random.default_rng(seed)
     in_c = int(rng.integers(1, 5))
     widths = (16, 32, 64) if seed % 3 else (16, int(rng.choice([16, 32])), int(rng.choice([16, 32, 64])))
@@ -153,8 +155,9 @@ def random_cifar_net(seed):
     narrow = seed % 2 == 0                 # half of the networks keep mid-range shifts so that deep layers stay lively
     sl, sh = (7, 12) if narrow else (1, 20)
     zp = lambda: int(rng.integers(-128, 128))
+    trunk = [zp(), zp(), zp()]
     zps = {0: int(rng.integers(0, 256))}
-    L = [_conv(rng, 0, in_c, widths[0], int(rng.choice([1, 3])), 1, int(rng.integers(0, 2)), zps[0], zp(), shift_lo=sl, shift_hi=sh)]
+    L = [_conv(rng, 0, in_c, widths[0], int(rng.choice([1, 3])), 1, int(rng.integers(0, 2)), zps[0], trunk[0], shift_lo=sl, shift_hi=sh)]
     zps[1] = L[0]["zp_out"]
     cur, cin = 1, widths[0]
     for si, width in enumerate(widths):
@@ -163,12 +166,12 @@ def random_cifar_net(seed):
             L.append(_conv(rng, cur, cin, width, 3, stride, int(rng.integers(0, 2)), zps[cur], zp(), shift_lo=sl, shift_hi=sh))
             y1 = len(L); zps[y1] = L[-1]["zp_out"]
             if stride != 1 or cin != width:
-                L.append(_conv(rng, cur, cin, width, 1, stride, int(rng.integers(0, 2)), zps[cur], zp(), shift_lo=sl, shift_hi=sh))
+                L.append(_conv(rng, cur, cin, width, 1, stride, int(rng.integers(0, 2)), zps[cur], trunk[si], shift_lo=sl, shift_hi=sh))
                 short = len(L); zps[short] = L[-1]["zp_out"]
             else:
                 short = cur
             zp_res = zps[short] if rng.integers(0, 2) else zp()
-            L.append(_conv(rng, y1, width, width, int(rng.choice([3, 3, 1])), 1, int(rng.integers(0, 2)), zps[y1], zp(),
+            L.append(_conv(rng, y1, width, width, int(rng.choice([3, 3, 1])), 1, int(rng.integers(0, 2)), zps[y1], trunk[si],
                            res_tensor=short, zp_res=zp_res, shift_lo=sl, shift_hi=sh))
             cur, cin = len(L), width
             zps[cur] = L[-1]["zp_out"]

@@ -138,3 +138,24 @@ def test_certified_metrics_equal_oracle():
     assert isc.certified_metrics([-1, -1], [0.0, 0.0], [1, 2], []) == (0.0, [])
     cp = C.c_double(9.0)
     assert isc.lib().isc_certified_metrics(None, None, None, 3, None, 0, C.byref(cp), None) == -1 and cp.value == 9.0
+
+
+def test_plan_resident_accepts_cifar_resnets_and_names_the_refusing_rule():
+    """Host-only planner query: the CIFAR-shaped networks fit the shared-memory-resident engine (227 KB per CTA at
+    most), the 224x224 bottleneck network does not."""
+    import workloads as wl
+    for model in (wl.tiny_cnn(), wl.resnet20(), wl.resnet110(), wl.spread_model("resnet20")):
+        fits, rule, smem = isc.plan_resident(model)
+        assert (fits, rule) == (1, 0) and 0 < smem <= 227 * 1024, model["name"]
+    fits, rule, smem = isc.plan_resident(wl.resnet50())
+    assert fits == 0 and rule > 0 and smem == 0
+    # a consumer whose zero-point differs from its producer's output zero-point reads wrong padding: refused
+    model = wl.resnet20()
+    model["layers"][1] = dict(model["layers"][1], zp_in=-100)
+    fits, rule, _ = isc.plan_resident(model)
+    assert fits == 0 and rule == 108
+    # a layer list that does not type-check is an error, not a refusal
+    model = wl.resnet20()
+    model["layers"][1] = dict(model["layers"][1], cin=8)
+    with pytest.raises(isc.IscError):
+        isc.plan_resident(model)
