@@ -8,6 +8,10 @@ device memory; `e2e` is the same call given host buffers (host->device copy of t
 device->host read of the vote counts inside the timed region).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+`--config 4` runs the throughput sweep (launch batch x sigma on the ResNet-110 model): one JSON
+line per cell, then the summary line.  `--samples N` replaces the workload's N by a smaller
+number (a short case for profilers; the line says so and is not a benchmark result).
 """
 from __future__ import annotations
 
@@ -79,11 +83,16 @@ class ClockSampler:
                     reasons=reasons, samples=len(self.samples))
 
 
-def workload(cfg_id):
+def workload(cfg_id, sigma=None):
     cfg = wl.CONFIGS[cfg_id]
     model = cfg["model"]()
-    sigma = 0.25 if 0.25 in cfg["sigmas"] else cfg["sigmas"][0]
+    if sigma is None:
+        sigma = 0.25 if 0.25 in cfg["sigmas"] else cfg["sigmas"][0]
     return cfg, model, sigma
+
+
+def workload_name(cfg_id, model):
+    return f"config {cfg_id}: {model['name']} CERTIFY"
 
 
 def oracle_rate(model, cfg, sigma, n_samples, x):
@@ -108,7 +117,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cfg, model, sigma = workload(args.config)
+    cfg, model, sigma = workload(args.config, args.sigma)
     x = wl.images(1, shape=cfg["shape"], seed=cfg["image_seed"])[0]
     import oracle
     om = oracle.Model(model)
@@ -126,7 +135,7 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": f"config {args.config}: {model['name']} CERTIFY", "sigma": sigma,
+        "config": {"workload": workload_name(args.config, model), "sigma": sigma,
                    "N0": cfg["N0"], "N": cfg["N"], "alpha": cfg["alpha"]},
         "cpu_baseline": {"value": value, "unit": "samples/s", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
@@ -142,8 +151,10 @@ def main():
     ap.add_argument("--config", type=int, default=2, choices=sorted(wl.CONFIGS))
     ap.add_argument("--images-per-step", type=int, default=0)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 layer-by-layer, 2 resident tensor-core (flat tiles), 3 resident tensor-core (line tiles)")
-    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 layer-by-layer, 3 resident tensor-core (line tiles)")
+    ap.add_argument("--batch", type=int, default=0, help="noisy samples per launch (0: the library chooses)")
+    ap.add_argument("--sigma", type=float, default=None, help="noise level (default: the workload's)")
+    ap.add_argument("--samples", type=int, default=0, help="replace the workload's N (short case for profilers)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -161,16 +172,52 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    cfg, model, sigma = workload(args.config)
+    cfg, model, sigma = workload(args.config, args.sigma)
     gm = isc.Model(model)
     gm.set_option("engine", args.engine)
-    gm.set_option("batch", args.batch)
-    N0, N, alpha = cfg["N0"], cfg["N"], cfg["alpha"]
+    ctx = dict(torch=torch, dist=dist, rank=rank, local_rank=local_rank, world=world, gm=gm, cfg=cfg, model=model)
+
+    if args.config == 4 and not args.samples:
+        # the sweep: launch batch x sigma, 20 images per cell (2 steps of 10), device-resident images
+        cells = []
+        for batch in cfg["batches"]:
+            for sg in cfg["sigmas"]:
+                r = measure(ctx, args, sg, batch, steps=2, warmup=1, ips=10, e2e_arm=False)
+                cell = {"cell": {"batch": batch, "sigma": sg}, "value": r["value"], "unit": r["unit"],
+                        "certified_images_per_sec": r["certified_images_per_sec"], "ms_per_step": r["ms_per_step"],
+                        "gpu_launches": r["gpu_launches"], "roofline_frac": r["roofline"]["frac"],
+                        "frac_of_nominal_int8": r["roofline"]["frac_of_nominal_int8"],
+                        "sampler_share": r.get("sampler_share"), "clocks": r["clocks"]}
+                cells.append(cell)
+                if rank == 0:
+                    print(json.dumps(cell), flush=True)
+        out = measure(ctx, args, sigma, args.batch, steps=args.steps, warmup=args.warmup, ips=args.images_per_step, e2e_arm=True)
+        out["sweep"] = cells
+    else:
+        out = measure(ctx, args, sigma, args.batch, steps=args.steps, warmup=args.warmup, ips=args.images_per_step, e2e_arm=True)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_or = oracle_sample_size(model)
+        probe = wl.images(1, shape=cfg["shape"], seed=cfg["image_seed"])
+        rate, cores, dt = oracle_rate(model, cfg, sigma, n_or, probe[0])
+        out["cpu_baseline"] = {"value": rate, "unit": "samples/s", "cores": cores, "kind": "oracle",
+                               "sample": f"{n_or} noisy samples of one image (estimation phase), {dt:.1f} s"}
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def measure(ctx, args, sigma, batch, steps, warmup, ips, e2e_arm):
+    """One measurement: `steps` timed steps of `ips` certified images each, after `warmup` untimed ones."""
+    torch, dist, rank, local_rank, world = ctx["torch"], ctx["dist"], ctx["rank"], ctx["local_rank"], ctx["world"]
+    gm, cfg, model = ctx["gm"], ctx["cfg"], ctx["model"]
+    gm.set_option("batch", batch)
+    N0, alpha = cfg["N0"], cfg["alpha"]
+    N = args.samples if args.samples else cfg["N"]
     macs = wl.macs_per_sample(model)
 
     # images per step: sized so that one step is about a second of GPU time
-    ips = args.images_per_step
-    total_steps = args.warmup + 2 * args.steps
+    total_steps = warmup + 2 * steps
     # every rank certifies its own images (weak scaling, no exchange)
     probe = wl.images(1, shape=cfg["shape"], seed=cfg["image_seed"])
     stream = torch.cuda.current_stream()
@@ -216,16 +263,24 @@ def main():
             total_ms += e0.elapsed_time(e1)
         return total_ms
 
-    for i in range(args.warmup):
+    def phase_cycles():
+        try:
+            return [gm.get_info(k) for k in ("cycles_fill", "cycles_noise", "cycles_conv", "cycles_tail")]
+        except Exception:
+            return None
+
+    for i in range(warmup):
         step(i, False)
     launches0 = gm.get_info("gpu_launches")
+    cyc0 = phase_cycles()
     barrier()
     with ClockSampler(local_rank) as clk:
-        ms = timed(args.warmup, args.steps, False)
+        ms = timed(warmup, steps, False)
         barrier()
     launches = gm.get_info("gpu_launches") - launches0
+    cyc1 = phase_cycles()
     barrier()
-    ms_e2e = timed(args.warmup + args.steps, args.steps, True)
+    ms_e2e = timed(warmup + steps, steps, True) if e2e_arm else ms
     barrier()
     if dist is not None:
         t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
@@ -233,23 +288,25 @@ def main():
         ms, ms_e2e = t.tolist()
 
     samples_per_step = ips * (N0 + N)
-    total_samples = samples_per_step * args.steps * world
+    total_samples = samples_per_step * steps * world
     value = total_samples / (ms * 1e-3)
     e2e = total_samples / (ms_e2e * 1e-3)
     peaks = load_peaks()
     int8_peak = 2.0 * peaks["bf16_sustained"]              # nominal int8 : bf16 ratio of the tensor cores is 2
-    achieved = 2.0 * macs * samples_per_step * args.steps / (ms * 1e-3) / 1e12   # per GPU
+    achieved = 2.0 * macs * samples_per_step * steps / (ms * 1e-3) / 1e12   # per GPU
     engine = gm.get_info("engine")
+    name = workload_name(args.config, model)
+    if args.samples:
+        name += f" (short case: N = {N} instead of {cfg['N']}; not a benchmark result)"
 
     out = {
         "metric": "noisy int8 samples/sec", "value": value, "unit": "samples/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "steps": steps, "warmup": warmup, "ms_per_step": ms / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
         "data": "synthetic",
-        "config": {"workload": f"config {args.config}: {model['name']} CERTIFY, {ips} images/step/GPU",
-                   "sigma": sigma, "N0": N0, "N": N, "alpha": alpha, "images_per_step": ips,
-                   "engine": {1: "layer-by-layer", 2: "resident tensor-core, flat tiles",
-                              3: "resident tensor-core, line tiles"}.get(engine, str(engine)),
+        "config": {"workload": name,
+                   "sigma": sigma, "N0": N0, "N": N, "alpha": alpha, "images_per_step": ips, "batch": batch,
+                   "engine": {1: "layer-by-layer", 3: "resident tensor-core, line tiles"}.get(engine, str(engine)),
                    "l2": "flushed between steps (256 MiB write)", "macs_per_sample": macs},
         "certified_images_per_sec": value / (N0 + N),
         "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(ips * np.prod(cfg["shape"])),
@@ -257,20 +314,19 @@ def main():
         "gpu_launches": int(launches),
         "clocks": clk.summary(),
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TFLOP/s",
-                     "frac": achieved / int8_peak, "traffic": None,
+                     "frac": achieved / int8_peak, "frac_of_nominal_int8": achieved / NOMINAL_INT8_TOPS, "traffic": None,
                      "peak_source": f"2 x {peaks['source']} sustained bf16 ({peaks['bf16_sustained']} TFLOP/s); "
                                     f"nominal dense int8 {NOMINAL_INT8_TOPS} TOP/s -> frac {achieved / NOMINAL_INT8_TOPS:.4f}",
                      "ops": "algorithmic: 2 x true MACs per noisy sample"},
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_or = oracle_sample_size(model)
-        rate, cores, dt = oracle_rate(model, cfg, sigma, n_or, probe[0])
-        out["cpu_baseline"] = {"value": rate, "unit": "samples/s", "cores": cores, "kind": "oracle",
-                               "sample": f"{n_or} noisy samples of one image (estimation phase), {dt:.1f} s"}
-    if rank == 0:
-        print(json.dumps(out))
-    if dist is not None:
-        dist.destroy_process_group()
+    if not e2e_arm:
+        del out["e2e"]
+    if cyc0 is not None and cyc1 is not None:
+        d = [b - a for a, b in zip(cyc0, cyc1)]
+        if sum(d) > 0:
+            out["sampler_share"] = d[1] / sum(d)
+            out["phase_shares"] = {"fill": d[0] / sum(d), "noise": d[1] / sum(d), "conv": d[2] / sum(d), "tail": d[3] / sum(d)}
+    return out
 
 
 if __name__ == "__main__":

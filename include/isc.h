@@ -255,8 +255,12 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
  *              tensor-core kernel (ISC_ERR_UNSUPPORTED at the next call if the model
  *              does not fit it).  2 is not an engine (ISC_ERR_ARG).
  * isc_get_info reads back: "engine" (the engine the last call used), "gpu_launches"
- * (kernel launches issued by this handle so far), "macs_per_sample" and
- * "has_line_engine" (1 if the model fits engine 3).
+ * (kernel launches issued by this handle so far), "macs_per_sample",
+ * "has_line_engine" (1 if the model fits engine 3) and, for engine 3, "cycles_fill",
+ * "cycles_noise", "cycles_conv", "cycles_tail": SM cycles summed over thread blocks and over
+ * all launches of this handle so far, spent in halo fills, in the noise phase (draw, add,
+ * saturate, store), in the convolutions and in pool / FC / argmax / vote -- the noise
+ * sampler's cost share is cycles_noise over their sum (these reads synchronise the device).
  */
 int isc_set_option(isc_model *m, const char *name, int64_t value);
 int isc_get_info(isc_model *m, const char *name, int64_t *out);

@@ -894,6 +894,16 @@ int isc_get_info(isc_model *m, const char *name, int64_t *out)
     else if (!strcmp(name, "gpu_launches")) *out = m->launches;
     else if (!strcmp(name, "macs_per_sample")) *out = m->macs;
     else if (!strcmp(name, "has_line_engine")) *out = m->line ? 1 : 0;
+    else if (!strncmp(name, "cycles_", 7)) {
+        static const char *const which[4] = {"cycles_fill", "cycles_noise", "cycles_conv", "cycles_tail"};
+        if (!m->line) return ISC_ERR_UNSUPPORTED;
+        unsigned long long c[4];
+        int rc = isc::line_phase_cycles(m->line, c);
+        if (rc) return rc;
+        for (int k = 0; k < 4; ++k)
+            if (!strcmp(name, which[k])) { *out = (int64_t)c[k]; return ISC_OK; }
+        return ISC_ERR_ARG;
+    }
     else return ISC_ERR_ARG;
     return ISC_OK;
 }

@@ -24,16 +24,17 @@
 // operand.  Strided and 1x1 convolutions, and those with cout = 64, run unstacked: one chain per output line
 // over all taps.
 //
-// Roles.  Four issuing warps (lane 0 of each) share the MMA chains of a convolution: the host prepares a table
-// of operations (accumulator columns, descriptor offsets, which units of the previous convolution must be stored,
+// Roles.  Three issuing warps (lane 0 of each) share the MMA chains of a convolution: the host prepares a table of
+// operations (accumulator columns, descriptor offsets, which units of the previous convolution must be stored,
 // which units complete) in the order in which their inputs become available; operation i belongs to issuing warp
-// i mod 4.  One thread alone cannot feed the tensor pipe: a chain costs it several hundred cycles of issue
-// latency.  Eight epilogue warps requantise: two sets of four warps (one per 32-lane quarter of tensor memory)
-// share the output lines of a convolution, two lines and one 16-channel chunk per pass, in the order in which
-// they complete; eight warps leave each thread 128 registers, which the unrolled requantisation needs (sixteen
-// warps at 80 registers spill and are slower).  A loader warp copies the next convolution's blob once its place is
-// free.  A unit (the lines of a pass) has two mbarriers "accumulators complete", used in turn by the convolutions
-// of a class, and a counter "stored"; consecutive convolutions overlap unit by unit.  Input noise (Def. 3.3,
+// i mod 3.  One thread alone cannot feed the tensor pipe: an MMA costs it about a hundred cycles of issue latency and
+// a commit as much again, so the loop is kept to the fewest instructions (dependency counters read together, the
+// timed wait out of line).  Sixteen epilogue warps requantise: four sets of four warps (one per 32-lane quarter of
+// tensor memory) share the items of a convolution, an item being one unit (two or four output lines: one
+// "accumulators complete" barrier pair, one "stored" counter) and one 16-channel chunk, in the order in which they
+// complete.  The requantisation is integer arithmetic on a pipe that issues multiplies, shifts and packs at half
+// rate: the pass is written for the fewest such instructions (see ChanConst4).  A loader warp copies the next
+// convolution's blob once its place is free.  Consecutive convolutions overlap unit by unit.  Input noise (Def. 3.3,
 // Eq. 2; Def. 3.4), halo fills and the pool / FC / argmax tail are CTA-wide phases between barriers.
 //
 // Every device-side wait is bounded by a wall-clock limit; on expiry the CTA raises an abort flag, all
@@ -58,17 +59,16 @@ using namespace tc;
 namespace {
 
 constexpr int kG = 4;                       // samples per group
-constexpr int kEpiWarps = 8;                // warps 0..7: epilogue; set = warp / 4, tensor-memory quarter = warp % 4
+constexpr int kEpiWarps = 16;               // the first warps: epilogue; set = warp / 4, tensor-memory quarter = warp % 4
 constexpr int kSets = kEpiWarps / 4;
-constexpr int kIssuers = 4;                 // the next four warps: lane 0 of each issues every fourth MMA chain of a convolution
+constexpr int kIssuers = 3;                 // the next warps: lane 0 of each issues every kIssuers-th MMA chain of a convolution
 constexpr int kLoaderWarp = kEpiWarps + kIssuers;   // the last warp: weight copies
 constexpr int kThreads = 32 * (kEpiWarps + kIssuers + 1);
-constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kMaxKsteps = 18;
 constexpr int kMaxPhases = 160;
 constexpr int kMaxBars = 128;
 constexpr int kMaxLines = 32;               // output lines of one convolution
-constexpr int kCtrlBytes = 9216;
+constexpr int kCtrlBytes = 10240;
 constexpr int kMaxConv = 128;
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kTmemCols = 512;
@@ -77,7 +77,9 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
 enum { ERR_NONE = 0, ERR_WAIT_DONE = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_READY = 3, ERR_WAIT_FULL = 4, ERR_WAIT_DRAIN = 5 };
 enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8, CF_GENERAL = 16 };     // CF_GENERAL: the pass that decides everything at run time
-enum { OPF_WAIT_ALL = 1, OPF_NULL = 4 };
+// OPF_WAIT_ALL: every unit of the previous convolution; OPF_NULL: no MMAs, arrivals only; OPF_WAITS / OPF_WAITS4: the
+// record names counters to test (two / four slots in use); bits 4-6: how many of them are distinct; bits 8-9: arrivals
+enum { OPF_WAIT_ALL = 1, OPF_WAITS = 2, OPF_NULL = 4, OPF_WAITS4 = 8 };
 
 // ---- what the kernel reads -------------------------------------------------------------------
 
@@ -102,7 +104,7 @@ struct alignas(16) LOp {
     uint32_t a_add, b_add;  // 16-byte units: (input line + 1) * pitch, first weight block * block size
     uint16_t wait[4];       // 8 * unit of the previous convolution that must be stored
     uint16_t commit[3];     // 8 * unit of this convolution whose accumulators are complete after the chain
-    uint16_t flags;         // OPF_WAIT_ALL: every unit of the previous convolution; OPF_NULL: no MMAs, arrivals only
+    uint16_t flags;         // OPF_* | distinct waits << 4 | arrivals << 8
 };
 static_assert(sizeof(LOp) == 32, "one operation is two 16-byte loads");
 
@@ -119,7 +121,7 @@ struct alignas(16) LConvDesc {
     uint32_t out_log_lines, out_nb, out_logI, res_base;
     uint32_t res_plane, in_logI, in_I, in_n_lines;
     int32_t lo; uint32_t res_m2, res_r2_lo, res_r2_hi;
-    uint32_t b_lo0, kstep16, pad0, pad1;       // low word of the first K-step's weight descriptor (shared-memory base 0)
+    uint32_t b_lo0, kstep16, recs_per_item, pad1;       // low word of the first K-step's weight descriptor (shared-memory base 0); records per (unit, chunk)
     uint32_t a_lo[kMaxKsteps + 2];             // low words of the operand descriptors of line -1 (shared-memory base 0)
 };
 static_assert(sizeof(LConvDesc) % 16 == 0, "blob sections stay 16-byte aligned");
@@ -145,6 +147,7 @@ struct LineParams {
     int32_t *counts;
     int8_t *logits;                   // [n_samples][n_classes] or null
     int32_t *err;
+    unsigned long long *phase_cycles; // [4]: SM cycles per CTA spent in FILL, INPUT, everything else, TAIL, summed over CTAs and launches
     // debug
     int32_t stop_phase;
     uint32_t dump_off, dump_bytes;
@@ -158,6 +161,8 @@ struct Ctrl {
     volatile int abort_flag;
     uint32_t stored[kMaxBars];              // per unit: stores of its 16-channel chunks by a warp, counted over the whole run
     int32_t hist[128];
+    int32_t pooled[kG][64];                 // the tail's pooled features, one row per sample of the group
+    long long cyc[4], cyc_mark;             // thread 0's phase clocks
     PhaseEntry ptab[kMaxPhases];
     ConvSrc csrc[kMaxConv];
 };
@@ -188,16 +193,27 @@ __device__ __forceinline__ long long mad_wide_u(uint32_t a, uint32_t b, long lon
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
     return d;
 }
-// Per-channel constants of a blob that is complete in shared memory (the address derives from a value read after
-// the wait for the blob): a plain load the compiler may schedule ahead of the tensor-memory wait.
-__device__ __forceinline__ ChanConst ld_chan_const_early(uint32_t addr)
+// Per-channel requantisation constants as stored in the blob (16 bytes): folded bias, multiplier, rounding addend
+// and shift.  With s = shift - 1 >= 1,
+//   rs((acc + bias) * mult, 31 + shift) + zp_out = (hi32((acc + bias) * mult) + c) >> s,   c = 2^(s-1) + zp_out * 2^s,
+// exactly: the rounding half 2^(31+s) is a multiple of 2^32, so the low word of the product cannot change the floor.
+// For s = 0 the half sits in the low word: the result is hi32 + (bit 31 of the low word) + c with c = zp_out.
+// The integer pipe issues multiplies, shifts and packs at half rate here, a 64-bit addend costs two more
+// instructions: this form is the cheapest exact one found (add, wide multiply, add, shift).
+struct ChanConst4 { int bias, mult, c, s; };
+// A plain load (the blob is complete in shared memory; the address derives from a value read after the wait for it)
+// that the compiler may schedule ahead of the tensor-memory wait.
+__device__ __forceinline__ ChanConst4 ld_chan_const_early(uint32_t addr)
 {
-    long long b, ms;
-    asm("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(b), "=l"(ms) : "r"(addr));
-    ChanConst c;
-    c.B = b;
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(c.mult), "=r"(c.s) : "l"(ms));
+    ChanConst4 c;
+    asm("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(c.bias), "=r"(c.mult), "=r"(c.c), "=r"(c.s) : "r"(addr));
     return c;
+}
+__device__ __forceinline__ long long mul_wide(int a, int b)
+{
+    long long d;
+    asm("mul.wide.s32 %0, %1, %2;" : "=l"(d) : "r"(a), "r"(b));
+    return d;
 }
 __device__ __forceinline__ void red_release_add(uint32_t addr, uint32_t v)
 {
@@ -276,8 +292,42 @@ struct IssueCtx {
     uint32_t desc, ops, n_ops, s16, b_lo0, kstep16, d0, stacked, full_addr, cg, issuer;
 };
 
-// The operations of one convolution that belong to one issuing thread (every kIssuers-th record).  The low words of the operand descriptors stay in registers; an operation adds
-// its line and block offsets to their start-address fields.
+// The first, cheap read of a "stored" counter by an issuing thread.  A plain load by default: an acquiring one costs
+// over a hundred cycles per test on the issue path.  What the counter guards was published by the storing warp with a
+// proxy fence and a releasing add; the MMAs that read it are issued after the value was seen (control dependency)
+// and after tcgen05.fence::after_thread_sync.  Building with -DISC_ACQUIRE_POLL takes the acquiring form instead, so
+// that a divergence could be traced to this choice.
+__device__ __forceinline__ uint32_t ld_counter(uint32_t addr)
+{
+#ifdef ISC_ACQUIRE_POLL
+    return ld_acquire_u32(addr);
+#else
+    return lds32(addr);
+#endif
+}
+
+// The dependency test of an operation when its first, cheap form did not pass (or the operation waits for the whole
+// previous convolution): bounded waits on every counter the record names.  Kept out of line: the issue loop is
+// latency-bound, every instruction on its path counts.
+__device__ __noinline__ bool wait_units_slow(Waiter w, const PrevConv &prev, uint4 r1)
+{
+    const uint32_t fl = r1.w >> 16;
+    if (fl & OPF_WAIT_ALL)
+        for (uint32_t l = 0; l < prev.n_lines; ++l)
+            if (!w.counter(prev.done_addr + 4 * l, prev.expected, ERR_WAIT_DONE)) return false;
+    const uint32_t nw = (fl >> 4) & 7u;
+    const uint32_t off[4] = {r1.x & 0xFFFFu, r1.x >> 16, r1.y & 0xFFFFu, r1.y >> 16};
+#pragma unroll
+    for (uint32_t k = 0; k < 4; ++k)
+        if (k < nw && !w.counter(prev.done_addr + off[k], prev.expected, ERR_WAIT_DONE)) return false;
+    return true;
+}
+
+// The operations of one convolution that belong to one issuing thread (every kIssuers-th record).  The low words of
+// the operand descriptors stay in registers; an operation adds its line and block offsets to their start-address
+// fields.  The counters an operation depends on are read together (unused slots repeat the first one) and compared
+// once; what the counters guard was made visible to the tensor cores' reads by the storing warp (proxy fence, then a
+// releasing add) and is read by MMAs that are issued only after the values have been seen.
 template <int KS>
 __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const PrevConv &prev, uint32_t n_ksteps)
 {
@@ -298,49 +348,49 @@ __device__ __forceinline__ bool issue_ops(Waiter w, const IssueCtx &ic, const Pr
     }
     uint32_t at = ic.ops + 32u * ic.issuer;           // the table ends with kIssuers spare records: reads run one ahead
     uint4 n0 = ld_shared_v4(at), n1 = ld_shared_v4(at + 16);
+    const uint32_t acc_first = ic.stacked;
     for (uint32_t i = ic.issuer; i < ic.n_ops; i += kIssuers) {
         const uint4 r0 = n0, r1 = n1;         // d_col, idesc, a_add, b_add | wait 0-1, wait 2-3, commit 0-1, commit 2 and flags
         at += 32u * kIssuers;
         n0 = ld_shared_v4(at); n1 = ld_shared_v4(at + 16);
+        const uint32_t fl = r1.w >> 16;
         // units of the previous convolution this operation depends on
-        if (prev.n_lines) {
-            if ((r1.w >> 16) & OPF_WAIT_ALL) {
-                for (uint32_t l = 0; l < prev.n_lines; ++l)
-                    if (!w.counter(prev.done_addr + 4 * l, prev.expected, ERR_WAIT_DONE)) return false;
+        if (fl & (OPF_WAIT_ALL | OPF_WAITS)) {
+            int32_t m = -1;
+            if (!(fl & OPF_WAIT_ALL)) {
+                m = min((int32_t)(ld_counter(prev.done_addr + (r1.x & 0xFFFFu)) - prev.expected),
+                        (int32_t)(ld_counter(prev.done_addr + (r1.x >> 16)) - prev.expected));
+                if (fl & OPF_WAITS4)
+                    m = min(m, min((int32_t)(ld_counter(prev.done_addr + (r1.y & 0xFFFFu)) - prev.expected),
+                                   (int32_t)(ld_counter(prev.done_addr + (r1.y >> 16)) - prev.expected)));
             }
-            if ((r1.x & 0xFFFFu) != 0xFFFFu) {
-                if (!w.counter(prev.done_addr + (r1.x & 0xFFFFu), prev.expected, ERR_WAIT_DONE)) return false;
-                if ((r1.x >> 16) != 0xFFFFu) {
-                    if (!w.counter(prev.done_addr + (r1.x >> 16), prev.expected, ERR_WAIT_DONE)) return false;
-                    if ((r1.y & 0xFFFFu) != 0xFFFFu && !w.counter(prev.done_addr + (r1.y & 0xFFFFu), prev.expected, ERR_WAIT_DONE)) return false;
-                    if ((r1.y >> 16) != 0xFFFFu && !w.counter(prev.done_addr + (r1.y >> 16), prev.expected, ERR_WAIT_DONE)) return false;
-                }
-            }
+            if (m < 0 && !wait_units_slow(w, prev, r1)) return false;
         }
         tc_fence_after();
         const uint32_t d = ic.d0 + r0.x;
-        if ((r1.w >> 16) & OPF_NULL) {
+        if (fl & OPF_NULL) {
             // a record that only carries this thread's arrivals on units it did not add to
         } else if (KS > 0) {
 #pragma unroll
             for (int k = 0; k < NK; ++k) {
                 const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(alo[k] + r0.z);
                 const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)(blo[k] + r0.w);
-                mma_i8(d, ad, bd, r0.y, ic.stacked | (uint32_t)(k > 0));
+                mma_i8(d, ad, bd, r0.y, k > 0 ? 1u : acc_first);
             }
         } else {
             for (uint32_t k = 0; k < n_ksteps; ++k) {
                 const uint32_t a_lo = lds32(ic.desc + offsetof(LConvDesc, a_lo) + 4 * k) + ic.s16;
                 const uint64_t ad = ((uint64_t)ahi << 32) | (uint64_t)(a_lo + r0.z);
                 const uint64_t bd = ((uint64_t)bhi << 32) | (uint64_t)(ic.b_lo0 + ic.s16 + k * ic.kstep16 + r0.w);
-                mma_i8(d, ad, bd, r0.y, ic.stacked | (uint32_t)(k > 0));
+                mma_i8(d, ad, bd, r0.y, k > 0 ? 1u : acc_first);
             }
         }
-        if ((r1.z & 0xFFFFu) != 0xFFFFu) {
+        const uint32_t nc = (fl >> 8) & 3u;
+        if (nc) {
             commit_to(ic.full_addr + (r1.z & 0xFFFFu));
-            if ((r1.z >> 16) != 0xFFFFu) {
+            if (nc > 1) {
                 commit_to(ic.full_addr + (r1.z >> 16));
-                if ((r1.w & 0xFFFFu) != 0xFFFFu) commit_to(ic.full_addr + (r1.w & 0xFFFFu));
+                if (nc > 2) commit_to(ic.full_addr + (r1.w & 0xFFFFu));
             }
         }
     }
@@ -446,15 +496,13 @@ struct alignas(16) LPass {
 };
 static_assert(sizeof(LPass) == 32, "one pass is two 16-byte loads");
 
-// Per-channel requantisation constants as stored in the blob: the 64-bit addend, then multiplier and shift.
-//   y = floor((acc * mult + B) / 2^(32 + s)); B holds the folded bias, the rounding half and the output
-//   zero-point, so this is rs(acc' * mult, 31 + shift) + zp_out exactly.
+// One output of the common pass (every channel has s >= 1).
 //   residual: y += floor((u * m2 + R2) / 2^32) with u = r + 128 the residual byte as an unsigned number,
 //   m2 = res_mult * 2^(32-n) and R2 the rounding half and the zero-points folded: rs((r - zp_res) * res_mult, n).
 template <bool kRes, int K>
-__device__ __forceinline__ int requant1(int acc, const ChanConst &cs, uint32_t rword, uint32_t res_m2, long long res_r2)
+__device__ __forceinline__ int requant1(int acc, const ChanConst4 &cs, uint32_t rword, uint32_t res_m2, long long res_r2)
 {
-    int y = hi32(mad_wide(acc, cs.mult, cs.B)) >> cs.s;
+    int y = (hi32(mul_wide(acc + cs.bias, cs.mult)) + cs.c) >> cs.s;
     if (kRes) y += hi32(mad_wide_u(ubyte<K>(rword), res_m2, res_r2));
     return y;
 }
@@ -511,8 +559,8 @@ __device__ __forceinline__ void epi_pass2(const EpiConv &E, const EpiCtx &c, uin
     uint32_t o0[4], o1[4];
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
-        const ChanConst c0 = ld_chan_const_early(cbase + (4 * g + 0) * 16), c1 = ld_chan_const_early(cbase + (4 * g + 1) * 16);
-        const ChanConst c2 = ld_chan_const_early(cbase + (4 * g + 2) * 16), c3 = ld_chan_const_early(cbase + (4 * g + 3) * 16);
+        const ChanConst4 c0 = ld_chan_const_early(cbase + (4 * g + 0) * 16), c1 = ld_chan_const_early(cbase + (4 * g + 1) * 16);
+        const ChanConst4 c2 = ld_chan_const_early(cbase + (4 * g + 2) * 16), c3 = ld_chan_const_early(cbase + (4 * g + 3) * 16);
         o0[g] = pack4_sat(requant1<kRes, 0>(acc0[4 * g + 0], c0, r0[g], m2, r2), requant1<kRes, 1>(acc0[4 * g + 1], c1, r0[g], m2, r2),
                           requant1<kRes, 2>(acc0[4 * g + 2], c2, r0[g], m2, r2), requant1<kRes, 3>(acc0[4 * g + 3], c3, r0[g], m2, r2));
         o1[g] = pack4_sat(requant1<kRes, 0>(acc1[4 * g + 0], c0, r1[g], m2, r2), requant1<kRes, 1>(acc1[4 * g + 1], c1, r1[g], m2, r2),
@@ -530,20 +578,28 @@ __device__ __forceinline__ void epi_pass2(const EpiConv &E, const EpiCtx &c, uin
         st_shared_v4_if(a1 + E.dup_delta, v1, (q0.x >> 18) & E.dup_up);
         st_shared_v4_if(a1 - E.dup_delta, v1, (q0.x >> 19) & E.dup_dn);
     }
-    tmem_st_wait();
-    pass_done(E, c, q0.x & 0xFFu);
 }
 
+// The items (unit, chunk) of a convolution that belong to this warp's set: one wait, one or two records of two lines
+// each, one arrival.
 template <bool kRes>
-__device__ __forceinline__ void epi_conv_fast(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_passes)
+__device__ __forceinline__ void epi_conv_fast(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_items,
+                                            uint32_t item_bytes)
 {
     const EpiConv E = E_in;
     const EpiCtx c = c_in;
 #pragma unroll 1
-    for (uint32_t i = (uint32_t)c.set; i < n_passes; i += kSets) {
-        const uint4 q0 = ld_shared_v4(passes + 32u * i), q1 = ld_shared_v4(passes + 32u * i + 16u);
+    for (uint32_t i = (uint32_t)c.set; i < n_items; i += kSets) {
+        const uint32_t rec = passes + item_bytes * i;
+        const uint4 q0 = ld_shared_v4(rec), q1 = ld_shared_v4(rec + 16u);
         if (!wait_full(w, E.full_addr + 8u * (q0.x & 0xFFu), E.parity)) return;     // aborted: every other wait falls through too
         epi_pass2<kRes>(E, c, q0, q1);
+        if (item_bytes > 32u) {
+            const uint4 p0 = ld_shared_v4(rec + 32u), p1 = ld_shared_v4(rec + 48u);
+            epi_pass2<kRes>(E, c, p0, p1);
+        }
+        tmem_st_wait();
+        pass_done(E, c, q0.x & 0xFFu);
     }
 }
 
@@ -593,8 +649,9 @@ __device__ __noinline__ void epi_conv_general(Waiter w, const EpiConv &E, const 
                 int y[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const ChanConst cs = ld_chan_const_early(E.const_addr + ch * 256u + (4 * g + k) * 16);
-                    int v = hi32(mad_wide(acc[4 * g + k], cs.mult, cs.B)) >> cs.s;
+                    const ChanConst4 cs = ld_chan_const_early(E.const_addr + ch * 256u + (4 * g + k) * 16);
+                    const long long prod = mul_wide(acc[4 * g + k] + cs.bias, cs.mult);
+                    int v = cs.s ? (hi32(prod) + cs.c) >> cs.s : hi32(prod) + (int)((uint32_t)lo32(prod) >> 31) + cs.c;
                     if (res) v += hi32(mad_wide_u((rw[g] >> (8 * k)) & 0xFFu, E.res_m2, E.res_r2));
                     y[k] = max(v, lo);
                 }
@@ -653,8 +710,9 @@ __device__ __forceinline__ void epi_conv(const LineParams &p, const EpiCtx &c, u
         epi_conv_general(w, E, c, desc, flags, (int32_t)h9.x, passes, n_passes);
         return;
     }
-    if (flags & CF_RES) epi_conv_fast<true>(w, E, c, passes, n_passes);
-    else epi_conv_fast<false>(w, E, c, passes, n_passes);
+    const uint32_t rpi = lds32(desc + offsetof(LConvDesc, recs_per_item));
+    if (flags & CF_RES) epi_conv_fast<true>(w, E, c, passes, n_passes / rpi, 32u * rpi);
+    else epi_conv_fast<false>(w, E, c, passes, n_passes / rpi, 32u * rpi);
 }
 
 // FILL: the region takes its halo value everywhere
@@ -717,36 +775,36 @@ __device__ void input_phase(const LineParams &p, const EpiCtx &c, int grp)
     }
 }
 
-// TAIL: global average pool, FC, argmax and vote; one warp carries one sample (Algorithm 1 steps 1-4).
+// TAIL, first half: global average pool.  One thread sums one (sample, channel) pair over the pixels and
+// requantises it; consecutive threads take the four samples of consecutive channels (one shared-memory wavefront).
+__device__ void tail_pool(const LineParams &p, const EpiCtx &c)
+{
+    const int tail_W = p.tail_W, n_lines = p.tail_n_lines, hw = p.tail_H * p.tail_W;
+    for (int q = c.tid; q < kG * p.tail_C; q += kThreads) {
+        const int s = q & (kG - 1), ch = q >> 2;
+        const uint32_t base = c.sbase + p.tail_base + (uint32_t)(ch >> 4) * p.tail_plane + (uint32_t)(ch & 15);
+        int sum = 0;
+        for (int i = 0; i < hw; ++i) {
+            const int y = i / tail_W, x = i - y * tail_W;
+            const int line = y % n_lines, band = y / n_lines;
+            const uint32_t pos = (uint32_t)line * p.tail_pitch16 + ((uint32_t)x << p.tail_logI) + (uint32_t)(band * 4 + s);
+            int v;
+            asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(base + pos * 16u));
+            sum += v - p.pool_zp_in;
+        }
+        long long v = ((long long)sum * p.pool_mult + (1ll << (p.pool_n - 1))) >> p.pool_n;
+        v += p.pool_zp_out;
+        v = v < p.pool_lo ? p.pool_lo : v;
+        v = v > 127 ? 127 : v;
+        c.ctrl->pooled[s][ch] = (int32_t)v;
+    }
+}
+
+// TAIL, second half: FC, argmax and vote; one warp carries one sample (Algorithm 1 steps 1-4).
 __device__ void tail_sample(const LineParams &p, const EpiCtx &c, int s, int grp)
 {
-    const int tail_H = p.tail_H, tail_W = p.tail_W, tail_C = p.tail_C, n_lines = p.tail_n_lines;
+    const int tail_C = p.tail_C;
     const int n_classes = p.n_classes;
-    const int hw = tail_H * tail_W;
-    int pooled[2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int ch = c.lane + 32 * h;
-        int q = 0;
-        if (ch < tail_C) {
-            const uint32_t base = c.sbase + p.tail_base + (uint32_t)(ch >> 4) * p.tail_plane + (ch & 15);
-            int sum = 0;
-            for (int i = 0; i < hw; ++i) {
-                const int y = i / tail_W, x = i - y * tail_W;
-                const int line = y % n_lines, band = y / n_lines;
-                const uint32_t pos = (uint32_t)line * p.tail_pitch16 + ((uint32_t)x << p.tail_logI) + (uint32_t)(band * 4 + s);
-                int v;
-                asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(base + pos * 16u));
-                sum += v - p.pool_zp_in;
-            }
-            long long v = ((long long)sum * p.pool_mult + (1ll << (p.pool_n - 1))) >> p.pool_n;
-            v += p.pool_zp_out;
-            v = v < p.pool_lo ? p.pool_lo : v;
-            v = v > 127 ? 127 : v;
-            q = (int)v;
-        }
-        pooled[h] = q;
-    }
     const long long sample = (long long)grp * kG + s;          // index within this launch
     const bool counted = sample < p.n_samples;
     int best_v = -1000, best_o = 0x7fffffff;
@@ -756,10 +814,7 @@ __device__ void tail_sample(const LineParams &p, const EpiCtx &c, int s, int grp
         const FcConst k = p.fc_c[live ? o : 0];
         const int8_t *wrow = p.fc_w + (size_t)(live ? o : 0) * 64;
         int acc = k.bias;
-        for (int cc = 0; cc < tail_C; ++cc) {
-            const int a = __shfl_sync(0xffffffffu, pooled[cc >> 5], cc & 31);
-            acc += a * (int)__ldg(wrow + cc);
-        }
+        for (int cc = 0; cc < tail_C; ++cc) acc += c.ctrl->pooled[s][cc] * (int)__ldg(wrow + cc);
         long long v = ((long long)acc * k.mult + (1ll << (k.n - 1))) >> k.n;
         v += k.zp_out;
         v = v < k.lo ? k.lo : v;
@@ -821,6 +876,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     const int n_phases = p.n_phases, stop_phase = p.stop_phase;
     bool role_ok = true;
     int it = 0;
+    // thread 0 keeps the time the CTA spends in its CTA-wide phases (they run between barriers, so one thread's clock
+    // measures them); what is left of the kernel's duration is the convolutions
+    if (threadIdx.x == 0) {
+        ctrl->cyc[PH_FILL] = ctrl->cyc[PH_INPUT] = ctrl->cyc[PH_TAIL] = 0;
+        ctrl->cyc[PH_CONV] = clock64();         // until the end: the start time
+    }
     for (int grp = blockIdx.x; grp < p.n_groups; grp += gridDim.x, ++it) {
         PrevConv prev{0u, 0u, 0u};
         int conv_index = 0;
@@ -855,17 +916,32 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
                     role_ok = loader_copy(p, ctrl, sbase, 0, (uint32_t)it * (uint32_t)p.n_conv, it);
                 first_phase = false;
             }
-            if (!ctrl->abort_flag) {           // every warp of the CTA takes part in these phases
+            // every warp of the CTA takes part in these phases; nothing inside them can raise the abort flag
+            const bool live = !ctrl->abort_flag;
+            if (threadIdx.x == 0) ctrl->cyc_mark = clock64();
+            if (live) {
                 if (e.x == PH_FILL) fill_phase(c, e.y, e.z, e.w);
                 else if (e.x == PH_INPUT) input_phase(p, c, grp);
-                else if (warp < kG) tail_sample(p, c, warp, grp);
+                else tail_pool(p, c);
+            }
+            if (e.x == PH_TAIL) {
+                __syncthreads();
+                if (live && warp < kG) tail_sample(p, c, warp, grp);
             }
             fence_proxy_async();
             __syncthreads();
+            if (threadIdx.x == 0) ctrl->cyc[e.x & 3u] += clock64() - ctrl->cyc_mark;
         }
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
+    }
+    if (threadIdx.x == 0 && p.phase_cycles) {
+        const long long total = clock64() - ctrl->cyc[PH_CONV];
+        atomicAdd(p.phase_cycles + PH_FILL, (unsigned long long)ctrl->cyc[PH_FILL]);
+        atomicAdd(p.phase_cycles + PH_INPUT, (unsigned long long)ctrl->cyc[PH_INPUT]);
+        atomicAdd(p.phase_cycles + PH_TAIL, (unsigned long long)ctrl->cyc[PH_TAIL]);
+        atomicAdd(p.phase_cycles + PH_CONV, (unsigned long long)(total - ctrl->cyc[PH_FILL] - ctrl->cyc[PH_INPUT] - ctrl->cyc[PH_TAIL]));
     }
     if (!ctrl->abort_flag)
         for (int i = threadIdx.x; i < p.n_classes; i += blockDim.x)
@@ -970,6 +1046,7 @@ struct LinePlan {
     int8_t *d_fc_w = nullptr;
     FcConst *d_fc_c = nullptr;
     int32_t *d_err = nullptr;
+    unsigned long long *d_phase_cycles = nullptr;
     uint8_t *d_dump = nullptr;
     int sm_count = 0;
     bool attr_set = false;
@@ -981,7 +1058,8 @@ namespace {
 struct ConvPlan {
     int layer = -1, phase = -1;
     int in_tensor = -1, out_tensor = -1;
-    bool stacked = false, scatter = false;
+    bool stacked = false, scatter = false, general = false;
+    int recs_per_item = 1;              // records of the pass table per (unit, chunk)
     int m = 0;                          // output lines (ordinals)
     int n_chunks = 0, cols = 0, n_banks = 1;
     int cls = -1, use_local = 0;
@@ -1198,12 +1276,20 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
         std::vector<int> order((size_t)cp.m);
         for (int y = 0; y < cp.m; ++y) order[(size_t)y] = y;
         std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return last_op[(size_t)a] < last_op[(size_t)b]; });
+        // A record of the pass table covers `sup` lines; a unit (one "accumulators complete" barrier, one "stored"
+        // counter) covers `upl` lines = one or two records.  Long convolutions take four-line units: every barrier
+        // arrival costs an issuing thread a tcgen05.commit and every unit costs an epilogue warp a wait and an arrival.
         const int sup = cp.m >= 2 ? 2 : 1;
-        cp.n_units = (cp.m + sup - 1) / sup;
+        bool general = cp.scatter || (cp.m & 1) || (L.relu && L.zp_out > -128);
+        for (int oc = 0; oc < L.cout; ++oc) general = general || layers[cp.layer].shift[oc] == 1;
+        cp.general = general;
+        const int upl = (!general && cp.m >= 16 && cp.m % 4 == 0) ? 4 : sup;
+        cp.recs_per_item = upl / sup;
+        cp.n_units = (cp.m + upl - 1) / upl;
         cp.unit_of.assign((size_t)cp.m, 0);
         std::vector<int> unit_last_op((size_t)cp.n_units, -1);
         for (int i = 0; i < cp.m; ++i) {
-            const int u = i / sup;
+            const int u = i / upl;
             cp.unit_of[(size_t)order[(size_t)i]] = u;
             unit_last_op[(size_t)u] = std::max(unit_last_op[(size_t)u], last_op[(size_t)order[(size_t)i]]);
         }
@@ -1292,6 +1378,12 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
                     all_waited[(size_t)u] = 1;
                 }
             for (int u : commits[i]) op.commit[n_commit++] = (uint16_t)(8 * u);
+            // unused wait slots repeat the first one, so that the kernel reads two (or four) counters without looking
+            if (n_wait) {
+                op.flags |= OPF_WAITS | (n_wait > 2 ? OPF_WAITS4 : 0);
+                for (int k = n_wait; k < 4; ++k) op.wait[k] = op.wait[0];
+            }
+            op.flags |= (uint16_t)(n_wait << 4) | (uint16_t)(n_commit << 8);
             cp.ops.push_back(op);
         }
         // "this convolution complete" must imply "the previous one complete": between them the threads wait for all its units
@@ -1300,14 +1392,17 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
                 if (!wtd) PLAN_FAIL(20);
         // ---- passes: unit by unit, chunk by chunk
         cp.done_time.assign((size_t)cp.m, 0);
+        int n_items = 0;
         for (int u = 0; u < cp.n_units; ++u)
-            for (int ch = 0; ch < cp.n_chunks; ++ch) {
-                const int n = std::min(sup, cp.m - u * sup);
+            for (int ch = 0; ch < cp.n_chunks; ++ch, ++n_items)
+              for (int rec = 0; rec < cp.recs_per_item; ++rec) {
+                const int first = u * upl + rec * sup;
+                const int n = std::min(sup, cp.m - first);
                 LPass P;
                 memset(&P, 0, sizeof(P));
                 P.meta = (uint32_t)u | ((uint32_t)n << 8) | ((uint32_t)ch << 12);
                 for (int q = 0; q < n; ++q) {
-                    const int line = order[(size_t)u * sup + q];
+                    const int line = order[(size_t)first + q];
                     P.lines |= (uint32_t)line << (8 * q);
                     P.tcol[q] = (uint32_t)(line * cp.cols + ch * 16);
                     P.out[q] = (uint32_t)(line * out.pitch) * 16u + (uint32_t)ch * out.plane_bytes;
@@ -1316,10 +1411,10 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
                         if (line == 0) P.meta |= 1u << (16 + 2 * q);
                         if (line == out.n_lines - 1) P.meta |= 1u << (17 + 2 * q);
                     }
-                    cp.done_time[(size_t)line] = (int)cp.passes.size() / kSets;
+                    cp.done_time[(size_t)line] = n_items / kSets;
                 }
                 cp.passes.push_back(P);
-            }
+              }
         convs.push_back(cp);
     }
     const int n_conv = (int)convs.size();
@@ -1414,7 +1509,8 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
         if (lo > -128) D.flags |= CF_LO;
         D.lo = lo;
         // the fast pass covers pairs of lines stored in place with the saturating pack as the only clamp
-        if (lo > -128 || cp.scatter || (cp.m & 1)) D.flags |= CF_GENERAL;
+        if (cp.general) D.flags |= CF_GENERAL;
+        D.recs_per_item = (uint32_t)cp.recs_per_item;
         // operand base: line -1, lane 0, plane 0 of the input
         D.a_base = plan->tensor_off[(size_t)cp.in_tensor] + in.line0 - (uint32_t)in.pitch * 16u;
         D.pitch16 = (uint32_t)in.pitch;
@@ -1485,17 +1581,21 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
                 }
             }
         }
+        bool any_shift_one = false;
         for (int oc = 0; oc < L.cout; ++oc) {
             long long wsum = 0;
             for (int q = 0; q < L.cin * taps; ++q) wsum += ML.w[(size_t)oc * L.cin * taps + q];
             const int sh = ML.shift[oc];
             if (sh < 1 || sh > 20) PLAN_FAIL(19);
-            const int nn = 31 + sh;
             const long long biasf = (long long)ML.bias[oc] - (long long)L.zp_in * wsum;
-            const long long B = biasf * ML.mult[oc] + (1ll << (nn - 1)) + ((long long)L.zp_out << nn);
-            int32_t cst[4] = {(int32_t)(uint32_t)(B & 0xFFFFFFFFll), (int32_t)(B >> 32), ML.mult[oc], nn - 32};
+            if (biasf < -(1ll << 31) || biasf >= (1ll << 31)) PLAN_FAIL(24);
+            const int sft = sh - 1;
+            const int32_t addend = sft ? (1 << (sft - 1)) + L.zp_out * (1 << sft) : L.zp_out;
+            int32_t cst[4] = {(int32_t)biasf, ML.mult[oc], addend, sft};
             memcpy(&blob[c_rel[(size_t)c] + (size_t)oc * 16], cst, 16);
+            if (sft == 0) any_shift_one = true;
         }
+        if (any_shift_one && !cp.general) PLAN_FAIL(25);      // a shift of one puts the rounding half in the product's low word
         (*blob_offsets)[(size_t)c] = (uint32_t)blob_out->size();
         blob_out->insert(blob_out->end(), blob.begin(), blob.end());
         (*csrc_out)[(size_t)c].bytes_phase = w_bytes[(size_t)c] | ((uint32_t)ph << 24);
@@ -1624,6 +1724,8 @@ int line_build(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w
     up((void **)&plan->d_fc_c, fcc.data(), fcc.size() * sizeof(FcConst));
     int32_t zero = 0;
     up((void **)&plan->d_err, &zero, sizeof(zero));
+    const unsigned long long zeros4[4] = {0, 0, 0, 0};
+    up((void **)&plan->d_phase_cycles, zeros4, sizeof(zeros4));
     if (cuda_ok && cudaMalloc((void **)&plan->d_dump, kSmemLimit) != cudaSuccess) cuda_ok = false;
     if (!cuda_ok) { cudaGetLastError(); line_free(plan); return ISC_ERR_NOMEM; }
 
@@ -1649,6 +1751,7 @@ int line_build(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_w
     b.fc_w = plan->d_fc_w; b.fc_c = plan->d_fc_c;
     b.n_classes = n_classes;
     b.err = plan->d_err;
+    b.phase_cycles = plan->d_phase_cycles;
     b.stop_phase = 1 << 30;
     *out = plan;
     return ISC_OK;
@@ -1658,7 +1761,7 @@ void line_free(LinePlan *p)
 {
     if (!p) return;
     cudaFree(p->d_ptab); cudaFree(p->d_conv_src); cudaFree(p->d_bar_counts); cudaFree(p->d_blob); cudaFree(p->d_fc_w);
-    cudaFree(p->d_fc_c); cudaFree(p->d_err); cudaFree(p->d_dump);
+    cudaFree(p->d_fc_c); cudaFree(p->d_err); cudaFree(p->d_phase_cycles); cudaFree(p->d_dump);
     delete p;
 }
 
@@ -1707,6 +1810,15 @@ int line_check(LinePlan *p)
         if (getenv("ISC_PLAN_DEBUG")) fprintf(stderr, "line engine: wait %d on barrier %d parity %d expired in CTA %d\n", e & 0xFF, (e >> 8) & 0xFFF, (e >> 20) & 1, (int)((unsigned)e >> 21));
         cudaMemset(p->d_err, 0, sizeof(e));
         return ISC_ERR_TIMEOUT;
+    }
+    return ISC_OK;
+}
+
+int line_phase_cycles(LinePlan *p, unsigned long long out[4])
+{
+    if (cudaMemcpy(out, p->d_phase_cycles, 4 * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return ISC_ERR_CUDA;
     }
     return ISC_OK;
 }

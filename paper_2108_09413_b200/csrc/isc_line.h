@@ -33,4 +33,8 @@ int line_debug_tensor(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, in
 // After the stream has been synchronised: ISC_OK, or ISC_ERR_TIMEOUT if a bounded wait expired.
 int line_check(LinePlan *p);
 
+// SM cycles, summed over CTAs and over every launch so far, spent in: [0] halo fills, [1] the noise phase (draw, add,
+// saturate, store: Def. 3.3, Def. 3.4), [2] the convolutions, [3] pool / FC / argmax / vote.  Synchronises the device.
+int line_phase_cycles(LinePlan *p, unsigned long long out[4]);
+
 }  // namespace isc
