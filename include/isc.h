@@ -250,13 +250,16 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
 /*
  * isc_set_option -- tuning knobs; none changes a result.
  *   "batch"  : noisy samples per launch (0 = choose automatically).
- *   "engine" : 0 = automatic (the fastest engine the model fits), 1 = layer-by-layer
- *              kernels only, 3 = require the line-tiled shared-memory-resident
- *              tensor-core kernel (ISC_ERR_UNSUPPORTED at the next call if the model
- *              does not fit it).  2 is not an engine (ISC_ERR_ARG).
+ *   "engine" : 0 = automatic (3 if the model fits it, else 2 if any layer fits it, else 1),
+ *              1 = layer-by-layer kernels without tensor cores, 2 = layer-by-layer with
+ *              the tcgen05 implicit-GEMM kernel for every convolution whose input and
+ *              output channels are multiples of 64, 3 = the line-tiled
+ *              shared-memory-resident tensor-core kernel (2 and 3 give
+ *              ISC_ERR_UNSUPPORTED at the next call if the model does not fit).
  * isc_get_info reads back: "engine" (the engine the last call used), "gpu_launches"
  * (kernel launches issued by this handle so far), "macs_per_sample",
- * "has_line_engine" (1 if the model fits engine 3) and, for engine 3, "cycles_fill",
+ * "has_line_engine" (1 if the model fits engine 3), "has_tensor_core_layers" (1 if
+ * engine 2 has a layer to run) and, for engine 3, "cycles_fill",
  * "cycles_noise", "cycles_conv", "cycles_tail": SM cycles summed over thread blocks and over
  * all launches of this handle so far, spent in halo fills, in the noise phase (draw, add,
  * saturate, store), in the convolutions and in pool / FC / argmax / vote -- the noise

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libisc.so")
-SOURCES = ["isc_api.cu", "isc_generic.cu", "isc_line.cu", "isc_decide.cpp"]
+SOURCES = ["isc_api.cu", "isc_generic.cu", "isc_igemm.cu", "isc_line.cu", "isc_decide.cpp"]
 
 
 def _newest_source() -> float:

@@ -44,6 +44,9 @@ struct isc_model {
     // device parameters of the layer-by-layer engine
     std::vector<GLayer> glayers;
     std::vector<void *> param_allocs;
+    std::vector<const int8_t *> wpacks;         // per layer: repacked weights of the tensor-core convolution, or null
+    bool has_tc = false;
+    int32_t *d_tc_err = nullptr;
 
     // activation buffers: tensor t lives in pool buffer tensor_buf[t] (bytes per sample buf_bytes[b])
     std::vector<int> tensor_buf;
@@ -195,6 +198,7 @@ int build_generic_engine(isc_model *m)
         if (m->layers[(size_t)i].d.in_tensor == 0) return ISC_ERR_UNSUPPORTED;
 
     m->glayers.resize((size_t)n);
+    m->wpacks.assign((size_t)n, nullptr);
     for (int i = 0; i < n; ++i) {
         const HostLayer &H = m->layers[(size_t)i];
         const isc_layer &L = H.d;
@@ -240,8 +244,20 @@ int build_generic_engine(isc_model *m)
                         }
             }
             rc = upload(m, w, &G.w); if (rc) return rc;
+            if (i > 0 && igemm_tile_n(G)) {                 // the same layer for the tensor-core kernel
+                std::vector<int8_t> wp(igemm_pack_bytes(G));
+                igemm_pack_weights(G, H.w.data(), wp.data());
+                rc = upload(m, wp, &m->wpacks[(size_t)i]); if (rc) return rc;
+                m->has_tc = true;
+            }
         }
         m->glayers[(size_t)i] = G;
+    }
+    if (m->has_tc) {
+        std::vector<int32_t> zero(1, 0);
+        const int32_t *p = nullptr;
+        int rc = upload(m, zero, &p); if (rc) return rc;
+        m->d_tc_err = const_cast<int32_t *>(p);
     }
 
     // buffer plan: greedy reuse by last use
@@ -352,14 +368,16 @@ NoiseStream make_stream(const isc_model *m, uint64_t seed, uint64_t image_id, in
 int choose_engine(isc_model *m)
 {
     if (m->opt_engine == 1) return 1;
+    if (m->opt_engine == 2) return m->has_tc ? 2 : ISC_ERR_UNSUPPORTED;
     if (m->opt_engine == 3) return m->line ? 3 : ISC_ERR_UNSUPPORTED;
     if (m->line) return 3;
+    if (m->has_tc) return 2;
     return 1;
 }
 
 // Layer-by-layer forward of `batch` samples; leaves the logits in the last tensor's buffer.
 int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int batch, cudaStream_t st,
-                    int stop_after_layer = -1)
+                    int stop_after_layer = -1, bool tensor_cores = false)
 {
     const int n = (int)m->glayers.size();
     for (int i = 0; i < n; ++i) {
@@ -370,6 +388,7 @@ int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int
         const int8_t *res = L.res_tensor >= 0 ? (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.res_tensor]].p : nullptr;
         cudaError_t e;
         if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, batch, out, st);
+        else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], batch, in, res, out, m->d_tc_err, st);
         else if (L.op == ISC_CONV2D || L.op == ISC_FC) e = launch_conv(G, batch, in, res, out, st);
         else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, batch, in, out, st);
         else e = launch_maxpool(G, batch, in, out, st);
@@ -412,7 +431,7 @@ int run_counts(isc_model *m, const uint8_t *d_x, uint64_t seed, uint64_t image_i
     for (int64_t done = 0; done < n; done += cap) {
         const int b = (int)std::min<int64_t>(cap, n - done);
         NoiseStream ns = make_stream(m, seed, image_id, phase, first + done);
-        rc = generic_forward(m, d_x, ns, b, st);
+        rc = generic_forward(m, d_x, ns, b, st, -1, engine == 2);
         if (rc) return rc;
         const int8_t *lg = (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)last]].p;
         cudaError_t e = launch_votes(lg, m->shapes[(size_t)last].cp, m->n_classes, b, d_counts,
@@ -433,6 +452,22 @@ int stage_image(isc_model *m, const uint8_t *x, size_t bytes, bool on_device, cu
     if (rc) return rc;
     CK(cudaMemcpyAsync(m->d_x, x, bytes, cudaMemcpyHostToDevice, st));
     *d_x = m->d_x;
+    return ISC_OK;
+}
+
+// After the stream has been synchronised: has a bounded wait of a tensor-core kernel expired?
+int check_engines(isc_model *m)
+{
+    int rc;
+    if (m->line && (rc = isc::line_check(m->line))) return rc;
+    if (m->d_tc_err && m->last_engine == 2) {
+        int32_t e = 0;
+        CK(cudaMemcpy(&e, m->d_tc_err, sizeof(e), cudaMemcpyDeviceToHost));
+        if (e != 0) {
+            cudaMemset(m->d_tc_err, 0, sizeof(e));
+            return ISC_ERR_TIMEOUT;
+        }
+    }
     return ISC_OK;
 }
 
@@ -574,7 +609,7 @@ int isc_sample_counts(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t
         CK(cudaMemcpyAsync(hl.data(), m->d_logits, hl.size(), cudaMemcpyDeviceToHost, st));
     }
     CK(cudaStreamSynchronize(st));
-    if (m->line && (rc = isc::line_check(m->line))) return rc;
+    if ((rc = check_engines(m))) return rc;
     memcpy(out_counts, h.data(), C * sizeof(int32_t));
     if (out_logits && n_samples > 0) memcpy(out_logits, hl.data(), hl.size());
     return ISC_OK;
@@ -621,7 +656,7 @@ int isc_certify_batch(isc_model *m, const uint8_t *x_u8, int x_on_device, int n_
     std::vector<int32_t> h(2 * C * (size_t)n_images);
     CK(cudaMemcpyAsync(h.data(), m->d_counts, h.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
-    if (m->line && (rc = isc::line_check(m->line))) return rc;
+    if ((rc = check_engines(m))) return rc;
     for (int i = 0; i < n_images; ++i) {
         const int32_t *c0 = h.data() + (size_t)i * 2 * C, *c1 = c0 + C;
         double radius = 0.0;
@@ -744,7 +779,7 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
         return e == cudaSuccess ? ISC_OK : ISC_ERR_CUDA;
     }
     if ((rc = ensure_workspace(m, 1))) return rc;
-    if ((rc = generic_forward(m, d_x, ns, 1, st, tensor - 1))) return rc;
+    if ((rc = generic_forward(m, d_x, ns, 1, st, tensor - 1, m->opt_engine == 2 || (m->opt_engine == 0 && m->has_tc)))) return rc;
     std::vector<int8_t> h((size_t)s.h * s.w * s.cp);
     CK(cudaMemcpyAsync(h.data(), m->bufs[(size_t)m->tensor_buf[(size_t)tensor]].p, h.size(),
                        cudaMemcpyDeviceToHost, st));
@@ -880,7 +915,7 @@ int isc_set_option(isc_model *m, const char *name, int64_t value)
         return ISC_OK;
     }
     if (!strcmp(name, "engine")) {
-        if (value != 0 && value != 1 && value != 3) return ISC_ERR_ARG;
+        if (value < 0 || value > 3) return ISC_ERR_ARG;
         m->opt_engine = value;
         return ISC_OK;
     }
@@ -894,6 +929,7 @@ int isc_get_info(isc_model *m, const char *name, int64_t *out)
     else if (!strcmp(name, "gpu_launches")) *out = m->launches;
     else if (!strcmp(name, "macs_per_sample")) *out = m->macs;
     else if (!strcmp(name, "has_line_engine")) *out = m->line ? 1 : 0;
+    else if (!strcmp(name, "has_tensor_core_layers")) *out = m->has_tc ? 1 : 0;
     else if (!strncmp(name, "cycles_", 7)) {
         static const char *const which[4] = {"cycles_fill", "cycles_noise", "cycles_conv", "cycles_tail"};
         if (!m->line) return ISC_ERR_UNSUPPORTED;

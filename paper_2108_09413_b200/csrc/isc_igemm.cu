@@ -1,0 +1,230 @@
+// Layer-by-layer implicit-GEMM convolution on the tensor cores (sm_100a): one launch per convolution over a batch of
+// noisy samples, for the networks whose activations do not fit in shared memory (the 224 x 224 bottleneck network of
+// the paper's second workload, Sec. 4.1).  Activations are the layer-by-layer engine's: int8, global memory,
+// [sample][y][x][channel padded to 16].
+//
+//   D[pixel, cout] = sum over (tap, cin) of A[pixel, (tap, cin)] * W[cout, (tap, cin)]
+//
+// A CTA owns a tile of 128 output pixels x N output channels (N = 64, 128 or 256) whose int32 accumulators live in
+// tensor memory.  The reduction runs in blocks of 64 input channels of one filter tap: the CTA's 128 threads gather
+// the block's operand rows (one thread = one pixel = 64 contiguous bytes, or the input zero-point outside the image)
+// into shared memory in the K-major core-matrix layout, one bulk copy brings the matching slice of the repacked
+// weights, and one thread issues two tcgen05.mma (kind::i8, K = 32 each).  Three stages of operands are in flight:
+// a stage is refilled when the commit of the MMAs that read it has arrived.  The epilogue reads the accumulators
+// back (one warp per 32-lane quarter), requantises (fixed-point multiplier, shift, zero-points, residual add, clamp)
+// and stores 16 channels per pixel at a time.  Every wait is bounded; on expiry the CTA sets an error word, frees its
+// tensor memory and returns.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "isc_epilogue.cuh"
+#include "isc_internal.h"
+#include "isc_tc.cuh"
+
+namespace isc {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kBlockK = 64;                  // bytes of K per stage: two MMA K-steps
+constexpr int kStages = 3;
+constexpr int kThreads = 128;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct IgemmParams {
+    GLayer L;
+    int batch, n_tile, tmem_cols;
+    long long m_total;                       // batch * hout * wout
+    const int8_t *in, *res;
+    int8_t *out;
+    const int8_t *wpack;                     // [cout tile][tap][cin block][4 K columns][n_tile rows][16 bytes]
+    int32_t *err;
+};
+
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void commit_to(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Bounded wait for a phase of an mbarrier; false after the limit (the caller raises the error word).
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity)
+{
+    if (mbar_test(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer();
+    for (int spin = 0;; ++spin) {
+        if (mbar_try(bar, parity)) return true;
+        if ((spin & 7) == 7 && globaltimer() - t0 > kWaitLimitNs) return false;
+    }
+}
+
+
+__global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ IgemmParams p)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ unsigned long long bar_w[kStages], bar_free[kStages], bar_done;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ volatile int abort_s;
+    const GLayer &L = p.L;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const uint32_t sbase = smem_u32(smem);
+    const int n_tile = p.n_tile;
+    const uint32_t a_bytes = kTileM * kBlockK, b_bytes = (uint32_t)n_tile * kBlockK, stage_bytes = a_bytes + b_bytes;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bar_w[s]), 1); mbar_init(smem_u32(&bar_free[s]), 1); }
+        mbar_init(smem_u32(&bar_done), 1);
+        abort_s = 0;
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_base_s), (uint32_t)p.tmem_cols);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+
+    // this thread's output pixel = row `tid` of the tile
+    const long long m = (long long)blockIdx.x * kTileM + tid;
+    const bool valid = m < p.m_total;
+    const long long mm = valid ? m : 0;
+    const int ox = (int)(mm % L.wout), oy = (int)((mm / L.wout) % L.hout);
+    const long long b = mm / ((long long)L.wout * L.hout);
+    const int n0 = blockIdx.y * n_tile;
+    const int cblocks = L.cinp / kBlockK, nkb = L.kh * L.kw * cblocks;
+    const int8_t *wtile = p.wpack + (size_t)blockIdx.y * (size_t)nkb * b_bytes;
+    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    const uint32_t zp4 = (uint32_t)(L.zp_in & 0xFF) * 0x01010101u;
+    const uint4 zpv = make_uint4(zp4, zp4, zp4, zp4);
+    bool ok = true;
+
+    for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % kStages, use = kb / kStages;
+        const uint32_t stage = sbase + (uint32_t)s * stage_bytes;
+        // the MMAs that read this stage last have completed
+        if (kb >= kStages && ok && !abort_s) ok = wait_bar(smem_u32(&bar_free[s]), (uint32_t)(use - 1) & 1u);
+        if (tid == 0) {
+            mbar_expect_tx(smem_u32(&bar_w[s]), b_bytes);
+            bulk_g2s(stage + a_bytes, wtile + (size_t)kb * b_bytes, b_bytes, smem_u32(&bar_w[s]));
+        }
+        const int tap = kb / cblocks, cb = kb - tap * cblocks;
+        const int r = tap / L.kw, sx = tap - r * L.kw;
+        const int iy = oy * L.stride + r - L.pad, ix = ox * L.stride + sx - L.pad;
+        const bool inside = valid && iy >= 0 && iy < L.hin && ix >= 0 && ix < L.win;
+        uint4 v0 = zpv, v1 = zpv, v2 = zpv, v3 = zpv;          // taps outside the image read the input zero-point
+        if (inside) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.in + ((b * L.hin + iy) * L.win + ix) * L.cinp + cb * kBlockK);
+            v0 = __ldg(src); v1 = __ldg(src + 1); v2 = __ldg(src + 2); v3 = __ldg(src + 3);
+        }
+        // K-major core matrices: 16-byte column j of row r at j * (128 rows * 16) + r * 16
+        st_shared_v4(stage + 0 * 2048 + tid * 16, v0);
+        st_shared_v4(stage + 1 * 2048 + tid * 16, v1);
+        st_shared_v4(stage + 2 * 2048 + tid * 16, v2);
+        st_shared_v4(stage + 3 * 2048 + tid * 16, v3);
+        fence_proxy_async();
+        __syncthreads();
+        if (tid == 0) {
+            if (ok && !abort_s) ok = wait_bar(smem_u32(&bar_w[s]), (uint32_t)use & 1u);
+            tc_fence_after();
+            if (ok) {
+#pragma unroll
+                for (int k2 = 0; k2 < 2; ++k2) {
+                    const uint64_t ad = make_desc(stage + (uint32_t)k2 * 4096u, 2048u, 128u);
+                    const uint64_t bd = make_desc(stage + a_bytes + (uint32_t)k2 * 2u * (uint32_t)n_tile * 16u, (uint32_t)n_tile * 16u, 128u);
+                    mma_i8(tmem, ad, bd, idesc, (kb > 0 || k2 > 0) ? 1u : 0u);
+                }
+            }
+            commit_to(smem_u32(&bar_free[s]));
+        }
+        if (!ok) abort_s = 1;
+    }
+    if (tid == 0) commit_to(smem_u32(&bar_done));
+    if (ok && !abort_s) ok = wait_bar(smem_u32(&bar_done), 0);
+    if (!ok) { abort_s = 1; atomicCAS(p.err, 0, 1 + (int)blockIdx.x); }
+    tc_fence_after();
+    __syncthreads();
+    if (!abort_s) {
+        const int8_t *res_px = (p.res && valid) ? p.res + (size_t)m * L.coutp : nullptr;
+        for (int c0 = 0; c0 < n_tile; c0 += 16) {
+            int acc[16];
+            tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc);
+            if (valid && n0 + c0 < L.coutp) {
+#pragma unroll
+                for (int o = 0; o < 16; ++o) acc[o] += __ldg(L.bias + n0 + c0 + o);
+                const uint4 v = epilogue16(acc, L, n0 + c0, res_px);
+                *reinterpret_cast<uint4 *>(p.out + (size_t)m * L.coutp + n0 + c0) = v;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc(tmem, (uint32_t)p.tmem_cols);
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ host side
+
+int igemm_tile_n(const GLayer &G)
+{
+    if ((G.op != ISC_CONV2D && G.op != ISC_FC) || G.cinp % kBlockK != 0 || G.cin != G.cinp) return 0;
+    if (G.coutp % 256 == 0) return 256;
+    if (G.coutp % 128 == 0) return 128;
+    if (G.coutp % 64 == 0) return 64;
+    return 0;
+}
+
+size_t igemm_pack_bytes(const GLayer &G)
+{
+    return (size_t)G.coutp * (size_t)(G.kh * G.kw) * (size_t)G.cinp;
+}
+
+// w: [cout][cin][kh][kw] as the model gives it -> [cout tile][tap][cin block][4 columns of 16 channels][n_tile rows][16]
+void igemm_pack_weights(const GLayer &G, const int8_t *w, int8_t *out)
+{
+    const int n_tile = igemm_tile_n(G), taps = G.kh * G.kw, cblocks = G.cinp / kBlockK;
+    size_t at = 0;
+    for (int t = 0; t < G.coutp / n_tile; ++t)
+        for (int tap = 0; tap < taps; ++tap)
+            for (int cb = 0; cb < cblocks; ++cb)
+                for (int j = 0; j < 4; ++j)
+                    for (int n = 0; n < n_tile; ++n)
+                        for (int e = 0; e < 16; ++e, ++at) {
+                            const int oc = t * n_tile + n, ci = cb * kBlockK + j * 16 + e;
+                            out[at] = (oc < G.cout && ci < G.cin) ? w[((size_t)oc * G.cin + ci) * taps + tap] : (int8_t)0;
+                        }
+}
+
+cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, int batch, const int8_t *in, const int8_t *res,
+                              int8_t *out, int32_t *err, cudaStream_t st)
+{
+    IgemmParams p;
+    p.L = G;
+    p.batch = batch;
+    p.n_tile = igemm_tile_n(G);
+    if (p.n_tile == 0) return cudaErrorInvalidValue;
+    p.tmem_cols = p.n_tile < 32 ? 32 : p.n_tile;
+    p.m_total = (long long)batch * G.hout * G.wout;
+    p.in = in; p.res = res; p.out = out; p.wpack = wpack; p.err = err;
+    const size_t smem = (size_t)kStages * ((size_t)kTileM * kBlockK + (size_t)p.n_tile * kBlockK);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_igemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kStages * (kTileM + 256) * kBlockK));
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const long long tiles_m = (p.m_total + kTileM - 1) / kTileM;
+    if (tiles_m <= 0) return cudaSuccess;
+    dim3 grid((unsigned)tiles_m, (unsigned)(G.coutp / p.n_tile));
+    k_igemm<<<grid, kThreads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace isc

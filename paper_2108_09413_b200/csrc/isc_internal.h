@@ -64,6 +64,16 @@ cudaError_t launch_maxpool(const GLayer &L, int batch, const int8_t *in, int8_t 
 cudaError_t launch_votes(const int8_t *logits_nhwc, int cp, int n_classes, int batch, int32_t *counts,
                          int8_t *logits_out, cudaStream_t st);
 
+// ---- layer-by-layer tensor-core convolutions (isc_igemm.cu) ----
+// Output-channel tile of the implicit-GEMM kernel for this layer (64, 128 or 256), or 0 when the layer does not fit
+// it (input channels not a multiple of 64, output channels not a multiple of 64, pools).
+int igemm_tile_n(const GLayer &G);
+size_t igemm_pack_bytes(const GLayer &G);
+void igemm_pack_weights(const GLayer &G, const int8_t *w_oihw, int8_t *out);
+// `err` (device) receives a non-zero word if a bounded wait inside the kernel expired.
+cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, int batch, const int8_t *in, const int8_t *res,
+                              int8_t *out, int32_t *err, cudaStream_t st);
+
 // ---- host decision rules (isc_decide.cpp) ----
 double lower_conf_bound(int64_t k, int64_t n, double alpha);
 double normal_quantile(double p);

@@ -116,9 +116,74 @@ def test_resnet110_logits_and_prefix_counts():
 
 
 def test_resnet50_logits():
+    """Config 3 (Sec. 4.1: ResNet-50 on 3 x 224 x 224 inputs, 101 classes): 64 samples on the tensor-core
+    layer-by-layer engine (the automatic choice), a few on the plain one."""
     cfg = wl.CONFIGS[3]
     x = wl.images(1, seed=cfg["image_seed"], shape=cfg["shape"])[0]
-    _logit_parity(cfg["model"](), x, 0, 1, 0, 6, 0.5, engines={"auto": 0})
+    model = cfg["model"]()
+    gm = isc.Model(model)
+    assert gm.get_info("has_tensor_core_layers") == 1
+    gm.sample_counts(x, SEED, 0, 1, 0, 2, 0.5)
+    assert gm.get_info("engine") == 2
+    gm.close()
+    _logit_parity(model, x, 0, 1, 0, 64, 0.5, engines={"auto": 0})
+    _logit_parity(model, x, 0, 1, 61, 6, 0.5, engines={"layerwise": 1, "tensorcore": 2})
+
+
+def test_resnet50_every_tensor_on_the_tensor_core_engine():
+    from concurrent.futures import ThreadPoolExecutor
+    cfg = wl.CONFIGS[3]
+    x = wl.images(2, seed=cfg["image_seed"], shape=cfg["shape"])[1]
+    model = cfg["model"]()
+    gm, om = _pair(model)
+    gm.set_option("engine", 2)
+    sizes = _tensor_sizes(om)
+    a0 = oracle.noisy_input(x, SEED, 1, 1, 5, 0.5)
+    with ThreadPoolExecutor(16) as pool:          # one oracle forward per tensor; the C call releases the GIL
+        expected = list(pool.map(lambda k: oracle.forward(om, a0, dump_tensor=k)[1], range(1, om.n_layers + 1)))
+    for k in range(1, om.n_layers + 1):
+        got = gm.debug_tensor(x, SEED, 1, 1, 5, 0.5, k, sizes[k])
+        bad = np.nonzero(got != expected[k - 1])[0]
+        assert bad.size == 0, f"tensor {k}: {bad.size} of {got.size} differ, first at {bad[:8]}"
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_bottleneck_nets_on_the_tensor_core_engine(seed):
+    """Small bottleneck networks with ragged sizes, strides, every zero-point and shift, residual rescales of all
+    allowed shifts: the implicit-GEMM kernel's tiles end inside rows and images, its padding is a non-trivial
+    zero-point."""
+    rng = np.random.default_rng(900 + seed)
+    h, w = int(rng.integers(9, 23)), int(rng.integers(2, 6)) * 4
+    zp = lambda: int(rng.integers(-128, 128))
+    c0, c1 = int(rng.choice([64, 128])), int(rng.choice([64, 128, 256]))
+    z = [int(rng.integers(0, 256)), zp(), zp(), zp(), zp(), zp()]
+    L = [_rand_conv(rng, 0, 3, c0, 3, 1, 1, 1, z[0], z[1]),
+         _rand_conv(rng, 1, c0, c0, 1, 1, 0, int(rng.integers(0, 2)), z[1], z[2]),
+         _rand_conv(rng, 2, c0, c0, 3, 2, 1, int(rng.integers(0, 2)), z[2], z[3]),
+         _rand_conv(rng, 1, c0, c1, 1, 2, 0, 0, z[1], z[4])]
+    L.append(_rand_conv(rng, 3, c0, c1, 1, 1, 0, 1, z[3], z[5], res_tensor=4, zp_res=z[4]))
+    L.append(_rand_conv(rng, 5, c1, c1, 3, 1, 1, 1, z[5], z[1], res_tensor=5, zp_res=z[5]))
+    model = dict(in_shape=(3, h, w), n_classes=5, layers=L)
+    om_tmp = oracle.Model(dict(model, n_classes=1))
+    hw = oracle.tensor_size(om_tmp, 6) // c1
+    L.append(wl._gavgpool(6, c1, hw, z[1]))
+    fc = _rand_conv(rng, 7, c1, 5, 1, 1, 0, 0, z[1], zp())
+    fc["op"] = wl.OP_FC
+    L.append(fc)
+    gm, om = _pair(model)
+    gm.set_option("engine", 2)
+    x = rng.integers(0, 256, (3, h, w)).astype(np.uint8)
+    sizes = _tensor_sizes(om)
+    a0 = oracle.noisy_input(x, 5, seed, 1, 2, 0.25)
+    for k in range(1, om.n_layers + 1):
+        _, exp = oracle.forward(om, a0, dump_tensor=k)
+        got = gm.debug_tensor(x, 5, seed, 1, 2, 0.25, k, sizes[k])
+        np.testing.assert_array_equal(got, exp, err_msg=f"tensor {k}")
+    ec, el = oracle.sample_counts(om, x, 5, seed, 1, 0, 37, 0.25, want_logits=True)
+    gc, gl = gm.sample_counts(x, 5, seed, 1, 0, 37, 0.25, want_logits=True)
+    assert gm.get_info("engine") == 2
+    np.testing.assert_array_equal(gl, el)
+    np.testing.assert_array_equal(gc, ec)
 
 
 def test_partition_and_batch_invariance():
