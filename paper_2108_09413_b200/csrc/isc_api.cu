@@ -45,6 +45,8 @@ struct isc_model {
     std::vector<GLayer> glayers;
     std::vector<void *> param_allocs;
     std::vector<const int8_t *> wpacks;         // per layer: repacked weights of the tensor-core convolution, or null
+    std::vector<const int32_t *> tc_cst;        // per layer: its epilogue constants
+    std::vector<char> tc_fast;
     bool has_tc = false;
     int32_t *d_tc_err = nullptr;
 
@@ -199,6 +201,8 @@ int build_generic_engine(isc_model *m)
 
     m->glayers.resize((size_t)n);
     m->wpacks.assign((size_t)n, nullptr);
+    m->tc_cst.assign((size_t)n, nullptr);
+    m->tc_fast.assign((size_t)n, 0);
     for (int i = 0; i < n; ++i) {
         const HostLayer &H = m->layers[(size_t)i];
         const isc_layer &L = H.d;
@@ -248,6 +252,9 @@ int build_generic_engine(isc_model *m)
                 std::vector<int8_t> wp(igemm_pack_bytes(G));
                 igemm_pack_weights(G, H.w.data(), wp.data());
                 rc = upload(m, wp, &m->wpacks[(size_t)i]); if (rc) return rc;
+                std::vector<int32_t> c4((size_t)G.coutp * 4);
+                m->tc_fast[(size_t)i] = igemm_constants(G, bias.data(), mult.data(), shift.data(), c4.data()) ? 1 : 0;
+                rc = upload(m, c4, &m->tc_cst[(size_t)i]); if (rc) return rc;
                 m->has_tc = true;
             }
         }
@@ -388,7 +395,7 @@ int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int
         const int8_t *res = L.res_tensor >= 0 ? (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.res_tensor]].p : nullptr;
         cudaError_t e;
         if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, batch, out, st);
-        else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], batch, in, res, out, m->d_tc_err, st);
+        else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], m->tc_cst[(size_t)i], m->tc_fast[(size_t)i] != 0, batch, in, res, out, m->d_tc_err, st);
         else if (L.op == ISC_CONV2D || L.op == ISC_FC) e = launch_conv(G, batch, in, res, out, st);
         else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, batch, in, out, st);
         else e = launch_maxpool(G, batch, in, out, st);

@@ -40,6 +40,10 @@ struct IgemmParams {
     const int8_t *in, *res;
     int8_t *out;
     const int8_t *wpack;                     // [cout tile][tap][cin block][4 K columns][n_tile rows][16 bytes]
+    const int4 *cst;                         // per output channel: folded bias, multiplier, rounding addend, shift - 1
+    int fast_requant, fast_residual, lo;     // every shift >= 2; residual rescale by 2^-31 or 2^-32; lower clamp
+    uint32_t res_m2;                         // residual multiplier and addend in the 2^-32 form (see requant16_fast)
+    long long res_r2;
     int32_t *err;
 };
 
@@ -52,6 +56,45 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t
 __device__ __forceinline__ void commit_to(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ long long mul_wide(int a, int b)
+{
+    long long d;
+    asm("mul.wide.s32 %0, %1, %2;" : "=l"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ long long mad_wide_u(uint32_t a, uint32_t b, long long c)
+{
+    long long d;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return d;
+}
+
+// 16 accumulators -> 16 int8 outputs with 32-bit arithmetic.  With s = shift - 1 >= 1,
+//   rs((acc + bias) * mult, 31 + shift) + zp_out = (hi32((acc + bias) * mult) + c) >> s,  c = 2^(s-1) + zp_out * 2^s,
+// exactly (the rounding half 2^(31+s) is a multiple of 2^32, so the product's low word cannot change the floor), and
+//   rs((r - zp_res) * res_mult, n) = hi32(u * m2 + R2),  u = r + 128, m2 = res_mult * 2^(32-n), n = 31 or 32,
+// with R2 = (2^(n-1) - (128 + zp_res) * res_mult) * 2^(32-n).  `cst` points at this block's constants in shared memory.
+template <bool kRes>
+__device__ __forceinline__ uint4 requant16_fast(const int *acc, uint32_t cst, uint4 rv, uint32_t m2, long long r2, int lo)
+{
+    const uint32_t rw[4] = {rv.x ^ 0x80808080u, rv.y ^ 0x80808080u, rv.z ^ 0x80808080u, rv.w ^ 0x80808080u};
+    uint32_t packed[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        int y[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int4 c;
+            asm("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(c.x), "=r"(c.y), "=r"(c.z), "=r"(c.w) : "r"(cst + (4 * g + k) * 16));
+            int v = (hi32(mul_wide(acc[4 * g + k] + c.x, c.y)) + c.z) >> c.w;
+            if (kRes) v += hi32(mad_wide_u((rw[g] >> (8 * k)) & 0xFFu, m2, r2));
+            y[k] = max(v, lo);
+        }
+        packed[g] = pack4_sat(y[0], y[1], y[2], y[3]);
+    }
+    return make_uint4(packed[0], packed[1], packed[2], packed[3]);
 }
 
 // Bounded wait for a phase of an mbarrier; false after the limit (the caller raises the error word).
@@ -72,6 +115,7 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
     __shared__ unsigned long long bar_w[kStages], bar_free[kStages], bar_done;
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_s;
+    __shared__ __align__(16) int4 cst_s[256];
     const GLayer &L = p.L;
     const int tid = threadIdx.x, warp = tid >> 5;
     const uint32_t sbase = smem_u32(smem);
@@ -83,6 +127,7 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
         abort_s = 0;
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_base_s), (uint32_t)p.tmem_cols);
+    for (int i = tid; i < n_tile; i += kThreads) cst_s[i] = __ldg(p.cst + blockIdx.y * n_tile + i);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
     tc_fence_before();
@@ -155,9 +200,16 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
             int acc[16];
             tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc);
             if (valid && n0 + c0 < L.coutp) {
+                uint4 v;
+                if (p.fast_requant && (!res_px || p.fast_residual)) {
+                    const uint32_t cst = smem_u32(cst_s + c0);
+                    if (res_px) v = requant16_fast<true>(acc, cst, __ldg(reinterpret_cast<const uint4 *>(res_px + n0 + c0)), p.res_m2, p.res_r2, p.lo);
+                    else v = requant16_fast<false>(acc, cst, make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
+                } else {
 #pragma unroll
-                for (int o = 0; o < 16; ++o) acc[o] += __ldg(L.bias + n0 + c0 + o);
-                const uint4 v = epilogue16(acc, L, n0 + c0, res_px);
+                    for (int o = 0; o < 16; ++o) acc[o] += __ldg(L.bias + n0 + c0 + o);
+                    v = epilogue16(acc, L, n0 + c0, res_px);
+                }
                 *reinterpret_cast<uint4 *>(p.out + (size_t)m * L.coutp + n0 + c0) = v;
             }
         }
@@ -202,11 +254,37 @@ void igemm_pack_weights(const GLayer &G, const int8_t *w, int8_t *out)
                         }
 }
 
-cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, int batch, const int8_t *in, const int8_t *res,
-                              int8_t *out, int32_t *err, cudaStream_t st)
+// Per output channel {folded bias, multiplier, rounding addend, shift - 1}; returns whether every shift is >= 2 (the
+// condition of the 32-bit form).  `bias_folded`, `mult`, `shift` are the layer's host arrays padded to coutp.
+bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t *mult, const int32_t *shift, int32_t *out4)
+{
+    bool fast = true;
+    for (int o = 0; o < G.coutp; ++o) {
+        const int s = shift[o] - 1;
+        if (s < 1) fast = false;
+        out4[4 * o + 0] = bias_folded[o];
+        out4[4 * o + 1] = mult[o];
+        out4[4 * o + 2] = s >= 1 ? (1 << (s - 1)) + G.zp_out * (1 << s) : 0;
+        out4[4 * o + 3] = s >= 1 ? s : 0;
+    }
+    return fast;
+}
+
+cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, int batch, const int8_t *in,
+                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st)
 {
     IgemmParams p;
     p.L = G;
+    p.cst = reinterpret_cast<const int4 *>(cst);
+    p.fast_requant = fast ? 1 : 0;
+    p.lo = G.relu ? (G.zp_out > -128 ? G.zp_out : -128) : -128;
+    const int res_n = 31 - G.res_shift;
+    p.fast_residual = (res_n == 31 || res_n == 32) ? 1 : 0;
+    p.res_m2 = 0; p.res_r2 = 0;
+    if (res && p.fast_residual) {
+        p.res_m2 = (uint32_t)((unsigned long long)(uint32_t)G.res_mult << (32 - res_n));
+        p.res_r2 = ((1ll << (res_n - 1)) - (128ll + G.zp_res) * (long long)G.res_mult) * (1ll << (32 - res_n));
+    }
     p.batch = batch;
     p.n_tile = igemm_tile_n(G);
     if (p.n_tile == 0) return cudaErrorInvalidValue;

@@ -70,9 +70,13 @@ cudaError_t launch_votes(const int8_t *logits_nhwc, int cp, int n_classes, int b
 int igemm_tile_n(const GLayer &G);
 size_t igemm_pack_bytes(const GLayer &G);
 void igemm_pack_weights(const GLayer &G, const int8_t *w_oihw, int8_t *out);
-// `err` (device) receives a non-zero word if a bounded wait inside the kernel expired.
-cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, int batch, const int8_t *in, const int8_t *res,
-                              int8_t *out, int32_t *err, cudaStream_t st);
+// Per-channel requantisation constants of the kernel's 32-bit epilogue (4 x int32 per padded output channel); returns
+// whether the layer qualifies for it (every shift >= 2).
+bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t *mult, const int32_t *shift, int32_t *out4);
+// `cst` / `fast`: what igemm_constants produced (device copy).  `err` (device) receives a non-zero word if a bounded
+// wait inside the kernel expired.
+cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, int batch, const int8_t *in,
+                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st);
 
 // ---- host decision rules (isc_decide.cpp) ----
 double lower_conf_bound(int64_t k, int64_t n, double alpha);
