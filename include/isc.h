@@ -224,6 +224,32 @@ int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_
 int isc_radius_integer(double sigma, uint32_t p_fx, int32_t *out_q, int64_t *out_q_squared);
 
 /*
+ * isc_certify_integer / isc_decide_certify_integer -- Algorithm 1 with the radius in the
+ * integer form of Theorem 3.2 (steps 2-3): class selection, vote count and the confidence
+ * bound p_A are Algorithm 1's (steps 1-6); the radius is then read off the cumulative table
+ * of the one-dimensional discrete Gaussian N_Z(0, (255 sigma)^2) (isc_noise_table) at
+ * floor(p_A * 2^32) instead of the normal quantile.
+ *   two_sided = 0 : out_q = Phi^-1_{N_H}(p_A) in pixel levels (q / 255 is the radius in the
+ *                   units of sigma), out_q_squared = q^2, the squared l2 radius the theorem
+ *                   compares integer perturbations with.
+ *   two_sided = 1 : Theorem 3.1's radius (sigma / 2)(Phi^-1(p_A^lb) - Phi^-1(p_B^ub)), with
+ *                   p_B^ub the one-sided (1 - alpha) Clopper-Pearson upper bound of the
+ *                   runner-up's votes: out_q = q_A - q_B (TWICE the radius, so that it stays an
+ *                   integer), out_q_squared = (q_A - q_B)^2 (four times the squared radius).
+ *                   Each bound holds with probability 1 - alpha on its own.
+ * ABSTAIN (class -1, q = 0) when p_A <= 1/2, or two-sided when p_A^lb < p_B^ub.
+ * isc_decide_certify_integer does the host part on given counts (no GPU work); arguments as
+ * isc_decide_certify.  out_q_squared, out_counts0, out_counts may be NULL.
+ */
+int isc_certify_integer(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id,
+                        int64_t N0, int64_t N, double sigma, double alpha, int two_sided,
+                        void *cuda_stream, int32_t *out_class, int32_t *out_q, int64_t *out_q_squared,
+                        int32_t *out_counts0, int32_t *out_counts);
+int isc_decide_certify_integer(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N,
+                               double sigma, double alpha, int two_sided, int32_t *out_class,
+                               int32_t *out_q, int64_t *out_q_squared);
+
+/*
  * isc_certified_metrics -- Certified Percentage and Certified Accuracy over a set of
  * certification results (Sec. 4.1, Evaluation Metrics, the two displayed equations); host only.
  *   classes, radii : what isc_certify returned for n inputs (class -1 = ABSTAIN), host arrays [n]

@@ -94,6 +94,9 @@ def lib():
         L.orc_predict_decide.restype = C.c_int32
         L.orc_dgauss_quantile_fx.argtypes = [C.c_uint32, C.c_void_p, C.c_int32]
         L.orc_dgauss_quantile_fx.restype = C.c_int32
+        L.orc_certify_integer_decide.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double, C.c_double,
+                                                 C.c_int, i32p, C.POINTER(C.c_int64)]
+        L.orc_certify_integer_decide.restype = C.c_int32
         L.orc_certify.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                   C.c_void_p, C.c_uint64, C.c_uint64, C.c_int64, C.c_int64,
                                   C.c_double, C.c_double, i32p, C.POINTER(C.c_double),
@@ -269,6 +272,17 @@ def predict_decide(counts, alpha):
 def dgauss_quantile_fx(p_fx, cum):
     T = (len(cum) - 1) // 2
     return int(lib().orc_dgauss_quantile_fx(int(p_fx), _ptr(cum), T))
+
+
+def certify_integer_decide(counts0, counts, N, sigma, alpha, two_sided=False):
+    """(class, q, q2): Algorithm 1's decision with the radius read off the discrete Gaussian's CDF table
+    (Theorem 3.2 steps 2-3); two_sided: Theorem 3.1's form, q = twice the radius in pixel levels."""
+    c0 = np.ascontiguousarray(counts0, dtype=np.int32)
+    c1 = np.ascontiguousarray(counts, dtype=np.int32)
+    q, q2 = C.c_int32(), C.c_int64()
+    cls = lib().orc_certify_integer_decide(_ptr(c0), _ptr(c1), c0.size, int(N), float(sigma), float(alpha),
+                                           int(bool(two_sided)), C.byref(q), C.byref(q2))
+    return int(cls), q.value, q2.value
 
 
 def certify(m: Model, x_u8, seed, image_id, N0, N, sigma, alpha):

@@ -546,6 +546,51 @@ int32_t orc_dgauss_quantile_fx(uint32_t p_fx, const uint32_t *cum, int32_t T)
     return T;
 }
 
+/* The integer-only form of the certification result (Theorem 3.2 steps 2-3; Theorem 3.1).
+ * Selection and the confidence bound are Algorithm 1's (steps 2, 4, 5, 6); the radius is then read off the
+ * precomputed CDF of the one-dimensional discrete Gaussian instead of the normal quantile:
+ *   one-sided  (two_sided = 0): q = Phi^-1_{N_H}(p_A) in pixel levels; returns q and q^2 (squared radius);
+ *   two-sided  (two_sided = 1): Theorem 3.1's radius (sigma/2)(Phi^-1(p_A^lb) - Phi^-1(p_B^ub)) with p_B^ub the
+ *              Clopper-Pearson upper bound of the runner-up's count; returns d = q_A - q_B (twice the radius, so that
+ *              it stays an integer) and d^2 (four times the squared radius).
+ * ABSTAIN (-1, 0, 0) when p_A <= 1/2 (Algorithm 1 step 6), or two-sided when p_A^lb < p_B^ub (Theorem 3.1's premise).
+ * Probabilities enter the table as floor(p * 2^32).                                                              */
+int32_t orc_certify_integer_decide(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N,
+                                   double sigma, double alpha, int two_sided, int32_t *out_q, int64_t *out_q2)
+{
+    *out_q = 0; *out_q2 = 0;
+    int32_t cA = orc_argmax(counts0, n_classes);
+    double pA = orc_lower_conf_bound(counts[cA], N, alpha);
+    if (!(pA > 0.5)) return -1;
+    int32_t T = orc_dgauss_halfwidth(sigma);
+    uint32_t *cum = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(2 * T + 1));
+    orc_dgauss_table(sigma, cum);
+    double scaled = floor(pA * 4294967296.0);
+    uint32_t pfx = scaled >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)scaled;
+    int32_t qA = orc_dgauss_quantile_fx(pfx, cum, T);
+    int32_t result = cA;
+    if (!two_sided) {
+        *out_q = qA;
+        *out_q2 = (int64_t)qA * qA;
+    } else {
+        int64_t nB = 0;
+        for (int c = 0; c < n_classes; ++c)
+            if (c != cA && counts[c] > nB) nB = counts[c];
+        double pB = 1.0 - orc_lower_conf_bound(N - nB, N, alpha);     /* upper bound of n_B out of N */
+        if (pA < pB) {
+            result = -1;
+        } else {
+            double sb = floor(pB * 4294967296.0);
+            uint32_t pbfx = sb >= 4294967295.0 ? 0xFFFFFFFFu : (sb < 0.0 ? 0u : (uint32_t)sb);
+            int32_t qB = orc_dgauss_quantile_fx(pbfx, cum, T);
+            *out_q = qA - qB;
+            *out_q2 = (int64_t)(qA - qB) * (qA - qB);
+        }
+    }
+    free(cum);
+    return result;
+}
+
 /* Whole CERTIFY (Algorithm 1) for one image; counts vectors may be NULL.       */
 int orc_certify(const orc_layer *layers, int n_layers, int in_c, int in_h, int in_w,
                 int n_classes, const uint8_t *x, uint64_t seed, uint64_t image_id,

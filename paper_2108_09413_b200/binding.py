@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
 EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_plan_resident", "isc_predict", "isc_certify", "isc_certify_batch",
-           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_noise_table", "isc_radius_integer", "isc_certified_metrics",
+           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_certify_integer", "isc_decide_certify_integer", "isc_noise_table", "isc_radius_integer", "isc_certified_metrics",
            "isc_debug_tensor", "isc_set_option", "isc_get_info", "isc_strerror"]
 
 
@@ -56,6 +56,10 @@ def lib():
                                                C.c_double, vp, vp]
         L.isc_decide_certify.argtypes = [vp, vp, C.c_int, C.c_int64, C.c_double, C.c_double, i32p, f64p, f64p]
         L.isc_decide_predict.argtypes = [vp, C.c_int, C.c_double, i32p]
+        L.isc_decide_certify_integer.argtypes = [vp, vp, C.c_int, C.c_int64, C.c_double, C.c_double, C.c_int, i32p, i32p,
+                                                 C.POINTER(C.c_int64)]
+        L.isc_certify_integer.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int64, C.c_int64, C.c_double, C.c_double,
+                                          C.c_int, vp, i32p, i32p, C.POINTER(C.c_int64), vp, vp]
         L.isc_noise_table.argtypes = [C.c_double, vp, C.c_int64, i32p]
         L.isc_radius_integer.argtypes = [C.c_double, C.c_uint32, i32p, C.POINTER(C.c_int64)]
         L.isc_certified_metrics.argtypes = [vp, vp, vp, C.c_int64, vp, C.c_int, C.POINTER(C.c_double), vp]
@@ -190,6 +194,17 @@ class Model:
                "isc_certify")
         return cls.value, rad.value, c0, c1
 
+    def certify_integer(self, x_u8, seed, image_id, N0, N, sigma, alpha, two_sided=False, stream=None):
+        """(class, q, q*q, counts0, counts): isc_certify_integer (Theorem 3.2 steps 2-3; Theorem 3.1 when two_sided)."""
+        x = self._x(x_u8)
+        cls, q, q2 = C.c_int32(), C.c_int32(), C.c_int64()
+        c0 = np.zeros(self.n_classes, dtype=np.int32)
+        c1 = np.zeros(self.n_classes, dtype=np.int32)
+        _check(lib().isc_certify_integer(self._h, _ptr(x), seed, image_id, N0, N, float(sigma), float(alpha),
+                                         int(bool(two_sided)), _stream_ptr(stream), C.byref(cls), C.byref(q), C.byref(q2),
+                                         _ptr(c0), _ptr(c1)), "isc_certify_integer")
+        return cls.value, q.value, q2.value, c0, c1
+
     def certify_batch(self, x_u8, n_images, seed, image_id0, N0, N, sigma, alpha, stream=None,
                       device_ptr=None):
         """x_u8: host array [n][C][H][W], or pass device_ptr (int) to read images resident on the GPU."""
@@ -222,6 +237,16 @@ def certify_decide(counts0, counts, N, sigma, alpha):
     _check(lib().isc_decide_certify(_ptr(c0), _ptr(c1), c0.size, int(N), float(sigma), float(alpha),
                                     C.byref(cls), C.byref(rad), C.byref(pl)), "isc_decide_certify")
     return cls.value, rad.value, pl.value
+
+
+def certify_integer_decide(counts0, counts, N, sigma, alpha, two_sided=False):
+    c0 = np.ascontiguousarray(counts0, dtype=np.int32)
+    c1 = np.ascontiguousarray(counts, dtype=np.int32)
+    cls, q, q2 = C.c_int32(), C.c_int32(), C.c_int64()
+    _check(lib().isc_decide_certify_integer(_ptr(c0), _ptr(c1), c0.size, int(N), float(sigma), float(alpha),
+                                            int(bool(two_sided)), C.byref(cls), C.byref(q), C.byref(q2)),
+           "isc_decide_certify_integer")
+    return cls.value, q.value, q2.value
 
 
 def predict_decide(counts, alpha):

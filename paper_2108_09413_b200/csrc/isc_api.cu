@@ -697,6 +697,41 @@ int isc_decide_certify(const int32_t *counts0, const int32_t *counts, int n_clas
     return ISC_OK;
 }
 
+int isc_decide_certify_integer(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N, double sigma,
+                               double alpha, int two_sided, int32_t *out_class, int32_t *out_q, int64_t *out_q_squared)
+{
+    if (!counts0 || !counts || !out_class || !out_q || n_classes < 1 || N < 1) return ISC_ERR_ARG;
+    if (!(alpha > 0.0 && alpha < 1.0) || !(sigma > 0.0) || !std::isfinite(sigma) || sigma > 64.0) return ISC_ERR_ARG;
+    for (int c = 0; c < n_classes; ++c)
+        if (counts0[c] < 0 || counts[c] < 0 || counts[c] > N) return ISC_ERR_ARG;
+    int32_t q = 0;
+    int64_t q2 = 0;
+    *out_class = decide_certify_integer(counts0, counts, n_classes, N, sigma, alpha, two_sided != 0, &q, &q2);
+    *out_q = q;
+    if (out_q_squared) *out_q_squared = q2;
+    return ISC_OK;
+}
+
+int isc_certify_integer(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t image_id, int64_t N0, int64_t N,
+                        double sigma, double alpha, int two_sided, void *cuda_stream, int32_t *out_class,
+                        int32_t *out_q, int64_t *out_q_squared, int32_t *out_counts0, int32_t *out_counts)
+{
+    if (!m || !x_u8 || !out_class || !out_q) return ISC_ERR_ARG;
+    const size_t C = (size_t)m->n_classes;
+    std::vector<int32_t> c0(C), c1(C);
+    int32_t cls = -1;
+    double radius = 0.0;
+    int rc = isc_certify_batch(m, x_u8, 0, 1, seed, image_id, N0, N, sigma, alpha, cuda_stream, &cls, &radius,
+                               c0.data(), c1.data());
+    if (rc) return rc;
+    rc = isc_decide_certify_integer(c0.data(), c1.data(), m->n_classes, N, sigma, alpha, two_sided, &cls, out_q, out_q_squared);
+    if (rc) return rc;
+    *out_class = cls;
+    if (out_counts0) memcpy(out_counts0, c0.data(), C * sizeof(int32_t));
+    if (out_counts) memcpy(out_counts, c1.data(), C * sizeof(int32_t));
+    return ISC_OK;
+}
+
 int isc_decide_predict(const int32_t *counts, int n_classes, double alpha, int32_t *out_class)
 {
     if (!counts || !out_class || n_classes < 1 || !(alpha > 0.0 && alpha < 1.0)) return ISC_ERR_ARG;

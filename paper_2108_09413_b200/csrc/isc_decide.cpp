@@ -1,6 +1,7 @@
 // Host side of Algorithm 1 (steps 2, 5-9) and Algorithm 2 (steps 2-6), and the cumulative
 // table of the noise law (Def. 3.3, Eq. 2).  IEEE doubles, fixed evaluation order, compiled
 // without contraction or fast-math so that the result is reproducible bit for bit.
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <vector>
@@ -93,6 +94,53 @@ int32_t decide_certify(const int32_t *counts0, const int32_t *counts, int n_clas
     }
     *radius = 0.0;                                          // step 8: ABSTAIN
     return -1;
+}
+
+namespace {
+
+// floor(p * 2^32) as the table's fixed-point probability, saturated to 32 bits
+uint32_t to_fixed32(double p)
+{
+    const double scaled = std::floor(p * 4294967296.0);
+    if (scaled <= 0.0) return 0u;
+    return scaled >= 4294967295.0 ? 4294967295u : (uint32_t)scaled;
+}
+
+// Theorem 3.2 step 2: the quantile of the discrete Gaussian by lookup, the first level whose cumulative entry reaches p
+int32_t table_quantile(const std::vector<uint32_t> &cum, uint32_t p_fx)
+{
+    const int32_t T = (int32_t)(cum.size() - 1) / 2;
+    const int32_t at = (int32_t)(std::lower_bound(cum.begin(), cum.end(), p_fx) - cum.begin());
+    return at > 2 * T ? T : at - T;
+}
+
+}  // namespace
+
+int32_t decide_certify_integer(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N, double sigma,
+                               double alpha, bool two_sided, int32_t *q, int64_t *q_squared)
+{
+    *q = 0; *q_squared = 0;
+    const int c_a = first_max(counts0, n_classes);           // Algorithm 1 steps 2, 4, 5, 6
+    const double p_a = lower_conf_bound(counts[c_a], N, alpha);
+    if (!(p_a > 0.5)) return -1;
+    std::vector<uint32_t> cum;
+    noise_table(sigma, cum);
+    const int32_t q_a = table_quantile(cum, to_fixed32(p_a));
+    if (!two_sided) {                                         // Theorem 3.2 steps 2-3: radius and squared radius in pixel levels
+        *q = q_a;
+        *q_squared = (int64_t)q_a * q_a;
+        return c_a;
+    }
+    // Theorem 3.1: the runner-up's upper bound enters as well; d = q_A - q_B is twice the radius
+    int64_t n_b = 0;
+    for (int c = 0; c < n_classes; ++c)
+        if (c != c_a && counts[c] > n_b) n_b = counts[c];
+    const double p_b = 1.0 - lower_conf_bound(N - n_b, N, alpha);
+    if (p_a < p_b) return -1;
+    const int32_t d = q_a - table_quantile(cum, to_fixed32(p_b));
+    *q = d;
+    *q_squared = (int64_t)d * d;
+    return c_a;
 }
 
 int32_t decide_predict(const int32_t *counts, int n_classes, double alpha)

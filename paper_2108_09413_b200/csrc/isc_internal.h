@@ -85,6 +85,8 @@ double binom_pvalue_half(int64_t n_a, int64_t m);
 int32_t decide_certify(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N,
                        double sigma, double alpha, double *radius, double *p_lower);
 int32_t decide_predict(const int32_t *counts, int n_classes, double alpha);
+int32_t decide_certify_integer(const int32_t *counts0, const int32_t *counts, int n_classes, int64_t N, double sigma,
+                               double alpha, bool two_sided, int32_t *q, int64_t *q_squared);
 int noise_halfwidth(double sigma);
 void noise_table(double sigma, std::vector<uint32_t> &cum);
 

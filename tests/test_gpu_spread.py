@@ -72,6 +72,24 @@ def test_spread_certify_and_predict_abstain_and_partial_radius(name, N):
     assert seen == {"abstain", "partial"}, seen
 
 
+def test_integer_certification_from_real_counts():
+    """isc_certify_integer (Theorem 3.2 steps 2-3, Theorem 3.1) from the votes of the GPU loop: counts, class, q and
+    q^2 equal the oracle's, for an abstaining image and for a majority that is not unanimous."""
+    x = wl.spread_image()
+    N = 4000
+    seen = set()
+    for boost in (0, BOOST["tiny_cnn"]):
+        model = wl.spread_model("tiny_cnn", boost=boost)
+        gm, om = isc.Model(model), oracle.Model(model)
+        _, _, ec0, ec1 = oracle.certify(om, x, SEED, 3, 100, N, 0.25, ALPHA)
+        for two in (False, True):
+            cls, q, q2, c0, c1 = gm.certify_integer(x, SEED, 3, 100, N, 0.25, ALPHA, two_sided=two)
+            np.testing.assert_array_equal(c0, ec0); np.testing.assert_array_equal(c1, ec1)
+            assert (cls, q, q2) == oracle.certify_integer_decide(ec0, ec1, N, 0.25, ALPHA, two)
+            seen.add(cls)
+    assert seen == {-1, 0}
+
+
 def test_resnet110_logits_where_a_cta_runs_several_groups():
     """One launch of 1776 samples = 444 groups of four: with one CTA per SM (148) every CTA carries three groups in
     turn.  Rows of the second and third turn are compared with the oracle; the counts of the whole launch follow from

@@ -159,3 +159,25 @@ def test_plan_resident_accepts_cifar_resnets_and_names_the_refusing_rule():
     model["layers"][1] = dict(model["layers"][1], cin=8)
     with pytest.raises(isc.IscError):
         isc.plan_resident(model)
+
+
+def test_integer_certify_decisions_equal_the_oracle():
+    rng = np.random.default_rng(11)
+    for _ in range(60):
+        n_classes = int(rng.integers(2, 12))
+        N = int(rng.choice([100, 1000, 100_000]))
+        top = int(rng.integers(N // 2 - N // 20, N + 1))
+        rest = rng.multinomial(N - top, np.ones(n_classes - 1) / (n_classes - 1))
+        counts = np.concatenate([[top], rest]).astype(np.int32)
+        rng.shuffle(counts)
+        counts0 = rng.integers(0, 50, n_classes).astype(np.int32)
+        sigma = float(rng.choice([0.12, 0.25, 0.5, 1.0]))
+        for two in (False, True):
+            assert isc.certify_integer_decide(counts0, counts, N, sigma, 0.001, two) == \
+                   oracle.certify_integer_decide(counts0, counts, N, sigma, 0.001, two)
+    L = isc.lib()
+    c = np.array([5, 5], np.int32)
+    cls, q = C.c_int32(7), C.c_int32(7)
+    assert L.isc_decide_certify_integer(c.ctypes.data, c.ctypes.data, 2, 10, 0.25, 1.5, 0, C.byref(cls), C.byref(q), None) == -1
+    assert L.isc_decide_certify_integer(c.ctypes.data, c.ctypes.data, 2, 4, 0.25, 0.001, 0, C.byref(cls), C.byref(q), None) == -1
+    assert (cls.value, q.value) == (7, 7)

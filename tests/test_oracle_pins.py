@@ -471,3 +471,44 @@ def test_workload_shapes():
     b = wl.images(2, seed=5)
     np.testing.assert_array_equal(a, b)
     assert a.dtype == np.uint8 and a.shape == (2, 3, 32, 32) and a.min() == 0 and a.max() == 255
+
+
+# ------------------------------------------------------------------ integer-only certification (Thm 3.2, Thm 3.1)
+
+def test_integer_certify_decide_against_the_normal_radius_and_symmetry():
+    """Theorem 3.2 steps 2-3: the table quantile q (pixel levels) must agree with Algorithm 1's sigma * Phi^-1(p_A)
+    within 1.5 levels once the lattice is fine (255 sigma >= 30), abstain exactly when Algorithm 1 abstains, grow with
+    the vote count; Theorem 3.1's two-sided form with a lone runner-up (n_B = N - n_A, so p_B^ub = 1 - p_A^lb) is the
+    symmetric quantile: q_A - q_B within one level of 2 q_A."""
+    N, alpha = 100_000, 0.001
+    for sigma in (0.12, 0.25, 0.5, 1.0):
+        prev_q = -1
+        for n_a in (50_000, 50_600, 52_000, 60_000, 80_000, 99_000, 99_990, N):
+            counts = [n_a, N - n_a, 0, 0]
+            cls, radius, p_l = oracle.certify_decide([7, 1, 0, 0], counts, N, sigma, alpha)
+            icls, q, q2 = oracle.certify_integer_decide([7, 1, 0, 0], counts, N, sigma, alpha)
+            assert icls == cls
+            if cls == -1:
+                assert (q, q2) == (0, 0)
+                continue
+            assert q2 == q * q and q >= prev_q
+            prev_q = q
+            assert abs(q / 255.0 - radius) <= 1.5 / 255.0, (sigma, n_a, q, radius)
+            tcls, d, d2 = oracle.certify_integer_decide([7, 1, 0, 0], counts, N, sigma, alpha, two_sided=True)
+            assert tcls == cls and d2 == d * d and abs(d - 2 * q) <= 1
+    # a runner-up weaker than the complement (votes spread over a third class): Theorem 3.1's radius exceeds
+    # Algorithm 1's, and equals the normal form (sigma / 2)(Phi^-1(p_A^lb) - Phi^-1(p_B^ub)) within the lattice step
+    from scipy.stats import norm
+    counts = [70_000, 29_000, 1_000, 0]
+    _, q, _ = oracle.certify_integer_decide([5, 1, 0, 0], counts, N, 0.5, alpha)
+    _, d, _ = oracle.certify_integer_decide([5, 1, 0, 0], counts, N, 0.5, alpha, two_sided=True)
+    p_a = oracle.lower_conf_bound(70_000, N, alpha)
+    p_b = 1.0 - oracle.lower_conf_bound(N - 29_000, N, alpha)
+    assert d > 2 * q
+    assert abs(d / 255.0 - 0.5 * (norm.ppf(p_a) - norm.ppf(p_b))) <= 3.0 / 255.0
+    # Theorem 3.1's premise fails (p_A^lb < p_B^ub) although Algorithm 1 would certify: cannot happen with p_A > 1/2
+    # and n_B <= N - n_A, so the two forms abstain together
+    for n_a in (50_100, 50_400):
+        counts = [n_a, N - n_a, 0, 0]
+        assert oracle.certify_integer_decide([3, 1, 0, 0], counts, N, 0.25, alpha, two_sided=True)[0] == \
+               oracle.certify_integer_decide([3, 1, 0, 0], counts, N, 0.25, alpha)[0]
