@@ -155,6 +155,9 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="noisy samples per launch (0: the library chooses)")
     ap.add_argument("--sigma", type=float, default=None, help="noise level (default: the workload's)")
     ap.add_argument("--samples", type=int, default=0, help="replace the workload's N (short case for profilers)")
+    ap.add_argument("--spread", action="store_true",
+                    help="the workload's network with the balanced final layer and its image (votes spread over the classes, "
+                         "so the host bound runs its bisection instead of the closed form of unanimous votes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -173,6 +176,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     cfg, model, sigma = workload(args.config, args.sigma)
+    if args.spread:
+        model = wl.spread_model(model["name"])
     gm = isc.Model(model)
     gm.set_option("engine", args.engine)
     ctx = dict(torch=torch, dist=dist, rank=rank, local_rank=local_rank, world=world, gm=gm, cfg=cfg, model=model)
@@ -234,6 +239,8 @@ def measure(ctx, args, sigma, batch, steps, warmup, ips, e2e_arm):
             ips = int(t.item())
     imgs = wl.images(ips * total_steps, shape=cfg["shape"], seed=cfg["image_seed"] + 7919 * rank)
     imgs = imgs.reshape(total_steps, ips, *cfg["shape"])
+    if args.spread:                      # the image the head was balanced on, under a different image id each time
+        imgs = np.broadcast_to(wl.spread_image(cfg["shape"]), imgs.shape).copy()
     dev_imgs = torch.from_numpy(imgs).cuda()
     pinned = torch.from_numpy(imgs).pin_memory()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
@@ -257,11 +264,22 @@ def measure(ctx, args, sigma, batch, steps, warmup, ips, e2e_arm):
             flush.zero_()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            step(i, host)
+            last_result[0] = step(i, host)
             e1.record(stream)
             e1.synchronize()
             total_ms += e0.elapsed_time(e1)
         return total_ms
+
+    last_result = [None]
+
+    def decide_ms():
+        """Host time of the bound and radius (Algorithm 1 steps 5-7) per image, on the counts of the last step."""
+        import paper_2108_09413_b200 as isc
+        _, _, c0, c1 = last_result[0]
+        t0 = time.perf_counter()
+        for i in range(len(c0)):
+            isc.certify_decide(c0[i], c1[i], N, sigma, alpha)
+        return 1e3 * (time.perf_counter() - t0) / max(1, len(c0))
 
     def phase_cycles():
         try:
@@ -296,6 +314,8 @@ def measure(ctx, args, sigma, batch, steps, warmup, ips, e2e_arm):
     achieved = 2.0 * macs * samples_per_step * steps / (ms * 1e-3) / 1e12   # per GPU
     engine = gm.get_info("engine")
     name = workload_name(args.config, model)
+    if args.spread:
+        name += " (spread-vote head)"
     if args.samples:
         name += f" (short case: N = {N} instead of {cfg['N']}; not a benchmark result)"
 
@@ -309,6 +329,7 @@ def measure(ctx, args, sigma, batch, steps, warmup, ips, e2e_arm):
                    "engine": {1: "layer-by-layer", 3: "resident tensor-core, line tiles"}.get(engine, str(engine)),
                    "l2": "flushed between steps (256 MiB write)", "macs_per_sample": macs},
         "certified_images_per_sec": value / (N0 + N),
+        "decide_ms_per_image": decide_ms(),
         "e2e": {"value": e2e, "unit": "samples/s", "h2d_bytes_per_step": int(ips * np.prod(cfg["shape"])),
                 "d2h_bytes_per_step": int(ips * 2 * model["n_classes"] * 4)},
         "gpu_launches": int(launches),

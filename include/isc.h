@@ -274,6 +274,20 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
                      int32_t *out, int64_t capacity);
 
 /*
+ * isc_debug_wait_timeout -- exercises the bounded-wait failure path of the resident engine
+ * without any failure: a one-thread kernel runs the engine's own wait code on a barrier and a
+ * counter that nothing ever completes, with `limit_ns` (1,000 .. 100,000,000) as the limit.
+ * The GPU keeps running; nothing faults or hangs.
+ *   returns : ISC_ERR_TIMEOUT when the path works as designed (the expired wait raised the
+ *             engine's error word, and reading it reported and cleared it); ISC_OK means the
+ *             wait did NOT expire; ISC_ERR_UNSUPPORTED if the model has no resident engine.
+ *   out4    : host, 4 int32: result of the first wait (0 = expired), result of the second wait
+ *             (0 = fell through because the abort flag was up), the abort flag, nanoseconds spent.
+ * The handle stays usable: the next call on it must succeed.
+ */
+int isc_debug_wait_timeout(isc_model *m, int64_t limit_ns, void *cuda_stream, int32_t *out4);
+
+/*
  * isc_set_option -- tuning knobs; none changes a result.
  *   "batch"  : noisy samples per launch (0 = choose automatically).
  *   "engine" : 0 = automatic (3 if the model fits it, else 2 if any layer fits it, else 1),

@@ -11,7 +11,7 @@ _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
 EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_plan_resident", "isc_predict", "isc_certify", "isc_certify_batch",
            "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_certify_integer", "isc_decide_certify_integer", "isc_noise_table", "isc_radius_integer", "isc_certified_metrics",
-           "isc_debug_tensor", "isc_set_option", "isc_get_info", "isc_strerror"]
+           "isc_debug_tensor", "isc_debug_wait_timeout", "isc_set_option", "isc_get_info", "isc_strerror"]
 
 
 class IscError(RuntimeError):
@@ -65,6 +65,7 @@ def lib():
         L.isc_certified_metrics.argtypes = [vp, vp, vp, C.c_int64, vp, C.c_int, C.POINTER(C.c_double), vp]
         L.isc_debug_tensor.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int32, C.c_int64, C.c_double,
                                        C.c_int, vp, vp, C.c_int64]
+        L.isc_debug_wait_timeout.argtypes = [vp, C.c_int64, vp, vp]
         L.isc_set_option.argtypes = [vp, C.c_char_p, C.c_int64]
         L.isc_get_info.argtypes = [vp, C.c_char_p, C.POINTER(C.c_int64)]
         L.isc_strerror.argtypes = [C.c_int]
@@ -221,6 +222,12 @@ class Model:
                                        float(alpha), _stream_ptr(stream), _ptr(cls), _ptr(rad), _ptr(c0),
                                        _ptr(c1)), "isc_certify_batch")
         return cls, rad, c0, c1
+
+    def debug_wait_timeout(self, limit_ns, stream=None):
+        """(status, [first wait, second wait, abort flag, ns]): isc_debug_wait_timeout; the status is returned, not raised."""
+        out = np.zeros(4, dtype=np.int32)
+        rc = lib().isc_debug_wait_timeout(self._h, int(limit_ns), _stream_ptr(stream), _ptr(out))
+        return rc, out.tolist()
 
     def debug_tensor(self, x_u8, seed, image_id, phase, j, sigma, tensor, size, stream=None):
         x = self._x(x_u8)

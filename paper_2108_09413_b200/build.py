@@ -22,7 +22,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC,-ffp-contract=off,-fno-fast-math,-Wall",
+           "-shared", "-Xcompiler", "-fPIC,-ffp-contract=off,-fno-fast-math,-Wall,-pthread",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]

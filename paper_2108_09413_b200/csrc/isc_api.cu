@@ -7,8 +7,10 @@
 #include <string.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <new>
+#include <thread>
 #include <vector>
 
 #include "isc.h"
@@ -65,6 +67,10 @@ struct isc_model {
     int cum_T = 0;
 
     isc::LinePlan *line = nullptr;
+
+    // isc_certify_batch: pinned copy of the vote counts, one event per image
+    int32_t *h_counts = nullptr;  size_t h_counts_bytes = 0;
+    std::vector<cudaEvent_t> events;
 
     int64_t opt_batch = 0, opt_engine = 0;
     int64_t last_engine = 0, launches = 0;
@@ -578,6 +584,8 @@ void isc_free_qmodel(isc_model *m)
     if (m->d_counts) cudaFree(m->d_counts);
     if (m->d_logits) cudaFree(m->d_logits);
     if (m->d_cum) cudaFree(m->d_cum);
+    if (m->h_counts) cudaFreeHost(m->h_counts);
+    for (cudaEvent_t ev : m->events) cudaEventDestroy(ev);
     isc::line_free(m->line);
     delete m;
 }
@@ -653,22 +661,69 @@ int isc_certify_batch(isc_model *m, const uint8_t *x_u8, int x_on_device, int n_
     const uint8_t *d_x;
     if ((rc = stage_image(m, x_u8, d * (size_t)n_images, x_on_device != 0, st, &d_x))) return rc;
     CK(cudaMemsetAsync(m->d_counts, 0, 2 * C * (size_t)n_images * sizeof(int32_t), st));
+    // Pinned staging for the counts and one event per image: the host bound of image i (Algorithm 1 steps 5-7, up to
+    // a hundred milliseconds of bisection at N = 100,000) runs on a worker thread while the kernels of the images
+    // after it are in flight.
+    const size_t need = 2 * C * (size_t)n_images * sizeof(int32_t);
+    if (m->h_counts_bytes < need) {
+        if (m->h_counts) cudaFreeHost(m->h_counts);
+        m->h_counts = nullptr; m->h_counts_bytes = 0;
+        CK(cudaHostAlloc((void **)&m->h_counts, need, cudaHostAllocDefault));
+        m->h_counts_bytes = need;
+    }
+    while ((int)m->events.size() < n_images) {
+        cudaEvent_t ev;
+        CK(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        m->events.push_back(ev);
+    }
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    std::vector<int32_t> cls((size_t)n_images, -1);
+    std::vector<double> rad((size_t)n_images, 0.0);
+    std::atomic<int> enqueued(0);
+    std::atomic<bool> failed(false);
+    int32_t *h = m->h_counts;
+    const int n_cls = m->n_classes;
+    // a few workers, image i on worker i mod n_workers: one bound can take longer than one image's kernels
+    const int n_workers = std::max(1, std::min(std::min(n_images, 4), (int)std::thread::hardware_concurrency()));
+    auto work = [&, dev, h, n_cls](int first) {
+        if (cudaSetDevice(dev) != cudaSuccess) { failed = true; return; }
+        for (int i = first; i < n_images; i += n_workers) {
+            while (enqueued.load(std::memory_order_acquire) <= i) {
+                if (failed.load()) return;
+                std::this_thread::yield();
+            }
+            if (cudaEventSynchronize(m->events[(size_t)i]) != cudaSuccess) { failed = true; return; }
+            const int32_t *c0 = h + (size_t)i * 2 * C, *c1 = c0 + C;
+            double radius = 0.0;
+            cls[(size_t)i] = decide_certify(c0, c1, n_cls, N, sigma, alpha, &radius, nullptr);
+            rad[(size_t)i] = radius;
+        }
+    };
+    std::vector<std::thread> workers;
+    for (int t = 0; t < n_workers; ++t) workers.emplace_back(work, t);
     for (int i = 0; i < n_images && rc == ISC_OK; ++i) {
         int32_t *c0 = m->d_counts + (size_t)i * 2 * C;
         rc = run_counts(m, d_x + (size_t)i * d, seed, image_id0 + (uint64_t)i, 0, 0, N0, st, c0, nullptr);
         if (rc == ISC_OK)
             rc = run_counts(m, d_x + (size_t)i * d, seed, image_id0 + (uint64_t)i, 1, 0, N, st, c0 + C, nullptr);
+        if (rc == ISC_OK && (cudaMemcpyAsync(h + (size_t)i * 2 * C, c0, 2 * C * sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+                             cudaEventRecord(m->events[(size_t)i], st) != cudaSuccess)) {
+            cudaGetLastError();
+            rc = ISC_ERR_CUDA;
+        }
+        if (rc == ISC_OK) enqueued.store(i + 1, std::memory_order_release);
     }
+    if (rc) failed = true;
+    for (std::thread &t : workers) t.join();
     if (rc) { cudaStreamSynchronize(st); return rc; }
-    std::vector<int32_t> h(2 * C * (size_t)n_images);
-    CK(cudaMemcpyAsync(h.data(), m->d_counts, h.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
+    if (failed.load()) return ISC_ERR_CUDA;
     if ((rc = check_engines(m))) return rc;
     for (int i = 0; i < n_images; ++i) {
-        const int32_t *c0 = h.data() + (size_t)i * 2 * C, *c1 = c0 + C;
-        double radius = 0.0;
-        out_class[i] = decide_certify(c0, c1, m->n_classes, N, sigma, alpha, &radius, nullptr);
-        out_radius[i] = radius;
+        const int32_t *c0 = h + (size_t)i * 2 * C, *c1 = c0 + C;
+        out_class[i] = cls[(size_t)i];
+        out_radius[i] = rad[(size_t)i];
         if (out_counts0) memcpy(out_counts0 + (size_t)i * C, c0, C * sizeof(int32_t));
         if (out_counts) memcpy(out_counts + (size_t)i * C, c1, C * sizeof(int32_t));
     }
@@ -831,6 +886,17 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
             for (int x = 0; x < s.w; ++x)
                 out[((size_t)c * s.h + y) * s.w + x] = h[((size_t)y * s.w + x) * s.cp + c];
     return ISC_OK;
+}
+
+int isc_debug_wait_timeout(isc_model *m, int64_t limit_ns, void *cuda_stream, int32_t *out4)
+{
+    if (!m || !out4) return ISC_ERR_ARG;
+    if (!m->line) return ISC_ERR_UNSUPPORTED;
+    int32_t tmp[4] = {0, 0, 0, 0};
+    const int rc = isc::line_wait_probe(m->line, limit_ns, tmp, (cudaStream_t)cuda_stream);
+    if (rc == ISC_ERR_ARG || rc == ISC_ERR_CUDA) return rc;
+    memcpy(out4, tmp, sizeof(tmp));
+    return rc;
 }
 
 }  // extern "C"

@@ -18,14 +18,15 @@ inline double log_choose(int64_t n, int64_t i)
     return std::lgamma((double)n + 1.0) - std::lgamma((double)i + 1.0) - std::lgamma((double)(n - i) + 1.0);
 }
 
-// P[Binomial(n, p) >= k], terms added for i = k, k+1, ..., n
-double upper_tail(int64_t k, int64_t n, double p)
+// P[Binomial(n, p) >= k], terms added for i = k, k+1, ..., n; log_c[i - k] = log_choose(n, i), computed once per
+// bound (the same value in the same place of the same expression, so the sum is what it was term by term)
+double upper_tail(int64_t k, int64_t n, double p, const std::vector<double> &log_c)
 {
     const double log_p = std::log(p);
     const double log_q = std::log1p(-p);
     double total = 0.0;
     for (int64_t i = k; i <= n; ++i)
-        total += std::exp(log_choose(n, i) + (double)i * log_p + (double)(n - i) * log_q);
+        total += std::exp(log_c[(size_t)(i - k)] + (double)i * log_p + (double)(n - i) * log_q);
     return total;
 }
 
@@ -45,10 +46,12 @@ double lower_conf_bound(int64_t k, int64_t n, double alpha)
 {
     if (k <= 0) return 0.0;
     if (k >= n) return std::exp(std::log(alpha) / (double)n);
+    std::vector<double> log_c((size_t)(n - k + 1));
+    for (int64_t i = k; i <= n; ++i) log_c[(size_t)(i - k)] = log_choose(n, i);
     double left = 0.0, right = (double)k / (double)n;
     for (int step = 0; step < 64; ++step) {
         const double mid = 0.5 * (left + right);
-        if (upper_tail(k, n, mid) < alpha)
+        if (upper_tail(k, n, mid, log_c) < alpha)
             left = mid;
         else
             right = mid;

@@ -243,6 +243,7 @@ __device__ __forceinline__ uint32_t ubyte(uint32_t w)
 struct Waiter {
     Ctrl *ctrl;
     int32_t *err;
+    unsigned long long limit_ns = kWaitLimitNs;
     __device__ __forceinline__ bool aborted() const { return ctrl->abort_flag != 0; }
     // the error word: wait kind | index of the barrier within the control block << 8 | parity waited for << 20 | CTA << 21
     __device__ __noinline__ void fail(int code, uint32_t bar, uint32_t parity)
@@ -262,7 +263,7 @@ struct Waiter {
             if (mbar_try(bar, parity)) return true;
             if ((spin & 7) == 7) {
                 if (aborted()) return false;
-                if (globaltimer() - t0 > kWaitLimitNs) { fail(code, bar, parity); return false; }
+                if (globaltimer() - t0 > limit_ns) { fail(code, bar, parity); return false; }
             }
         }
     }
@@ -278,7 +279,7 @@ struct Waiter {
             if ((int32_t)(ld_acquire_u32(addr) - expected) >= 0) return true;
             if ((spin & 15) == 15) {
                 if (aborted()) return false;
-                if (globaltimer() - t0 > kWaitLimitNs) { fail(code, addr, 0); return false; }
+                if (globaltimer() - t0 > limit_ns) { fail(code, addr, 0); return false; }
             }
         }
     }
@@ -959,6 +960,30 @@ __global__ void __launch_bounds__(kThreads, 1) k_line(const __grid_constant__ Li
     __syncthreads();
     tc_fence_after();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// The engine's wait code on a barrier and a counter that nothing ever completes: one CTA, one thread, the limit given by
+// the caller.  The first wait must run out and raise the abort flag and the error word; the second must then fall
+// through at once.  out[0..1] = what the two waits returned, out[2] = the abort flag, out[3] = nanoseconds spent.
+__global__ void k_wait_probe(int32_t *err, unsigned long long limit_ns, int32_t *out)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&ctrl->bars[0]), 1);
+        ctrl->abort_flag = 0;
+        ctrl->stored[0] = 0;
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Waiter w{ctrl, err, limit_ns};
+        const unsigned long long t0 = globaltimer();
+        out[0] = w.barrier(smem_u32(&ctrl->bars[0]), 0, ERR_WAIT_FULL) ? 1 : 0;
+        out[1] = w.counter(smem_u32(&ctrl->stored[0]), 1u, ERR_WAIT_DONE) ? 1 : 0;
+        out[2] = ctrl->abort_flag;
+        out[3] = (int32_t)min(globaltimer() - t0, 0x7FFFFFFFull);
+    }
 }
 
 // =============================================================================== host planner
@@ -1812,6 +1837,17 @@ int line_check(LinePlan *p)
         return ISC_ERR_TIMEOUT;
     }
     return ISC_OK;
+}
+
+int line_wait_probe(LinePlan *p, long long limit_ns, int32_t out[4], cudaStream_t st)
+{
+    if (limit_ns < 1000 || limit_ns > 100000000ll) return ISC_ERR_ARG;          // 1 us .. 100 ms
+    int32_t *d_out = reinterpret_cast<int32_t *>(p->d_dump);                   // the debug read-back buffer
+    k_wait_probe<<<1, 32, kCtrlBytes, st>>>(p->d_err, (unsigned long long)limit_ns, d_out);
+    if (cudaGetLastError() != cudaSuccess) return ISC_ERR_CUDA;
+    if (cudaMemcpyAsync(out, d_out, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ISC_ERR_CUDA; }
+    return line_check(p);
 }
 
 int line_phase_cycles(LinePlan *p, unsigned long long out[4])

@@ -33,6 +33,11 @@ int line_debug_tensor(LinePlan *p, const uint8_t *d_x, const NoiseStream &ns, in
 // After the stream has been synchronised: ISC_OK, or ISC_ERR_TIMEOUT if a bounded wait expired.
 int line_check(LinePlan *p);
 
+// Failure-path check without a failure: runs the engine's wait code (one thread) on a barrier and a counter that nothing
+// completes, with `limit_ns` as the wait limit.  Returns what line_check returns afterwards (ISC_ERR_TIMEOUT when the
+// path works) and out[] = {first wait's result, second wait's result, abort flag, nanoseconds spent}.
+int line_wait_probe(LinePlan *p, long long limit_ns, int32_t out[4], cudaStream_t st);
+
 // SM cycles, summed over CTAs and over every launch so far, spent in: [0] halo fills, [1] the noise phase (draw, add,
 // saturate, store: Def. 3.3, Def. 3.4), [2] the convolutions, [3] pool / FC / argmax / vote.  Synchronises the device.
 int line_phase_cycles(LinePlan *p, unsigned long long out[4]);

@@ -316,3 +316,24 @@ def test_argument_errors_leave_outputs_untouched():
     assert L.isc_predict(gm._h, None, 1, 0, 10, 0.25, 0.001, None, C.byref(cls), None) == -1
     assert cls.value == 9 and rad.value == 9.0
     assert gm.get_info("gpu_launches") >= 0
+
+
+def test_expired_wait_is_reported_and_the_handle_recovers():
+    """Every device-side wait of the resident engine is bounded.  The harness runs the engine's own wait code on a
+    barrier and a counter that nothing completes, with a 1 ms limit: the first wait must expire, raise the abort flag
+    and the error word (ISC_ERR_TIMEOUT = -6 from the check), the second must fall through at once, and the handle must
+    work afterwards.  Nothing here faults, traps or hangs the GPU."""
+    model = wl.spread_model("resnet20")
+    gm, om = _pair(model)
+    x = wl.spread_image()
+    before = gm.sample_counts(x, SEED, 0, 1, 0, 64, 0.25)
+    rc, (first, second, abort_flag, ns) = gm.debug_wait_timeout(1_000_000)
+    assert rc == -6
+    assert (first, second, abort_flag) == (0, 0, 1)
+    assert 1_000_000 <= ns < 200_000_000
+    after, logits = gm.sample_counts(x, SEED, 0, 1, 0, 64, 0.25, want_logits=True)
+    np.testing.assert_array_equal(after, before)
+    np.testing.assert_array_equal(logits, oracle.sample_counts(om, x, SEED, 0, 1, 0, 64, 0.25, want_logits=True)[1])
+    # out-of-range limits are refused before anything is launched
+    assert gm.debug_wait_timeout(10)[0] == -1 and gm.debug_wait_timeout(10 ** 10)[0] == -1
+    assert isc.Model(wl.resnet50()).debug_wait_timeout(1_000_000)[0] == -3
