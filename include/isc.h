@@ -211,6 +211,16 @@ int isc_decide_predict(const int32_t *counts, int n_classes, double alpha, int32
 int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_T);
 
 /*
+ * isc_noise_table_rounded -- the same table for the noise of the paper's comparison method
+ * "FloatRS-quant" (Sec. 4.1, comparison methods: continuous Gaussian noise is added to the image
+ * and the sum is quantised): on integer pixels delta = round(255 sigma g), g ~ N(0, 1), so
+ * cum[z + T] = floor(2^32 * Phi((z + 1/2) / (255 sigma))).  A model handle draws from this law
+ * instead of Eq. 2 after isc_set_option(m, "noise", 1); nothing else changes (same random
+ * stream, same inverse-CDF rule, same kernels).  Arguments as isc_noise_table.
+ */
+int isc_noise_table_rounded(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_T);
+
+/*
  * isc_radius_integer -- the integer-only form of the radius (Theorem 3.2 steps 2-3,
  * Theorem 3.1): the quantile of the one-dimensional discrete Gaussian N_Z(0, (255 sigma)^2)
  * by lookup in the cumulative table above, for a probability given as a 32-bit fixed-point
@@ -288,7 +298,10 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
 int isc_debug_wait_timeout(isc_model *m, int64_t limit_ns, void *cuda_stream, int32_t *out4);
 
 /*
- * isc_set_option -- tuning knobs; none changes a result.
+ * isc_set_option -- "batch" and "engine" are tuning knobs that change no result; "noise" selects
+ * the noise law and therefore changes the samples.
+ *   "noise"  : 0 = the discrete Gaussian of Def. 3.3 / Eq. 2 (IntRS, the default), 1 = the
+ *              rounded continuous Gaussian of the comparison method (isc_noise_table_rounded).
  *   "batch"  : noisy samples per launch (0 = choose automatically).
  *   "engine" : 0 = automatic (3 if the model fits it, else 2 if any layer fits it, else 1),
  *              1 = layer-by-layer kernels without tensor cores, 2 = layer-by-layer with

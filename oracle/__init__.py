@@ -15,6 +15,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "intrs_oracle.c")
+_SRC2 = os.path.join(_HERE, "dgauss_rejection.c")
 _LIB = os.path.join(_HERE, "libintrs_oracle.so")
 
 OP_CONV2D, OP_FC, OP_GAVGPOOL, OP_MAXPOOL = 0, 1, 2, 3
@@ -22,9 +23,9 @@ OP_CONV2D, OP_FC, OP_GAVGPOOL, OP_MAXPOOL = 0, 1, 2, 3
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (no fast-math, no contraction)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC2)):
         cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
-               "-fno-fast-math", "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
+               "-fno-fast-math", "-Wall", "-Wextra", "-o", _LIB, _SRC, _SRC2, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 
@@ -56,6 +57,12 @@ def lib():
         L.orc_dgauss_pmf.restype = None
         L.orc_dgauss_table.argtypes = [C.c_double, C.c_void_p]
         L.orc_dgauss_table.restype = None
+        L.rej_dgauss_draws.argtypes = [C.c_double, C.c_uint64, C.c_int64, C.c_void_p]
+        L.rej_dgauss_draws.restype = C.c_int64
+        L.orc_rgauss_table.argtypes = [C.c_double, C.c_void_p]
+        L.orc_rgauss_table.restype = None
+        L.orc_set_noise_kind.argtypes = [C.c_int]
+        L.orc_set_noise_kind.restype = None
         for f in (L.orc_dgauss_from_uniform, L.orc_dgauss_from_uniform_fast):
             f.argtypes = [C.c_uint32, C.c_void_p, C.c_int32]
             f.restype = C.c_int32
@@ -176,6 +183,27 @@ def dgauss_table(sigma):
     t = np.zeros(2 * T + 1, dtype=np.uint32)
     lib().orc_dgauss_table(float(sigma), _ptr(t))
     return t
+
+
+def rgauss_table(sigma):
+    """Cumulative table of the rounded continuous Gaussian (the FloatRS-quant comparison method's noise, Sec. 4.1)."""
+    T = dgauss_halfwidth(sigma)
+    t = np.zeros(2 * T + 1, dtype=np.uint32)
+    lib().orc_rgauss_table(float(sigma), _ptr(t))
+    return t
+
+
+def rejection_dgauss(sigma, seed, n):
+    """n draws of the discrete Gaussian with std 255 * sigma pixel levels from the table-free rejection sampler
+    (dgauss_rejection.c); returns (draws, proposals made)."""
+    out = np.zeros(n, dtype=np.int32)
+    proposals = lib().rej_dgauss_draws(255.0 * float(sigma), int(seed), int(n), _ptr(out))
+    return out, int(proposals)
+
+
+def set_noise_kind(kind):
+    """0: discrete Gaussian of Eq. 2 (default); 1: rounded continuous Gaussian.  Process-wide."""
+    lib().orc_set_noise_kind(int(kind))
 
 
 def dgauss_from_uniform(u, cum, fast=False):

@@ -148,6 +148,32 @@ void orc_dgauss_table(double sigma, uint32_t *cum)
     cum[2 * T] = 4294967295u;
 }
 
+/* The comparison method's noise (Sec. 4.1, "FloatRS-quant": continuous Gaussian noise added to the image, the sum
+ * then quantised): on integer pixels that is delta = round(sigma_int * g), g ~ N(0, 1), whose law is
+ * P[delta = z] = Phi((z + 1/2) / sigma_int) - Phi((z - 1/2) / sigma_int).  Same table form as above:
+ * cum[z+T] = floor(Phi((z + 1/2) / sigma_int) * 2^32), the last entry forced to 2^32-1.                        */
+void orc_rgauss_table(double sigma, uint32_t *cum)
+{
+    double sigma_int = 255.0 * sigma;
+    int32_t T = orc_dgauss_halfwidth(sigma);
+    for (int32_t z = -T; z <= T; ++z) {
+        double cdf = 0.5 * erfc(-(((double)z + 0.5) / sigma_int) / sqrt(2.0));
+        double v = floor(cdf * 4294967296.0);
+        if (v > 4294967295.0) v = 4294967295.0;
+        cum[z + T] = (uint32_t)v;
+    }
+    cum[2 * T] = 4294967295u;
+}
+
+/* Which noise law the sampling functions below use: 0 = the discrete Gaussian of Eq. 2 (IntRS, the default),
+ * 1 = the rounded continuous Gaussian (FloatRS-quant).  Process-wide; set it before a call, not during one.     */
+static int g_noise_kind = 0;
+void orc_set_noise_kind(int kind) { g_noise_kind = kind ? 1 : 0; }
+static void sampling_table(double sigma, uint32_t *cum)
+{
+    if (g_noise_kind) orc_rgauss_table(sigma, cum); else orc_dgauss_table(sigma, cum);
+}
+
 /* Inverse-CDF draw by plain linear scan of the table.                          */
 int32_t orc_dgauss_from_uniform(uint32_t u, const uint32_t *cum, int32_t T)
 {
@@ -180,7 +206,7 @@ void orc_noise(uint64_t seed, uint64_t image_id, uint32_t phase, uint64_t j,
 {
     int32_t T = orc_dgauss_halfwidth(sigma);
     uint32_t *cum = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(2 * T + 1));
-    orc_dgauss_table(sigma, cum);
+    sampling_table(sigma, cum);
     for (int64_t i = 0; i < n_draws; ++i) {
         uint32_t u = orc_uniform_u32(seed, image_id, phase, j, e0 + (uint64_t)i);
         delta[i] = dgauss_bisect(u, cum, T);
@@ -210,7 +236,7 @@ void orc_noisy_input(const uint8_t *x, int64_t d, uint64_t seed, uint64_t image_
     int32_t T = orc_dgauss_halfwidth(sigma);
     uint32_t *cum = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(2 * T + 1));
     int32_t *a0 = (int32_t *)malloc(sizeof(int32_t) * (size_t)d);
-    orc_dgauss_table(sigma, cum);
+    sampling_table(sigma, cum);
     noisy_input(x, d, seed, image_id, phase, j, cum, T, a0);
     for (int64_t e = 0; e < d; ++e) out[e] = (uint8_t)a0[e];
     free(a0);
@@ -413,7 +439,7 @@ int orc_sample_counts(const orc_layer *layers, int n_layers, int in_c, int in_h,
     if (orc_tensor_size(layers, n_layers, in_c, in_h, in_w, n_layers) != n_classes) return -1;
     int32_t T = orc_dgauss_halfwidth(sigma);
     uint32_t *cum = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(2 * T + 1));
-    orc_dgauss_table(sigma, cum);
+    sampling_table(sigma, cum);
     int32_t *labels = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
     int bad = 0;
 #pragma omp parallel

@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
 EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_plan_resident", "isc_predict", "isc_certify", "isc_certify_batch",
-           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_certify_integer", "isc_decide_certify_integer", "isc_noise_table", "isc_radius_integer", "isc_certified_metrics",
+           "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_certify_integer", "isc_decide_certify_integer", "isc_noise_table", "isc_noise_table_rounded", "isc_radius_integer", "isc_certified_metrics",
            "isc_debug_tensor", "isc_debug_wait_timeout", "isc_set_option", "isc_get_info", "isc_strerror"]
 
 
@@ -61,6 +61,7 @@ def lib():
         L.isc_certify_integer.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int64, C.c_int64, C.c_double, C.c_double,
                                           C.c_int, vp, i32p, i32p, C.POINTER(C.c_int64), vp, vp]
         L.isc_noise_table.argtypes = [C.c_double, vp, C.c_int64, i32p]
+        L.isc_noise_table_rounded.argtypes = [C.c_double, vp, C.c_int64, i32p]
         L.isc_radius_integer.argtypes = [C.c_double, C.c_uint32, i32p, C.POINTER(C.c_int64)]
         L.isc_certified_metrics.argtypes = [vp, vp, vp, C.c_int64, vp, C.c_int, C.POINTER(C.c_double), vp]
         L.isc_debug_tensor.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int32, C.c_int64, C.c_double,
@@ -284,9 +285,11 @@ def radius_integer(sigma, p_fx):
     return q.value, q2.value
 
 
-def noise_table(sigma):
+def noise_table(sigma, rounded=False):
+    """Cumulative table of the noise law: Eq. 2, or the rounded continuous Gaussian when `rounded`."""
+    f = lib().isc_noise_table_rounded if rounded else lib().isc_noise_table
     T = C.c_int32()
-    _check(lib().isc_noise_table(float(sigma), None, 0, C.byref(T)), "isc_noise_table")
+    _check(f(float(sigma), None, 0, C.byref(T)), "isc_noise_table")
     cum = np.zeros(2 * T.value + 1, dtype=np.uint32)
-    _check(lib().isc_noise_table(float(sigma), _ptr(cum), cum.size, C.byref(T)), "isc_noise_table")
+    _check(f(float(sigma), _ptr(cum), cum.size, C.byref(T)), "isc_noise_table")
     return cum

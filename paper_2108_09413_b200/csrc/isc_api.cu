@@ -64,7 +64,7 @@ struct isc_model {
     int8_t *d_logits = nullptr;   size_t d_logits_bytes = 0;
     uint32_t *d_cum = nullptr;    size_t d_cum_n = 0;
     double cum_sigma = -1.0;
-    int cum_T = 0;
+    int cum_T = 0, cum_kind = -1;
 
     isc::LinePlan *line = nullptr;
 
@@ -72,7 +72,7 @@ struct isc_model {
     int32_t *h_counts = nullptr;  size_t h_counts_bytes = 0;
     std::vector<cudaEvent_t> events;
 
-    int64_t opt_batch = 0, opt_engine = 0;
+    int64_t opt_batch = 0, opt_engine = 0, opt_noise = 0;
     int64_t last_engine = 0, launches = 0;
 };
 
@@ -332,9 +332,9 @@ int ensure_workspace(isc_model *m, int batch)
 
 int ensure_noise_table(isc_model *m, double sigma, cudaStream_t st)
 {
-    if (m->d_cum && m->cum_sigma == sigma) return ISC_OK;
+    if (m->d_cum && m->cum_sigma == sigma && m->cum_kind == (int)m->opt_noise) return ISC_OK;
     std::vector<uint32_t> cum;
-    noise_table(sigma, cum);
+    if (m->opt_noise) noise_table_rounded(sigma, cum); else noise_table(sigma, cum);
     // the guide table follows the cumulative one in the same allocation
     const size_t n_cum = cum.size();
     for (int j = 0; j <= isc::kNoiseGuide; ++j) {
@@ -351,6 +351,7 @@ int ensure_noise_table(isc_model *m, double sigma, cudaStream_t st)
     CK(cudaMemcpyAsync(m->d_cum, cum.data(), cum.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
     CK(cudaStreamSynchronize(st));                       // cum is a local vector
     m->cum_sigma = sigma;
+    m->cum_kind = (int)m->opt_noise;
     m->cum_T = (int)(n_cum - 1) / 2;
     return ISC_OK;
 }
@@ -810,6 +811,20 @@ int isc_noise_table(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_
     return ISC_OK;
 }
 
+int isc_noise_table_rounded(double sigma, uint32_t *cum, int64_t capacity, int32_t *out_T)
+{
+    if (!out_T || !(sigma > 0.0) || !std::isfinite(sigma) || sigma > 64.0) return ISC_ERR_ARG;
+    const int T = noise_halfwidth(sigma);
+    if (cum) {
+        if (capacity < 2 * (int64_t)T + 1) return ISC_ERR_ARG;
+        std::vector<uint32_t> t;
+        noise_table_rounded(sigma, t);
+        memcpy(cum, t.data(), t.size() * sizeof(uint32_t));
+    }
+    *out_T = T;
+    return ISC_OK;
+}
+
 int isc_certified_metrics(const int32_t *classes, const double *radii, const int32_t *labels, int64_t n,
                           const double *r, int n_r, double *out_cp, double *out_ca)
 {
@@ -973,7 +988,7 @@ extern "C" int isc_sample_counts_static(isc_model *m, const uint8_t *x_u8, uint6
     }
 
     std::vector<uint32_t> cum;
-    noise_table(sigma, cum);
+    if (m->opt_noise) noise_table_rounded(sigma, cum); else noise_table(sigma, cum);
     m->last_engine = 1;
     // the array keeps whatever the previous call left: the vote counts must start from zero
     CK(cudaMemsetAsync(d_counts, 0, C * sizeof(int32_t), st));
@@ -1020,6 +1035,11 @@ int isc_set_option(isc_model *m, const char *name, int64_t value)
     if (!strcmp(name, "batch")) {
         if (value < 0 || value > (1 << 20)) return ISC_ERR_ARG;
         m->opt_batch = value;
+        return ISC_OK;
+    }
+    if (!strcmp(name, "noise")) {
+        if (value != 0 && value != 1) return ISC_ERR_ARG;
+        m->opt_noise = value;
         return ISC_OK;
     }
     if (!strcmp(name, "engine")) {

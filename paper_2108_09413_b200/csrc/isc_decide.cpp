@@ -188,4 +188,21 @@ void noise_table(double sigma, std::vector<uint32_t> &cum)
     cum[(size_t)(2 * T)] = 4294967295u;
 }
 
+// The same table form for the rounded continuous Gaussian: delta = round(255 sigma g), g ~ N(0, 1), the noise of the
+// paper's comparison method that perturbs with continuous noise and then quantises (Sec. 4.1, comparison methods):
+// cum[z + T] = floor(2^32 * Phi((z + 1/2) / (255 sigma))).
+void noise_table_rounded(double sigma, std::vector<uint32_t> &cum)
+{
+    const double s = 255.0 * sigma;
+    const int T = noise_halfwidth(sigma);
+    cum.resize((size_t)(2 * T + 1));
+    for (int z = -T; z <= T; ++z) {
+        const double cdf = 0.5 * std::erfc(-(((double)z + 0.5) / s) / std::sqrt(2.0));
+        double scaled = std::floor(cdf * 4294967296.0);
+        if (scaled > 4294967295.0) scaled = 4294967295.0;
+        cum[(size_t)(z + T)] = (uint32_t)scaled;
+    }
+    cum[(size_t)(2 * T)] = 4294967295u;
+}
+
 }  // namespace isc

@@ -89,5 +89,6 @@ int32_t decide_certify_integer(const int32_t *counts0, const int32_t *counts, in
                                double alpha, bool two_sided, int32_t *q, int64_t *q_squared);
 int noise_halfwidth(double sigma);
 void noise_table(double sigma, std::vector<uint32_t> &cum);
+void noise_table_rounded(double sigma, std::vector<uint32_t> &cum);
 
 }  // namespace isc

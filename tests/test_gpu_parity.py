@@ -337,3 +337,31 @@ def test_expired_wait_is_reported_and_the_handle_recovers():
     # out-of-range limits are refused before anything is launched
     assert gm.debug_wait_timeout(10)[0] == -1 and gm.debug_wait_timeout(10 ** 10)[0] == -1
     assert isc.Model(wl.resnet50()).debug_wait_timeout(1_000_000)[0] == -3
+
+
+def test_rounded_gaussian_noise_path():
+    """The comparison method's noise (Sec. 4.1, FloatRS-quant: continuous Gaussian, then quantised) behind the same
+    staging: with isc_set_option("noise", 1) every engine draws from the rounded-Gaussian table; noisy inputs, logits
+    and counts equal the oracle's under the same law, and differ from the discrete-Gaussian ones."""
+    model = wl.spread_model("resnet20")
+    gm, om = _pair(model)
+    x = wl.spread_image()
+    base = gm.sample_counts(x, SEED, 0, 1, 0, 600, 0.5)
+    gm.set_option("noise", 1)
+    oracle.set_noise_kind(1)
+    try:
+        exp_in = oracle.noisy_input(x, SEED, 4, 1, 9, 0.5).ravel()
+        ecounts, elog = oracle.sample_counts(om, x, SEED, 0, 1, 0, 600, 0.5, want_logits=True)
+    finally:
+        oracle.set_noise_kind(0)
+    for eng in (1, 2, 3):
+        gm.set_option("engine", eng)
+        np.testing.assert_array_equal(gm.debug_tensor(x, SEED, 4, 1, 9, 0.5, 0, x.size), exp_in)
+        counts, log = gm.sample_counts(x, SEED, 0, 1, 0, 600, 0.5, want_logits=True)
+        np.testing.assert_array_equal(log, elog)
+        np.testing.assert_array_equal(counts, ecounts)
+    np.testing.assert_array_equal(gm.sample_counts_static(x, SEED, 0, 1, 0, 600, 0.5), ecounts)
+    assert (ecounts != base).any()
+    gm.set_option("noise", 0)
+    gm.set_option("engine", 0)
+    np.testing.assert_array_equal(gm.sample_counts(x, SEED, 0, 1, 0, 600, 0.5), base)

@@ -181,3 +181,9 @@ def test_integer_certify_decisions_equal_the_oracle():
     assert L.isc_decide_certify_integer(c.ctypes.data, c.ctypes.data, 2, 10, 0.25, 1.5, 0, C.byref(cls), C.byref(q), None) == -1
     assert L.isc_decide_certify_integer(c.ctypes.data, c.ctypes.data, 2, 4, 0.25, 0.001, 0, C.byref(cls), C.byref(q), None) == -1
     assert (cls.value, q.value) == (7, 7)
+
+
+def test_rounded_noise_table_equals_the_oracle():
+    for sigma in (0.12, 0.25, 0.5, 1.0):
+        np.testing.assert_array_equal(isc.noise_table(sigma, rounded=True), oracle.rgauss_table(sigma))
+        np.testing.assert_array_equal(isc.noise_table(sigma), oracle.dgauss_table(sigma))

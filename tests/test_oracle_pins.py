@@ -512,3 +512,65 @@ def test_integer_certify_decide_against_the_normal_radius_and_symmetry():
         counts = [n_a, N - n_a, 0, 0]
         assert oracle.certify_integer_decide([3, 1, 0, 0], counts, N, 0.25, alpha, two_sided=True)[0] == \
                oracle.certify_integer_decide([3, 1, 0, 0], counts, N, 0.25, alpha)[0]
+
+
+# ------------------------------------------------------------------ second samplers (Sec. 3.3, Sec. 4.1)
+
+def _pooled_chi2_p(obs, exp, n):
+    keep = exp >= 5.0
+    lo, hi = np.argmax(keep), len(keep) - np.argmax(keep[::-1])
+    o = np.concatenate(([obs[:lo].sum()], obs[lo:hi], [obs[hi:].sum()]))
+    e = np.concatenate(([exp[:lo].sum()], exp[lo:hi], [exp[hi:].sum()]))
+    e[0] += n - e.sum()
+    return st.chi2.sf(((o - e) ** 2 / e).sum(), df=len(o) - 1)
+
+
+@pytest.mark.parametrize("sigma", [0.12, 0.5])
+def test_table_sampler_agrees_with_the_rejection_sampler(sigma):
+    """The table-free rejection sampler the paper cites for its noise (Sec. 3.3) and the oracle's inverse-CDF table
+    draw from the same law: each passes the exact-pmf chi-square of Eq. 2, and their two histograms pass a
+    two-sample chi-square against each other."""
+    n = 2_000_000
+    T = oracle.dgauss_halfwidth(sigma)
+    rej, proposals = oracle.rejection_dgauss(sigma, seed=4242, n=n)
+    assert n <= proposals < 4 * n                       # the publication bounds the expected number of proposals
+    assert np.abs(rej).max() <= T
+    pmf = _pmf_direct(sigma, np.arange(-T, T + 1))
+    h_rej = np.bincount(rej + T, minlength=2 * T + 1).astype(np.float64)
+    assert _pooled_chi2_p(h_rej, pmf * n, n) > 1e-3
+    tab = oracle.noise(seed=5, image_id=1, phase=0, j=77, sigma=sigma, e0=0, n=n)
+    h_tab = np.bincount(tab + T, minlength=2 * T + 1).astype(np.float64)
+    both = h_rej + h_tab
+    use = both >= 10
+    chi2 = (((h_rej - h_tab) ** 2)[use] / both[use]).sum()
+    assert st.chi2.sf(chi2, df=int(use.sum()) - 1) > 1e-3
+    s_int = 255.0 * sigma
+    assert abs(rej.mean()) < 5 * s_int / math.sqrt(n)
+    assert abs(rej.astype(np.float64).var() - s_int ** 2) < 5 * s_int ** 2 * math.sqrt(2.0 / n)
+
+
+@pytest.mark.parametrize("sigma", [0.12, 1.0])
+def test_rounded_gaussian_noise_of_the_comparison_method(sigma):
+    """FloatRS-quant's noise (Sec. 4.1): continuous Gaussian, then quantised.  The oracle's table must be the CDF of
+    round(255 sigma g) at the half-integers (SciPy's normal CDF), the draws must pass the chi-square of that law, and
+    their variance must carry the rounding's 1/12 that the discrete Gaussian of Eq. 2 does not have."""
+    s_int = 255.0 * sigma
+    T = oracle.dgauss_halfwidth(sigma)
+    cum = oracle.rgauss_table(sigma).astype(np.float64)
+    z = np.arange(-T, T + 1)
+    ref = np.floor(st.norm.cdf((z + 0.5) / s_int) * 2.0 ** 32)
+    assert np.abs(cum[:-1] - ref[:-1]).max() <= 64           # the two erfc implementations differ in the last bits
+    assert cum[-1] == 2.0 ** 32 - 1 and (np.diff(cum) >= 0).all()
+    n = 2_000_000
+    oracle.set_noise_kind(1)
+    try:
+        draws = oracle.noise(seed=8, image_id=2, phase=1, j=5, sigma=sigma, e0=0, n=n)
+    finally:
+        oracle.set_noise_kind(0)
+    pmf = st.norm.cdf((z + 0.5) / s_int) - st.norm.cdf((z - 0.5) / s_int)
+    obs = np.bincount(draws + T, minlength=2 * T + 1).astype(np.float64)
+    assert _pooled_chi2_p(obs, pmf * n, n) > 1e-3
+    var = draws.astype(np.float64).var()
+    assert abs(var - (s_int ** 2 + 1.0 / 12.0)) < 5 * s_int ** 2 * math.sqrt(2.0 / n)
+    # and it is not the law of Eq. 2: the default kind draws something else from the same uniforms
+    assert (oracle.noise(seed=8, image_id=2, phase=1, j=5, sigma=sigma, e0=0, n=20000) != draws[:20000]).any()
