@@ -254,6 +254,14 @@ int build_generic_engine(isc_model *m)
                         }
             }
             rc = upload(m, w, &G.w); if (rc) return rc;
+            if (i == 0 && stem_fits(G, m->in_c)) {          // the stem for the tensor-core kernel
+                std::vector<int8_t> wp(stem_pack_bytes(G));
+                stem_pack_weights(G, H.w.data(), wp.data());
+                rc = upload(m, wp, &m->wpacks[0]); if (rc) return rc;
+                std::vector<int32_t> c4((size_t)G.coutp * 4);
+                m->tc_fast[0] = igemm_constants(G, bias.data(), mult.data(), shift.data(), c4.data()) ? 1 : 0;
+                rc = upload(m, c4, &m->tc_cst[0]); if (rc) return rc;
+            }
             if (i > 0 && igemm_tile_n(G)) {                 // the same layer for the tensor-core kernel
                 std::vector<int8_t> wp(igemm_pack_bytes(G));
                 igemm_pack_weights(G, H.w.data(), wp.data());
@@ -401,7 +409,9 @@ int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int
         const int8_t *in = i == 0 ? nullptr : (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.in_tensor]].p;
         const int8_t *res = L.res_tensor >= 0 ? (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.res_tensor]].p : nullptr;
         cudaError_t e;
-        if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, batch, out, st);
+        if (i == 0 && tensor_cores && m->wpacks[0])
+            e = launch_stem_conv(G, m->wpacks[0], m->tc_cst[0], m->tc_fast[0] != 0, d_x, m->in_c, ns, batch, out, m->d_tc_err, st);
+        else if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, batch, out, st);
         else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], m->tc_cst[(size_t)i], m->tc_fast[(size_t)i] != 0, batch, in, res, out, m->d_tc_err, st);
         else if (L.op == ISC_CONV2D || L.op == ISC_FC) e = launch_conv(G, batch, in, res, out, st);
         else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, batch, in, out, st);

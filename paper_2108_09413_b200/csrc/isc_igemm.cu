@@ -220,6 +220,164 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
     if (warp == 0) tmem_dealloc(tmem, (uint32_t)p.tmem_cols);
 }
 
+
+// ------------------------------------------------------------------ first convolution on the tensor cores
+//
+// The stem of a network whose input is the noisy image (Def. 3.4): a k x k convolution over <= 4 input channels.
+// One CTA = one sample x one band of output rows.  The band's input rows are drawn (Philox -> inverse-CDF table ->
+// add -> saturate to 0..255, Def. 3.3 / Eq. 2) into a shared-memory patch as 4 bytes per pixel, padded with the input
+// zero-point, and never written to memory.  The GEMM takes one filter row per K-step: eight horizontally adjacent
+// pixels x 4 bytes = 32 bytes of K (pixels beyond the filter width meet zero weights), so a tile of 128 output pixels
+// is `kh` MMAs.  Each thread copies its pixel's `kh` windows from the patch into the K-major operand stage; tiles
+// alternate between two stages and two halves of the accumulator columns, so the requantisation of one tile runs
+// while the MMAs of the next are in flight.
+struct StemParams {
+    GLayer L;
+    int in_c, band_rows, n_bands, tiles_per_band, tmem_cols;
+    uint32_t patch_bytes, w_bytes;
+    const uint8_t *x;                        // clean image, CHW
+    NoiseStream ns;
+    const int8_t *wpack;                     // [filter row][2 K columns][coutp rows][16 bytes]
+    const int4 *cst;
+    int fast_requant, lo;
+    int8_t *out;
+    int32_t *err;
+};
+
+__global__ void __launch_bounds__(kThreads) k_stem(const __grid_constant__ StemParams p)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ unsigned long long bar_w, bar_full[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ volatile int abort_s;
+    __shared__ __align__(16) int4 cst_s[256];
+    const GLayer &L = p.L;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const uint32_t sbase = smem_u32(smem);
+    const int N = L.coutp, kh = L.kh;
+    const uint32_t a_bytes = (uint32_t)kh * kTileM * 32u;
+    const uint32_t w_off = 0, a_off = p.w_bytes, patch_off = a_off + 2u * a_bytes;        // weights | two operand stages | patch
+    if (tid == 0) {
+        mbar_init(smem_u32(&bar_w), 1);
+        mbar_init(smem_u32(&bar_full[0]), 1);
+        mbar_init(smem_u32(&bar_full[1]), 1);
+        abort_s = 0;
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_base_s), (uint32_t)p.tmem_cols);
+    for (int i = tid; i < N; i += kThreads) cst_s[i] = __ldg(p.cst + i);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    if (tid == 0) {
+        mbar_expect_tx(smem_u32(&bar_w), p.w_bytes);
+        bulk_g2s(sbase + w_off, p.wpack, p.w_bytes, smem_u32(&bar_w));
+    }
+
+    // ---- the band's noisy input rows
+    const int b = blockIdx.y;
+    const int64_t j = p.ns.first_sample + b;
+    const int oy0 = blockIdx.x * p.band_rows, oy1 = min(L.hout, oy0 + p.band_rows);
+    const int wpad = L.win + 2 * L.pad + 8;                     // 8 more pixels: the windows of the last columns stay inside
+    const int iy0 = oy0 * L.stride - L.pad;
+    const int rows_in = (oy1 - oy0 - 1) * L.stride + kh;
+    uint32_t *patch = reinterpret_cast<uint32_t *>(smem + patch_off);
+    const uint32_t zp_fill = (uint32_t)(L.zp_in & 0xFF) * (0x01010101u >> (8 * (4 - p.in_c)));
+    for (int i = tid; i < rows_in * wpad; i += kThreads) patch[i] = zp_fill;
+    __syncthreads();
+    const int vy0 = max(0, iy0), vy1 = min(L.hin, iy0 + rows_in);
+    if (vy1 > vy0) {
+        uint8_t *pb = reinterpret_cast<uint8_t *>(patch);
+        const uint32_t ctr3 = p.ns.ctr3_fixed | (uint32_t)(((j >> 32) & 0xFF) << 8);
+        for (int c = 0; c < p.in_c; ++c) {
+            const int64_t e_begin = ((int64_t)c * L.hin + vy0) * L.win, e_end = ((int64_t)c * L.hin + vy1) * L.win;
+            for (int64_t q = (e_begin >> 2) + tid; q < ((e_end + 3) >> 2); q += kThreads) {
+                const uint4 r = philox4x32_10(make_uint4((uint32_t)q, (uint32_t)(j & 0xFFFFFFFFll), p.ns.ctr2, ctr3), p.ns.key0, p.ns.key1);
+                const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int64_t e = q * 4 + k;
+                    if (e < e_begin || e >= e_end) continue;
+                    const int rem = (int)(e - (int64_t)c * L.hin * L.win);
+                    const int h = rem / L.win, w = rem - h * L.win;
+                    int v = (int)__ldg(p.x + e) + noise_level(u[k], p.ns.cum, p.ns.T);
+                    v = min(255, max(0, v));
+                    pb[((h - iy0) * wpad + (w + L.pad)) * 4 + c] = (uint8_t)v;
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- tiles of 128 output pixels of the band
+    const int band_px = (oy1 - oy0) * L.wout;
+    const int n_tiles = (band_px + kTileM - 1) / kTileM;
+    const uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    bool ok = true;
+    if (tid == 0) ok = wait_bar(smem_u32(&bar_w), 0);
+    for (int t = 0; t <= n_tiles; ++t) {
+        if (t < n_tiles) {
+            // operand stage of tile t: free once the MMAs of tile t - 2 are complete (waited for by its epilogue below)
+            const uint32_t stage = sbase + a_off + (uint32_t)(t & 1) * a_bytes;
+            const int px = t * kTileM + tid;
+            const int pp = px < band_px ? px : 0;
+            const int oyl = pp / L.wout, ox = pp - oyl * L.wout;
+            for (int r = 0; r < kh; ++r) {
+                const uint32_t *src = patch + (oyl * L.stride + r) * wpad + ox * L.stride;
+                st_shared_v4(stage + (uint32_t)r * 4096u + 0u * 2048u + tid * 16, make_uint4(src[0], src[1], src[2], src[3]));
+                st_shared_v4(stage + (uint32_t)r * 4096u + 1u * 2048u + tid * 16, make_uint4(src[4], src[5], src[6], src[7]));
+            }
+            fence_proxy_async();
+        }
+        __syncthreads();
+        if (t < n_tiles && tid == 0) {
+            tc_fence_after();
+            if (ok && !abort_s) {
+                const uint32_t stage = sbase + a_off + (uint32_t)(t & 1) * a_bytes;
+                for (int r = 0; r < kh; ++r) {
+                    const uint64_t ad = make_desc(stage + (uint32_t)r * 4096u, 2048u, 128u);
+                    const uint64_t bd = make_desc(sbase + w_off + (uint32_t)r * 2u * (uint32_t)N * 16u, (uint32_t)N * 16u, 128u);
+                    mma_i8(tmem + (uint32_t)(t & 1) * (uint32_t)N, ad, bd, idesc, r > 0 ? 1u : 0u);
+                }
+            }
+            commit_to(smem_u32(&bar_full[t & 1]));
+        }
+        if (t >= 1) {
+            // epilogue of tile t - 1 while the MMAs of tile t run
+            const int tt = t - 1;
+            if (ok && !abort_s) ok = wait_bar(smem_u32(&bar_full[tt & 1]), (uint32_t)(tt >> 1) & 1u);
+            if (!ok) abort_s = 1;
+            tc_fence_after();
+            const int px = tt * kTileM + tid;
+            const bool valid = px < band_px;
+            const size_t m = ((size_t)b * L.hout + oy0) * L.wout + (size_t)(valid ? px : 0);
+            for (int c0 = 0; c0 < N; c0 += 16) {
+                int acc[16];
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(tt & 1) * (uint32_t)N + (uint32_t)c0, acc);
+                if (valid && !abort_s) {
+                    uint4 v;
+                    if (p.fast_requant) {
+                        v = requant16_fast<false>(acc, smem_u32(cst_s + c0), make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
+                    } else {
+#pragma unroll
+                        for (int o = 0; o < 16; ++o) acc[o] += __ldg(L.bias + c0 + o);
+                        v = epilogue16(acc, L, c0, nullptr);
+                    }
+                    *reinterpret_cast<uint4 *>(p.out + m * L.coutp + c0) = v;
+                }
+            }
+            tc_fence_before();
+        }
+    }
+    if (!ok) atomicCAS(p.err, 0, 1 + (int)blockIdx.x);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc(tmem, (uint32_t)p.tmem_cols);
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------ host side
@@ -305,4 +463,75 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
     return cudaGetLastError();
 }
 
+// ---- the stem
+
+namespace {
+
+int stem_band_rows(const GLayer &G)
+{
+    const int wpad = G.win + 2 * G.pad + 8;
+    int rows = 8;
+    while (rows > 1 && (size_t)((rows - 1) * G.stride + G.kh) * wpad * 4 > 24 * 1024) rows >>= 1;
+    return rows;
+}
+
+}  // namespace
+
+bool stem_fits(const GLayer &G, int in_c)
+{
+    if (G.op != ISC_CONV2D || in_c > 4 || G.kw > 8 || G.kh > 8 || G.coutp % 16 != 0 || G.coutp > 256) return false;
+    const int rows = stem_band_rows(G);
+    const size_t patch = (size_t)((rows - 1) * G.stride + G.kh) * (G.win + 2 * G.pad + 8) * 4;
+    const size_t total = (size_t)G.kh * G.coutp * 32 + 2 * (size_t)G.kh * kTileM * 32 + patch;
+    return total <= 100 * 1024;
+}
+
+size_t stem_pack_bytes(const GLayer &G) { return (size_t)G.kh * G.coutp * 32; }
+
+// w: [cout][cin][kh][kw] -> [filter row][2 columns of 16 bytes][coutp rows][16]: byte pix * 4 + ch of a row's 32
+void stem_pack_weights(const GLayer &G, const int8_t *w, int8_t *out)
+{
+    size_t at = 0;
+    for (int r = 0; r < G.kh; ++r)
+        for (int j = 0; j < 2; ++j)
+            for (int n = 0; n < G.coutp; ++n)
+                for (int e = 0; e < 16; ++e, ++at) {
+                    const int c32 = j * 16 + e, pix = c32 >> 2, ch = c32 & 3;
+                    out[at] = (n < G.cout && pix < G.kw && ch < G.cin) ? w[(((size_t)n * G.cin + ch) * G.kh + r) * G.kw + pix] : (int8_t)0;
+                }
+}
+
+cudaError_t launch_stem_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, const uint8_t *x_chw, int in_c,
+                             const NoiseStream &ns, int batch, int8_t *out, int32_t *err, cudaStream_t st)
+{
+    StemParams p;
+    p.L = G;
+    p.in_c = in_c;
+    p.band_rows = stem_band_rows(G);
+    p.n_bands = (G.hout + p.band_rows - 1) / p.band_rows;
+    p.tiles_per_band = (p.band_rows * G.wout + kTileM - 1) / kTileM;
+    int cols = 32;
+    while (cols < 2 * G.coutp) cols <<= 1;
+    p.tmem_cols = cols;
+    p.w_bytes = (uint32_t)stem_pack_bytes(G);
+    p.patch_bytes = (uint32_t)(((p.band_rows - 1) * G.stride + G.kh) * (G.win + 2 * G.pad + 8) * 4);
+    p.x = x_chw; p.ns = ns; p.wpack = wpack;
+    p.cst = reinterpret_cast<const int4 *>(cst);
+    p.fast_requant = fast ? 1 : 0;
+    p.lo = G.relu ? (G.zp_out > -128 ? G.zp_out : -128) : -128;
+    p.out = out; p.err = err;
+    const size_t smem = (size_t)p.w_bytes + 2 * (size_t)G.kh * kTileM * 32 + p.patch_bytes;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_stem, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    if (batch <= 0) return cudaSuccess;
+    dim3 grid((unsigned)p.n_bands, (unsigned)batch);
+    k_stem<<<grid, kThreads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
 }  // namespace isc
+

@@ -78,6 +78,13 @@ bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t 
 cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, int batch, const int8_t *in,
                               const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st);
 
+// The first convolution (<= 4 input channels, filter at most 8 x 8) on the tensor cores, noise drawn into its staging.
+bool stem_fits(const GLayer &G, int in_c);
+size_t stem_pack_bytes(const GLayer &G);
+void stem_pack_weights(const GLayer &G, const int8_t *w_oihw, int8_t *out);
+cudaError_t launch_stem_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, const uint8_t *x_chw, int in_c,
+                             const NoiseStream &ns, int batch, int8_t *out, int32_t *err, cudaStream_t st);
+
 // ---- host decision rules (isc_decide.cpp) ----
 double lower_conf_bound(int64_t k, int64_t n, double alpha);
 double normal_quantile(double p);
