@@ -196,21 +196,33 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
     __syncthreads();
     if (!abort_s) {
         const int8_t *res_px = (p.res && valid) ? p.res + (size_t)m * L.coutp : nullptr;
-        for (int c0 = 0; c0 < n_tile; c0 += 16) {
-            int acc[16];
-            tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc);
-            if (valid && n0 + c0 < L.coutp) {
-                uint4 v;
-                if (p.fast_requant && (!res_px || p.fast_residual)) {
-                    const uint32_t cst = smem_u32(cst_s + c0);
-                    if (res_px) v = requant16_fast<true>(acc, cst, __ldg(reinterpret_cast<const uint4 *>(res_px + n0 + c0)), p.res_m2, p.res_r2, p.lo);
-                    else v = requant16_fast<false>(acc, cst, make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
-                } else {
+        // 32 channels per step: two accumulator loads in flight, 32 contiguous bytes per pixel read and written
+        for (int c0 = 0; c0 < n_tile; c0 += 32) {
+            int acc[2][16];
+            tmem_ld16_issue(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc[0]);
+            tmem_ld16_issue(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0 + 16u, acc[1]);
+            uint4 rv[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+            if (res_px && p.fast_requant && p.fast_residual) {
+                rv[0] = __ldg(reinterpret_cast<const uint4 *>(res_px + n0 + c0));
+                rv[1] = __ldg(reinterpret_cast<const uint4 *>(res_px + n0 + c0) + 1);
+            }
+            tmem_ld_wait();
+            if (valid) {
 #pragma unroll
-                    for (int o = 0; o < 16; ++o) acc[o] += __ldg(L.bias + n0 + c0 + o);
-                    v = epilogue16(acc, L, n0 + c0, res_px);
+                for (int h = 0; h < 2; ++h) {
+                    const int cc = c0 + 16 * h;
+                    uint4 v;
+                    if (p.fast_requant && (!res_px || p.fast_residual)) {
+                        const uint32_t cst = smem_u32(cst_s + cc);
+                        if (res_px) v = requant16_fast<true>(acc[h], cst, rv[h], p.res_m2, p.res_r2, p.lo);
+                        else v = requant16_fast<false>(acc[h], cst, make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
+                    } else {
+#pragma unroll
+                        for (int o = 0; o < 16; ++o) acc[h][o] += __ldg(L.bias + n0 + cc + o);
+                        v = epilogue16(acc[h], L, n0 + cc, res_px);
+                    }
+                    *reinterpret_cast<uint4 *>(p.out + (size_t)m * L.coutp + n0 + cc) = v;
                 }
-                *reinterpret_cast<uint4 *>(p.out + (size_t)m * L.coutp + n0 + c0) = v;
             }
         }
     }
@@ -302,7 +314,7 @@ __global__ void __launch_bounds__(kThreads) k_stem(const __grid_constant__ StemP
                     if (e < e_begin || e >= e_end) continue;
                     const int rem = (int)(e - (int64_t)c * L.hin * L.win);
                     const int h = rem / L.win, w = rem - h * L.win;
-                    int v = (int)__ldg(p.x + e) + noise_level(u[k], p.ns.cum, p.ns.T);
+                    int v = (int)__ldg(p.x + e) + (p.ns.guide ? noise_level_guided(u[k], p.ns.cum, p.ns.guide, p.ns.T) : noise_level(u[k], p.ns.cum, p.ns.T));
                     v = min(255, max(0, v));
                     pb[((h - iy0) * wpad + (w + L.pad)) * 4 + c] = (uint8_t)v;
                 }

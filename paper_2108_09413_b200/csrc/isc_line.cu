@@ -724,20 +724,6 @@ __device__ void fill_phase(const EpiCtx &c, uint32_t off, uint32_t bytes, uint32
     for (uint32_t o = (uint32_t)c.tid * 16u; o < bytes; o += kThreads * 16u) st_shared_v4(c.sbase + off + o, v);
 }
 
-// Inverse-CDF search min{ z : u < cum[z] } (the last entry always matches) by bisection between the guide table's
-// results for the two uniforms that bracket u's top bits: the same result as the bisection over the whole table,
-// in one or two steps for the bulk of the distribution.
-__device__ __forceinline__ int noise_level_guided(uint32_t u, const uint32_t *__restrict__ cum, const uint32_t *__restrict__ guide, int T)
-{
-    const uint32_t j = u >> (32 - kNoiseGuideBits);
-    uint32_t lo = __ldg(guide + j), hi = __ldg(guide + j + 1);
-    while (lo < hi) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (u < __ldg(cum + mid)) hi = mid; else lo = mid + 1;
-    }
-    return (int)lo - T;
-}
-
 // INPUT: one thread = four horizontally adjacent pixels of one sample, all input channels (Def. 3.3, Def. 3.4).
 __device__ void input_phase(const LineParams &p, const EpiCtx &c, int grp)
 {

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "isc_internal.h"
+
 namespace isc {
 namespace tc {
 
@@ -228,6 +230,20 @@ __device__ __forceinline__ int noise_level(uint32_t u, const uint32_t *__restric
         if (u < __ldg(cum + mid)) hi = mid; else lo = mid + 1;
     }
     return lo - T;
+}
+
+// Inverse-CDF search min{ z : u < cum[z] } (the last entry always matches) by bisection between the guide table's
+// results for the two uniforms that bracket u's top bits: the same result as the bisection over the whole table,
+// in one or two steps for the bulk of the distribution.
+__device__ __forceinline__ int noise_level_guided(uint32_t u, const uint32_t *__restrict__ cum, const uint32_t *__restrict__ guide, int T)
+{
+    const uint32_t j = u >> (32 - kNoiseGuideBits);
+    uint32_t lo = __ldg(guide + j), hi = __ldg(guide + j + 1);
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (u < __ldg(cum + mid)) hi = mid; else lo = mid + 1;
+    }
+    return (int)lo - T;
 }
 
 }  // namespace tc
