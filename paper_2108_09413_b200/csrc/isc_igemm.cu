@@ -149,6 +149,21 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
     const uint4 zpv = make_uint4(zp4, zp4, zp4, zp4);
     bool ok = true;
 
+    // the operand rows of block kb + 1 are requested before block kb's are stored: their latency hides behind the
+    // barrier and the MMA issue of the current block
+    auto gather = [&](int kb, uint4 &v0, uint4 &v1, uint4 &v2, uint4 &v3) {
+        const int tap = kb / cblocks, cb = kb - tap * cblocks;
+        const int r = tap / L.kw, sx = tap - r * L.kw;
+        const int iy = oy * L.stride + r - L.pad, ix = ox * L.stride + sx - L.pad;
+        const bool inside = valid && iy >= 0 && iy < L.hin && ix >= 0 && ix < L.win;
+        v0 = zpv; v1 = zpv; v2 = zpv; v3 = zpv;                 // taps outside the image read the input zero-point
+        if (inside) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.in + ((b * L.hin + iy) * L.win + ix) * L.cinp + cb * kBlockK);
+            v0 = __ldg(src); v1 = __ldg(src + 1); v2 = __ldg(src + 2); v3 = __ldg(src + 3);
+        }
+    };
+    uint4 n0v, n1v, n2v, n3v;
+    gather(0, n0v, n1v, n2v, n3v);
     for (int kb = 0; kb < nkb; ++kb) {
         const int s = kb % kStages, use = kb / kStages;
         const uint32_t stage = sbase + (uint32_t)s * stage_bytes;
@@ -158,15 +173,8 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
             mbar_expect_tx(smem_u32(&bar_w[s]), b_bytes);
             bulk_g2s(stage + a_bytes, wtile + (size_t)kb * b_bytes, b_bytes, smem_u32(&bar_w[s]));
         }
-        const int tap = kb / cblocks, cb = kb - tap * cblocks;
-        const int r = tap / L.kw, sx = tap - r * L.kw;
-        const int iy = oy * L.stride + r - L.pad, ix = ox * L.stride + sx - L.pad;
-        const bool inside = valid && iy >= 0 && iy < L.hin && ix >= 0 && ix < L.win;
-        uint4 v0 = zpv, v1 = zpv, v2 = zpv, v3 = zpv;          // taps outside the image read the input zero-point
-        if (inside) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.in + ((b * L.hin + iy) * L.win + ix) * L.cinp + cb * kBlockK);
-            v0 = __ldg(src); v1 = __ldg(src + 1); v2 = __ldg(src + 2); v3 = __ldg(src + 3);
-        }
+        const uint4 v0 = n0v, v1 = n1v, v2 = n2v, v3 = n3v;
+        if (kb + 1 < nkb) gather(kb + 1, n0v, n1v, n2v, n3v);
         // K-major core matrices: 16-byte column j of row r at j * (128 rows * 16) + r * 16
         st_shared_v4(stage + 0 * 2048 + tid * 16, v0);
         st_shared_v4(stage + 1 * 2048 + tid * 16, v1);
