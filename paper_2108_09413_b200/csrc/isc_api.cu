@@ -64,7 +64,7 @@ struct isc_model {
     int8_t *d_logits = nullptr;   size_t d_logits_bytes = 0;
     uint32_t *d_cum = nullptr;    size_t d_cum_n = 0;
     double cum_sigma = -1.0;
-    int cum_T = 0, cum_kind = -1;
+    int cum_T = 0, cum_kind = -1, cum_steps = 0;
 
     isc::LinePlan *line = nullptr;
 
@@ -361,6 +361,11 @@ int ensure_noise_table(isc_model *m, double sigma, cudaStream_t st)
     m->cum_sigma = sigma;
     m->cum_kind = (int)m->opt_noise;
     m->cum_T = (int)(n_cum - 1) / 2;
+    // bisection steps that close the widest guide interval
+    uint32_t span = 0;
+    for (int j = 0; j < isc::kNoiseGuide; ++j) span = std::max(span, cum[n_cum + j + 1] - cum[n_cum + j]);
+    m->cum_steps = 0;
+    while ((1u << m->cum_steps) < span + 1) ++m->cum_steps;
     return ISC_OK;
 }
 
@@ -384,6 +389,7 @@ NoiseStream make_stream(const isc_model *m, uint64_t seed, uint64_t image_id, in
     ns.cum = m->d_cum;
     ns.T = m->cum_T;
     ns.guide = m->d_cum ? m->d_cum + (2 * m->cum_T + 1) : nullptr;
+    ns.guide_steps = m->cum_steps;
     return ns;
 }
 
@@ -1011,6 +1017,7 @@ extern "C" int isc_sample_counts_static(isc_model *m, const uint8_t *x_u8, uint6
         ns.cum = d_cum;
         ns.T = T;
         ns.guide = nullptr;
+        ns.guide_steps = 0;
         for (int i = 0; i < n_layers; ++i) {
             const GLayer &G = m->glayers[(size_t)i];
             const isc_layer &L = m->layers[(size_t)i].d;

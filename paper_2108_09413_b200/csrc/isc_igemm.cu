@@ -5,17 +5,25 @@
 //
 //   D[pixel, cout] = sum over (tap, cin) of A[pixel, (tap, cin)] * W[cout, (tap, cin)]
 //
-// A CTA owns a tile of 128 output pixels x N output channels (N = 64, 128 or 256) whose int32 accumulators live in
-// tensor memory.  The reduction runs in blocks of 64 input channels of one filter tap: the CTA's 128 threads gather
-// the block's operand rows (one thread = one pixel = 64 contiguous bytes, or the input zero-point outside the image)
-// into shared memory in the K-major core-matrix layout, one bulk copy brings the matching slice of the repacked
-// weights, and one thread issues two tcgen05.mma (kind::i8, K = 32 each).  Three stages of operands are in flight:
-// a stage is refilled when the commit of the MMAs that read it has arrived.  The epilogue reads the accumulators
-// back (one warp per 32-lane quarter), requantises (fixed-point multiplier, shift, zero-points, residual add, clamp)
-// and stores 16 channels per pixel at a time.  Every wait is bounded; on expiry the CTA sets an error word, frees its
-// tensor memory and returns.
+// A tile is 128 output pixels x N output channels (N = 64, 128 or 256) whose int32 accumulators live in tensor
+// memory.  The kernel is persistent (one CTA per SM, tiles dealt round-robin) and its warps have fixed roles that
+// meet only at mbarriers:
+//   * four warps gather operand rows: one thread = one pixel, per reduction block (64 input channels of one filter
+//     tap) four asynchronous 16-byte copies into the K-major core-matrix layout whose completion arrives on the
+//     stage's barrier; pixels outside the image are stored as the input zero-point;
+//   * one thread streams the matching slices of the repacked weights with bulk copies into the same stages;
+//   * one thread issues two tcgen05.mma (kind::i8, K = 32) per stage and commits the stage back to the loaders;
+//     accumulators alternate between two column ranges, so a tile's reduction runs under the previous one's
+//     epilogue;
+//   * two teams of four warps requantise (fixed-point multiplier, shift, zero-points, residual add, clamp), one
+//     accumulator each: a thread owns one tile row, the rows pass through a per-warp scratch area so that the
+//     residual operand is read and the result written in contiguous runs.
+// Every wait is bounded; on expiry a role raises the CTA's abort flag and the error word, the others leave their
+// loops, and the CTA frees its tensor memory and returns.
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include <algorithm>
 
 #include "isc_epilogue.cuh"
 #include "isc_internal.h"
@@ -29,14 +37,19 @@ namespace {
 
 constexpr int kTileM = 128;
 constexpr int kBlockK = 64;                  // bytes of K per stage: two MMA K-steps
-constexpr int kStages = 3;
-constexpr int kThreads = 128;
+constexpr unsigned kSleepLoad = 200, kSleepEpi = 100, kSleepMma = 0;      // ns between barrier polls, by role
+constexpr int kMaxStages = 16;
+constexpr int kStemThreads = 512;           // k_stem: four threads per tile row
+constexpr int kEpiWarps = 4, kEpiTeams = 2, kGatherWarps = 4;          // a team of epilogue warps takes every other tile
+constexpr int kAllEpiWarps = kEpiWarps * kEpiTeams;
+constexpr int kGemmThreads = 32 * (kAllEpiWarps + kGatherWarps + 2);      // k_igemm: + the MMA warp + the weights warp
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct IgemmParams {
     GLayer L;
-    int batch, n_tile, tmem_cols;
-    long long m_total;                       // batch * hout * wout
+    int batch, n_tile, tmem_cols, stages;
+    uint32_t scratch_off;                    // the epilogue warps' row scratch within the dynamic shared memory
+    long long m_total, tiles_m;              // batch * hout * wout; tiles of 128 of them
     const int8_t *in, *res;
     int8_t *out;
     const int8_t *wpack;                     // [cout tile][tap][cin block][4 K columns][n_tile rows][16 bytes]
@@ -89,7 +102,7 @@ __device__ __forceinline__ uint4 requant16_fast(const int *acc, uint32_t cst, ui
             int4 c;
             asm("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(c.x), "=r"(c.y), "=r"(c.z), "=r"(c.w) : "r"(cst + (4 * g + k) * 16));
             int v = (hi32(mul_wide(acc[4 * g + k] + c.x, c.y)) + c.z) >> c.w;
-            if (kRes) v += hi32(mad_wide_u((rw[g] >> (8 * k)) & 0xFFu, m2, r2));
+            if (kRes) v += hi32(mad_wide_u(__byte_perm(rw[g], 0u, 0x4440u | (uint32_t)k), m2, r2));
             y[k] = max(v, lo);
         }
         packed[g] = pack4_sat(y[0], y[1], y[2], y[3]);
@@ -107,27 +120,60 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity)
         if ((spin & 7) == 7 && globaltimer() - t0 > kWaitLimitNs) return false;
     }
 }
-
-
-__global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ IgemmParams p)
+// The same for the roles of k_igemm, which also give up when another role has raised the CTA's abort flag.  A role
+// that is far ahead of the others sleeps `kSleepNs` between polls so that its polling does not take issue slots
+// from the warps that do the arithmetic.
+template <unsigned kSleepNs>
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const volatile int *abort_flag)
 {
-    extern __shared__ __align__(128) uint8_t smem[];
-    __shared__ unsigned long long bar_w[kStages], bar_free[kStages], bar_done;
+    if (mbar_test(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer();
+    for (int spin = 0;; ++spin) {
+        if (mbar_try(bar, parity)) return true;
+        if (kSleepNs) __nanosleep(kSleepNs);
+        if ((spin & 7) == 7 && (*abort_flag || globaltimer() - t0 > kWaitLimitNs)) return false;
+    }
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// one arrival on `bar` (counted in its initial count) once every cp.async this thread has issued so far is complete
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// all of this thread's copy groups but the newest are complete
+__device__ __forceinline__ void cp_async_wait_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
+// A stage ring position: index and how many times the ring has wrapped.
+struct Ring {
+    int s = 0, use = 0;
+    __device__ __forceinline__ void advance(int stages) { if (++s == stages) { s = 0; ++use; } }
+};
+
+__global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant__ IgemmParams p)
+{
+    extern __shared__ __align__(128) uint8_t smem[];            // operand stages | requantisation constants | epilogue scratch
+    __shared__ unsigned long long bar_full[kMaxStages], bar_free[kMaxStages], bar_acc_full[2], bar_acc_free[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_s;
-    __shared__ __align__(16) int4 cst_s[256];
     const GLayer &L = p.L;
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t sbase = smem_u32(smem);
-    const int n_tile = p.n_tile;
+    const int n_tile = p.n_tile, stages = p.stages;
     const uint32_t a_bytes = kTileM * kBlockK, b_bytes = (uint32_t)n_tile * kBlockK, stage_bytes = a_bytes + b_bytes;
+    int4 *cst_s = reinterpret_cast<int4 *>(smem + (size_t)stages * stage_bytes);
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bar_w[s]), 1); mbar_init(smem_u32(&bar_free[s]), 1); }
-        mbar_init(smem_u32(&bar_done), 1);
+        for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&bar_full[s]), kGatherWarps * 32 + 1); mbar_init(smem_u32(&bar_free[s]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_free[i]), kEpiWarps * 32); }
         abort_s = 0;
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_base_s), (uint32_t)p.tmem_cols);
-    for (int i = tid; i < n_tile; i += kThreads) cst_s[i] = __ldg(p.cst + blockIdx.y * n_tile + i);
+    for (int i = tid; i < L.coutp; i += kGemmThreads) cst_s[i] = __ldg(p.cst + i);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
     tc_fence_before();
@@ -135,104 +181,191 @@ __global__ void __launch_bounds__(kThreads) k_igemm(const __grid_constant__ Igem
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
 
-    // this thread's output pixel = row `tid` of the tile
-    const long long m = (long long)blockIdx.x * kTileM + tid;
-    const bool valid = m < p.m_total;
-    const long long mm = valid ? m : 0;
-    const int ox = (int)(mm % L.wout), oy = (int)((mm / L.wout) % L.hout);
-    const long long b = mm / ((long long)L.wout * L.hout);
-    const int n0 = blockIdx.y * n_tile;
+    // tiles in m-major order (the CTAs of one wave share operand rows in L2), dealt round-robin to the CTAs
+    const int tiles_n = L.coutp / n_tile;
+    const long long n_tiles = p.tiles_m * tiles_n;
     const int cblocks = L.cinp / kBlockK, nkb = L.kh * L.kw * cblocks;
-    const int8_t *wtile = p.wpack + (size_t)blockIdx.y * (size_t)nkb * b_bytes;
-    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-    const uint32_t zp4 = (uint32_t)(L.zp_in & 0xFF) * 0x01010101u;
-    const uint4 zpv = make_uint4(zp4, zp4, zp4, zp4);
     bool ok = true;
 
-    // the operand rows of block kb + 1 are requested before block kb's are stored: their latency hides behind the
-    // barrier and the MMA issue of the current block
-    auto gather = [&](int kb, uint4 &v0, uint4 &v1, uint4 &v2, uint4 &v3) {
-        const int tap = kb / cblocks, cb = kb - tap * cblocks;
-        const int r = tap / L.kw, sx = tap - r * L.kw;
-        const int iy = oy * L.stride + r - L.pad, ix = ox * L.stride + sx - L.pad;
-        const bool inside = valid && iy >= 0 && iy < L.hin && ix >= 0 && ix < L.win;
-        v0 = zpv; v1 = zpv; v2 = zpv; v3 = zpv;                 // taps outside the image read the input zero-point
-        if (inside) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.in + ((b * L.hin + iy) * L.win + ix) * L.cinp + cb * kBlockK);
-            v0 = __ldg(src); v1 = __ldg(src + 1); v2 = __ldg(src + 2); v3 = __ldg(src + 3);
-        }
-    };
-    uint4 n0v, n1v, n2v, n3v;
-    gather(0, n0v, n1v, n2v, n3v);
-    for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % kStages, use = kb / kStages;
-        const uint32_t stage = sbase + (uint32_t)s * stage_bytes;
-        // the MMAs that read this stage last have completed
-        if (kb >= kStages && ok && !abort_s) ok = wait_bar(smem_u32(&bar_free[s]), (uint32_t)(use - 1) & 1u);
-        if (tid == 0) {
-            mbar_expect_tx(smem_u32(&bar_w[s]), b_bytes);
-            bulk_g2s(stage + a_bytes, wtile + (size_t)kb * b_bytes, b_bytes, smem_u32(&bar_w[s]));
-        }
-        const uint4 v0 = n0v, v1 = n1v, v2 = n2v, v3 = n3v;
-        if (kb + 1 < nkb) gather(kb + 1, n0v, n1v, n2v, n3v);
-        // K-major core matrices: 16-byte column j of row r at j * (128 rows * 16) + r * 16
-        st_shared_v4(stage + 0 * 2048 + tid * 16, v0);
-        st_shared_v4(stage + 1 * 2048 + tid * 16, v1);
-        st_shared_v4(stage + 2 * 2048 + tid * 16, v2);
-        st_shared_v4(stage + 3 * 2048 + tid * 16, v3);
-        fence_proxy_async();
-        __syncthreads();
-        if (tid == 0) {
-            if (ok && !abort_s) ok = wait_bar(smem_u32(&bar_w[s]), (uint32_t)use & 1u);
+    if (warp < kAllEpiWarps) {
+        // ---- epilogue: warp w owns lanes 32 (w mod 4) .. +31 of the accumulator (= 32 tile rows) and one group of
+        // `cpg` of its columns.  A thread requantises its own row; the rows pass through a per-warp scratch area in
+        // shared memory (row stride cpg + 16 bytes: conflict-free both ways) so that the residual operand is read
+        // and the result is written as runs of `cpg` contiguous bytes per row instead of 16 bytes per lane and row.
+        const int q = warp & 3;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const int team = warp / kEpiWarps;
+        const int cpg = n_tile / (kEpiWarps / 4), c_begin = ((warp >> 2) % (kEpiWarps / 4)) * cpg;
+        const uint32_t row_stride = (uint32_t)cpg + 16u;
+        const uint32_t scr0 = sbase + p.scratch_off + (uint32_t)warp * 32u * row_stride;
+        const int lpr = cpg >> 4, rpi = 32 / lpr;                       // lanes per row, rows per instruction
+        const int crow = lane / lpr, cchunk = lane - crow * lpr;
+        const bool fast = p.fast_requant && (!p.res || p.fast_residual);
+        const bool res_fast = p.res && fast;
+        auto residual_fetch = [&](long long t) {
+            const long long m_idx = t / tiles_n;
+            const long long m0 = m_idx * kTileM + q * 32;
+            const int8_t *src = p.res + (size_t)m0 * L.coutp + (int)(t - m_idx * tiles_n) * n_tile + c_begin + cchunk * 16;
+            const uint32_t dst = scr0 + (uint32_t)cchunk * 16u;
+            for (int k = 0; k < lpr; ++k) {
+                const int row = k * rpi + crow;
+                if (m0 + row < p.m_total) cp_async16(dst + (uint32_t)row * row_stride, src + (size_t)row * L.coutp);
+            }
+        };
+        // the team's tiles: every kEpiTeams-th of the CTA's, accumulator `team`
+        const long long t_step = (long long)kEpiTeams * gridDim.x;
+        long long t = blockIdx.x + (long long)team * gridDim.x;
+        if (res_fast && t < n_tiles) residual_fetch(t);
+        for (int au = 0; t < n_tiles; t += t_step, ++au) {
+            const long long m_idx = t / tiles_n;
+            const int n0 = (int)(t - m_idx * tiles_n) * n_tile;
+            const long long m0 = m_idx * kTileM + q * 32, m = m0 + lane;
+            const bool valid = m < p.m_total;
+            const int8_t *res_px = (p.res && valid) ? p.res + (size_t)m * L.coutp : nullptr;
+            const int buf = team;
+            cp_async_wait_all();                                // the tile's residual rows, requested after the previous tile
+            __syncwarp();
+            ok = wait_bar<kSleepEpi>(smem_u32(&bar_acc_full[buf]), (uint32_t)au & 1u, &abort_s);
+            if (!ok) break;
             tc_fence_after();
-            if (ok) {
-#pragma unroll
-                for (int k2 = 0; k2 < 2; ++k2) {
-                    const uint64_t ad = make_desc(stage + (uint32_t)k2 * 4096u, 2048u, 128u);
-                    const uint64_t bd = make_desc(stage + a_bytes + (uint32_t)k2 * 2u * (uint32_t)n_tile * 16u, (uint32_t)n_tile * 16u, 128u);
-                    mma_i8(tmem, ad, bd, idesc, (kb > 0 || k2 > 0) ? 1u : 0u);
+            const uint32_t acc_base = tmem + lane_base + (uint32_t)(buf * n_tile + c_begin);
+            const uint32_t scr_row = scr0 + (uint32_t)lane * row_stride;
+            for (int c0 = 0; c0 < cpg; c0 += 32) {
+                int acc[2][16];
+                tmem_ld16_issue(acc_base + (uint32_t)c0, acc[0]);
+                tmem_ld16_issue(acc_base + (uint32_t)c0 + 16u, acc[1]);
+                uint4 rv[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+                if (res_fast) {
+                    rv[0] = ld_shared_v4(scr_row + (uint32_t)c0);
+                    rv[1] = ld_shared_v4(scr_row + (uint32_t)c0 + 16u);
                 }
-            }
-            commit_to(smem_u32(&bar_free[s]));
-        }
-        if (!ok) abort_s = 1;
-    }
-    if (tid == 0) commit_to(smem_u32(&bar_done));
-    if (ok && !abort_s) ok = wait_bar(smem_u32(&bar_done), 0);
-    if (!ok) { abort_s = 1; atomicCAS(p.err, 0, 1 + (int)blockIdx.x); }
-    tc_fence_after();
-    __syncthreads();
-    if (!abort_s) {
-        const int8_t *res_px = (p.res && valid) ? p.res + (size_t)m * L.coutp : nullptr;
-        // 32 channels per step: two accumulator loads in flight, 32 contiguous bytes per pixel read and written
-        for (int c0 = 0; c0 < n_tile; c0 += 32) {
-            int acc[2][16];
-            tmem_ld16_issue(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc[0]);
-            tmem_ld16_issue(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0 + 16u, acc[1]);
-            uint4 rv[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-            if (res_px && p.fast_requant && p.fast_residual) {
-                rv[0] = __ldg(reinterpret_cast<const uint4 *>(res_px + n0 + c0));
-                rv[1] = __ldg(reinterpret_cast<const uint4 *>(res_px + n0 + c0) + 1);
-            }
-            tmem_ld_wait();
-            if (valid) {
+                tmem_ld_wait();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const int cc = c0 + 16 * h;
+                    const int cc = n0 + c_begin + c0 + 16 * h;
                     uint4 v;
-                    if (p.fast_requant && (!res_px || p.fast_residual)) {
+                    if (fast) {
                         const uint32_t cst = smem_u32(cst_s + cc);
-                        if (res_px) v = requant16_fast<true>(acc[h], cst, rv[h], p.res_m2, p.res_r2, p.lo);
+                        if (res_fast) v = requant16_fast<true>(acc[h], cst, rv[h], p.res_m2, p.res_r2, p.lo);
                         else v = requant16_fast<false>(acc[h], cst, make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
                     } else {
 #pragma unroll
-                        for (int o = 0; o < 16; ++o) acc[h][o] += __ldg(L.bias + n0 + cc + o);
-                        v = epilogue16(acc[h], L, n0 + cc, res_px);
+                        for (int o = 0; o < 16; ++o) acc[h][o] += __ldg(L.bias + cc + o);
+                        v = epilogue16(acc[h], L, cc, res_px);
                     }
-                    *reinterpret_cast<uint4 *>(p.out + (size_t)m * L.coutp + n0 + cc) = v;
+                    st_shared_v4(scr_row + (uint32_t)(c0 + 16 * h), v);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bar_acc_free[buf]));
+            __syncwarp();
+            {
+                int8_t *dst = p.out + (size_t)m0 * L.coutp + n0 + c_begin + cchunk * 16;
+                const uint32_t src = scr0 + (uint32_t)cchunk * 16u;
+                for (int k = 0; k < lpr; ++k) {
+                    const int row = k * rpi + crow;
+                    if (m0 + row < p.m_total) *reinterpret_cast<uint4 *>(dst + (size_t)row * L.coutp) = ld_shared_v4(src + (uint32_t)row * row_stride);
+                }
+            }
+            __syncwarp();
+            if (res_fast && t + t_step < n_tiles) residual_fetch(t + t_step);
+        }
+        cp_async_wait_all();
+    } else if (warp < kAllEpiWarps + kGatherWarps) {
+        // ---- operand rows: one thread per tile row, 64 bytes per block as four asynchronous 16-byte copies whose
+        // completion arrives on the stage's barrier; rows outside the image are stored as the input zero-point
+        const int row = tid - kAllEpiWarps * 32;
+        const uint32_t zp4 = (uint32_t)(L.zp_in & 0xFF) * 0x01010101u;
+        const uint4 zpv = make_uint4(zp4, zp4, zp4, zp4);
+        Ring ring;
+        for (long long t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+            const long long m = (t / tiles_n) * kTileM + row;
+            const bool valid = m < p.m_total;
+            const long long mm = valid ? m : 0;
+            const int ox = (int)(mm % L.wout), oy = (int)((mm / L.wout) % L.hout);
+            const int8_t *in_b = p.in + (mm / ((long long)L.wout * L.hout)) * ((long long)L.hin * L.win * L.cinp);
+            for (int tap = 0; tap < L.kh * L.kw && ok; ++tap) {
+                const int r = tap / L.kw, sx = tap - r * L.kw;
+                const int iy = oy * L.stride + r - L.pad, ix = ox * L.stride + sx - L.pad;
+                const bool inside = valid && iy >= 0 && iy < L.hin && ix >= 0 && ix < L.win;
+                const int8_t *src = in_b + ((long long)iy * L.win + ix) * L.cinp;
+                for (int cb = 0; cb < cblocks; ++cb, ring.advance(stages)) {
+                    if (ring.use >= 1) {
+                        ok = wait_bar<kSleepLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
+                        if (!ok) break;
+                    }
+                    // K-major core matrices: 16-byte column j of row r at j * (128 rows * 16) + r * 16
+                    const uint32_t dst = sbase + (uint32_t)ring.s * stage_bytes + (uint32_t)row * 16u;
+                    if (inside) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) cp_async16(dst + (uint32_t)c * 2048u, src + cb * kBlockK + c * 16);
+                        cp_async_arrive(smem_u32(&bar_full[ring.s]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) st_shared_v4(dst + (uint32_t)c * 2048u, zpv);
+                        fence_proxy_async();
+                        mbar_arrive(smem_u32(&bar_full[ring.s]));
+                    }
                 }
             }
         }
+        cp_async_wait_all();
+    } else if (warp == kAllEpiWarps + kGatherWarps) {
+        // ---- one thread issues the MMAs: two K-steps per stage, accumulators alternate between two column ranges
+        if (lane == 0) {
+            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            Ring ring;
+            int j = 0;
+            for (long long t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++j) {
+                const int buf = j & 1, au = j >> 1;
+                if (au >= 1) {
+                    ok = wait_bar<kSleepMma>(smem_u32(&bar_acc_free[buf]), (uint32_t)(au - 1) & 1u, &abort_s);
+                    if (!ok) break;
+                }
+                for (int kb = 0; kb < nkb; ++kb, ring.advance(stages)) {
+                    ok = wait_bar<kSleepMma>(smem_u32(&bar_full[ring.s]), (uint32_t)ring.use & 1u, &abort_s);
+                    if (!ok) break;
+                    fence_proxy_async();                        // the operand rows were written through the generic proxy
+                    tc_fence_after();
+                    const uint32_t stage = sbase + (uint32_t)ring.s * stage_bytes;
+#pragma unroll
+                    for (int k2 = 0; k2 < 2; ++k2) {
+                        const uint64_t ad = make_desc(stage + (uint32_t)k2 * 4096u, 2048u, 128u);
+                        const uint64_t bd = make_desc(stage + a_bytes + (uint32_t)k2 * 2u * (uint32_t)n_tile * 16u, (uint32_t)n_tile * 16u, 128u);
+                        mma_i8(tmem + (uint32_t)(buf * n_tile), ad, bd, idesc, (kb > 0 || k2 > 0) ? 1u : 0u);
+                    }
+                    commit_to(smem_u32(&bar_free[ring.s]));
+                }
+                if (ok) commit_to(smem_u32(&bar_acc_full[buf]));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---- one thread streams the repacked weights: one bulk copy per block into the stage's second part
+        if (lane == 0) {
+            Ring ring;
+            for (long long t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+                const int8_t *wtile = p.wpack + (size_t)(t % tiles_n) * (size_t)nkb * b_bytes;
+                for (int kb = 0; kb < nkb; ++kb, ring.advance(stages)) {
+                    if (ring.use >= 1) {
+                        ok = wait_bar<kSleepLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
+                        if (!ok) break;
+                    }
+                    mbar_expect_tx(smem_u32(&bar_full[ring.s]), b_bytes);
+                    bulk_g2s(sbase + (uint32_t)ring.s * stage_bytes + a_bytes, wtile + (size_t)kb * b_bytes, b_bytes, smem_u32(&bar_full[ring.s]));
+                }
+            }
+            if (!ok) {
+                // copies already issued may still be landing in this CTA's shared memory: give them time before the exit
+                const unsigned long long t0 = globaltimer();
+                while (globaltimer() - t0 < 50000ull) __nanosleep(1000);
+            }
+        }
+        __syncwarp();
+    }
+    if (!ok) {
+        if (!abort_s) atomicCAS(p.err, 0, 1 + (int)blockIdx.x);
+        abort_s = 1;
     }
     tc_fence_before();
     __syncthreads();
@@ -264,7 +397,7 @@ struct StemParams {
     int32_t *err;
 };
 
-__global__ void __launch_bounds__(kThreads) k_stem(const __grid_constant__ StemParams p)
+__global__ void __launch_bounds__(kStemThreads, 2) k_stem(const __grid_constant__ StemParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ unsigned long long bar_w, bar_full[2];
@@ -284,7 +417,7 @@ __global__ void __launch_bounds__(kThreads) k_stem(const __grid_constant__ StemP
         abort_s = 0;
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_base_s), (uint32_t)p.tmem_cols);
-    for (int i = tid; i < N; i += kThreads) cst_s[i] = __ldg(p.cst + i);
+    for (int i = tid; i < N; i += kStemThreads) cst_s[i] = __ldg(p.cst + i);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
     tc_fence_before();
@@ -305,49 +438,71 @@ __global__ void __launch_bounds__(kThreads) k_stem(const __grid_constant__ StemP
     const int rows_in = (oy1 - oy0 - 1) * L.stride + kh;
     uint32_t *patch = reinterpret_cast<uint32_t *>(smem + patch_off);
     const uint32_t zp_fill = (uint32_t)(L.zp_in & 0xFF) * (0x01010101u >> (8 * (4 - p.in_c)));
-    for (int i = tid; i < rows_in * wpad; i += kThreads) patch[i] = zp_fill;
+    for (int i = tid; i < rows_in * wpad; i += kStemThreads) patch[i] = zp_fill;
     __syncthreads();
     const int vy0 = max(0, iy0), vy1 = min(L.hin, iy0 + rows_in);
     if (vy1 > vy0) {
         uint8_t *pb = reinterpret_cast<uint8_t *>(patch);
         const uint32_t ctr3 = p.ns.ctr3_fixed | (uint32_t)(((j >> 32) & 0xFF) << 8);
-        for (int c = 0; c < p.in_c; ++c) {
-            const int64_t e_begin = ((int64_t)c * L.hin + vy0) * L.win, e_end = ((int64_t)c * L.hin + vy1) * L.win;
-            for (int64_t q = (e_begin >> 2) + tid; q < ((e_end + 3) >> 2); q += kThreads) {
-                const uint4 r = philox4x32_10(make_uint4((uint32_t)q, (uint32_t)(j & 0xFFFFFFFFll), p.ns.ctr2, ctr3), p.ns.key0, p.ns.key1);
-                const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+        const uint32_t ctr1 = (uint32_t)(j & 0xFFFFFFFFll);
+        if ((L.win & 3) == 0 && p.ns.guide) {
+            // every Philox block (four consecutive elements of the CHW order) lies within one image row: a thread
+            // takes whole blocks, all channels of the band's rows as one index space, the four searches interleaved
+            const int qpr = L.win >> 2, qpc = (vy1 - vy0) * qpr;
+            for (int i = tid; i < p.in_c * qpc; i += kStemThreads) {
+                const int c = i / qpc, ic = i - c * qpc;
+                const int hr = ic / qpr, wq = ic - hr * qpr;
+                const int h = vy0 + hr;
+                const uint32_t e = (uint32_t)((c * L.hin + h) * L.win) + 4u * (uint32_t)wq;
+                const uint4 r = philox4x32_10(make_uint4(e >> 2, ctr1, p.ns.ctr2, ctr3), p.ns.key0, p.ns.key1);
+                const uint32_t clean = __ldg(reinterpret_cast<const uint32_t *>(p.x + e));
+                int z[4];
+                noise_levels4(r, p.ns.cum, p.ns.guide, p.ns.T, p.ns.guide_steps, z);
+                uint8_t *dst = pb + ((h - iy0) * wpad + (4 * wq + L.pad)) * 4 + c;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int64_t e = q * 4 + k;
-                    if (e < e_begin || e >= e_end) continue;
-                    const int rem = (int)(e - (int64_t)c * L.hin * L.win);
-                    const int h = rem / L.win, w = rem - h * L.win;
-                    int v = (int)__ldg(p.x + e) + (p.ns.guide ? noise_level_guided(u[k], p.ns.cum, p.ns.guide, p.ns.T) : noise_level(u[k], p.ns.cum, p.ns.T));
-                    v = min(255, max(0, v));
-                    pb[((h - iy0) * wpad + (w + L.pad)) * 4 + c] = (uint8_t)v;
+                for (int k = 0; k < 4; ++k) dst[4 * k] = (uint8_t)min(255, max(0, (int)((clean >> (8 * k)) & 0xFFu) + z[k]));
+            }
+        } else {
+            for (int c = 0; c < p.in_c; ++c) {
+                const int64_t e_begin = ((int64_t)c * L.hin + vy0) * L.win, e_end = ((int64_t)c * L.hin + vy1) * L.win;
+                for (int64_t q = (e_begin >> 2) + tid; q < ((e_end + 3) >> 2); q += kStemThreads) {
+                    const uint4 r = philox4x32_10(make_uint4((uint32_t)q, ctr1, p.ns.ctr2, ctr3), p.ns.key0, p.ns.key1);
+                    const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int64_t e = q * 4 + k;
+                        if (e < e_begin || e >= e_end) continue;
+                        const int rem = (int)(e - (int64_t)c * L.hin * L.win);
+                        const int h = rem / L.win, w = rem - h * L.win;
+                        int v = (int)__ldg(p.x + e) + (p.ns.guide ? noise_level_guided(u[k], p.ns.cum, p.ns.guide, p.ns.T) : noise_level(u[k], p.ns.cum, p.ns.T));
+                        v = min(255, max(0, v));
+                        pb[((h - iy0) * wpad + (w + L.pad)) * 4 + c] = (uint8_t)v;
+                    }
                 }
             }
         }
     }
     __syncthreads();
 
-    // ---- tiles of 128 output pixels of the band
+    // ---- tiles of 128 output pixels of the band.  Thread = tile row `px` x one of four groups: a group copies every
+    // fourth filter row's windows and requantises every fourth 16-channel chunk.
     const int band_px = (oy1 - oy0) * L.wout;
     const int n_tiles = (band_px + kTileM - 1) / kTileM;
     const uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    const int px_row = tid & (kTileM - 1), grp = tid >> 7;
     bool ok = true;
     if (tid == 0) ok = wait_bar(smem_u32(&bar_w), 0);
     for (int t = 0; t <= n_tiles; ++t) {
         if (t < n_tiles) {
             // operand stage of tile t: free once the MMAs of tile t - 2 are complete (waited for by its epilogue below)
             const uint32_t stage = sbase + a_off + (uint32_t)(t & 1) * a_bytes;
-            const int px = t * kTileM + tid;
+            const int px = t * kTileM + px_row;
             const int pp = px < band_px ? px : 0;
             const int oyl = pp / L.wout, ox = pp - oyl * L.wout;
-            for (int r = 0; r < kh; ++r) {
+            for (int r = grp; r < kh; r += kStemThreads / kTileM) {
                 const uint32_t *src = patch + (oyl * L.stride + r) * wpad + ox * L.stride;
-                st_shared_v4(stage + (uint32_t)r * 4096u + 0u * 2048u + tid * 16, make_uint4(src[0], src[1], src[2], src[3]));
-                st_shared_v4(stage + (uint32_t)r * 4096u + 1u * 2048u + tid * 16, make_uint4(src[4], src[5], src[6], src[7]));
+                st_shared_v4(stage + (uint32_t)r * 4096u + 0u * 2048u + px_row * 16, make_uint4(src[0], src[1], src[2], src[3]));
+                st_shared_v4(stage + (uint32_t)r * 4096u + 1u * 2048u + px_row * 16, make_uint4(src[4], src[5], src[6], src[7]));
             }
             fence_proxy_async();
         }
@@ -370,12 +525,12 @@ __global__ void __launch_bounds__(kThreads) k_stem(const __grid_constant__ StemP
             if (ok && !abort_s) ok = wait_bar(smem_u32(&bar_full[tt & 1]), (uint32_t)(tt >> 1) & 1u);
             if (!ok) abort_s = 1;
             tc_fence_after();
-            const int px = tt * kTileM + tid;
+            const int px = tt * kTileM + px_row;
             const bool valid = px < band_px;
             const size_t m = ((size_t)b * L.hout + oy0) * L.wout + (size_t)(valid ? px : 0);
-            for (int c0 = 0; c0 < N; c0 += 16) {
+            for (int c0 = 16 * grp; c0 < N; c0 += 16 * (kStemThreads / kTileM)) {
                 int acc[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(tt & 1) * (uint32_t)N + (uint32_t)c0, acc);
+                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(tt & 1) * (uint32_t)N + (uint32_t)c0, acc);
                 if (valid && !abort_s) {
                     uint4 v;
                     if (p.fast_requant) {
@@ -466,20 +621,31 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
     p.batch = batch;
     p.n_tile = igemm_tile_n(G);
     if (p.n_tile == 0) return cudaErrorInvalidValue;
-    p.tmem_cols = p.n_tile < 32 ? 32 : p.n_tile;
+    p.tmem_cols = 2 * p.n_tile;                                  // two accumulators: 128, 256 or 512 columns
     p.m_total = (long long)batch * G.hout * G.wout;
+    p.tiles_m = (p.m_total + kTileM - 1) / kTileM;
     p.in = in; p.res = res; p.out = out; p.wpack = wpack; p.err = err;
-    const size_t smem = (size_t)kStages * ((size_t)kTileM * kBlockK + (size_t)p.n_tile * kBlockK);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_igemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kStages * (kTileM + 256) * kBlockK));
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    if (p.tiles_m <= 0) return cudaSuccess;
+    // as many operand stages as fit beside the constants, at most kMaxStages
+    const size_t stage_bytes = (size_t)kTileM * kBlockK + (size_t)p.n_tile * kBlockK, cst_bytes = (size_t)G.coutp * 16;
+    const size_t scratch_bytes = (size_t)kAllEpiWarps * 32 * ((size_t)p.n_tile / (kEpiWarps / 4) + 16);
+    const size_t smem_limit = 226 * 1024;
+    if (cst_bytes + scratch_bytes + 2 * stage_bytes > smem_limit) return cudaErrorInvalidValue;
+    p.stages = (int)std::min<size_t>(kMaxStages, (smem_limit - cst_bytes - scratch_bytes) / stage_bytes);
+    p.scratch_off = (uint32_t)((size_t)p.stages * stage_bytes + cst_bytes);
+    const size_t smem = (size_t)p.stages * stage_bytes + cst_bytes + scratch_bytes;
+    static int n_sms = 0;
+    if (n_sms == 0) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_igemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_limit);
+        if (e != cudaSuccess) { n_sms = 0; return e; }
     }
-    const long long tiles_m = (p.m_total + kTileM - 1) / kTileM;
-    if (tiles_m <= 0) return cudaSuccess;
-    dim3 grid((unsigned)tiles_m, (unsigned)(G.coutp / p.n_tile));
-    k_igemm<<<grid, kThreads, smem, st>>>(p);
+    // persistent: one CTA per SM (shared memory and the 512 tensor-memory columns allow no second one at N = 256)
+    const long long n_tiles = p.tiles_m * (G.coutp / p.n_tile);
+    const unsigned grid = (unsigned)std::min<long long>(n_tiles, n_sms);
+    k_igemm<<<grid, kGemmThreads, smem, st>>>(p);
     return cudaGetLastError();
 }
 
@@ -549,7 +715,7 @@ cudaError_t launch_stem_conv(const GLayer &G, const int8_t *wpack, const int32_t
     }
     if (batch <= 0) return cudaSuccess;
     dim3 grid((unsigned)p.n_bands, (unsigned)batch);
-    k_stem<<<grid, kThreads, smem, st>>>(p);
+    k_stem<<<grid, kStemThreads, smem, st>>>(p);
     return cudaGetLastError();
 }
 

@@ -28,6 +28,7 @@ struct NoiseStream {
     // Optional guide table (device, kNoiseGuide + 1 entries, or null): guide[j] is the search result for the
     // uniform j << (32 - kNoiseGuideBits), a lower bound of the result for every uniform with these top bits.
     const uint32_t *guide;
+    int guide_steps;          // bisection steps that close the widest interval [guide[j], guide[j+1]]
 };
 
 // One layer as the layer-by-layer kernels see it (device pointers).

@@ -246,5 +246,32 @@ __device__ __forceinline__ int noise_level_guided(uint32_t u, const uint32_t *__
     return (int)lo - T;
 }
 
+// The same search for the four uniforms of one Philox block with a fixed number of bisection steps (`steps` covers the
+// widest guide interval; a step on an interval that has already closed changes nothing, since u < cum[result]), so
+// that the four dependent load chains run interleaved.
+__device__ __forceinline__ void noise_levels4(uint4 u4, const uint32_t *__restrict__ cum, const uint32_t *__restrict__ guide, int T,
+                                              int steps, int (&z)[4])
+{
+    const uint32_t u[4] = {u4.x, u4.y, u4.z, u4.w};
+    uint32_t lo[4], hi[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t j = u[k] >> (32 - kNoiseGuideBits);
+        lo[k] = __ldg(guide + j);
+        hi[k] = __ldg(guide + j + 1);
+    }
+    for (int s = 0; s < steps; ++s) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t mid = (lo[k] + hi[k]) >> 1;
+            const bool below = u[k] < __ldg(cum + mid);
+            hi[k] = below ? mid : hi[k];
+            lo[k] = below ? lo[k] : min(mid + 1, hi[k]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) z[k] = (int)lo[k] - T;
+}
+
 }  // namespace tc
 }  // namespace isc
