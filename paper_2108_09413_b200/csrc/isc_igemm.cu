@@ -8,9 +8,10 @@
 // A tile is 128 output pixels x N output channels (N = 64, 128 or 256) whose int32 accumulators live in tensor
 // memory.  The kernel is persistent (one CTA per SM, tiles dealt round-robin) and its warps have fixed roles that
 // meet only at mbarriers:
-//   * four warps gather operand rows: one thread = one pixel, per reduction block (64 input channels of one filter
-//     tap) four asynchronous 16-byte copies into the K-major core-matrix layout whose completion arrives on the
-//     stage's barrier; pixels outside the image are stored as the input zero-point;
+//   * four warps gather operand rows: per reduction block (64 input channels of one filter tap) a lane issues four
+//     asynchronous 16-byte copies into the K-major core-matrix layout (four lanes read one pixel's 64 bytes) whose
+//     completion arrives on the stage's barrier; a pixel outside the image is copied from a run of the input
+//     zero-point kept behind the repacked weights;
 //   * one thread streams the matching slices of the repacked weights with bulk copies into the same stages;
 //   * one thread issues two tcgen05.mma (kind::i8, K = 32) per stage and commits the stage back to the loaders;
 //     accumulators alternate between two column ranges, so a tile's reduction runs under the previous one's
@@ -49,7 +50,7 @@ struct IgemmParams {
     GLayer L;
     int batch, n_tile, tmem_cols, stages;
     uint32_t scratch_off;                    // the epilogue warps' row scratch within the dynamic shared memory
-    long long m_total, tiles_m;              // batch * hout * wout; tiles of 128 of them
+    uint32_t m_total, tiles_m;               // batch * hout * wout (< 2^31); tiles of 128 of them
     const int8_t *in, *res;
     int8_t *out;
     const int8_t *wpack;                     // [cout tile][tap][cin block][4 K columns][n_tile rows][16 bytes]
@@ -139,6 +140,11 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+// the same through L1: for a source that every CTA reads again and again
+__device__ __forceinline__ void cp_async16_cached(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
 // one arrival on `bar` (counted in its initial count) once every cp.async this thread has issued so far is complete
 __device__ __forceinline__ void cp_async_arrive(uint32_t bar)
 {
@@ -183,7 +189,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
 
     // tiles in m-major order (the CTAs of one wave share operand rows in L2), dealt round-robin to the CTAs
     const int tiles_n = L.coutp / n_tile;
-    const long long n_tiles = p.tiles_m * tiles_n;
+    const uint32_t n_tiles = p.tiles_m * (uint32_t)tiles_n, grid_n = gridDim.x;
     const int cblocks = L.cinp / kBlockK, nkb = L.kh * L.kw * cblocks;
     bool ok = true;
 
@@ -202,9 +208,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
         const int crow = lane / lpr, cchunk = lane - crow * lpr;
         const bool fast = p.fast_requant && (!p.res || p.fast_residual);
         const bool res_fast = p.res && fast;
-        auto residual_fetch = [&](long long t) {
-            const long long m_idx = t / tiles_n;
-            const long long m0 = m_idx * kTileM + q * 32;
+        auto residual_fetch = [&](uint32_t t) {
+            const uint32_t m_idx = t / (uint32_t)tiles_n;
+            const uint32_t m0 = m_idx * kTileM + (uint32_t)q * 32u;
             const int8_t *src = p.res + (size_t)m0 * L.coutp + (int)(t - m_idx * tiles_n) * n_tile + c_begin + cchunk * 16;
             const uint32_t dst = scr0 + (uint32_t)cchunk * 16u;
             for (int k = 0; k < lpr; ++k) {
@@ -213,13 +219,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
             }
         };
         // the team's tiles: every kEpiTeams-th of the CTA's, accumulator `team`
-        const long long t_step = (long long)kEpiTeams * gridDim.x;
-        long long t = blockIdx.x + (long long)team * gridDim.x;
+        const uint32_t t_step = (uint32_t)kEpiTeams * grid_n;
+        uint32_t t = blockIdx.x + (uint32_t)team * grid_n;
         if (res_fast && t < n_tiles) residual_fetch(t);
         for (int au = 0; t < n_tiles; t += t_step, ++au) {
-            const long long m_idx = t / tiles_n;
+            const uint32_t m_idx = t / (uint32_t)tiles_n;
             const int n0 = (int)(t - m_idx * tiles_n) * n_tile;
-            const long long m0 = m_idx * kTileM + q * 32, m = m0 + lane;
+            const uint32_t m0 = m_idx * kTileM + (uint32_t)q * 32u, m = m0 + (uint32_t)lane;
             const bool valid = m < p.m_total;
             const int8_t *res_px = (p.res && valid) ? p.res + (size_t)m * L.coutp : nullptr;
             const int buf = team;
@@ -272,40 +278,48 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
         }
         cp_async_wait_all();
     } else if (warp < kAllEpiWarps + kGatherWarps) {
-        // ---- operand rows: one thread per tile row, 64 bytes per block as four asynchronous 16-byte copies whose
-        // completion arrives on the stage's barrier; rows outside the image are stored as the input zero-point
-        const int row = tid - kAllEpiWarps * 32;
-        const uint32_t zp4 = (uint32_t)(L.zp_in & 0xFF) * 0x01010101u;
-        const uint4 zpv = make_uint4(zp4, zp4, zp4, zp4);
+        // ---- operand rows: per reduction block a warp copies 32 tile rows x 64 bytes with four asynchronous 16-byte
+        // copies per lane (lane = 16-byte column x row within a group of eight, so that an instruction reads whole
+        // 64-byte rows) whose completion arrives on the stage's barrier.  A row outside the image is copied from a
+        // 64-byte run of the input zero-point that follows the repacked weights, so every row takes the same path.
+        const int gw = warp - kAllEpiWarps, chunk = lane & 3, rsub = lane >> 2;
+        const int8_t *zp_src = p.wpack + (size_t)L.coutp * (size_t)(L.kh * L.kw) * (size_t)L.cinp + chunk * 16;
+        const int8_t *in_c = p.in + chunk * 16;
+        // K-major core matrices: 16-byte column j of row r at j * (128 rows * 16) + r * 16
+        const uint32_t dst0 = sbase + (uint32_t)chunk * 2048u + (uint32_t)(32 * gw + rsub) * 16u;
         Ring ring;
-        for (long long t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-            const long long m = (t / tiles_n) * kTileM + row;
-            const bool valid = m < p.m_total;
-            const long long mm = valid ? m : 0;
-            const int ox = (int)(mm % L.wout), oy = (int)((mm / L.wout) % L.hout);
-            const int8_t *in_b = p.in + (mm / ((long long)L.wout * L.hout)) * ((long long)L.hin * L.win * L.cinp);
-            for (int tap = 0; tap < L.kh * L.kw && ok; ++tap) {
-                const int r = tap / L.kw, sx = tap - r * L.kw;
-                const int iy = oy * L.stride + r - L.pad, ix = ox * L.stride + sx - L.pad;
-                const bool inside = valid && iy >= 0 && iy < L.hin && ix >= 0 && ix < L.win;
-                const int8_t *src = in_b + ((long long)iy * L.win + ix) * L.cinp;
+        const uint32_t px_per_sample = (uint32_t)(L.hout * L.wout);
+        for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += grid_n) {
+            const uint32_t m0 = (t / (uint32_t)tiles_n) * kTileM + (uint32_t)(32 * gw + rsub);
+            int iy0[4], ix0[4], off[4];                         // this lane's four rows: 8 apart
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t m = m0 + 8u * (uint32_t)i;
+                const bool valid = m < p.m_total;
+                const uint32_t mm = valid ? m : 0u;
+                const uint32_t b = mm / px_per_sample, pp = mm - b * px_per_sample;
+                const int oy = (int)(pp / (uint32_t)L.wout), ox = (int)pp - oy * L.wout;
+                iy0[i] = valid ? oy * L.stride - L.pad : -0x100000;             // an invalid row is outside for every tap
+                ix0[i] = ox * L.stride - L.pad;
+                off[i] = (((int)b * L.hin + oy * L.stride - L.pad) * L.win + ix0[i]) * L.cinp;    // the tensor is < 2^31 bytes
+            }
+            for (int tap = 0, r = 0, sx = 0; tap < L.kh * L.kw && ok; ++tap, sx = (sx + 1 == L.kw) ? 0 : sx + 1, r += (sx == 0)) {
+                const int tap_off = (r * L.win + sx) * L.cinp;
+                bool inside[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) inside[i] = (unsigned)(iy0[i] + r) < (unsigned)L.hin && (unsigned)(ix0[i] + sx) < (unsigned)L.win;
                 for (int cb = 0; cb < cblocks; ++cb, ring.advance(stages)) {
                     if (ring.use >= 1) {
                         ok = wait_bar<kSleepLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
                         if (!ok) break;
                     }
-                    // K-major core matrices: 16-byte column j of row r at j * (128 rows * 16) + r * 16
-                    const uint32_t dst = sbase + (uint32_t)ring.s * stage_bytes + (uint32_t)row * 16u;
-                    if (inside) {
+                    const uint32_t dst = dst0 + (uint32_t)ring.s * stage_bytes;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) cp_async16(dst + (uint32_t)c * 2048u, src + cb * kBlockK + c * 16);
-                        cp_async_arrive(smem_u32(&bar_full[ring.s]));
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) st_shared_v4(dst + (uint32_t)c * 2048u, zpv);
-                        fence_proxy_async();
-                        mbar_arrive(smem_u32(&bar_full[ring.s]));
+                    for (int i = 0; i < 4; ++i) {
+                        if (inside[i]) cp_async16(dst + (uint32_t)i * 128u, in_c + (off[i] + tap_off + cb * kBlockK));
+                        else cp_async16_cached(dst + (uint32_t)i * 128u, zp_src);
                     }
+                    cp_async_arrive(smem_u32(&bar_full[ring.s]));
                 }
             }
         }
@@ -316,7 +330,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             Ring ring;
             int j = 0;
-            for (long long t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++j) {
+            for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += grid_n, ++j) {
                 const int buf = j & 1, au = j >> 1;
                 if (au >= 1) {
                     ok = wait_bar<kSleepMma>(smem_u32(&bar_acc_free[buf]), (uint32_t)(au - 1) & 1u, &abort_s);
@@ -325,7 +339,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
                 for (int kb = 0; kb < nkb; ++kb, ring.advance(stages)) {
                     ok = wait_bar<kSleepMma>(smem_u32(&bar_full[ring.s]), (uint32_t)ring.use & 1u, &abort_s);
                     if (!ok) break;
-                    fence_proxy_async();                        // the operand rows were written through the generic proxy
                     tc_fence_after();
                     const uint32_t stage = sbase + (uint32_t)ring.s * stage_bytes;
 #pragma unroll
@@ -344,7 +357,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
         // ---- one thread streams the repacked weights: one bulk copy per block into the stage's second part
         if (lane == 0) {
             Ring ring;
-            for (long long t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+            for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += grid_n) {
                 const int8_t *wtile = p.wpack + (size_t)(t % tiles_n) * (size_t)nkb * b_bytes;
                 for (int kb = 0; kb < nkb; ++kb, ring.advance(stages)) {
                     if (ring.use >= 1) {
@@ -566,9 +579,10 @@ int igemm_tile_n(const GLayer &G)
     return 0;
 }
 
+// the repacked weights, then 64 bytes of the input zero-point (the operand row of a pixel outside the image)
 size_t igemm_pack_bytes(const GLayer &G)
 {
-    return (size_t)G.coutp * (size_t)(G.kh * G.kw) * (size_t)G.cinp;
+    return (size_t)G.coutp * (size_t)(G.kh * G.kw) * (size_t)G.cinp + kBlockK;
 }
 
 // w: [cout][cin][kh][kw] as the model gives it -> [cout tile][tap][cin block][4 columns of 16 channels][n_tile rows][16]
@@ -585,6 +599,7 @@ void igemm_pack_weights(const GLayer &G, const int8_t *w, int8_t *out)
                             const int oc = t * n_tile + n, ci = cb * kBlockK + j * 16 + e;
                             out[at] = (oc < G.cout && ci < G.cin) ? w[((size_t)oc * G.cin + ci) * taps + tap] : (int8_t)0;
                         }
+    for (int e = 0; e < kBlockK; ++e) out[at + e] = (int8_t)G.zp_in;
 }
 
 // Per output channel {folded bias, multiplier, rounding addend, shift - 1}; returns whether every shift is >= 2 (the
@@ -622,10 +637,12 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
     p.n_tile = igemm_tile_n(G);
     if (p.n_tile == 0) return cudaErrorInvalidValue;
     p.tmem_cols = 2 * p.n_tile;                                  // two accumulators: 128, 256 or 512 columns
-    p.m_total = (long long)batch * G.hout * G.wout;
+    const long long m_total = (long long)batch * G.hout * G.wout;
+    if (m_total >= (1ll << 31) / (G.coutp / p.n_tile) || (long long)batch * G.hin * G.win * G.cinp >= (1ll << 31)) return cudaErrorInvalidValue;
+    p.m_total = (uint32_t)m_total;
     p.tiles_m = (p.m_total + kTileM - 1) / kTileM;
     p.in = in; p.res = res; p.out = out; p.wpack = wpack; p.err = err;
-    if (p.tiles_m <= 0) return cudaSuccess;
+    if (p.tiles_m == 0) return cudaSuccess;
     // as many operand stages as fit beside the constants, at most kMaxStages
     const size_t stage_bytes = (size_t)kTileM * kBlockK + (size_t)p.n_tile * kBlockK, cst_bytes = (size_t)G.coutp * 16;
     const size_t scratch_bytes = (size_t)kAllEpiWarps * 32 * ((size_t)p.n_tile / (kEpiWarps / 4) + 16);
@@ -643,8 +660,8 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
         if (e != cudaSuccess) { n_sms = 0; return e; }
     }
     // persistent: one CTA per SM (shared memory and the 512 tensor-memory columns allow no second one at N = 256)
-    const long long n_tiles = p.tiles_m * (G.coutp / p.n_tile);
-    const unsigned grid = (unsigned)std::min<long long>(n_tiles, n_sms);
+    const uint32_t n_tiles = p.tiles_m * (uint32_t)(G.coutp / p.n_tile);
+    const unsigned grid = std::min<uint32_t>(n_tiles, (uint32_t)n_sms);
     k_igemm<<<grid, kGemmThreads, smem, st>>>(p);
     return cudaGetLastError();
 }
