@@ -423,7 +423,10 @@ int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int
         else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, batch, in, out, st);
         else e = launch_maxpool(G, batch, in, out, st);
         m->launches += 1;
-        if (e != cudaSuccess) return ISC_ERR_CUDA;
+        if (e != cudaSuccess) {
+            if (getenv("ISC_DEBUG_CUDA")) fprintf(stderr, "isc: layer %d launch: %s\n", i, cudaGetErrorString(e));
+            return ISC_ERR_CUDA;
+        }
         if (i == stop_after_layer) break;
     }
     return ISC_OK;

@@ -17,8 +17,9 @@
 //     accumulators alternate between two column ranges, so a tile's reduction runs under the previous one's
 //     epilogue;
 //   * two teams of four warps requantise (fixed-point multiplier, shift, zero-points, residual add, clamp), one
-//     accumulator each: a thread owns one tile row, the rows pass through a per-warp scratch area so that the
-//     residual operand is read and the result written in contiguous runs.
+//     accumulator each: a thread owns one tile row, 32 columns per step with the next step's accumulators already
+//     requested; the rows pass through a per-warp scratch area so that, every 64 columns, the results leave and the
+//     next tile's residual rows arrive as contiguous runs, under the arithmetic of the following columns.
 // Every wait is bounded; on expiry a role raises the CTA's abort flag and the error word, the others leave their
 // loops, and the CTA frees its tensor memory and returns.
 #include <cuda_runtime.h>
@@ -38,11 +39,12 @@ namespace {
 
 constexpr int kTileM = 128;
 constexpr int kBlockK = 64;                  // bytes of K per stage: two MMA K-steps
-constexpr unsigned kSleepLoad = 200, kSleepEpi = 100, kSleepMma = 0;      // ns between barrier polls, by role
+constexpr unsigned kSleepLoad = 20000, kSleepEpi = 20000, kSleepMma = 20000;      // suspend-time hint of a barrier wait (ns), by role
 constexpr int kMaxStages = 16;
 constexpr int kStemThreads = 512;           // k_stem: four threads per tile row
 constexpr int kEpiWarps = 4, kEpiTeams = 2, kGatherWarps = 4;          // a team of epilogue warps takes every other tile
 constexpr int kAllEpiWarps = kEpiWarps * kEpiTeams;
+static_assert(kEpiWarps == 4, "an epilogue warp owns all N columns of its 32 rows");
 constexpr int kGemmThreads = 32 * (kAllEpiWarps + kGatherWarps + 2);      // k_igemm: + the MMA warp + the weights warp
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -111,6 +113,23 @@ __device__ __forceinline__ uint4 requant16_fast(const int *acc, uint32_t cst, ui
     return make_uint4(packed[0], packed[1], packed[2], packed[3]);
 }
 
+// 32 accumulator columns of this thread's lane, asynchronously; the registers are valid after tmem_ld32_wait(),
+// which names them so that no use can move above it
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, int (&v)[2][16])
+{
+    tmem_ld16_issue(taddr, v[0]);
+    tmem_ld16_issue(taddr + 16u, v[1]);
+}
+__device__ __forceinline__ void tmem_ld32_wait(int (&v)[2][16])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0][0]), "+r"(v[0][1]), "+r"(v[0][2]), "+r"(v[0][3]), "+r"(v[0][4]), "+r"(v[0][5]), "+r"(v[0][6]), "+r"(v[0][7]),
+                   "+r"(v[0][8]), "+r"(v[0][9]), "+r"(v[0][10]), "+r"(v[0][11]), "+r"(v[0][12]), "+r"(v[0][13]), "+r"(v[0][14]), "+r"(v[0][15]),
+                   "+r"(v[1][0]), "+r"(v[1][1]), "+r"(v[1][2]), "+r"(v[1][3]), "+r"(v[1][4]), "+r"(v[1][5]), "+r"(v[1][6]), "+r"(v[1][7]),
+                   "+r"(v[1][8]), "+r"(v[1][9]), "+r"(v[1][10]), "+r"(v[1][11]), "+r"(v[1][12]), "+r"(v[1][13]), "+r"(v[1][14]), "+r"(v[1][15])
+                 :: "memory");
+}
+
 // Bounded wait for a phase of an mbarrier; false after the limit (the caller raises the error word).
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity)
 {
@@ -130,8 +149,17 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const vo
     if (mbar_test(bar, parity)) return true;
     const unsigned long long t0 = globaltimer();
     for (int spin = 0;; ++spin) {
-        if (mbar_try(bar, parity)) return true;
-        if (kSleepNs) __nanosleep(kSleepNs);
+        if (kSleepNs) {
+            // parked in hardware until the phase completes or the hint runs out
+            uint32_t done;
+            asm volatile("{\n\t.reg .pred p;\n\t"
+                         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+                         "selp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(done) : "r"(bar), "r"(parity), "r"(kSleepNs) : "memory");
+            if (done) return true;
+        } else if (mbar_try(bar, parity)) {
+            return true;
+        }
         if ((spin & 7) == 7 && (*abort_flag || globaltimer() - t0 > kWaitLimitNs)) return false;
     }
 }
@@ -160,6 +188,118 @@ struct Ring {
     int s = 0, use = 0;
     __device__ __forceinline__ void advance(int stages) { if (++s == stages) { s = 0; ++use; } }
 };
+
+// What an epilogue warp needs from the kernel's prologue.
+struct EpiCtx {
+    uint32_t sbase, tmem, n_tiles, grid_n;
+    int tiles_n, warp, lane;
+    uint32_t cst_s, acc_full, acc_free;       // shared-memory addresses: constants, the two accumulators' barriers
+    const volatile int *abort_flag;
+};
+
+// The epilogue of k_igemm.  Warp w owns lanes 32 (w mod 4) .. +31 of an accumulator (= 32 tile rows) and all N
+// columns; team w / 4 takes every other tile of the CTA (accumulator `team`).  A thread requantises its own row in
+// place in a per-warp scratch area in shared memory (row stride N + 16 bytes: conflict-free for the row-wise and
+// for the coalesced access).  After every 64 columns the warp writes those columns of its 32 rows out as runs of
+// 64 contiguous bytes per row and requests the same columns of the residual rows of its next tile into the
+// space that has just been read, so memory traffic runs under the arithmetic of the following columns.
+// kMode 0: 64-bit requantisation (any shift), 1: 32-bit form, 2: 32-bit form with the residual add.
+template <int kMode>
+__device__ __forceinline__ bool epilogue_role(const IgemmParams &p, const EpiCtx &c)
+{
+    const GLayer &L = p.L;
+    const int warp = c.warp, lane = c.lane, n_tile = p.n_tile, tiles_n = c.tiles_n;
+    const int q = warp & 3, team = warp / kEpiWarps;
+    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+    const uint32_t row_stride = (uint32_t)n_tile + 16u;
+    const uint32_t scr0 = c.sbase + p.scratch_off + (uint32_t)warp * 32u * row_stride;
+    const uint32_t scr_row = scr0 + (uint32_t)lane * row_stride;
+    // coalesced access to 64 columns of the 32 rows: four lanes per row, eight rows per instruction
+    const int crow = lane >> 2, cchunk = lane & 3;
+    const uint32_t scr_co = scr0 + (uint32_t)crow * row_stride + (uint32_t)cchunk * 16u;
+    const size_t co_step = (size_t)8 * L.coutp;
+    // where tile t's rows start in the output / residual tensors, for this lane's coalesced position; null when the
+    // row is beyond the last pixel (the rows of a warp that are valid are its first ones)
+    auto tile_ptr = [&](const int8_t *base, uint32_t t, uint32_t &rows) {
+        const uint32_t m_idx = t / (uint32_t)tiles_n;
+        const uint32_t m0 = m_idx * kTileM + (uint32_t)q * 32u;
+        rows = m0 < p.m_total ? min(32u, p.m_total - m0) : 0u;
+        return base + (size_t)(m0 + (uint32_t)crow) * L.coutp + (int)(t - m_idx * tiles_n) * n_tile + cchunk * 16;
+    };
+    auto residual_fetch = [&](const int8_t *src, uint32_t rows, int c0) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if ((uint32_t)(8 * k + crow) < rows) cp_async16(scr_co + (uint32_t)(8 * k) * row_stride + (uint32_t)c0, src + (size_t)k * co_step + c0);
+    };
+    // the team's tiles: every kEpiTeams-th of the CTA's
+    const uint32_t t_step = (uint32_t)kEpiTeams * c.grid_n;
+    uint32_t t = blockIdx.x + (uint32_t)team * c.grid_n;
+    if (kMode == 2 && t < c.n_tiles) {
+        uint32_t rows;
+        const int8_t *src = tile_ptr(p.res, t, rows);
+        for (int c0 = 0; c0 < n_tile; c0 += 64) residual_fetch(src, rows, c0);
+    }
+    for (int au = 0; t < c.n_tiles; t += t_step, ++au) {
+        const uint32_t m_idx = t / (uint32_t)tiles_n;
+        const int n0 = (int)(t - m_idx * tiles_n) * n_tile;
+        const uint32_t m = m_idx * kTileM + (uint32_t)q * 32u + (uint32_t)lane;
+        const int8_t *res_px = (kMode == 0 && p.res && m < p.m_total) ? p.res + (size_t)m * L.coutp : nullptr;
+        uint32_t rows, rows_next = 0;
+        int8_t *dst = const_cast<int8_t *>(tile_ptr(p.out, t, rows));
+        const int8_t *res_next = (kMode == 2 && t + t_step < c.n_tiles) ? tile_ptr(p.res, t + t_step, rows_next) : nullptr;
+        cp_async_wait_all();                                        // the tile's residual rows, requested during the previous tile
+        __syncwarp();
+        if (!wait_bar<kSleepEpi>(c.acc_full + 8u * (uint32_t)team, (uint32_t)au & 1u, c.abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t acc_base = c.tmem + lane_base + (uint32_t)(team * n_tile);
+        const uint32_t cst0 = c.cst_s + (uint32_t)n0 * 16u;
+        // 32 columns per step, the accumulators of the next step requested before this step's arithmetic
+        auto step = [&](int (&acc)[2][16], int c0) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int cc = c0 + 16 * h;
+                uint4 v;
+                if (kMode == 2) {
+                    v = requant16_fast<true>(acc[h], cst0 + (uint32_t)cc * 16u, ld_shared_v4(scr_row + (uint32_t)cc), p.res_m2, p.res_r2, p.lo);
+                } else if (kMode == 1) {
+                    v = requant16_fast<false>(acc[h], cst0 + (uint32_t)cc * 16u, make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
+                } else {
+#pragma unroll
+                    for (int o = 0; o < 16; ++o) acc[h][o] += __ldg(L.bias + n0 + cc + o);
+                    v = epilogue16(acc[h], L, n0 + cc, res_px);
+                }
+                st_shared_v4(scr_row + (uint32_t)cc, v);
+            }
+        };
+        int acc_a[2][16], acc_b[2][16];
+        tmem_ld32_issue(acc_base, acc_a);
+#pragma unroll 1
+        for (int c0 = 0; c0 < n_tile; c0 += 64) {                   // N is a multiple of 64
+            tmem_ld32_wait(acc_a);
+            tmem_ld32_issue(acc_base + (uint32_t)c0 + 32u, acc_b);
+            step(acc_a, c0);
+            tmem_ld32_wait(acc_b);
+            if (c0 + 64 < n_tile) {
+                tmem_ld32_issue(acc_base + (uint32_t)c0 + 64u, acc_a);
+            } else {
+                tc_fence_before();
+                mbar_arrive(c.acc_free + 8u * (uint32_t)team);      // the accumulator is in registers: the next tile may overwrite it
+            }
+            step(acc_b, c0 + 32);
+            __syncwarp();
+            uint4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v[k] = ld_shared_v4(scr_co + (uint32_t)(8 * k) * row_stride + (uint32_t)c0);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if ((uint32_t)(8 * k + crow) < rows) *reinterpret_cast<uint4 *>(dst + (size_t)k * co_step + c0) = v[k];
+            __syncwarp();
+            if (res_next) residual_fetch(res_next, rows_next, c0);
+        }
+    }
+    cp_async_wait_all();
+    return true;
+}
 
 __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant__ IgemmParams p)
 {
@@ -194,89 +334,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
     bool ok = true;
 
     if (warp < kAllEpiWarps) {
-        // ---- epilogue: warp w owns lanes 32 (w mod 4) .. +31 of the accumulator (= 32 tile rows) and one group of
-        // `cpg` of its columns.  A thread requantises its own row; the rows pass through a per-warp scratch area in
-        // shared memory (row stride cpg + 16 bytes: conflict-free both ways) so that the residual operand is read
-        // and the result is written as runs of `cpg` contiguous bytes per row instead of 16 bytes per lane and row.
-        const int q = warp & 3;
-        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        const int team = warp / kEpiWarps;
-        const int cpg = n_tile / (kEpiWarps / 4), c_begin = ((warp >> 2) % (kEpiWarps / 4)) * cpg;
-        const uint32_t row_stride = (uint32_t)cpg + 16u;
-        const uint32_t scr0 = sbase + p.scratch_off + (uint32_t)warp * 32u * row_stride;
-        const int lpr = cpg >> 4, rpi = 32 / lpr;                       // lanes per row, rows per instruction
-        const int crow = lane / lpr, cchunk = lane - crow * lpr;
+        EpiCtx c;
+        c.sbase = sbase; c.tmem = tmem; c.n_tiles = n_tiles; c.grid_n = grid_n; c.tiles_n = tiles_n; c.warp = warp; c.lane = lane;
+        c.cst_s = smem_u32(cst_s);
+        c.acc_full = smem_u32(&bar_acc_full[0]); c.acc_free = smem_u32(&bar_acc_free[0]);
+        c.abort_flag = &abort_s;
         const bool fast = p.fast_requant && (!p.res || p.fast_residual);
-        const bool res_fast = p.res && fast;
-        auto residual_fetch = [&](uint32_t t) {
-            const uint32_t m_idx = t / (uint32_t)tiles_n;
-            const uint32_t m0 = m_idx * kTileM + (uint32_t)q * 32u;
-            const int8_t *src = p.res + (size_t)m0 * L.coutp + (int)(t - m_idx * tiles_n) * n_tile + c_begin + cchunk * 16;
-            const uint32_t dst = scr0 + (uint32_t)cchunk * 16u;
-            for (int k = 0; k < lpr; ++k) {
-                const int row = k * rpi + crow;
-                if (m0 + row < p.m_total) cp_async16(dst + (uint32_t)row * row_stride, src + (size_t)row * L.coutp);
-            }
-        };
-        // the team's tiles: every kEpiTeams-th of the CTA's, accumulator `team`
-        const uint32_t t_step = (uint32_t)kEpiTeams * grid_n;
-        uint32_t t = blockIdx.x + (uint32_t)team * grid_n;
-        if (res_fast && t < n_tiles) residual_fetch(t);
-        for (int au = 0; t < n_tiles; t += t_step, ++au) {
-            const uint32_t m_idx = t / (uint32_t)tiles_n;
-            const int n0 = (int)(t - m_idx * tiles_n) * n_tile;
-            const uint32_t m0 = m_idx * kTileM + (uint32_t)q * 32u, m = m0 + (uint32_t)lane;
-            const bool valid = m < p.m_total;
-            const int8_t *res_px = (p.res && valid) ? p.res + (size_t)m * L.coutp : nullptr;
-            const int buf = team;
-            cp_async_wait_all();                                // the tile's residual rows, requested after the previous tile
-            __syncwarp();
-            ok = wait_bar<kSleepEpi>(smem_u32(&bar_acc_full[buf]), (uint32_t)au & 1u, &abort_s);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t acc_base = tmem + lane_base + (uint32_t)(buf * n_tile + c_begin);
-            const uint32_t scr_row = scr0 + (uint32_t)lane * row_stride;
-            for (int c0 = 0; c0 < cpg; c0 += 32) {
-                int acc[2][16];
-                tmem_ld16_issue(acc_base + (uint32_t)c0, acc[0]);
-                tmem_ld16_issue(acc_base + (uint32_t)c0 + 16u, acc[1]);
-                uint4 rv[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-                if (res_fast) {
-                    rv[0] = ld_shared_v4(scr_row + (uint32_t)c0);
-                    rv[1] = ld_shared_v4(scr_row + (uint32_t)c0 + 16u);
-                }
-                tmem_ld_wait();
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int cc = n0 + c_begin + c0 + 16 * h;
-                    uint4 v;
-                    if (fast) {
-                        const uint32_t cst = smem_u32(cst_s + cc);
-                        if (res_fast) v = requant16_fast<true>(acc[h], cst, rv[h], p.res_m2, p.res_r2, p.lo);
-                        else v = requant16_fast<false>(acc[h], cst, make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
-                    } else {
-#pragma unroll
-                        for (int o = 0; o < 16; ++o) acc[h][o] += __ldg(L.bias + cc + o);
-                        v = epilogue16(acc[h], L, cc, res_px);
-                    }
-                    st_shared_v4(scr_row + (uint32_t)(c0 + 16 * h), v);
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bar_acc_free[buf]));
-            __syncwarp();
-            {
-                int8_t *dst = p.out + (size_t)m0 * L.coutp + n0 + c_begin + cchunk * 16;
-                const uint32_t src = scr0 + (uint32_t)cchunk * 16u;
-                for (int k = 0; k < lpr; ++k) {
-                    const int row = k * rpi + crow;
-                    if (m0 + row < p.m_total) *reinterpret_cast<uint4 *>(dst + (size_t)row * L.coutp) = ld_shared_v4(src + (uint32_t)row * row_stride);
-                }
-            }
-            __syncwarp();
-            if (res_fast && t + t_step < n_tiles) residual_fetch(t + t_step);
-        }
-        cp_async_wait_all();
+        if (fast && p.res) ok = epilogue_role<2>(p, c);
+        else if (fast) ok = epilogue_role<1>(p, c);
+        else ok = epilogue_role<0>(p, c);
     } else if (warp < kAllEpiWarps + kGatherWarps) {
         // ---- operand rows: per reduction block a warp copies 32 tile rows x 64 bytes with four asynchronous 16-byte
         // copies per lane (lane = 16-byte column x row within a group of eight, so that an instruction reads whole
