@@ -168,7 +168,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
-// the same through L1: for a source that every CTA reads again and again
+// the same through L1: the taps of a 3 x 3 filter read a pixel's row nine times, and every CTA reads the zero-point run
 __device__ __forceinline__ void cp_async16_cached(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -382,8 +382,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
                     const uint32_t dst = dst0 + (uint32_t)ring.s * stage_bytes;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        if (inside[i]) cp_async16(dst + (uint32_t)i * 128u, in_c + (off[i] + tap_off + cb * kBlockK));
-                        else cp_async16_cached(dst + (uint32_t)i * 128u, zp_src);
+                        cp_async16_cached(dst + (uint32_t)i * 128u, inside[i] ? in_c + (off[i] + tap_off + cb * kBlockK) : zp_src);
                     }
                     cp_async_arrive(smem_u32(&bar_full[ring.s]));
                 }
