@@ -298,6 +298,17 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
 int isc_debug_wait_timeout(isc_model *m, int64_t limit_ns, void *cuda_stream, int32_t *out4);
 
 /*
+ * isc_debug_residual_form -- host only.  The tensor-core engines compute the residual operand's
+ * rescale rs((r - zp_res) * res_mult, 31 - res_shift) (the skip path's term of the residual add)
+ * as floor((u * m2 + R2) / 2^32), u = r + 128, and, where an offset k < 4096 exists for which
+ * floor((256 k + u) * m2 / 2^32) - c equals that for all 256 values of u, in this shorter form.
+ * This call runs the search the engines run.
+ *   returns : 1 and *k / *c when the form exists, 0 when the engines keep the long form
+ *             (including res_shift other than 0 or -1), ISC_ERR_ARG for a null pointer.
+ */
+int isc_debug_residual_form(int32_t res_mult, int32_t res_shift, int32_t zp_res, int32_t *k, int32_t *c);
+
+/*
  * isc_set_option -- "batch" and "engine" are tuning knobs that change no result; "noise" selects
  * the noise law and therefore changes the samples.
  *   "noise"  : 0 = the discrete Gaussian of Def. 3.3 / Eq. 2 (IntRS, the default), 1 = the

@@ -11,7 +11,7 @@ _LIB_PATH = os.path.join(_HERE, "libisc.so")
 
 EXPORTS = ["isc_load_qmodel", "isc_free_qmodel", "isc_plan_resident", "isc_predict", "isc_certify", "isc_certify_batch",
            "isc_sample_counts", "isc_sample_counts_static", "isc_decide_certify", "isc_decide_predict", "isc_certify_integer", "isc_decide_certify_integer", "isc_noise_table", "isc_noise_table_rounded", "isc_radius_integer", "isc_certified_metrics",
-           "isc_debug_tensor", "isc_debug_wait_timeout", "isc_set_option", "isc_get_info", "isc_strerror"]
+           "isc_debug_tensor", "isc_debug_wait_timeout", "isc_debug_residual_form", "isc_set_option", "isc_get_info", "isc_strerror"]
 
 
 class IscError(RuntimeError):
@@ -67,6 +67,7 @@ def lib():
         L.isc_debug_tensor.argtypes = [vp, vp, C.c_uint64, C.c_uint64, C.c_int32, C.c_int64, C.c_double,
                                        C.c_int, vp, vp, C.c_int64]
         L.isc_debug_wait_timeout.argtypes = [vp, C.c_int64, vp, vp]
+        L.isc_debug_residual_form.argtypes = [C.c_int32, C.c_int32, C.c_int32, vp, vp]
         L.isc_set_option.argtypes = [vp, C.c_char_p, C.c_int64]
         L.isc_get_info.argtypes = [vp, C.c_char_p, C.POINTER(C.c_int64)]
         L.isc_strerror.argtypes = [C.c_int]
@@ -283,6 +284,15 @@ def radius_integer(sigma, p_fx):
     q, q2 = C.c_int32(), C.c_int64()
     _check(lib().isc_radius_integer(float(sigma), int(p_fx), C.byref(q), C.byref(q2)), "isc_radius_integer")
     return q.value, q2.value
+
+
+def residual_form(res_mult, res_shift, zp_res):
+    """(k, c) of isc_debug_residual_form when the short form of the residual rescale exists, else None; host only."""
+    k, c = C.c_int32(), C.c_int32()
+    rc = lib().isc_debug_residual_form(int(res_mult), int(res_shift), int(zp_res), C.byref(k), C.byref(c))
+    if rc < 0:
+        raise IscError(rc, "isc_debug_residual_form")
+    return (k.value, c.value) if rc == 1 else None
 
 
 def noise_table(sigma, rounded=False):

@@ -49,6 +49,7 @@ struct isc_model {
     std::vector<const int8_t *> wpacks;         // per layer: repacked weights of the tensor-core convolution, or null
     std::vector<const int32_t *> tc_cst;        // per layer: its epilogue constants
     std::vector<char> tc_fast;
+    std::vector<uint32_t> tc_resk;           // per layer: offset of the residual term's two-instruction form, or 0xFFFFFFFF
     bool has_tc = false;
     int32_t *d_tc_err = nullptr;
 
@@ -209,6 +210,7 @@ int build_generic_engine(isc_model *m)
     m->wpacks.assign((size_t)n, nullptr);
     m->tc_cst.assign((size_t)n, nullptr);
     m->tc_fast.assign((size_t)n, 0);
+    m->tc_resk.assign((size_t)n, 0xFFFFFFFFu);
     for (int i = 0; i < n; ++i) {
         const HostLayer &H = m->layers[(size_t)i];
         const isc_layer &L = H.d;
@@ -259,7 +261,7 @@ int build_generic_engine(isc_model *m)
                 stem_pack_weights(G, H.w.data(), wp.data());
                 rc = upload(m, wp, &m->wpacks[0]); if (rc) return rc;
                 std::vector<int32_t> c4((size_t)G.coutp * 4);
-                m->tc_fast[0] = igemm_constants(G, bias.data(), mult.data(), shift.data(), c4.data()) ? 1 : 0;
+                m->tc_fast[0] = igemm_constants(G, bias.data(), mult.data(), shift.data(), c4.data(), false, nullptr) ? 1 : 0;
                 rc = upload(m, c4, &m->tc_cst[0]); if (rc) return rc;
             }
             if (i > 0 && igemm_tile_n(G)) {                 // the same layer for the tensor-core kernel
@@ -267,7 +269,7 @@ int build_generic_engine(isc_model *m)
                 igemm_pack_weights(G, H.w.data(), wp.data());
                 rc = upload(m, wp, &m->wpacks[(size_t)i]); if (rc) return rc;
                 std::vector<int32_t> c4((size_t)G.coutp * 4);
-                m->tc_fast[(size_t)i] = igemm_constants(G, bias.data(), mult.data(), shift.data(), c4.data()) ? 1 : 0;
+                m->tc_fast[(size_t)i] = igemm_constants(G, bias.data(), mult.data(), shift.data(), c4.data(), H.d.res_tensor >= 0, &m->tc_resk[(size_t)i]) ? 1 : 0;
                 rc = upload(m, c4, &m->tc_cst[(size_t)i]); if (rc) return rc;
                 m->has_tc = true;
             }
@@ -418,7 +420,7 @@ int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int
         if (i == 0 && tensor_cores && m->wpacks[0])
             e = launch_stem_conv(G, m->wpacks[0], m->tc_cst[0], m->tc_fast[0] != 0, d_x, m->in_c, ns, batch, out, m->d_tc_err, st);
         else if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, batch, out, st);
-        else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], m->tc_cst[(size_t)i], m->tc_fast[(size_t)i] != 0, batch, in, res, out, m->d_tc_err, st);
+        else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], m->tc_cst[(size_t)i], m->tc_fast[(size_t)i] != 0, m->tc_resk[(size_t)i], batch, in, res, out, m->d_tc_err, st);
         else if (L.op == ISC_CONV2D || L.op == ISC_FC) e = launch_conv(G, batch, in, res, out, st);
         else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, batch, in, out, st);
         else e = launch_maxpool(G, batch, in, out, st);
@@ -920,6 +922,17 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
             for (int x = 0; x < s.w; ++x)
                 out[((size_t)c * s.h + y) * s.w + x] = h[((size_t)y * s.w + x) * s.cp + c];
     return ISC_OK;
+}
+
+int isc_debug_residual_form(int32_t res_mult, int32_t res_shift, int32_t zp_res, int32_t *k, int32_t *c)
+{
+    if (!k || !c) return ISC_ERR_ARG;
+    uint32_t k8 = 0;
+    int32_t cc = 0;
+    if (!isc::residual_short_form(res_mult, res_shift, zp_res, &k8, &cc)) return 0;
+    *k = (int32_t)(k8 >> 8);
+    *c = cc;
+    return 1;
 }
 
 int isc_debug_wait_timeout(isc_model *m, int64_t limit_ns, void *cuda_stream, int32_t *out4)

@@ -58,7 +58,8 @@ struct IgemmParams {
     const int8_t *wpack;                     // [cout tile][tap][cin block][4 K columns][n_tile rows][16 bytes]
     const int4 *cst;                         // per output channel: folded bias, multiplier, rounding addend, shift - 1
     int fast_requant, fast_residual, lo;     // every shift >= 2; residual rescale by 2^-31 or 2^-32; lower clamp
-    uint32_t res_m2;                         // residual multiplier and addend in the 2^-32 form (see requant16_fast)
+    uint32_t res_m2, res_k8;                 // residual multiplier and addend in the 2^-32 form; offset of the two-instruction form
+    int res_short;                           // the two-instruction form reproduces the residual term (see requant16_fast)
     long long res_r2;
     int32_t *err;
 };
@@ -91,9 +92,12 @@ __device__ __forceinline__ long long mad_wide_u(uint32_t a, uint32_t b, long lon
 //   rs((acc + bias) * mult, 31 + shift) + zp_out = (hi32((acc + bias) * mult) + c) >> s,  c = 2^(s-1) + zp_out * 2^s,
 // exactly (the rounding half 2^(31+s) is a multiple of 2^32, so the product's low word cannot change the floor), and
 //   rs((r - zp_res) * res_mult, n) = hi32(u * m2 + R2),  u = r + 128, m2 = res_mult * 2^(32-n), n = 31 or 32,
-// with R2 = (2^(n-1) - (128 + zp_res) * res_mult) * 2^(32-n).  `cst` points at this block's constants in shared memory.
-template <bool kRes>
-__device__ __forceinline__ uint4 requant16_fast(const int *acc, uint32_t cst, uint4 rv, uint32_t m2, long long r2, int lo)
+// with R2 = (2^(n-1) - (128 + zp_res) * res_mult) * 2^(32-n) (kRes = 1).  kRes = 2 is the same term without the
+// 64-bit addend: hi32((256 k + u) * m2) - c_r for an offset k that the host has checked on all 256 values of u
+// (residual_short_form); 256 k is merged into u by the byte permute that extracts u, and c_r is folded into c.
+// `cst` points at this block's constants in shared memory.
+template <int kRes>
+__device__ __forceinline__ uint4 requant16_fast(const int *acc, uint32_t cst, uint4 rv, uint32_t m2, long long r2, uint32_t k8, int lo)
 {
     const uint32_t rw[4] = {rv.x ^ 0x80808080u, rv.y ^ 0x80808080u, rv.z ^ 0x80808080u, rv.w ^ 0x80808080u};
     uint32_t packed[4];
@@ -105,7 +109,8 @@ __device__ __forceinline__ uint4 requant16_fast(const int *acc, uint32_t cst, ui
             int4 c;
             asm("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(c.x), "=r"(c.y), "=r"(c.z), "=r"(c.w) : "r"(cst + (4 * g + k) * 16));
             int v = (hi32(mul_wide(acc[4 * g + k] + c.x, c.y)) + c.z) >> c.w;
-            if (kRes) v += hi32(mad_wide_u(__byte_perm(rw[g], 0u, 0x4440u | (uint32_t)k), m2, r2));
+            if (kRes == 1) v += hi32(mad_wide_u(__byte_perm(rw[g], 0u, 0x4440u | (uint32_t)k), m2, r2));
+            if (kRes == 2) v += hi32(mad_wide_u(__byte_perm(rw[g], k8, 0x7650u | (uint32_t)k), m2, 0ll));
             y[k] = max(v, lo);
         }
         packed[g] = pack4_sat(y[0], y[1], y[2], y[3]);
@@ -203,7 +208,8 @@ struct EpiCtx {
 // for the coalesced access).  After every 64 columns the warp writes those columns of its 32 rows out as runs of
 // 64 contiguous bytes per row and requests the same columns of the residual rows of its next tile into the
 // space that has just been read, so memory traffic runs under the arithmetic of the following columns.
-// kMode 0: 64-bit requantisation (any shift), 1: 32-bit form, 2: 32-bit form with the residual add.
+// kMode 0: 64-bit requantisation (any shift), 1: 32-bit form, 2 / 3: 32-bit form with the residual add (3: its
+// two-instruction form).
 template <int kMode>
 __device__ __forceinline__ bool epilogue_role(const IgemmParams &p, const EpiCtx &c)
 {
@@ -234,7 +240,7 @@ __device__ __forceinline__ bool epilogue_role(const IgemmParams &p, const EpiCtx
     // the team's tiles: every kEpiTeams-th of the CTA's
     const uint32_t t_step = (uint32_t)kEpiTeams * c.grid_n;
     uint32_t t = blockIdx.x + (uint32_t)team * c.grid_n;
-    if (kMode == 2 && t < c.n_tiles) {
+    if (kMode >= 2 && t < c.n_tiles) {
         uint32_t rows;
         const int8_t *src = tile_ptr(p.res, t, rows);
         for (int c0 = 0; c0 < n_tile; c0 += 64) residual_fetch(src, rows, c0);
@@ -246,7 +252,7 @@ __device__ __forceinline__ bool epilogue_role(const IgemmParams &p, const EpiCtx
         const int8_t *res_px = (kMode == 0 && p.res && m < p.m_total) ? p.res + (size_t)m * L.coutp : nullptr;
         uint32_t rows, rows_next = 0;
         int8_t *dst = const_cast<int8_t *>(tile_ptr(p.out, t, rows));
-        const int8_t *res_next = (kMode == 2 && t + t_step < c.n_tiles) ? tile_ptr(p.res, t + t_step, rows_next) : nullptr;
+        const int8_t *res_next = (kMode >= 2 && t + t_step < c.n_tiles) ? tile_ptr(p.res, t + t_step, rows_next) : nullptr;
         cp_async_wait_all();                                        // the tile's residual rows, requested during the previous tile
         __syncwarp();
         if (!wait_bar<kSleepEpi>(c.acc_full + 8u * (uint32_t)team, (uint32_t)au & 1u, c.abort_flag)) return false;
@@ -259,10 +265,12 @@ __device__ __forceinline__ bool epilogue_role(const IgemmParams &p, const EpiCtx
             for (int h = 0; h < 2; ++h) {
                 const int cc = c0 + 16 * h;
                 uint4 v;
-                if (kMode == 2) {
-                    v = requant16_fast<true>(acc[h], cst0 + (uint32_t)cc * 16u, ld_shared_v4(scr_row + (uint32_t)cc), p.res_m2, p.res_r2, p.lo);
+                if (kMode == 3) {
+                    v = requant16_fast<2>(acc[h], cst0 + (uint32_t)cc * 16u, ld_shared_v4(scr_row + (uint32_t)cc), p.res_m2, 0ll, p.res_k8, p.lo);
+                } else if (kMode == 2) {
+                    v = requant16_fast<1>(acc[h], cst0 + (uint32_t)cc * 16u, ld_shared_v4(scr_row + (uint32_t)cc), p.res_m2, p.res_r2, 0u, p.lo);
                 } else if (kMode == 1) {
-                    v = requant16_fast<false>(acc[h], cst0 + (uint32_t)cc * 16u, make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
+                    v = requant16_fast<0>(acc[h], cst0 + (uint32_t)cc * 16u, make_uint4(0, 0, 0, 0), 0u, 0ll, 0u, p.lo);
                 } else {
 #pragma unroll
                     for (int o = 0; o < 16; ++o) acc[h][o] += __ldg(L.bias + n0 + cc + o);
@@ -340,7 +348,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
         c.acc_full = smem_u32(&bar_acc_full[0]); c.acc_free = smem_u32(&bar_acc_free[0]);
         c.abort_flag = &abort_s;
         const bool fast = p.fast_requant && (!p.res || p.fast_residual);
-        if (fast && p.res) ok = epilogue_role<2>(p, c);
+        if (fast && p.res && p.res_short) ok = epilogue_role<3>(p, c);
+        else if (fast && p.res) ok = epilogue_role<2>(p, c);
         else if (fast) ok = epilogue_role<1>(p, c);
         else ok = epilogue_role<0>(p, c);
     } else if (warp < kAllEpiWarps + kGatherWarps) {
@@ -612,7 +621,7 @@ __global__ void __launch_bounds__(kStemThreads, 2) k_stem(const __grid_constant_
                 if (valid && !abort_s) {
                     uint4 v;
                     if (p.fast_requant) {
-                        v = requant16_fast<false>(acc, smem_u32(cst_s + c0), make_uint4(0, 0, 0, 0), 0u, 0ll, p.lo);
+                        v = requant16_fast<0>(acc, smem_u32(cst_s + c0), make_uint4(0, 0, 0, 0), 0u, 0ll, 0u, p.lo);
                     } else {
 #pragma unroll
                         for (int o = 0; o < 16; ++o) acc[o] += __ldg(L.bias + c0 + o);
@@ -667,23 +676,60 @@ void igemm_pack_weights(const GLayer &G, const int8_t *w, int8_t *out)
     for (int e = 0; e < kBlockK; ++e) out[at + e] = (int8_t)G.zp_in;
 }
 
+// The residual term F(u) = floor((u * m2 + R2) / 2^32), u = r + 128 in 0..255 (see requant16_fast), as
+// hi32((256 k + u) * m2) - c: the smallest k < 4096 for which the two agree on all 256 inputs, or false.
+bool residual_short_form(int res_mult, int res_shift, int zp_res, uint32_t *k8, int32_t *c_out)
+{
+    const int n = 31 - res_shift;
+    if (n != 31 && n != 32) return false;
+    if (res_mult <= 0) return false;
+    const uint64_t m2 = (uint64_t)(uint32_t)res_mult << (32 - n);
+    if (m2 >= (1ull << 32)) return false;
+    const int64_t r2 = ((1ll << (n - 1)) - (128ll + zp_res) * (int64_t)res_mult) * (1ll << (32 - n));
+    for (uint32_t k = 0; k < 4096; ++k) {
+        int64_t c = 0;
+        bool same = true;
+        for (uint32_t u = 0; u < 256 && same; ++u) {
+            const int64_t want = ((int64_t)(u * m2) + r2) >> 32;                 // arithmetic shift: floor
+            const int64_t got = (int64_t)(((uint64_t)(256u * k + u) * m2) >> 32);
+            if (u == 0) c = got - want;
+            same = got - want == c;
+        }
+        if (same) { *k8 = k << 8; *c_out = (int32_t)c; return true; }
+    }
+    return false;
+}
+
 // Per output channel {folded bias, multiplier, rounding addend, shift - 1}; returns whether every shift is >= 2 (the
-// condition of the 32-bit form).  `bias_folded`, `mult`, `shift` are the layer's host arrays padded to coutp.
-bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t *mult, const int32_t *shift, int32_t *out4)
+// condition of the 32-bit form).  `bias_folded`, `mult`, `shift` are the layer's host arrays padded to coutp.  For a
+// layer with a residual operand whose term has the two-instruction form, that form's constant is folded into the
+// rounding addends and *res_k8 is its offset; otherwise *res_k8 = 0xFFFFFFFF.
+bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t *mult, const int32_t *shift, int32_t *out4,
+                     bool has_residual, uint32_t *res_k8)
 {
     bool fast = true;
+    for (int o = 0; o < G.coutp; ++o) fast = fast && shift[o] - 1 >= 1;
+    uint32_t k8 = 0;
+    int32_t c_res = 0;
+    bool short_form = fast && has_residual && residual_short_form(G.res_mult, G.res_shift, G.zp_res, &k8, &c_res);
+    for (int o = 0; o < G.coutp && short_form; ++o) {
+        const int s = shift[o] - 1;
+        const long long add = (1ll << (s - 1)) + ((long long)G.zp_out - c_res) * (1ll << s);
+        short_form = add > -(1ll << 31) && add < (1ll << 31);
+    }
+    if (!short_form) c_res = 0;
+    if (res_k8) *res_k8 = short_form ? k8 : 0xFFFFFFFFu;
     for (int o = 0; o < G.coutp; ++o) {
         const int s = shift[o] - 1;
-        if (s < 1) fast = false;
         out4[4 * o + 0] = bias_folded[o];
         out4[4 * o + 1] = mult[o];
-        out4[4 * o + 2] = s >= 1 ? (1 << (s - 1)) + G.zp_out * (1 << s) : 0;
+        out4[4 * o + 2] = s >= 1 ? (int32_t)((1ll << (s - 1)) + ((long long)G.zp_out - c_res) * (1ll << s)) : 0;
         out4[4 * o + 3] = s >= 1 ? s : 0;
     }
     return fast;
 }
 
-cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, int batch, const int8_t *in,
+cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, uint32_t res_k8, int batch, const int8_t *in,
                               const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st)
 {
     IgemmParams p;
@@ -694,6 +740,8 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
     const int res_n = 31 - G.res_shift;
     p.fast_residual = (res_n == 31 || res_n == 32) ? 1 : 0;
     p.res_m2 = 0; p.res_r2 = 0;
+    p.res_short = (res && res_k8 != 0xFFFFFFFFu) ? 1 : 0;
+    p.res_k8 = p.res_short ? res_k8 : 0u;
     if (res && p.fast_residual) {
         p.res_m2 = (uint32_t)((unsigned long long)(uint32_t)G.res_mult << (32 - res_n));
         p.res_r2 = ((1ll << (res_n - 1)) - (128ll + G.zp_res) * (long long)G.res_mult) * (1ll << (32 - res_n));

@@ -71,12 +71,16 @@ cudaError_t launch_votes(const int8_t *logits_nhwc, int cp, int n_classes, int b
 int igemm_tile_n(const GLayer &G);
 size_t igemm_pack_bytes(const GLayer &G);
 void igemm_pack_weights(const GLayer &G, const int8_t *w_oihw, int8_t *out);
+// The residual term F(u) = floor((u * m2 + R2) / 2^32), u = r + 128 in 0..255, of the 32-bit epilogues as
+// hi32((256 k + u) * m2) - c: the smallest k < 4096 for which the two agree on all 256 inputs (*k8 = 256 k), or false.
+bool residual_short_form(int res_mult, int res_shift, int zp_res, uint32_t *k8, int32_t *c);
 // Per-channel requantisation constants of the kernel's 32-bit epilogue (4 x int32 per padded output channel); returns
 // whether the layer qualifies for it (every shift >= 2).
-bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t *mult, const int32_t *shift, int32_t *out4);
+bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t *mult, const int32_t *shift, int32_t *out4,
+                     bool has_residual, uint32_t *res_k8);
 // `cst` / `fast`: what igemm_constants produced (device copy).  `err` (device) receives a non-zero word if a bounded
 // wait inside the kernel expired.
-cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, int batch, const int8_t *in,
+cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, uint32_t res_k8, int batch, const int8_t *in,
                               const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st);
 
 // The first convolution (<= 4 input channels, filter at most 8 x 8) on the tensor cores, noise drawn into its staging.

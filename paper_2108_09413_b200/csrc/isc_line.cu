@@ -76,7 +76,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
 enum { PH_FILL = 0, PH_INPUT = 1, PH_CONV = 2, PH_TAIL = 3 };
 enum { ERR_NONE = 0, ERR_WAIT_DONE = 1, ERR_WAIT_WEIGHTS = 2, ERR_WAIT_READY = 3, ERR_WAIT_FULL = 4, ERR_WAIT_DRAIN = 5 };
-enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8, CF_GENERAL = 16 };     // CF_GENERAL: the pass that decides everything at run time
+enum { CF_STACKED = 1, CF_RES = 2, CF_LO = 4, CF_SCATTER = 8, CF_GENERAL = 16, CF_RSHORT = 32 };     // CF_GENERAL: the pass that decides everything at run time; CF_RSHORT: residual term without the 64-bit addend
 // OPF_WAIT_ALL: every unit of the previous convolution; OPF_NULL: no MMAs, arrivals only; OPF_WAITS / OPF_WAITS4: the
 // record names counters to test (two / four slots in use); bits 4-6: how many of them are distinct; bits 8-9: arrivals
 enum { OPF_WAIT_ALL = 1, OPF_WAITS = 2, OPF_NULL = 4, OPF_WAITS4 = 8 };
@@ -500,11 +500,19 @@ static_assert(sizeof(LPass) == 32, "one pass is two 16-byte loads");
 // One output of the common pass (every channel has s >= 1).
 //   residual: y += floor((u * m2 + R2) / 2^32) with u = r + 128 the residual byte as an unsigned number,
 //   m2 = res_mult * 2^(32-n) and R2 the rounding half and the zero-points folded: rs((r - zp_res) * res_mult, n).
-template <bool kRes, int K>
+//   kRes = 2: the same term as hi32((256 k + u) * m2) - c_r, for an offset k that the planner has checked on all 256
+//   values of u (residual_short_form): `res_r2` then holds 256 k, which the byte permute that extracts u merges
+//   into it, and c_r is folded into the channel's rounding addend.
+template <int kRes, int K>
 __device__ __forceinline__ int requant1(int acc, const ChanConst4 &cs, uint32_t rword, uint32_t res_m2, long long res_r2)
 {
     int y = (hi32(mul_wide(acc + cs.bias, cs.mult)) + cs.c) >> cs.s;
-    if (kRes) y += hi32(mad_wide_u(ubyte<K>(rword), res_m2, res_r2));
+    if (kRes == 1) y += hi32(mad_wide_u(ubyte<K>(rword), res_m2, res_r2));
+    if (kRes == 2) {
+        uint32_t u;
+        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(u) : "r"(rword), "r"((uint32_t)lo32(res_r2)), "n"(0x7650 | K));
+        y += hi32(mad_wide_u(u, res_m2, 0ll));
+    }
     return y;
 }
 
@@ -537,7 +545,7 @@ __device__ __forceinline__ void pass_done(const EpiConv &E, const EpiCtx &c, uin
 
 // The common pass: two output lines, one 16-channel chunk, results stored where the next convolution reads them.
 // The accumulator columns are left at zero: stacked chains accumulate from their first K-step on.
-template <bool kRes>
+template <int kRes>
 __device__ __forceinline__ void epi_pass2(const EpiConv &E, const EpiCtx &c, uint4 q0, uint4 q1)
 {
     const uint32_t ch = (q0.x >> 12) & 0xFu;
@@ -583,7 +591,7 @@ __device__ __forceinline__ void epi_pass2(const EpiConv &E, const EpiCtx &c, uin
 
 // The items (unit, chunk) of a convolution that belong to this warp's set: one wait, one or two records of two lines
 // each, one arrival.
-template <bool kRes>
+template <int kRes>
 __device__ __forceinline__ void epi_conv_fast(Waiter w, const EpiConv &E_in, const EpiCtx &c_in, uint32_t passes, uint32_t n_items,
                                             uint32_t item_bytes)
 {
@@ -712,8 +720,9 @@ __device__ __forceinline__ void epi_conv(const LineParams &p, const EpiCtx &c, u
         return;
     }
     const uint32_t rpi = lds32(desc + offsetof(LConvDesc, recs_per_item));
-    if (flags & CF_RES) epi_conv_fast<true>(w, E, c, passes, n_passes / rpi, 32u * rpi);
-    else epi_conv_fast<false>(w, E, c, passes, n_passes / rpi, 32u * rpi);
+    if (flags & CF_RSHORT) epi_conv_fast<2>(w, E, c, passes, n_passes / rpi, 32u * rpi);
+    else if (flags & CF_RES) epi_conv_fast<1>(w, E, c, passes, n_passes / rpi, 32u * rpi);
+    else epi_conv_fast<0>(w, E, c, passes, n_passes / rpi, 32u * rpi);
 }
 
 // FILL: the region takes its halo value everywhere
@@ -1514,6 +1523,7 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
         std::vector<uint8_t> blob(w_bytes[(size_t)c], 0);
         LConvDesc D;
         memset(&D, 0, sizeof(D));
+        int32_t res_c = 0;                    // constant of the residual term's short form, folded into the rounding addends
         D.n_ops = (uint32_t)cp.ops.size(); D.n_passes = (uint32_t)cp.passes.size(); D.n_ksteps = (uint32_t)cp.kunits.size();
         D.flags = (cp.stacked ? CF_STACKED : 0u) | (L.res_tensor >= 0 ? CF_RES : 0u) | (cp.scatter ? CF_SCATTER : 0u);
         const int lo = L.relu ? std::max(-128, L.zp_out) : -128;
@@ -1553,6 +1563,22 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
             D.res_m2 = (uint32_t)m2;
             D.res_r2_lo = (uint32_t)((unsigned long long)r2 & 0xFFFFFFFFull);
             D.res_r2_hi = (uint32_t)((unsigned long long)r2 >> 32);
+            // the fast pass takes the term without the 64-bit addend when that form exists and its constant fits into
+            // every channel's rounding addend
+            uint32_t k8 = 0;
+            bool short_form = !cp.general && residual_short_form(L.res_mult, L.res_shift, L.zp_res, &k8, &res_c);
+            for (int oc = 0; oc < L.cout && short_form; ++oc) {
+                const int sft = ML.shift[oc] - 1;
+                const long long add = sft >= 1 ? (1ll << (sft - 1)) + ((long long)L.zp_out - res_c) * (1ll << sft) : (1ll << 40);
+                short_form = add > -(1ll << 31) && add < (1ll << 31);
+            }
+            if (short_form) {
+                D.flags |= CF_RSHORT;
+                D.res_r2_lo = k8;
+                D.res_r2_hi = 0;
+            } else {
+                res_c = 0;
+            }
         }
         for (size_t k = 0; k < cp.kunits.size(); ++k) {
             const long long a = (long long)D.a_base + cp.a_delta[k];
@@ -1601,7 +1627,7 @@ bool build_plan(const LayerIn *layers, int n_layers, int in_c, int in_h, int in_
             const long long biasf = (long long)ML.bias[oc] - (long long)L.zp_in * wsum;
             if (biasf < -(1ll << 31) || biasf >= (1ll << 31)) PLAN_FAIL(24);
             const int sft = sh - 1;
-            const int32_t addend = sft ? (1 << (sft - 1)) + L.zp_out * (1 << sft) : L.zp_out;
+            const int32_t addend = sft ? (int32_t)((1ll << (sft - 1)) + ((long long)L.zp_out - res_c) * (1ll << sft)) : L.zp_out;
             int32_t cst[4] = {(int32_t)biasf, ML.mult[oc], addend, sft};
             memcpy(&blob[c_rel[(size_t)c] + (size_t)oc * 16], cst, 16);
             if (sft == 0) any_shift_one = true;

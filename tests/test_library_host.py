@@ -187,3 +187,26 @@ def test_rounded_noise_table_equals_the_oracle():
     for sigma in (0.12, 0.25, 0.5, 1.0):
         np.testing.assert_array_equal(isc.noise_table(sigma, rounded=True), oracle.rgauss_table(sigma))
         np.testing.assert_array_equal(isc.noise_table(sigma), oracle.dgauss_table(sigma))
+
+
+def test_residual_short_form_reproduces_the_rescale_on_every_byte():
+    """The offset form of the residual rescale, floor((256 k + u) m2 / 2^32) - c, is used by the tensor-core engines only
+    when it equals rs((r - zp_res) * res_mult, 31 - res_shift) for all 256 bytes: checked here with exact integers."""
+    rng = np.random.default_rng(0x15174000)
+    found = 0
+    cases = [(1 << 30, 0, 0), (1 << 30, -1, -128), ((1 << 31) - 1, 0, 127), ((1 << 31) - 1, -1, -128)]
+    cases += [(int(rng.integers(1 << 30, 1 << 31)), int(rng.integers(-1, 1)), int(rng.integers(-128, 128))) for _ in range(60)]
+    for res_mult, res_shift, zp_res in cases:
+        form = isc.residual_form(res_mult, res_shift, zp_res)
+        if form is None:
+            continue
+        found += 1
+        k, c = form
+        assert 0 <= k < 4096
+        n = 31 - res_shift
+        m2 = res_mult << (32 - n)
+        for r in range(-128, 128):
+            want = ((r - zp_res) * res_mult + (1 << (n - 1))) >> n           # rs(): round half up, floor division
+            assert (((256 * k + r + 128) * m2) >> 32) - c == want, (res_mult, res_shift, zp_res, r)
+    assert found >= 50                                                        # the form exists for nearly every multiplier
+    assert isc.residual_form(1 << 30, -3, 0) is None                         # rescale shifts the engines do not take
