@@ -147,22 +147,26 @@ def test_resnet50_every_tensor_on_the_tensor_core_engine():
         assert bad.size == 0, f"tensor {k}: {bad.size} of {got.size} differ, first at {bad[:8]}"
 
 
-@pytest.mark.parametrize("seed", range(4))
-def test_random_bottleneck_nets_on_the_tensor_core_engine(seed):
-    """Small bottleneck networks with ragged sizes, strides, every zero-point and shift, residual rescales of all
-    allowed shifts: the implicit-GEMM kernel's tiles end inside rows and images, its padding is a non-trivial
-    zero-point."""
-    rng = np.random.default_rng(900 + seed)
+def _bottleneck_net(rng, fast=None):
+    """Two bottleneck-style residual blocks on a small ragged image.  `fast` = (res_mult, res_shift, zp_res): every
+    shift >= 2 and that residual rescale on both blocks, so that the 32-bit epilogue runs."""
     h, w = int(rng.integers(9, 23)), int(rng.integers(2, 6)) * 4
     zp = lambda: int(rng.integers(-128, 128))
     c0, c1 = int(rng.choice([64, 128])), int(rng.choice([64, 128, 256]))
     z = [int(rng.integers(0, 256)), zp(), zp(), zp(), zp(), zp()]
+    if fast:
+        z[4] = z[5] = fast[2]
     L = [_rand_conv(rng, 0, 3, c0, 3, 1, 1, 1, z[0], z[1]),
          _rand_conv(rng, 1, c0, c0, 1, 1, 0, int(rng.integers(0, 2)), z[1], z[2]),
          _rand_conv(rng, 2, c0, c0, 3, 2, 1, int(rng.integers(0, 2)), z[2], z[3]),
          _rand_conv(rng, 1, c0, c1, 1, 2, 0, 0, z[1], z[4])]
     L.append(_rand_conv(rng, 3, c0, c1, 1, 1, 0, 1, z[3], z[5], res_tensor=4, zp_res=z[4]))
     L.append(_rand_conv(rng, 5, c1, c1, 3, 1, 1, 1, z[5], z[1], res_tensor=5, zp_res=z[5]))
+    if fast:
+        for layer in L:
+            layer["shift"] = np.maximum(layer["shift"], 2).astype(np.int8)
+            if layer["res_tensor"] >= 0:
+                layer["res_mult"], layer["res_shift"] = fast[0], fast[1]
     model = dict(in_shape=(3, h, w), n_classes=5, layers=L)
     om_tmp = oracle.Model(dict(model, n_classes=1))
     hw = oracle.tensor_size(om_tmp, 6) // c1
@@ -170,9 +174,13 @@ def test_random_bottleneck_nets_on_the_tensor_core_engine(seed):
     fc = _rand_conv(rng, 7, c1, 5, 1, 1, 0, 0, z[1], zp())
     fc["op"] = wl.OP_FC
     L.append(fc)
+    return model
+
+
+def _bottleneck_parity(model, rng, seed):
     gm, om = _pair(model)
     gm.set_option("engine", 2)
-    x = rng.integers(0, 256, (3, h, w)).astype(np.uint8)
+    x = rng.integers(0, 256, model["in_shape"]).astype(np.uint8)
     sizes = _tensor_sizes(om)
     a0 = oracle.noisy_input(x, 5, seed, 1, 2, 0.25)
     for k in range(1, om.n_layers + 1):
@@ -184,6 +192,26 @@ def test_random_bottleneck_nets_on_the_tensor_core_engine(seed):
     assert gm.get_info("engine") == 2
     np.testing.assert_array_equal(gl, el)
     np.testing.assert_array_equal(gc, ec)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_bottleneck_nets_on_the_tensor_core_engine(seed):
+    """Small bottleneck networks with ragged sizes, strides, every zero-point and shift, residual rescales of all
+    allowed shifts: the implicit-GEMM kernel's tiles end inside rows and images, its padding is a non-trivial
+    zero-point."""
+    rng = np.random.default_rng(900 + seed)
+    _bottleneck_parity(_bottleneck_net(rng), rng, seed)
+
+
+@pytest.mark.parametrize("res", [(1304428746, 0, 77), (1334892440, -1, -63), (1 << 30, 0, 0),         # no offset form
+                                 (1979951843, 0, 0), (1435772024, -1, -128)])                           # offset form
+def test_bottleneck_nets_32_bit_epilogue_both_residual_forms(res):
+    """The same networks with every shift >= 2, so that the kernel's 32-bit epilogue runs, and residual rescales
+    with and without the offset form (isc_debug_residual_form): both forms of the residual term against the oracle."""
+    has_form = isc.residual_form(*res) is not None
+    assert has_form == (res[0] in (1979951843, 1435772024))
+    rng = np.random.default_rng(950 + res[0] % 97)
+    _bottleneck_parity(_bottleneck_net(rng, fast=res), rng, res[0] % 5)
 
 
 def test_partition_and_batch_invariance():
