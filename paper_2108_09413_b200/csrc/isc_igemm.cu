@@ -41,7 +41,8 @@ constexpr int kTileM = 128;
 constexpr int kBlockK = 64;                  // bytes of K per stage: two MMA K-steps
 constexpr unsigned kSleepLoad = 20000, kSleepEpi = 20000, kSleepMma = 20000;      // suspend-time hint of a barrier wait (ns), by role
 constexpr int kMaxStages = 16;
-constexpr int kStemThreads = 512;           // k_stem: four threads per tile row
+constexpr int kStemThreads = 256;           // k_stem: two threads per tile row; two CTAs per SM (registers allow no third, nor two of 512 threads)
+constexpr size_t kStemSmemLimit = 108 * 1024;          // dynamic shared memory of k_stem: two CTAs per SM
 constexpr int kEpiWarps = 4, kEpiTeams = 2, kGatherWarps = 4;          // a team of epilogue warps takes every other tile
 constexpr int kAllEpiWarps = kEpiWarps * kEpiTeams;
 static_assert(kEpiWarps == 4, "an epilogue warp owns all N columns of its 32 rows");
@@ -475,6 +476,7 @@ struct StemParams {
     GLayer L;
     int in_c, band_rows, n_bands, tiles_per_band, tmem_cols;
     uint32_t patch_bytes, w_bytes;
+    uint32_t tab_off;                        // the noise tables' copy in shared memory (after the patch), 0: searched in global memory
     const uint8_t *x;                        // clean image, CHW
     NoiseStream ns;
     const int8_t *wpack;                     // [filter row][2 K columns][coutp rows][16 bytes]
@@ -526,6 +528,11 @@ __global__ void __launch_bounds__(kStemThreads, 2) k_stem(const __grid_constant_
     uint32_t *patch = reinterpret_cast<uint32_t *>(smem + patch_off);
     const uint32_t zp_fill = (uint32_t)(L.zp_in & 0xFF) * (0x01010101u >> (8 * (4 - p.in_c)));
     for (int i = tid; i < rows_in * wpad; i += kStemThreads) patch[i] = zp_fill;
+    if (p.tab_off && p.ns.guide) {
+        // cumulative table, then the guide table that follows it in memory
+        uint32_t *tab = reinterpret_cast<uint32_t *>(smem + p.tab_off);
+        for (int i = tid; i < 2 * p.ns.T + 1 + kNoiseGuide + 1; i += kStemThreads) tab[i] = __ldg(p.ns.cum + i);
+    }
     __syncthreads();
     const int vy0 = max(0, iy0), vy1 = min(L.hin, iy0 + rows_in);
     if (vy1 > vy0) {
@@ -544,7 +551,8 @@ __global__ void __launch_bounds__(kStemThreads, 2) k_stem(const __grid_constant_
                 const uint4 r = philox4x32_10(make_uint4(e >> 2, ctr1, p.ns.ctr2, ctr3), p.ns.key0, p.ns.key1);
                 const uint32_t clean = __ldg(reinterpret_cast<const uint32_t *>(p.x + e));
                 int z[4];
-                noise_levels4(r, p.ns.cum, p.ns.guide, p.ns.T, p.ns.guide_steps, z);
+                if (p.tab_off) noise_levels4_shared(r, sbase + p.tab_off, sbase + p.tab_off + 4u * (uint32_t)(2 * p.ns.T + 1), p.ns.T, p.ns.guide_steps, z);
+                else noise_levels4(r, p.ns.cum, p.ns.guide, p.ns.T, p.ns.guide_steps, z);
                 uint8_t *dst = pb + ((h - iy0) * wpad + (4 * wq + L.pad)) * 4 + c;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) dst[4 * k] = (uint8_t)min(255, max(0, (int)((clean >> (8 * k)) & 0xFFu) + z[k]));
@@ -571,8 +579,8 @@ __global__ void __launch_bounds__(kStemThreads, 2) k_stem(const __grid_constant_
     }
     __syncthreads();
 
-    // ---- tiles of 128 output pixels of the band.  Thread = tile row `px` x one of four groups: a group copies every
-    // fourth filter row's windows and requantises every fourth 16-channel chunk.
+    // ---- tiles of 128 output pixels of the band.  Thread = tile row `px` x one of kStemThreads / 128 groups: the
+    // groups share the filter rows' windows and the 16-channel chunks round-robin.
     const int band_px = (oy1 - oy0) * L.wout;
     const int n_tiles = (band_px + kTileM - 1) / kTileM;
     const uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
@@ -836,10 +844,17 @@ cudaError_t launch_stem_conv(const GLayer &G, const int8_t *wpack, const int32_t
     p.fast_requant = fast ? 1 : 0;
     p.lo = G.relu ? (G.zp_out > -128 ? G.zp_out : -128) : -128;
     p.out = out; p.err = err;
-    const size_t smem = (size_t)p.w_bytes + 2 * (size_t)G.kh * kTileM * 32 + p.patch_bytes;
+    size_t smem = (size_t)p.w_bytes + 2 * (size_t)G.kh * kTileM * 32 + p.patch_bytes;
+    // the noise tables go to shared memory when two CTAs per SM still fit and the guide table follows the cumulative one
+    const size_t tab_bytes = ((size_t)(2 * ns.T + 1 + kNoiseGuide + 1) * 4 + 15) & ~(size_t)15;
+    p.tab_off = 0;
+    if (ns.guide == ns.cum + (2 * ns.T + 1) && smem + tab_bytes <= kStemSmemLimit) {
+        p.tab_off = (uint32_t)smem;
+        smem += tab_bytes;
+    }
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_stem, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_stem, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStemSmemLimit);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }

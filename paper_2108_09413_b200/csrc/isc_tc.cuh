@@ -273,5 +273,31 @@ __device__ __forceinline__ void noise_levels4(uint4 u4, const uint32_t *__restri
     for (int k = 0; k < 4; ++k) z[k] = (int)lo[k] - T;
 }
 
+// The same with both tables in shared memory (`cum_s`, `guide_s`: shared-memory addresses).  Thirty-two lanes searching
+// a table in global memory touch up to thirty-two cache lines per load; in shared memory the same load costs its bank
+// conflicts only.
+__device__ __forceinline__ void noise_levels4_shared(uint4 u4, uint32_t cum_s, uint32_t guide_s, int T, int steps, int (&z)[4])
+{
+    const uint32_t u[4] = {u4.x, u4.y, u4.z, u4.w};
+    uint32_t lo[4], hi[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t j = u[k] >> (32 - kNoiseGuideBits);
+        lo[k] = lds32(guide_s + 4u * j);
+        hi[k] = lds32(guide_s + 4u * j + 4u);
+    }
+    for (int s = 0; s < steps; ++s) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t mid = (lo[k] + hi[k]) >> 1;
+            const bool below = u[k] < lds32(cum_s + 4u * mid);
+            hi[k] = below ? mid : hi[k];
+            lo[k] = below ? lo[k] : min(mid + 1, hi[k]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) z[k] = (int)lo[k] - T;
+}
+
 }  // namespace tc
 }  // namespace isc
