@@ -9,7 +9,7 @@
 // memory.  The kernel is persistent (one CTA per SM, tiles dealt round-robin) and its warps have fixed roles that
 // meet only at mbarriers:
 //   * four warps gather operand rows: per reduction block (64 input channels of one filter tap) a lane issues four
-//     asynchronous 16-byte copies into the K-major core-matrix layout (four lanes read one pixel's 64 bytes) whose
+//     asynchronous 16-byte copies (through L1) into the K-major core-matrix layout (four lanes read one pixel's 64 bytes) whose
 //     completion arrives on the stage's barrier; a pixel outside the image is copied from a run of the input
 //     zero-point kept behind the repacked weights;
 //   * one thread streams the matching slices of the repacked weights with bulk copies into the same stages;
@@ -39,7 +39,7 @@ namespace {
 
 constexpr int kTileM = 128;
 constexpr int kBlockK = 64;                  // bytes of K per stage: two MMA K-steps
-constexpr unsigned kSleepLoad = 20000, kSleepEpi = 20000, kSleepMma = 20000;      // suspend-time hint of a barrier wait (ns), by role
+constexpr unsigned kHintLoad = 20000, kHintEpi = 20000, kHintMma = 20000;      // suspend-time hint of a barrier wait (ns), by role
 constexpr int kMaxStages = 16;
 constexpr int kStemThreads = 256;           // k_stem: two threads per tile row; two CTAs per SM (registers allow no third, nor two of 512 threads)
 constexpr size_t kStemSmemLimit = 108 * 1024;          // dynamic shared memory of k_stem: two CTAs per SM
@@ -146,22 +146,22 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity)
         if ((spin & 7) == 7 && globaltimer() - t0 > kWaitLimitNs) return false;
     }
 }
-// The same for the roles of k_igemm, which also give up when another role has raised the CTA's abort flag.  A role
-// that is far ahead of the others sleeps `kSleepNs` between polls so that its polling does not take issue slots
-// from the warps that do the arithmetic.
-template <unsigned kSleepNs>
+// The same for the roles of k_igemm, which also give up when another role has raised the CTA's abort flag.  With
+// `kHintNs` the wait is parked in hardware for up to that long per attempt instead of polling (the abort flag and
+// the time limit are looked at every eighth attempt).
+template <unsigned kHintNs>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const volatile int *abort_flag)
 {
     if (mbar_test(bar, parity)) return true;
     const unsigned long long t0 = globaltimer();
     for (int spin = 0;; ++spin) {
-        if (kSleepNs) {
+        if (kHintNs) {
             // parked in hardware until the phase completes or the hint runs out
             uint32_t done;
             asm volatile("{\n\t.reg .pred p;\n\t"
                          "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
                          "selp.u32 %0, 1, 0, p;\n\t}"
-                         : "=r"(done) : "r"(bar), "r"(parity), "r"(kSleepNs) : "memory");
+                         : "=r"(done) : "r"(bar), "r"(parity), "r"(kHintNs) : "memory");
             if (done) return true;
         } else if (mbar_try(bar, parity)) {
             return true;
@@ -256,7 +256,7 @@ __device__ __forceinline__ bool epilogue_role(const IgemmParams &p, const EpiCtx
         const int8_t *res_next = (kMode >= 2 && t + t_step < c.n_tiles) ? tile_ptr(p.res, t + t_step, rows_next) : nullptr;
         cp_async_wait_all();                                        // the tile's residual rows, requested during the previous tile
         __syncwarp();
-        if (!wait_bar<kSleepEpi>(c.acc_full + 8u * (uint32_t)team, (uint32_t)au & 1u, c.abort_flag)) return false;
+        if (!wait_bar<kHintEpi>(c.acc_full + 8u * (uint32_t)team, (uint32_t)au & 1u, c.abort_flag)) return false;
         tc_fence_after();
         const uint32_t acc_base = c.tmem + lane_base + (uint32_t)(team * n_tile);
         const uint32_t cst0 = c.cst_s + (uint32_t)n0 * 16u;
@@ -386,7 +386,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
                 for (int i = 0; i < 4; ++i) inside[i] = (unsigned)(iy0[i] + r) < (unsigned)L.hin && (unsigned)(ix0[i] + sx) < (unsigned)L.win;
                 for (int cb = 0; cb < cblocks; ++cb, ring.advance(stages)) {
                     if (ring.use >= 1) {
-                        ok = wait_bar<kSleepLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
+                        ok = wait_bar<kHintLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
                         if (!ok) break;
                     }
                     const uint32_t dst = dst0 + (uint32_t)ring.s * stage_bytes;
@@ -408,11 +408,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
             for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += grid_n, ++j) {
                 const int buf = j & 1, au = j >> 1;
                 if (au >= 1) {
-                    ok = wait_bar<kSleepMma>(smem_u32(&bar_acc_free[buf]), (uint32_t)(au - 1) & 1u, &abort_s);
+                    ok = wait_bar<kHintMma>(smem_u32(&bar_acc_free[buf]), (uint32_t)(au - 1) & 1u, &abort_s);
                     if (!ok) break;
                 }
                 for (int kb = 0; kb < nkb; ++kb, ring.advance(stages)) {
-                    ok = wait_bar<kSleepMma>(smem_u32(&bar_full[ring.s]), (uint32_t)ring.use & 1u, &abort_s);
+                    ok = wait_bar<kHintMma>(smem_u32(&bar_full[ring.s]), (uint32_t)ring.use & 1u, &abort_s);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t stage = sbase + (uint32_t)ring.s * stage_bytes;
@@ -436,7 +436,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
                 const int8_t *wtile = p.wpack + (size_t)(t % tiles_n) * (size_t)nkb * b_bytes;
                 for (int kb = 0; kb < nkb; ++kb, ring.advance(stages)) {
                     if (ring.use >= 1) {
-                        ok = wait_bar<kSleepLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
+                        ok = wait_bar<kHintLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
                         if (!ok) break;
                     }
                     mbar_expect_tx(smem_u32(&bar_full[ring.s]), b_bytes);
