@@ -293,6 +293,12 @@ int isc_debug_tensor(isc_model *m, const uint8_t *x_u8, uint64_t seed, uint64_t 
  *             wait did NOT expire; ISC_ERR_UNSUPPORTED if the model has no resident engine.
  *   out4    : host, 4 int32: result of the first wait (0 = expired), result of the second wait
  *             (0 = fell through because the abort flag was up), the abort flag, nanoseconds spent.
+ * A model without the resident engine but with tensor-core layers (the layer-by-layer tensor-core
+ * engine) is probed through that engine instead: one launch of its first implicit-GEMM layer on one
+ * sample's work space with the weights held back, so that the kernel's own waits run out (after
+ * their fixed limit of two seconds; `limit_ns` is not used) and every role leaves through the abort
+ * path.  out4 = {0, 0, the kernel's error word (non-zero = 1 + the CTA that raised it), host
+ * nanoseconds of the launch, saturated}.
  * The handle stays usable: the next call on it must succeed.
  */
 int isc_debug_wait_timeout(isc_model *m, int64_t limit_ns, void *cuda_stream, int32_t *out4);

@@ -1,6 +1,8 @@
 // Host side of libisc: argument checks, model repacking and upload, launch sequencing of the
 // Monte-Carlo loop (Algorithm 1 steps 1-4, Algorithm 2 steps 1-2) and the decision rules.
 #include <cuda_runtime.h>
+
+#include <chrono>
 #include <stdint.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -938,6 +940,32 @@ int isc_debug_residual_form(int32_t res_mult, int32_t res_shift, int32_t zp_res,
 int isc_debug_wait_timeout(isc_model *m, int64_t limit_ns, void *cuda_stream, int32_t *out4)
 {
     if (!m || !out4) return ISC_ERR_ARG;
+    if (!m->line && m->has_tc) {
+        // The layer-by-layer tensor-core engine: one launch of its first implicit-GEMM layer on one sample's work
+        // space with the weights held back, so that the kernel's own waits run out and its CTAs leave through the
+        // abort path; the error word must be up afterwards.
+        cudaStream_t st = (cudaStream_t)cuda_stream;
+        size_t li = 1;
+        while (li < m->glayers.size() && !m->wpacks[li]) ++li;
+        if (li >= m->glayers.size()) return ISC_ERR_UNSUPPORTED;
+        int rc = ensure_workspace(m, 1);
+        if (rc) return rc;
+        const GLayer &G = m->glayers[li];
+        const isc_layer &L = m->layers[li].d;
+        int8_t *out = (int8_t *)m->bufs[(size_t)m->tensor_buf[li + 1]].p;
+        const int8_t *in = (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.in_tensor]].p;
+        const int8_t *res = L.res_tensor >= 0 ? (const int8_t *)m->bufs[(size_t)m->tensor_buf[(size_t)L.res_tensor]].p : nullptr;
+        const auto t0 = std::chrono::steady_clock::now();
+        if (launch_igemm_conv(G, m->wpacks[li], m->tc_cst[li], m->tc_fast[li] != 0, m->tc_resk[li], 1, in, res, out, m->d_tc_err, st, true) != cudaSuccess)
+            return ISC_ERR_CUDA;
+        CK(cudaStreamSynchronize(st));
+        const long long ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+        int32_t e = 0;
+        CK(cudaMemcpy(&e, m->d_tc_err, sizeof(e), cudaMemcpyDeviceToHost));
+        CK(cudaMemset(m->d_tc_err, 0, sizeof(e)));
+        out4[0] = 0; out4[1] = 0; out4[2] = e; out4[3] = (int32_t)std::min<long long>(ns, 0x7FFFFFFF);
+        return e != 0 ? ISC_ERR_TIMEOUT : ISC_OK;
+    }
     if (!m->line) return ISC_ERR_UNSUPPORTED;
     int32_t tmp[4] = {0, 0, 0, 0};
     const int rc = isc::line_wait_probe(m->line, limit_ns, tmp, (cudaStream_t)cuda_stream);

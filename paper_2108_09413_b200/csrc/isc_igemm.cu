@@ -61,6 +61,7 @@ struct IgemmParams {
     int fast_requant, fast_residual, lo;     // every shift >= 2; residual rescale by 2^-31 or 2^-32; lower clamp
     uint32_t res_m2, res_k8;                 // residual multiplier and addend in the 2^-32 form; offset of the two-instruction form
     int res_short;                           // the two-instruction form reproduces the residual term (see requant16_fast)
+    int debug_stall;                         // test hook: the weights are never sent, so every wait of the kernel runs out
     long long res_r2;
     int32_t *err;
 };
@@ -256,7 +257,10 @@ __device__ __forceinline__ bool epilogue_role(const IgemmParams &p, const EpiCtx
         const int8_t *res_next = (kMode >= 2 && t + t_step < c.n_tiles) ? tile_ptr(p.res, t + t_step, rows_next) : nullptr;
         cp_async_wait_all();                                        // the tile's residual rows, requested during the previous tile
         __syncwarp();
-        if (!wait_bar<kHintEpi>(c.acc_full + 8u * (uint32_t)team, (uint32_t)au & 1u, c.abort_flag)) return false;
+        if (!wait_bar<kHintEpi>(c.acc_full + 8u * (uint32_t)team, (uint32_t)au & 1u, c.abort_flag)) {
+            cp_async_wait_all();                                    // the next tile's residual rows may still be landing
+            return false;
+        }
         tc_fence_after();
         const uint32_t acc_base = c.tmem + lane_base + (uint32_t)(team * n_tile);
         const uint32_t cst0 = c.cst_s + (uint32_t)n0 * 16u;
@@ -430,7 +434,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
         __syncwarp();
     } else {
         // ---- one thread streams the repacked weights: one bulk copy per block into the stage's second part
-        if (lane == 0) {
+        if (lane == 0 && !p.debug_stall) {
             Ring ring;
             for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += grid_n) {
                 const int8_t *wtile = p.wpack + (size_t)(t % tiles_n) * (size_t)nkb * b_bytes;
@@ -738,7 +742,7 @@ bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t 
 }
 
 cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, uint32_t res_k8, int batch, const int8_t *in,
-                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st)
+                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st, bool debug_stall)
 {
     IgemmParams p;
     p.L = G;
@@ -747,6 +751,7 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
     p.lo = G.relu ? (G.zp_out > -128 ? G.zp_out : -128) : -128;
     const int res_n = 31 - G.res_shift;
     p.fast_residual = (res_n == 31 || res_n == 32) ? 1 : 0;
+    p.debug_stall = debug_stall ? 1 : 0;
     p.res_m2 = 0; p.res_r2 = 0;
     p.res_short = (res && res_k8 != 0xFFFFFFFFu) ? 1 : 0;
     p.res_k8 = p.res_short ? res_k8 : 0u;

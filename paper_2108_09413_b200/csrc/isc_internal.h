@@ -79,9 +79,10 @@ bool residual_short_form(int res_mult, int res_shift, int zp_res, uint32_t *k8, 
 bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t *mult, const int32_t *shift, int32_t *out4,
                      bool has_residual, uint32_t *res_k8);
 // `cst` / `fast`: what igemm_constants produced (device copy).  `err` (device) receives a non-zero word if a bounded
-// wait inside the kernel expired.
+// wait inside the kernel expired.  `debug_stall`: the kernel's weights are never sent, so that its waits run out
+// (after their 2 s limit) and the CTAs leave through the abort path -- nothing faults or hangs.
 cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, uint32_t res_k8, int batch, const int8_t *in,
-                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st);
+                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st, bool debug_stall = false);
 
 // The first convolution (<= 4 input channels, filter at most 8 x 8) on the tensor cores, noise drawn into its staging.
 bool stem_fits(const GLayer &G, int in_c);

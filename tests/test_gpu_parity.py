@@ -364,7 +364,26 @@ def test_expired_wait_is_reported_and_the_handle_recovers():
     np.testing.assert_array_equal(logits, oracle.sample_counts(om, x, SEED, 0, 1, 0, 64, 0.25, want_logits=True)[1])
     # out-of-range limits are refused before anything is launched
     assert gm.debug_wait_timeout(10)[0] == -1 and gm.debug_wait_timeout(10 ** 10)[0] == -1
-    assert isc.Model(wl.resnet50()).debug_wait_timeout(1_000_000)[0] == -3
+
+
+def test_stalled_implicit_gemm_kernel_leaves_through_its_abort_path():
+    """The layer-by-layer tensor-core engine: one launch of k_igemm whose weights are held back.  Every role's wait
+    runs out after the kernel's own two-second limit (or sees the abort flag another role raised), in-flight copies
+    are waited for, the tensor memory is freed, the error word is up (ISC_ERR_TIMEOUT = -6), and the same handle
+    then computes the right logits.  Nothing here faults, traps or hangs the GPU."""
+    model = wl.resnet50(hw=64, blocks=(1, 1, 1, 1))
+    gm, om = _pair(model)
+    gm.set_option("engine", 2)
+    x = wl.images(1, shape=(3, 64, 64))[0]
+    rc, (first, second, err_word, ns) = gm.debug_wait_timeout(1_000_000)
+    assert rc == -6
+    assert err_word >= 1
+    assert 1_900_000_000 <= ns or ns == 0x7FFFFFFF
+    got = gm.sample_counts(x, SEED, 3, 1, 0, 5, 0.5, want_logits=True)
+    exp = oracle.sample_counts(om, x, SEED, 3, 1, 0, 5, 0.5, want_logits=True)
+    assert gm.get_info("engine") == 2
+    np.testing.assert_array_equal(got[1], exp[1])
+    np.testing.assert_array_equal(got[0], exp[0])
 
 
 def test_rounded_gaussian_noise_path():
