@@ -12,7 +12,9 @@
 //     asynchronous 16-byte copies (through L1) into the K-major core-matrix layout (four lanes read one pixel's 64 bytes) whose
 //     completion arrives on the stage's barrier; a pixel outside the image is copied from a run of the input
 //     zero-point kept behind the repacked weights;
-//   * one thread streams the matching slices of the repacked weights with bulk copies into the same stages;
+//   * one thread streams the matching slices of the repacked weights with bulk copies into the same stages; for a
+//     1 x 1 stride-1 layer it also brings the operand rows, one tensor copy (cp.async.bulk.tensor) per block, and
+//     the gather warps idle;
 //   * one thread issues two tcgen05.mma (kind::i8, K = 32) per stage and commits the stage back to the loaders;
 //     accumulators alternate between two column ranges, so a tile's reduction runs under the previous one's
 //     epilogue;
@@ -22,10 +24,14 @@
 //     next tile's residual rows arrive as contiguous runs, under the arithmetic of the following columns.
 // Every wait is bounded; on expiry a role raises the CTA's abort flag and the error word, the others leave their
 // loops, and the CTA frees its tensor memory and returns.
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
 
 #include "isc_epilogue.cuh"
 #include "isc_internal.h"
@@ -50,7 +56,9 @@ constexpr int kGemmThreads = 32 * (kAllEpiWarps + kGatherWarps + 2);      // k_i
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct IgemmParams {
+    alignas(64) CUtensorMap tmap_a;          // the input as (16 bytes, pixel, 16-byte column of the channels): see tma_a
     GLayer L;
+    int tma_a;                               // 1 x 1 stride 1: the operand rows arrive by one tensor copy per block, the gather warps idle
     int batch, n_tile, tmem_cols, stages;
     uint32_t scratch_off;                    // the epilogue warps' row scratch within the dynamic shared memory
     uint32_t m_total, tiles_m;               // batch * hout * wout (< 2^31); tiles of 128 of them
@@ -327,7 +335,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
     const uint32_t a_bytes = kTileM * kBlockK, b_bytes = (uint32_t)n_tile * kBlockK, stage_bytes = a_bytes + b_bytes;
     int4 *cst_s = reinterpret_cast<int4 *>(smem + (size_t)stages * stage_bytes);
     if (tid == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&bar_full[s]), kGatherWarps * 32 + 1); mbar_init(smem_u32(&bar_free[s]), 1); }
+        for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&bar_full[s]), p.tma_a ? 1 : kGatherWarps * 32 + 1); mbar_init(smem_u32(&bar_free[s]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_free[i]), kEpiWarps * 32); }
         abort_s = 0;
     }
@@ -369,7 +377,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
         const uint32_t dst0 = sbase + (uint32_t)chunk * 2048u + (uint32_t)(32 * gw + rsub) * 16u;
         Ring ring;
         const uint32_t px_per_sample = (uint32_t)(L.hout * L.wout);
-        for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += grid_n) {
+        for (uint32_t t = blockIdx.x; t < n_tiles && ok && !p.tma_a; t += grid_n) {
             const uint32_t m0 = (t / (uint32_t)tiles_n) * kTileM + (uint32_t)(32 * gw + rsub);
             int iy0[4], ix0[4], off[4];                         // this lane's four rows: 8 apart
 #pragma unroll
@@ -443,7 +451,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_igemm(const __grid_constant
                         ok = wait_bar<kHintLoad>(smem_u32(&bar_free[ring.s]), (uint32_t)(ring.use - 1) & 1u, &abort_s);
                         if (!ok) break;
                     }
-                    mbar_expect_tx(smem_u32(&bar_full[ring.s]), b_bytes);
+                    mbar_expect_tx(smem_u32(&bar_full[ring.s]), p.tma_a ? a_bytes + b_bytes : b_bytes);
+                    if (p.tma_a) {
+                        // box {16 bytes, 128 pixels, 4 columns} of the 3-D view lands as [column][pixel][16 bytes], which is
+                        // the K-major core-matrix layout; pixels beyond the last one are filled with zeros and never stored
+                        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                                     ::"r"(sbase + (uint32_t)ring.s * stage_bytes), "l"(reinterpret_cast<uint64_t>(&p.tmap_a)), "r"(0),
+                                       "r"((int)((t / (uint32_t)tiles_n) * kTileM)), "r"(kb * 4), "r"(smem_u32(&bar_full[ring.s])) : "memory");
+                    }
                     bulk_g2s(sbase + (uint32_t)ring.s * stage_bytes + a_bytes, wtile + (size_t)kb * b_bytes, b_bytes, smem_u32(&bar_full[ring.s]));
                 }
             }
@@ -752,6 +767,36 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
     const int res_n = 31 - G.res_shift;
     p.fast_residual = (res_n == 31 || res_n == 32) ? 1 : 0;
     p.debug_stall = debug_stall ? 1 : 0;
+    // A 1 x 1 stride-1 layer reads its input as the matrix [pixel][channel]: the tile's operand rows are a box of the
+    // view (16 bytes, pixel, 16-byte column) and come by tensor copy.  The encoder is the driver's, looked up at run
+    // time; without it (or if it refuses the view) the gather warps do the work.
+    p.tma_a = 0;
+    memset(&p.tmap_a, 0, sizeof(p.tmap_a));
+    if (G.kh == 1 && G.kw == 1 && G.stride == 1 && G.pad == 0) {
+        typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                     const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+        static EncodeFn encode = nullptr;
+        static bool looked_up = false;
+        if (!looked_up) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult qr;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
+                encode = (EncodeFn)fn;
+            else
+                cudaGetLastError();
+            looked_up = true;
+        }
+        if (encode) {
+            const cuuint64_t dims[3] = {16, (cuuint64_t)batch * G.hin * G.win, (cuuint64_t)(G.cinp / 16)};
+            const cuuint64_t strides[2] = {(cuuint64_t)G.cinp, 16};
+            const cuuint32_t box[3] = {16, (cuuint32_t)kTileM, (cuuint32_t)(kBlockK / 16)}, estr[3] = {1, 1, 1};
+            const CUresult r = encode(&p.tmap_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t *>(in), dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r == CUDA_SUCCESS) p.tma_a = 1;
+            else if (getenv("ISC_DEBUG_CUDA")) fprintf(stderr, "isc: cuTensorMapEncodeTiled: %d\n", (int)r);
+        }
+    }
     p.res_m2 = 0; p.res_r2 = 0;
     p.res_short = (res && res_k8 != 0xFFFFFFFFu) ? 1 : 0;
     p.res_k8 = p.res_short ? res_k8 : 0u;
