@@ -317,6 +317,9 @@ int isc_debug_residual_form(int32_t res_mult, int32_t res_shift, int32_t zp_res,
 /*
  * isc_set_option -- "batch" and "engine" are tuning knobs that change no result; "noise" selects
  * the noise law and therefore changes the samples.
+ *   "tensor_copy" : 1 (default) = the layer-by-layer tensor-core engine brings the operand rows of
+ *              1 x 1 stride-1 convolutions by tensor copy, 0 = by the copies every other layer uses;
+ *              changes no result.
  *   "noise"  : 0 = the discrete Gaussian of Def. 3.3 / Eq. 2 (IntRS, the default), 1 = the
  *              rounded continuous Gaussian of the comparison method (isc_noise_table_rounded).
  *   "batch"  : noisy samples per launch (0 = choose automatically).

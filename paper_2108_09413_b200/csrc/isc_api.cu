@@ -75,7 +75,7 @@ struct isc_model {
     int32_t *h_counts = nullptr;  size_t h_counts_bytes = 0;
     std::vector<cudaEvent_t> events;
 
-    int64_t opt_batch = 0, opt_engine = 0, opt_noise = 0;
+    int64_t opt_batch = 0, opt_engine = 0, opt_noise = 0, opt_tensor_copy = 1;
     int64_t last_engine = 0, launches = 0;
 };
 
@@ -422,7 +422,7 @@ int generic_forward(isc_model *m, const uint8_t *d_x, const NoiseStream &ns, int
         if (i == 0 && tensor_cores && m->wpacks[0])
             e = launch_stem_conv(G, m->wpacks[0], m->tc_cst[0], m->tc_fast[0] != 0, d_x, m->in_c, ns, batch, out, m->d_tc_err, st);
         else if (i == 0) e = launch_first_conv(G, d_x, m->in_c, ns, batch, out, st);
-        else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], m->tc_cst[(size_t)i], m->tc_fast[(size_t)i] != 0, m->tc_resk[(size_t)i], batch, in, res, out, m->d_tc_err, st);
+        else if (tensor_cores && m->wpacks[(size_t)i]) e = launch_igemm_conv(G, m->wpacks[(size_t)i], m->tc_cst[(size_t)i], m->tc_fast[(size_t)i] != 0, m->tc_resk[(size_t)i], batch, in, res, out, m->d_tc_err, st, false, m->opt_tensor_copy != 0);
         else if (L.op == ISC_CONV2D || L.op == ISC_FC) e = launch_conv(G, batch, in, res, out, st);
         else if (L.op == ISC_GAVGPOOL) e = launch_gavgpool(G, batch, in, out, st);
         else e = launch_maxpool(G, batch, in, out, st);
@@ -1101,6 +1101,11 @@ int isc_set_option(isc_model *m, const char *name, int64_t value)
     if (!strcmp(name, "noise")) {
         if (value != 0 && value != 1) return ISC_ERR_ARG;
         m->opt_noise = value;
+        return ISC_OK;
+    }
+    if (!strcmp(name, "tensor_copy")) {
+        if (value != 0 && value != 1) return ISC_ERR_ARG;
+        m->opt_tensor_copy = value;
         return ISC_OK;
     }
     if (!strcmp(name, "engine")) {

@@ -757,7 +757,7 @@ bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t 
 }
 
 cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, uint32_t res_k8, int batch, const int8_t *in,
-                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st, bool debug_stall)
+                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st, bool debug_stall, bool tensor_copy)
 {
     IgemmParams p;
     p.L = G;
@@ -772,7 +772,7 @@ cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_
     // time; without it (or if it refuses the view) the gather warps do the work.
     p.tma_a = 0;
     memset(&p.tmap_a, 0, sizeof(p.tmap_a));
-    if (G.kh == 1 && G.kw == 1 && G.stride == 1 && G.pad == 0) {
+    if (tensor_copy && G.kh == 1 && G.kw == 1 && G.stride == 1 && G.pad == 0) {
         typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
                                      const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
         static EncodeFn encode = nullptr;

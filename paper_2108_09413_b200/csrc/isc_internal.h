@@ -80,9 +80,12 @@ bool igemm_constants(const GLayer &G, const int32_t *bias_folded, const int32_t 
                      bool has_residual, uint32_t *res_k8);
 // `cst` / `fast`: what igemm_constants produced (device copy).  `err` (device) receives a non-zero word if a bounded
 // wait inside the kernel expired.  `debug_stall`: the kernel's weights are never sent, so that its waits run out
-// (after their 2 s limit) and the CTAs leave through the abort path -- nothing faults or hangs.
+// (after their 2 s limit) and the CTAs leave through the abort path -- nothing faults or hangs.  `tensor_copy`: a
+// 1 x 1 stride-1 layer may take its operand rows by tensor copy (false: the gather warps bring them, as for every
+// other layer).
 cudaError_t launch_igemm_conv(const GLayer &G, const int8_t *wpack, const int32_t *cst, bool fast, uint32_t res_k8, int batch, const int8_t *in,
-                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st, bool debug_stall = false);
+                              const int8_t *res, int8_t *out, int32_t *err, cudaStream_t st, bool debug_stall = false,
+                              bool tensor_copy = true);
 
 // The first convolution (<= 4 input channels, filter at most 8 x 8) on the tensor cores, noise drawn into its staging.
 bool stem_fits(const GLayer &G, int in_c);

@@ -177,9 +177,10 @@ def _bottleneck_net(rng, fast=None):
     return model
 
 
-def _bottleneck_parity(model, rng, seed):
+def _bottleneck_parity(model, rng, seed, tensor_copy=1):
     gm, om = _pair(model)
     gm.set_option("engine", 2)
+    gm.set_option("tensor_copy", tensor_copy)
     x = rng.integers(0, 256, model["in_shape"]).astype(np.uint8)
     sizes = _tensor_sizes(om)
     a0 = oracle.noisy_input(x, 5, seed, 1, 2, 0.25)
@@ -200,7 +201,7 @@ def test_random_bottleneck_nets_on_the_tensor_core_engine(seed):
     allowed shifts: the implicit-GEMM kernel's tiles end inside rows and images, its padding is a non-trivial
     zero-point."""
     rng = np.random.default_rng(900 + seed)
-    _bottleneck_parity(_bottleneck_net(rng), rng, seed)
+    _bottleneck_parity(_bottleneck_net(rng), rng, seed, tensor_copy=seed & 1)      # both ways of bringing 1 x 1 operand rows
 
 
 @pytest.mark.parametrize("res", [(1304428746, 0, 77), (1334892440, -1, -63), (1 << 30, 0, 0),         # no offset form
@@ -211,7 +212,7 @@ def test_bottleneck_nets_32_bit_epilogue_both_residual_forms(res):
     has_form = isc.residual_form(*res) is not None
     assert has_form == (res[0] in (1979951843, 1435772024))
     rng = np.random.default_rng(950 + res[0] % 97)
-    _bottleneck_parity(_bottleneck_net(rng, fast=res), rng, res[0] % 5)
+    _bottleneck_parity(_bottleneck_net(rng, fast=res), rng, res[0] % 5, tensor_copy=res[0] % 2)
 
 
 def test_partition_and_batch_invariance():
